@@ -1,0 +1,190 @@
+/*
+ * esp.h -- C ABI of the B200 (sm_100a) implementation of the ESP
+ * (Embedding-Space Probing) decode-and-verify step.
+ *
+ * One handle owns one model replica on one GPU.  Every device buffer
+ * (weights, workspace) is allocated by the caller and outlives the handle;
+ * the library allocates and frees no device memory.  All work is enqueued on
+ * the CUDA stream given to esp_init.  Every call returns ESP_OK (0) or a
+ * negative ESP_E_* code; nothing throws, aborts or exits.  Device-side
+ * problems (a bounded wait that ran out, an index outside its range) set an
+ * error word that esp_read / esp_step / esp_get_stats report as
+ * ESP_E_DEVICE.
+ *
+ * Pointers are marked [host] or [device].  Matrices are row-major
+ * [out_features][in_features]; dtype 0 = fp32, 1 = bf16 (weights,
+ * activations fed to matrix products and the KV cache share the dtype;
+ * accumulation, normalisation, softmax, the residual stream, the mask vector
+ * and all selection logic are fp32).
+ */
+#ifndef ESP_B200_H
+#define ESP_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    ESP_OK = 0,
+    ESP_E_BADCFG = -1,    /* unsupported or inconsistent configuration */
+    ESP_E_WORKSPACE = -2, /* workspace missing, misaligned or too small */
+    ESP_E_PROMPT = -3,    /* prompt empty, too long, or token id out of range */
+    ESP_E_FULL = -4,      /* the sequence has no room left for another block */
+    ESP_E_DEVICE = -5,    /* device error word set (see esp_stats.device_error) */
+    ESP_E_CUDA = -6,      /* a CUDA runtime/driver call failed */
+    ESP_E_STATE = -7,     /* call out of order (e.g. step before prefill) */
+    ESP_E_ARG = -8        /* NULL or out-of-range argument */
+};
+
+#define ESP_MAX_ROWS 80   /* rows of one block per sequence: tree nodes + mask probes */
+#define ESP_MAX_PROBES 8  /* k */
+#define ESP_MAX_KPRIME 32 /* Top-K entries kept per probe, K + pruner refills */
+
+/* The frozen decoder f_theta (Section 2; LLaMA3 / Qwen3 shapes, Section 4 "Models"). */
+typedef struct {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    int32_t dtype;           /* 0 = fp32 (CUDA-core path), 1 = bf16 (tcgen05 path) */
+    int32_t tied_embeddings; /* informational; lm_head may simply alias embed */
+    int32_t qk_norm;         /* per-head RMSNorm on q and k before RoPE (Qwen3) */
+    float rope_base, rms_eps;
+    int32_t max_seq_len;     /* cached positions per sequence (prompt + generated) */
+    int32_t max_batch;       /* independent sequences sharing one forward pass */
+} esp_model_cfg;
+
+/* Speculation hyper-parameters (Section 3.3-3.5, Section 4 "Block Complexity", "Mask token design"). */
+typedef struct {
+    int32_t n_probes;      /* k mask tokens per anchored node; 0 = plain greedy decoding */
+    int32_t topk;          /* K candidates per probe (Algorithm 1's pool is min(K, B-i)) */
+    int32_t max_nodes;     /* B tree nodes including the last accepted token */
+    int32_t expand_width;  /* nodes per depth that get children: 1 = Top-1 expansion, 0 = all */
+    int32_t n_anchor;      /* nodes (tree order) carrying a probe chain; 0 = every node (paper) */
+    int32_t prune_parent;  /* Section 3.5: drop a candidate equal to its parent's token */
+    int32_t prune_root;    /* also drop a candidate equal to the last generated token */
+    int32_t ema_per_token; /* mask update per emitted token (1) or once per step (0) */
+    float lambda;          /* mask update rate, Eq. (mask_update_mean); 0.1 in the paper */
+} esp_spec_cfg;
+
+/* Model weights. [device] matrices; the per-layer members are [host] arrays of
+ * n_layers [device] pointers.  q_norm / k_norm may be NULL unless qk_norm. */
+typedef struct {
+    const void* embed;      /* [vocab][d_model] */
+    const void* lm_head;    /* [vocab][d_model]; may equal embed */
+    const void* final_norm; /* [d_model] */
+    const void* const* wq;  /* [n_q_heads*head_dim][d_model] */
+    const void* const* wk;  /* [n_kv_heads*head_dim][d_model] */
+    const void* const* wv;  /* [n_kv_heads*head_dim][d_model] */
+    const void* const* wo;  /* [d_model][n_q_heads*head_dim] */
+    const void* const* w_gate; /* [d_ffn][d_model] */
+    const void* const* w_up;   /* [d_ffn][d_model] */
+    const void* const* w_down; /* [d_model][d_ffn] */
+    const void* const* norm_attn; /* [d_model] */
+    const void* const* norm_ffn;  /* [d_model] */
+    const void* const* q_norm;    /* [head_dim] */
+    const void* const* k_norm;    /* [head_dim] */
+} esp_weights;
+
+typedef struct {
+    int64_t steps;          /* decode-and-verify calls so far (all sequences) */
+    int64_t emitted;        /* tokens emitted by those calls (bonus tokens included) */
+    int64_t accept_hist[ESP_MAX_PROBES + 1]; /* [a] = steps that accepted a draft tokens */
+    int32_t device_error;   /* 0, or the first device-side error code recorded */
+    int32_t kernels_per_step; /* kernel launches one esp_step enqueues */
+} esp_stats;
+
+typedef struct esp_handle esp_handle;
+
+/* Bytes of [device] workspace esp_init needs (KV cache for max_batch sequences of
+ * max_seq_len + ESP_MAX_ROWS positions, activations, split-K and attention
+ * partials, per-sequence state).  ESP_E_BADCFG if the configuration is unsupported. */
+int esp_workspace_bytes(const esp_model_cfg* model, const esp_spec_cfg* spec, size_t* bytes_out);
+
+/* Create a handle.  `workspace` [device] must be 256-byte aligned and at least
+ * esp_workspace_bytes large; it is zeroed here.  `cuda_stream` is a cudaStream_t
+ * (NULL = default stream).  Builds the rotary table and TMA descriptors.
+ * The frozen model is the f_theta of Section 2. */
+int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_weights* weights, void* workspace,
+             size_t workspace_bytes, void* cuda_stream, esp_handle** handle_out);
+
+/* Prefill of sequence `seq` (Figure 1 middle; Section 3.3: generation only).
+ * prompt [host] n_prompt ids.  Sets the mask vector to the mean prompt
+ * embedding (Eq. mask_init_mean), runs the prompt in causal blocks with the
+ * k mask rows appended to the last one, caches the prompt rows, emits the
+ * first token (written to *first_token_out [host], may be NULL), applies the
+ * mask update and builds the first draft tree (Algorithm 1).  Synchronises. */
+int esp_prefill(esp_handle* h, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t* first_token_out);
+
+/* One decode-and-verify step for every prefilled sequence (Figure 1 right):
+ * forward over [last accepted token, draft-tree nodes, mask probes] under the
+ * tree mask, argmax / Top-K' + log-sum-exp, lossless verification (Section 2),
+ * KV compaction of the accepted path, mask update (Eq. mask_update_mean) and
+ * the next tree (Algorithm 1 + pruner).  esp_step = esp_step_async + esp_read.
+ * tokens_out [host] [max_batch][ESP_MAX_PROBES+1], n_out [host] [max_batch]. */
+int esp_step(esp_handle* h, int32_t* tokens_out, int32_t* n_out);
+int esp_step_async(esp_handle* h);
+int esp_read(esp_handle* h, int32_t* tokens_out, int32_t* n_out);
+
+/* Test hook: replace the draft tree of sequence `seq` for the next step.
+ * tokens/parents [host] n nodes in breadth-first order (parents[0] = -1,
+ * parents[i] < i); node 0 must carry the current root token.  Has no
+ * counterpart in the paper; it exists to drive acceptance lengths that
+ * random-init models never produce. */
+int esp_set_tree(esp_handle* h, int32_t seq, const int32_t* tokens, const int32_t* parents, int32_t n);
+
+/* Debug/parity access to device state of sequence `seq`, copied to [host] buffers (any may be NULL):
+ *   row_token/row_parent/row_depth [ESP_MAX_ROWS], n_nodes, n_rows, L of the block the NEXT step will run;
+ *   topk_ids/topk_vals [ESP_MAX_ROWS][ESP_MAX_KPRIME], lse [ESP_MAX_ROWS] from the LAST forward;
+ *   mask_vec [d_model].  Synchronises. */
+int esp_debug_state(esp_handle* h, int32_t seq, int32_t* row_token, int32_t* row_parent, int32_t* row_depth,
+                    int32_t* n_nodes, int32_t* n_rows, int32_t* L, int32_t* topk_ids, float* topk_vals, float* lse,
+                    float* mask_vec);
+
+/* Debug/parity: when `logits` [device] fp32 [max_batch*ESP_MAX_ROWS][vocab] is non-NULL, every later forward also
+ * stores the full logits there (the product path never materialises them).  `hidden` [device] fp32
+ * [max_batch*ESP_MAX_ROWS][d_model], if non-NULL, receives the residual stream after the last layer. */
+int esp_debug_capture(esp_handle* h, float* logits, float* hidden);
+
+/* Selects the matrix-product implementation for bf16 models: 0 = tcgen05 tensor-core kernels (default),
+ * 1 = CUDA-core reference kernels (same epilogues; for A/B checks on the GPU).  fp32 models always use 1. */
+int esp_debug_set_gemm(esp_handle* h, int32_t impl);
+
+int esp_get_stats(esp_handle* h, esp_stats* out);
+
+/* Releases host-side bookkeeping only. */
+void esp_free(esp_handle* h);
+
+/* ---- stand-alone operators (the same kernels the step uses), for operator-level parity and timing ---- */
+
+/* Tree-masked GQA attention (Figure 1 right / Figure 3: every row sees the cache and its own
+ * root-to-self path).  All pointers [device].
+ *   q        [batch][ESP_MAX_ROWS][n_q_heads][head_dim]
+ *   kcache,vcache [batch][n_kv_heads][cap][head_dim]; positions 0..L-1 are the cache, the block
+ *            row i's key/value sit at position L+i (the caller writes them there)
+ *   anc      [batch][ESP_MAX_ROWS][2] uint64 ancestor-or-self bitmask over block rows
+ *   depth    [batch][ESP_MAX_ROWS] int32, position of the row minus L
+ *   out      [batch][ESP_MAX_ROWS][n_q_heads][head_dim]
+ *   scratch  esp_tree_attention_scratch_bytes bytes
+ * dtype as in esp_model_cfg; n_rows <= ESP_MAX_ROWS rows are real; L + ESP_MAX_ROWS <= cap.
+ * dcap (a multiple of 16, >= the largest depth) sets where each row's key list switches from the
+ * tensor-core chunks to the position-by-position tail: keys at positions below
+ * floor((L + depth - dcap) / 16) * 16 go through the chunked path, the rest through the tail. */
+int esp_tree_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t cap,
+                                     size_t* bytes_out);
+int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, int32_t cap, int32_t n_q_heads,
+                       int32_t n_kv_heads, int32_t head_dim, int32_t dcap, const void* q, const void* kcache,
+                       const void* vcache, const uint64_t* anc, const int32_t* depth, void* out, void* scratch,
+                       size_t scratch_bytes, void* cuda_stream);
+
+/* y[rows][n_out] (fp32) = x[rows][k_in] (bf16) * w[n_out][k_in]^T (bf16) on the tcgen05 path
+ * (impl 0) or the CUDA-core path (impl 1).  All pointers [device]; x must hold ESP_MAX_ROWS
+ * rows (rows beyond `rows` are ignored); scratch as esp_gemm_scratch_bytes says. */
+int esp_gemm_scratch_bytes(size_t* bytes_out);
+int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const void* x, const void* w, float* y,
+                  void* scratch, size_t scratch_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ESP_B200_H */

@@ -1,0 +1,646 @@
+// C ABI of the ESP B200 library: configuration checks, workspace carving,
+// prefill, the decode-and-verify step and the stand-alone operators.
+#include <math.h>
+#include <new>
+#include <string.h>
+#include <vector>
+
+#include "esp_launch.h"
+
+using namespace esp;
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carve {
+    size_t off = 0;
+    char* base = nullptr;
+    template <typename T> T* take(size_t n) {
+        off = align_up(off, 256);
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+struct Buffers {
+    void *kcache, *vcache;
+    float* hres;
+    void *xn, *qbuf, *attn_out, *act;
+    float* part_o;
+    float2* part_ml;
+    Cand* cand;
+    float2* cand_ms;
+    Cand* topk;
+    float* lse;
+    float* mvec;
+    SeqState* states;
+    int* err;
+    int32_t* out_ring;
+    int32_t* prompt_dev;
+    int32_t* tree_dev;
+    float *rope_cos, *rope_sin;
+    void* gemm_partials;
+    int* gemm_counters;
+};
+
+
+int spec_rows(const esp_spec_cfg& s) {
+    int nA = s.n_probes > 0 ? (s.n_anchor == 0 ? s.max_nodes : (s.n_anchor < s.max_nodes ? s.n_anchor : s.max_nodes)) : 0;
+    return s.max_nodes + s.n_probes * nA;
+}
+
+int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
+    if (!m || !s) return ESP_E_ARG;
+    if (m->dtype != 0 && m->dtype != 1) return ESP_E_BADCFG;
+    if (m->n_layers < 1 || m->d_model < 8 || m->d_ffn < 8 || m->vocab < 2) return ESP_E_BADCFG;
+    if (m->head_dim != 32 && m->head_dim != 64 && m->head_dim != 128) return ESP_E_BADCFG;
+    if (m->n_kv_heads < 1 || m->n_q_heads % m->n_kv_heads) return ESP_E_BADCFG;
+    if ((m->n_q_heads * m->head_dim) % TILE_N || (m->n_kv_heads * m->head_dim) % TILE_N) return ESP_E_BADCFG;
+    if (m->d_model % 8 || m->d_ffn % 8) return ESP_E_BADCFG;  // 16-byte rows for TMA and vector loads
+    if (m->vocab > 2048 * TILE_N) return ESP_E_BADCFG;
+    if (m->max_batch < 1 || m->max_seq_len < 1) return ESP_E_BADCFG;
+    if (s->n_probes < 0 || s->n_probes > PROBES_MAX) return ESP_E_BADCFG;
+    if (s->max_nodes < 1) return ESP_E_BADCFG;
+    const int KP = s->topk + (s->prune_parent ? 1 : 0) + (s->prune_root ? 1 : 0);
+    if (s->n_probes > 0 && (s->topk < 1 || KP > KP_MAX || KP > m->vocab)) return ESP_E_BADCFG;
+    if (spec_rows(*s) > RT) return ESP_E_BADCFG;
+    if (2 * s->n_probes > DCAP_STEP) return ESP_E_BADCFG;
+    if (s->expand_width < 0 || s->n_anchor < 0) return ESP_E_BADCFG;
+    // Algorithm 1 must not create more than MAX_CAND nodes
+    long created = 1, n_exp = 1;
+    for (int i = 1; i <= s->n_probes; ++i) {
+        long pool = s->topk < s->max_nodes - i ? s->topk : s->max_nodes - i;
+        if (pool <= 0) break;
+        long n_new = n_exp * pool;
+        created += n_new;
+        long width = s->expand_width == 0 ? s->max_nodes - i : (s->expand_width < s->max_nodes - i ? s->expand_width : s->max_nodes - i);
+        n_exp = width < n_new ? width : n_new;
+    }
+    if (created > MAX_CAND) return ESP_E_BADCFG;
+    if (D) {
+        D->n_layers = m->n_layers; D->d = m->d_model; D->Hq = m->n_q_heads; D->Hkv = m->n_kv_heads; D->h = m->head_dim;
+        D->F = m->d_ffn; D->V = m->vocab; D->qk_norm = m->qk_norm;
+        D->cap = m->max_seq_len + RT;
+        D->batch = m->max_batch;
+        int S = 256;
+        while ((m->max_seq_len + S - 1) / S > 64) S *= 2;
+        D->split_len = S;
+        D->n_split_max = (m->max_seq_len + S - 1) / S + 1;
+        D->rms_eps = m->rms_eps;
+        D->k = s->n_probes; D->K = s->topk; D->KP = s->n_probes > 0 ? KP : 1; D->B = s->max_nodes; D->W = s->expand_width;
+        D->n_anchor = s->n_anchor; D->prune_parent = s->prune_parent; D->prune_root = s->prune_root;
+        D->ema_per_token = s->ema_per_token; D->lambda = s->lambda;
+    }
+    return ESP_OK;
+}
+
+size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
+    Carve c;
+    c.base = base;
+    const size_t es = dtype ? 2 : 4;
+    const size_t Mtot = (size_t)D.batch * RT;
+    const size_t kv = (size_t)D.n_layers * D.batch * D.Hkv * D.cap * D.h * es;
+    const int n_tiles_v = (D.V + TILE_N - 1) / TILE_N;
+    Buffers tmp;
+    Buffers& o = b ? *b : tmp;
+    o.kcache = c.take<char>(kv);
+    o.vcache = c.take<char>(kv);
+    o.hres = c.take<float>(Mtot * D.d);
+    o.xn = c.take<char>(Mtot * D.d * es);
+    o.qbuf = c.take<char>(Mtot * D.Hq * D.h * es);
+    o.attn_out = c.take<char>(Mtot * D.Hq * D.h * es);
+    o.act = c.take<char>(Mtot * D.F * es);
+    o.part_o = c.take<float>(Mtot * D.Hq * D.n_split_max * D.h);
+    o.part_ml = c.take<float2>(Mtot * D.Hq * D.n_split_max);
+    o.cand = c.take<Cand>((size_t)n_tiles_v * Mtot * D.KP);
+    o.cand_ms = c.take<float2>((size_t)n_tiles_v * Mtot);
+    o.topk = c.take<Cand>(Mtot * KP_MAX);
+    o.lse = c.take<float>(Mtot);
+    o.mvec = c.take<float>((size_t)D.batch * D.d);
+    o.states = c.take<SeqState>(D.batch);
+    o.err = c.take<int>(4);
+    o.out_ring = c.take<int32_t>((size_t)D.batch * RING);
+    o.prompt_dev = c.take<int32_t>(D.cap);
+    o.tree_dev = c.take<int32_t>(2 * RT);
+    o.rope_cos = c.take<float>((size_t)D.cap * (D.h / 2));
+    o.rope_sin = c.take<float>((size_t)D.cap * (D.h / 2));
+    o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm));
+    o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
+    return align_up(c.off, 256);
+}
+
+}  // namespace
+
+struct esp_handle {
+    esp_model_cfg mc;
+    esp_spec_cfg sc;
+    Dims D;
+    Buffers b;
+    cudaStream_t stream;
+    int dtype, gemm_impl, n_sm;
+    const void *embed, *lm_head, *final_norm;
+    std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, na, nf, qn, kn;
+    std::vector<TcGemm*> p_qkv, p_o, p_gu, p_down;
+    TcGemm* p_lm = nullptr;
+    std::vector<int> L_host, ready;
+    int32_t* pinned = nullptr;  // [batch][RING] + 4 ints (error words)
+    float *dbg_logits = nullptr, *dbg_hidden = nullptr;
+    int launches = 0, kernels_per_step = 0;
+    size_t layer_kv_stride = 0;  // bytes
+};
+
+namespace {
+
+int cuda_ok(cudaError_t e) { return e == cudaSuccess ? ESP_OK : ESP_E_CUDA; }
+
+void* layer_ptr(void* base, size_t stride_bytes, int l) { return reinterpret_cast<char*>(base) + stride_bytes * l; }
+
+EpiArgs base_epi(esp_handle* h, int n_out) {
+    EpiArgs a;
+    memset(&a, 0, sizeof(a));
+    a.n_out = n_out;
+    a.st = h->b.states;
+    a.batch = h->D.batch;
+    a.Hq = h->D.Hq; a.Hkv = h->D.Hkv; a.h = h->D.h; a.cap = h->D.cap; a.qk_norm = h->D.qk_norm;
+    a.rms_eps = h->D.rms_eps;
+    a.rope_cos = h->b.rope_cos; a.rope_sin = h->b.rope_sin;
+    a.KP = h->D.KP;
+    return a;
+}
+
+int run_gemm(esp_handle* h, TcGemm* plan, int epi, int n_tiles, const void* const w[3], const int32_t rows_w[3],
+             const void* x, int K, const EpiArgs& a) {
+    h->launches++;
+    if (h->dtype == 1 && h->gemm_impl == 0 && plan) return tc_gemm_launch(plan, a, h->stream);
+    launch_gemm_simt(h->dtype, epi, n_tiles, h->D.batch, w, rows_w, x, K, a, h->stream);
+    return ESP_OK;
+}
+
+int forward(esp_handle* h, bool with_lm, int dcap) {
+    const Dims& D = h->D;
+    Buffers& b = h->b;
+    cudaStream_t s = h->stream;
+    const int dq = D.Hq * D.h, dkv = D.Hkv * D.h;
+    int Lmax = 0;
+    for (int i = 0; i < D.batch; ++i) Lmax = h->L_host[i] > Lmax ? h->L_host[i] : Lmax;
+    const int n_split_launch = (Lmax + D.split_len - 1) / D.split_len;
+    launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.batch, s);
+    h->launches++;
+    for (int l = 0; l < D.n_layers; ++l) {
+        launch_rmsnorm(h->dtype, b.states, b.hres, h->na[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s);
+        h->launches++;
+        {
+            EpiArgs a = base_epi(h, dq + 2 * dkv);
+            a.q_out = b.qbuf;
+            a.kcache = layer_ptr(b.kcache, h->layer_kv_stride, l);
+            a.vcache = layer_ptr(b.vcache, h->layer_kv_stride, l);
+            a.q_norm = D.qk_norm ? h->qn[l] : nullptr;
+            a.k_norm = D.qk_norm ? h->kn[l] : nullptr;
+            const void* w[3] = {h->wq[l], h->wk[l], h->wv[l]};
+            const int32_t rows[3] = {dq, dkv, dkv};
+            int rc = run_gemm(h, h->p_qkv.empty() ? nullptr : h->p_qkv[l], EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a);
+            if (rc) return rc;
+        }
+        {
+            AttnArgs a;
+            memset(&a, 0, sizeof(a));
+            a.q = b.qbuf;
+            a.kc = layer_ptr(b.kcache, h->layer_kv_stride, l);
+            a.vc = layer_ptr(b.vcache, h->layer_kv_stride, l);
+            a.out = b.attn_out;
+            a.part_o = b.part_o; a.part_ml = b.part_ml;
+            a.st = b.states;
+            a.Hq = D.Hq; a.Hkv = D.Hkv; a.h = D.h; a.cap = D.cap; a.split_len = D.split_len; a.n_split_max = D.n_split_max;
+            a.dcap = dcap;
+            a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
+            a.err = b.err;
+            const bool mma = h->dtype == 1 && D.h == 128 && h->gemm_impl == 0;
+            if (mma && n_split_launch > 0) {
+                if (launch_attn_bulk_mma(a, D.batch, n_split_launch, s)) return ESP_E_BADCFG;
+                h->launches++;
+            }
+            if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, !mma, s)) return ESP_E_BADCFG;
+            h->launches += (!mma && n_split_launch > 0) ? 2 : 1;
+        }
+        {
+            EpiArgs a = base_epi(h, D.d);
+            a.hres = b.hres;
+            const void* w[3] = {h->wo[l], nullptr, nullptr};
+            const int32_t rows[3] = {D.d, 0, 0};
+            int rc = run_gemm(h, h->p_o.empty() ? nullptr : h->p_o[l], EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.attn_out, dq, a);
+            if (rc) return rc;
+        }
+        launch_rmsnorm(h->dtype, b.states, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s);
+        h->launches++;
+        {
+            EpiArgs a = base_epi(h, D.F);
+            a.act_out = b.act;
+            const void* w[3] = {h->wg[l], h->wu[l], nullptr};
+            const int32_t rows[3] = {D.F, D.F, 0};
+            int rc = run_gemm(h, h->p_gu.empty() ? nullptr : h->p_gu[l], EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a);
+            if (rc) return rc;
+        }
+        {
+            EpiArgs a = base_epi(h, D.d);
+            a.hres = b.hres;
+            const void* w[3] = {h->wd[l], nullptr, nullptr};
+            const int32_t rows[3] = {D.d, 0, 0};
+            int rc = run_gemm(h, h->p_down.empty() ? nullptr : h->p_down[l], EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.act, D.F, a);
+            if (rc) return rc;
+        }
+    }
+    if (with_lm) {
+        launch_rmsnorm(h->dtype, b.states, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, D.batch, h->dbg_hidden, s);
+        h->launches++;
+        const int n_tiles = (D.V + TILE_N - 1) / TILE_N;
+        EpiArgs a = base_epi(h, D.V);
+        a.cand = b.cand; a.cand_ms = b.cand_ms; a.n_tiles = n_tiles; a.logits_dump = h->dbg_logits;
+        const void* w[3] = {h->lm_head, nullptr, nullptr};
+        const int32_t rows[3] = {D.V, 0, 0};
+        int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a);
+        if (rc) return rc;
+        launch_topk_merge(b.states, b.cand, b.cand_ms, n_tiles, D.KP, D.batch, b.topk, b.lse, s);
+        h->launches++;
+    }
+    return cuda_ok(cudaGetLastError());
+}
+
+int tree_step(esp_handle* h) {
+    TreeArgs A;
+    A.D = h->D;
+    A.states = h->b.states;
+    A.topk = h->b.topk;
+    A.lse = h->b.lse;
+    A.mvec = h->b.mvec;
+    A.embed = h->embed;
+    A.kcache = h->b.kcache;
+    A.vcache = h->b.vcache;
+    A.err = h->b.err;
+    A.out_ring = h->b.out_ring;
+    launch_tree_step(h->dtype, A, h->stream);
+    h->launches++;
+    return cuda_ok(cudaGetLastError());
+}
+
+__global__ void k_select(SeqState* st, int batch, int seq_only) {
+    int i = threadIdx.x;
+    if (i < batch) st[i].active = seq_only < 0 ? st[i].ready : (i == seq_only);
+}
+__global__ void k_mark_ready(SeqState* st, int seq) { st[seq].ready = 1; }
+
+int read_ring(esp_handle* h) {
+    const int n = h->D.batch * RING;
+    if (cudaMemcpyAsync(h->pinned, h->b.out_ring, sizeof(int32_t) * n, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return ESP_E_CUDA;
+    if (cudaMemcpyAsync(h->pinned + n, h->b.err, sizeof(int), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return ESP_E_CUDA;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return ESP_E_CUDA;
+    return h->pinned[n] ? ESP_E_DEVICE : ESP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int esp_workspace_bytes(const esp_model_cfg* model, const esp_spec_cfg* spec, size_t* bytes_out) {
+    if (!bytes_out) return ESP_E_ARG;
+    Dims D;
+    int rc = check_cfg(model, spec, &D);
+    if (rc) return rc;
+    *bytes_out = carve_all(D, model->dtype, 148, nullptr, nullptr);
+    return ESP_OK;
+}
+
+int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_weights* w, void* workspace,
+             size_t workspace_bytes, void* cuda_stream, esp_handle** handle_out) {
+    if (!handle_out || !w || !workspace) return ESP_E_ARG;
+    Dims D;
+    int rc = check_cfg(model, spec, &D);
+    if (rc) return rc;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256) return ESP_E_WORKSPACE;
+    size_t need = carve_all(D, model->dtype, 148, nullptr, nullptr);
+    if (workspace_bytes < need) return ESP_E_WORKSPACE;
+    if (!w->embed || !w->lm_head || !w->final_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up ||
+        !w->w_down || !w->norm_attn || !w->norm_ffn)
+        return ESP_E_ARG;
+    if (model->qk_norm && (!w->q_norm || !w->k_norm)) return ESP_E_ARG;
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ESP_E_CUDA;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ESP_E_CUDA;
+    if (n_sm > 148) n_sm = 148;
+    esp_handle* h = new (std::nothrow) esp_handle();
+    if (!h) return ESP_E_ARG;
+    h->mc = *model; h->sc = *spec; h->D = D;
+    h->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    h->dtype = model->dtype;
+    h->gemm_impl = model->dtype == 0 ? 1 : 0;
+    h->n_sm = n_sm;
+    carve_all(D, model->dtype, 148, reinterpret_cast<char*>(workspace), &h->b);
+    h->embed = w->embed; h->lm_head = w->lm_head; h->final_norm = w->final_norm;
+    for (int l = 0; l < D.n_layers; ++l) {
+        h->wq.push_back(w->wq[l]); h->wk.push_back(w->wk[l]); h->wv.push_back(w->wv[l]); h->wo.push_back(w->wo[l]);
+        h->wg.push_back(w->w_gate[l]); h->wu.push_back(w->w_up[l]); h->wd.push_back(w->w_down[l]);
+        h->na.push_back(w->norm_attn[l]); h->nf.push_back(w->norm_ffn[l]);
+        h->qn.push_back(model->qk_norm ? w->q_norm[l] : nullptr); h->kn.push_back(model->qk_norm ? w->k_norm[l] : nullptr);
+    }
+    h->L_host.assign(D.batch, 0);
+    h->ready.assign(D.batch, 0);
+    h->layer_kv_stride = (size_t)D.batch * D.Hkv * D.cap * D.h * (model->dtype ? 2 : 4);
+    if (cudaMemsetAsync(workspace, 0, need, h->stream) != cudaSuccess) { delete h; return ESP_E_CUDA; }
+    if (cudaHostAlloc(reinterpret_cast<void**>(&h->pinned), sizeof(int32_t) * (D.batch * RING + 4), cudaHostAllocDefault) != cudaSuccess) {
+        delete h;
+        return ESP_E_CUDA;
+    }
+    launch_rope_table(h->b.rope_cos, h->b.rope_sin, D.cap, D.h, model->rope_base, h->stream);
+    if (model->dtype == 1 && D.batch == 1) {
+        const int dq = D.Hq * D.h, dkv = D.Hkv * D.h;
+        bool ok = true;
+        for (int l = 0; l < D.n_layers && ok; ++l) {
+            TcGemm* p = nullptr;
+            const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
+            const int32_t r1[3] = {dq, dkv, dkv};
+            ok = ok && !tc_gemm_create(&p, EPI_QKV, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            h->p_qkv.push_back(p);
+            const void* w2[3] = {h->wo[l], nullptr, nullptr};
+            const int32_t r2[3] = {D.d, 0, 0};
+            p = nullptr;
+            ok = ok && !tc_gemm_create(&p, EPI_RESID, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            h->p_o.push_back(p);
+            const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
+            const int32_t r3[3] = {D.F, D.F, 0};
+            p = nullptr;
+            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, w3, r3, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            h->p_gu.push_back(p);
+            const void* w4[3] = {h->wd[l], nullptr, nullptr};
+            const int32_t r4[3] = {D.d, 0, 0};
+            p = nullptr;
+            ok = ok && !tc_gemm_create(&p, EPI_RESID, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            h->p_down.push_back(p);
+        }
+        const void* w5[3] = {h->lm_head, nullptr, nullptr};
+        const int32_t r5[3] = {D.V, 0, 0};
+        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+        if (!ok) { esp_free(h); return ESP_E_CUDA; }
+    } else if (model->dtype == 1) {
+        h->gemm_impl = 1;  // batched rows: CUDA-core path until the tensor-core kernel tiles over sequences
+    }
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) { esp_free(h); return ESP_E_CUDA; }
+    *handle_out = h;
+    return ESP_OK;
+}
+
+int esp_prefill(esp_handle* h, int32_t seq, const int32_t* prompt, int32_t n_prompt, int32_t* first_token_out) {
+    if (!h || !prompt) return ESP_E_ARG;
+    if (seq < 0 || seq >= h->D.batch) return ESP_E_ARG;
+    if (n_prompt < 1 || n_prompt > h->mc.max_seq_len) return ESP_E_PROMPT;
+    for (int i = 0; i < n_prompt; ++i)
+        if (prompt[i] < 0 || prompt[i] >= h->D.V) return ESP_E_PROMPT;
+    cudaStream_t s = h->stream;
+    if (cudaMemcpyAsync(h->b.prompt_dev, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, s) != cudaSuccess) return ESP_E_CUDA;
+    launch_mask_mean(h->dtype, h->embed, h->b.prompt_dev, n_prompt, h->D.d, h->b.mvec + (size_t)seq * h->D.d, s);
+    k_select<<<1, 32, 0, s>>>(h->b.states, h->D.batch, seq);
+    std::vector<int> saved = h->L_host;
+    for (int i = 0; i < h->D.batch; ++i) h->L_host[i] = 0;
+    for (int off = 0; off < n_prompt; off += PREFILL_CHUNK) {
+        const int cn = n_prompt - off < PREFILL_CHUNK ? n_prompt - off : PREFILL_CHUNK;
+        const int last = off + cn == n_prompt;
+        launch_setup_chain(h->b.states, seq, h->b.prompt_dev, off, cn, last, h->D.k, s);
+        h->L_host[seq] = off;
+        int rc = forward(h, last, DCAP_PREFILL);
+        if (rc) return rc;
+        rc = tree_step(h);
+        if (rc) return rc;
+    }
+    k_mark_ready<<<1, 1, 0, s>>>(h->b.states, seq);
+    k_select<<<1, 32, 0, s>>>(h->b.states, h->D.batch, -1);
+    int rc = read_ring(h);
+    h->L_host = saved;
+    h->L_host[seq] = n_prompt;
+    h->ready[seq] = 1;
+    if (rc) return rc;
+    if (first_token_out) *first_token_out = h->pinned[seq * RING + 2];
+    return ESP_OK;
+}
+
+int esp_step_async(esp_handle* h) {
+    if (!h) return ESP_E_ARG;
+    bool any = false;
+    for (int i = 0; i < h->D.batch; ++i) {
+        if (!h->ready[i]) continue;
+        any = true;
+        if (h->L_host[i] + h->D.k + 1 + RT > h->D.cap) return ESP_E_FULL;
+    }
+    if (!any) return ESP_E_STATE;
+    const int before = h->launches;
+    int rc = forward(h, true, DCAP_STEP);
+    if (rc) return rc;
+    rc = tree_step(h);
+    h->kernels_per_step = h->launches - before;
+    // until the result is read the host only knows an upper bound of each cache length
+    for (int i = 0; i < h->D.batch; ++i)
+        if (h->ready[i]) h->L_host[i] += h->D.k + 1;
+    return rc;
+}
+
+int esp_read(esp_handle* h, int32_t* tokens_out, int32_t* n_out) {
+    if (!h) return ESP_E_ARG;
+    int rc = read_ring(h);
+    for (int i = 0; i < h->D.batch; ++i) {
+        if (!h->ready[i]) { if (n_out) n_out[i] = 0; continue; }
+        const int32_t* r = h->pinned + i * RING;
+        h->L_host[i] = r[1];
+        if (n_out) n_out[i] = r[0];
+        if (tokens_out)
+            for (int j = 0; j < r[0] && j <= PROBES_MAX; ++j) tokens_out[i * (PROBES_MAX + 1) + j] = r[2 + j];
+    }
+    return rc;
+}
+
+int esp_step(esp_handle* h, int32_t* tokens_out, int32_t* n_out) {
+    int rc = esp_step_async(h);
+    if (rc) return rc;
+    return esp_read(h, tokens_out, n_out);
+}
+
+int esp_set_tree(esp_handle* h, int32_t seq, const int32_t* tokens, const int32_t* parents, int32_t n) {
+    if (!h || !tokens || !parents) return ESP_E_ARG;
+    if (seq < 0 || seq >= h->D.batch || !h->ready[seq]) return ESP_E_STATE;
+    const int k = h->D.k;
+    const int nA = k > 0 ? (h->D.n_anchor == 0 ? n : (h->D.n_anchor < n ? h->D.n_anchor : n)) : 0;
+    if (n < 1 || n + nA * k > RT) return ESP_E_ARG;
+    std::vector<int> depth(n, 0);
+    for (int i = 0; i < n; ++i) {
+        if (tokens[i] < 0 || tokens[i] >= h->D.V) return ESP_E_ARG;
+        if (i == 0 ? parents[i] != -1 : (parents[i] < 0 || parents[i] >= i)) return ESP_E_ARG;
+        if (i) depth[i] = depth[parents[i]] + 1;
+        if (depth[i] + k > DCAP_STEP || depth[i] > PROBES_MAX) return ESP_E_ARG;
+    }
+    cudaStream_t s = h->stream;
+    if (cudaMemcpyAsync(h->b.tree_dev, tokens, sizeof(int32_t) * n, cudaMemcpyHostToDevice, s) != cudaSuccess) return ESP_E_CUDA;
+    if (cudaMemcpyAsync(h->b.tree_dev + RT, parents, sizeof(int32_t) * n, cudaMemcpyHostToDevice, s) != cudaSuccess) return ESP_E_CUDA;
+    launch_set_tree(h->b.states, seq, h->b.tree_dev, h->b.tree_dev + RT, n, k, h->D.n_anchor, h->b.err, s);
+    return cuda_ok(cudaStreamSynchronize(s));
+}
+
+int esp_debug_state(esp_handle* h, int32_t seq, int32_t* row_token, int32_t* row_parent, int32_t* row_depth,
+                    int32_t* n_nodes, int32_t* n_rows, int32_t* L, int32_t* topk_ids, float* topk_vals, float* lse,
+                    float* mask_vec) {
+    if (!h || seq < 0 || seq >= h->D.batch) return ESP_E_ARG;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return ESP_E_CUDA;
+    SeqState st;
+    if (cudaMemcpy(&st, h->b.states + seq, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+    if (row_token) memcpy(row_token, st.row_token, sizeof(st.row_token));
+    if (row_parent) memcpy(row_parent, st.row_parent, sizeof(st.row_parent));
+    if (row_depth) memcpy(row_depth, st.row_depth, sizeof(st.row_depth));
+    if (n_nodes) *n_nodes = st.n_nodes;
+    if (n_rows) *n_rows = st.n_rows;
+    if (L) *L = st.L;
+    if (topk_ids || topk_vals) {
+        std::vector<Cand> c((size_t)RT * KP_MAX);
+        if (cudaMemcpy(c.data(), h->b.topk + (size_t)seq * RT * KP_MAX, sizeof(Cand) * c.size(), cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+        for (size_t i = 0; i < c.size(); ++i) {
+            if (topk_ids) topk_ids[i] = c[i].id;
+            if (topk_vals) topk_vals[i] = c[i].val;
+        }
+    }
+    if (lse && cudaMemcpy(lse, h->b.lse + (size_t)seq * RT, sizeof(float) * RT, cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+    if (mask_vec && cudaMemcpy(mask_vec, h->b.mvec + (size_t)seq * h->D.d, sizeof(float) * h->D.d, cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+    return ESP_OK;
+}
+
+int esp_debug_capture(esp_handle* h, float* logits, float* hidden) {
+    if (!h) return ESP_E_ARG;
+    h->dbg_logits = logits;
+    h->dbg_hidden = hidden;
+    return ESP_OK;
+}
+
+int esp_debug_set_gemm(esp_handle* h, int32_t impl) {
+    if (!h || (impl != 0 && impl != 1)) return ESP_E_ARG;
+    if (h->dtype == 0 && impl == 0) return ESP_E_BADCFG;
+    if (impl == 0 && !h->p_lm) return ESP_E_BADCFG;
+    h->gemm_impl = impl;
+    return ESP_OK;
+}
+
+int esp_get_stats(esp_handle* h, esp_stats* out) {
+    if (!h || !out) return ESP_E_ARG;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return ESP_E_CUDA;
+    memset(out, 0, sizeof(*out));
+    for (int i = 0; i < h->D.batch; ++i) {
+        SeqState st;
+        if (cudaMemcpy(&st, h->b.states + i, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+        out->steps += (int64_t)st.steps;
+        out->emitted += (int64_t)st.emitted;
+        for (int a = 0; a <= PROBES_MAX; ++a) out->accept_hist[a] += (int64_t)st.accept_hist[a];
+    }
+    int e = 0;
+    if (cudaMemcpy(&e, h->b.err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+    out->device_error = e;
+    out->kernels_per_step = h->kernels_per_step;
+    return ESP_OK;
+}
+
+void esp_free(esp_handle* h) {
+    if (!h) return;
+    for (auto* p : h->p_qkv) tc_gemm_destroy(p);
+    for (auto* p : h->p_o) tc_gemm_destroy(p);
+    for (auto* p : h->p_gu) tc_gemm_destroy(p);
+    for (auto* p : h->p_down) tc_gemm_destroy(p);
+    tc_gemm_destroy(h->p_lm);
+    if (h->pinned) cudaFreeHost(h->pinned);
+    delete h;
+}
+
+// ------------------------------------------------------------------ stand-alone operators
+int esp_tree_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t cap, size_t* bytes_out) {
+    if (!bytes_out || batch < 1 || n_q_heads < 1 || cap < RT) return ESP_E_ARG;
+    int S = 256;
+    while ((cap + S - 1) / S > 64) S *= 2;
+    const size_t ns = (cap + S - 1) / S + 1;
+    const size_t rows = (size_t)batch * RT * n_q_heads * ns;
+    *bytes_out = align_up(rows * head_dim * sizeof(float), 256) + align_up(rows * sizeof(float2), 256) + 256;
+    return ESP_OK;
+}
+
+int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, int32_t cap, int32_t n_q_heads,
+                       int32_t n_kv_heads, int32_t head_dim, int32_t dcap, const void* q, const void* kcache,
+                       const void* vcache, const uint64_t* anc, const int32_t* depth, void* out, void* scratch,
+                       size_t scratch_bytes, void* cuda_stream) {
+    if (!q || !kcache || !vcache || !anc || !depth || !out || !scratch) return ESP_E_ARG;
+    if (dtype != 0 && dtype != 1) return ESP_E_BADCFG;
+    if (head_dim != 32 && head_dim != 64 && head_dim != 128) return ESP_E_BADCFG;
+    if (n_kv_heads < 1 || n_q_heads % n_kv_heads || batch < 1) return ESP_E_BADCFG;
+    if (n_rows < 1 || n_rows > RT || L < 0 || L + RT > cap || dcap < 16 || dcap % 16) return ESP_E_ARG;
+    size_t need = 0;
+    esp_tree_attention_scratch_bytes(batch, n_q_heads, head_dim, cap, &need);
+    if (scratch_bytes < need || reinterpret_cast<uintptr_t>(scratch) % 256) return ESP_E_WORKSPACE;
+    int S = 256;
+    while ((cap + S - 1) / S > 64) S *= 2;
+    const size_t ns = (cap + S - 1) / S + 1;
+    const size_t rows = (size_t)batch * RT * n_q_heads * ns;
+    AttnArgs a;
+    memset(&a, 0, sizeof(a));
+    a.q = q; a.kc = kcache; a.vc = vcache; a.out = out;
+    a.part_o = reinterpret_cast<float*>(scratch);
+    a.part_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(scratch) + align_up(rows * head_dim * sizeof(float), 256));
+    a.st = nullptr;
+    a.anc = reinterpret_cast<const unsigned long long*>(anc);
+    a.depth = depth;
+    a.n_rows_fixed = n_rows; a.L_fixed = L;
+    a.Hq = n_q_heads; a.Hkv = n_kv_heads; a.h = head_dim; a.cap = cap; a.split_len = S; a.n_split_max = (int)ns; a.dcap = dcap;
+    a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)head_dim));
+    a.err = reinterpret_cast<int*>(reinterpret_cast<char*>(scratch) + need - 256);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const int n_split_launch = (L + S - 1) / S;
+    const bool mma = dtype == 1 && head_dim == 128;
+    if (mma && n_split_launch > 0 && launch_attn_bulk_mma(a, batch, n_split_launch, s)) return ESP_E_BADCFG;
+    if (launch_attn_simt(dtype, a, batch, n_split_launch, !mma, s)) return ESP_E_BADCFG;
+    return cuda_ok(cudaGetLastError());
+}
+
+int esp_gemm_scratch_bytes(size_t* bytes_out) {
+    if (!bytes_out) return ESP_E_ARG;
+    *bytes_out = align_up(tc_gemm_partial_bytes(148), 256) + align_up(sizeof(int) * tc_gemm_counter_ints(), 256) + 256;
+    return ESP_OK;
+}
+
+int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const void* x, const void* w, float* y,
+                  void* scratch, size_t scratch_bytes, void* cuda_stream) {
+    if (!x || !w || !y || !scratch) return ESP_E_ARG;
+    if (rows < 1 || rows > RT || n_out < 1 || k_in < 8 || k_in % 8) return ESP_E_ARG;
+    size_t need = 0;
+    esp_gemm_scratch_bytes(&need);
+    if (scratch_bytes < need || reinterpret_cast<uintptr_t>(scratch) % 256) return ESP_E_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    EpiArgs a;
+    memset(&a, 0, sizeof(a));
+    a.n_out = n_out; a.st = nullptr; a.rows_fixed = rows; a.batch = 1; a.y_f32 = y;
+    const void* wv[3] = {w, nullptr, nullptr};
+    const int32_t rw[3] = {n_out, 0, 0};
+    const int n_tiles = (n_out + TILE_N - 1) / TILE_N;
+    if (impl == 1) {
+        launch_gemm_simt(1, EPI_STORE_F32, n_tiles, 1, wv, rw, x, k_in, a, s);
+        return cuda_ok(cudaGetLastError());
+    }
+    if (impl != 0) return ESP_E_ARG;
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ESP_E_CUDA;
+    if (n_sm > 148) n_sm = 148;
+    char* sc = reinterpret_cast<char*>(scratch);
+    int* counters = reinterpret_cast<int*>(sc + align_up(tc_gemm_partial_bytes(148), 256));
+    int* err = reinterpret_cast<int*>(sc + need - 256);
+    if (cudaMemsetAsync(counters, 0, sizeof(int) * tc_gemm_counter_ints() , s) != cudaSuccess) return ESP_E_CUDA;
+    if (cudaMemsetAsync(err, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
+    TcGemm* plan = nullptr;
+    if (tc_gemm_create(&plan, EPI_STORE_F32, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err)) return ESP_E_CUDA;
+    int rc = tc_gemm_launch(plan, a, s);
+    int e = 0;
+    if (!rc && cudaMemcpyAsync(&e, err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) rc = ESP_E_CUDA;
+    if (!rc && cudaStreamSynchronize(s) != cudaSuccess) rc = ESP_E_CUDA;
+    tc_gemm_destroy(plan);
+    if (!rc && e) rc = ESP_E_DEVICE;
+    return rc;
+}
+
+}  // extern "C"

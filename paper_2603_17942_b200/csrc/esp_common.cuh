@@ -1,0 +1,136 @@
+// Shared declarations of the ESP B200 library: device state layout, launch
+// parameters and small device helpers.  Everything here is device/product
+// code; the CPU oracle shares none of it.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/esp.h"
+
+namespace esp {
+
+constexpr int RT = ESP_MAX_ROWS;        // rows of one block per sequence
+constexpr int KP_MAX = ESP_MAX_KPRIME;  // Top-K' entries kept per row
+constexpr int PROBES_MAX = ESP_MAX_PROBES;
+constexpr int TILE_N = 128;             // output features per GEMM tile
+constexpr int MAX_CAND = 4096;          // nodes Algorithm 1 may create in one step
+constexpr int PREFILL_CHUNK = 64;       // prompt rows per prefill block
+constexpr int DCAP_STEP = 16;           // tail cap of decode steps (>= 2k)
+constexpr int DCAP_PREFILL = 80;        // tail cap of prefill chain blocks
+constexpr int RING = ESP_MAX_PROBES + 4; // per-sequence result record: n_out, L, tokens
+
+// device error codes (first one recorded wins)
+enum : int {
+    DEV_OK = 0,
+    DEV_E_WAIT_TIMEOUT = 1,   // a bounded mbarrier wait ran out
+    DEV_E_INDEX = 2,          // an index left its range
+    DEV_E_TREE_OVERFLOW = 3,  // Algorithm 1 would create more than MAX_CAND nodes
+    DEV_E_CAPACITY = 4        // KV cache would overflow
+};
+
+// Per-sequence device state.  The row table describes the block the next
+// forward pass runs: tree nodes first (breadth-first, parent < child), then
+// the mask-probe rows (Figure 3 of the paper: all mask rows at the end).
+struct SeqState {
+    int32_t L;         // cached positions
+    int32_t n_nodes;   // N, tree nodes incl. root
+    int32_t n_rows;    // N + probe rows
+    int32_t mode;      // 0 decode step, 1 prefill chunk (not last), 2 last prefill chunk
+    int32_t active;    // takes part in the next forward pass
+    int32_t ready;     // prefilled
+    int32_t n_out;     // tokens emitted by the last step
+    int32_t out_tokens[PROBES_MAX + 2];
+    int32_t forced;    // next tree was set by the caller (informational)
+    int32_t row_token[RT];   // -1 for probe rows
+    int32_t row_parent[RT];  // parent row (probe j>1: previous probe; probe 1: its anchor)
+    int32_t row_depth[RT];   // position of the row minus L
+    unsigned long long row_anc[RT][2];  // ancestor-or-self bitmask over rows
+    float row_logp[RT];
+    unsigned long long steps, emitted;
+    unsigned long long accept_hist[PROBES_MAX + 1];
+};
+
+struct Cand {  // one Top-K' entry
+    float val;
+    int32_t id;
+};
+
+// Geometry + spec needed by device code.
+struct Dims {
+    int32_t n_layers, d, Hq, Hkv, h, F, V, qk_norm;
+    int32_t cap;        // KV positions allocated per sequence (max_seq_len + RT)
+    int32_t batch;
+    int32_t split_len;  // attention split length in positions (multiple of 64)
+    int32_t n_split_max;
+    float rms_eps;
+    // speculation
+    int32_t k, K, KP, B, W, n_anchor, prune_parent, prune_root, ema_per_token;
+    float lambda;
+};
+
+// epilogue selectors of the small-M GEMMs
+enum Epi : int { EPI_STORE_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, EPI_LOGITS = 4 };
+
+// Everything an epilogue may need.  One struct for all variants keeps the
+// GEMM kernels identical across call sites.
+struct EpiArgs {
+    int32_t n_out;            // valid output features (ragged last tile is masked)
+    const SeqState* st;       // per-sequence state (row counts, L, depths); may be NULL -> rows_fixed
+    int32_t rows_fixed;       // used when st == NULL
+    int32_t batch;
+    // EPI_STORE_F32
+    float* y_f32;             // [batch*RT][n_out]
+    // EPI_RESID
+    float* hres;              // [batch*RT][n_out]
+    // EPI_QKV
+    void* q_out;              // [batch*RT][Hq*h] T
+    void* kcache;             // this layer: [batch][Hkv][cap][h] T
+    void* vcache;
+    const void* q_norm;       // [h] T or NULL
+    const void* k_norm;
+    const float* rope_cos;    // [cap][h/2]
+    const float* rope_sin;
+    int32_t Hq, Hkv, h, cap, qk_norm;
+    float rms_eps;
+    // EPI_SWIGLU
+    void* act_out;            // [batch*RT][F] T
+    // EPI_LOGITS
+    Cand* cand;               // [n_tiles][batch*RT][KP]
+    float2* cand_ms;          // [n_tiles][batch*RT] (max, sum exp)
+    int32_t KP;
+    int32_t n_tiles;
+    float* logits_dump;       // optional [batch*RT][V]
+};
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// (value descending, id ascending) strict order used by argmax / Top-K everywhere
+__device__ __forceinline__ bool cand_before(float va, int ia, float vb, int ib) {
+    return va > vb || (va == vb && ia < ib);
+}
+
+__device__ __forceinline__ void set_error(int* err, int code) {
+    if (err) atomicCAS(err, 0, code);
+}
+
+// ---- launchers implemented in the .cu files (all enqueue on `s`) ----
+struct GemmPlan;  // tcgen05 launch plan, see esp_gemm_tc.cu
+
+}  // namespace esp

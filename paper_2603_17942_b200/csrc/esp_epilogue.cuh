@@ -1,0 +1,147 @@
+// Epilogues of the small-M GEMMs.  Both GEMM implementations (tcgen05 and
+// CUDA-core) finish a 128-feature tile by placing the fp32 accumulators in
+// shared memory as s_acc[row][feature] and calling run_epilogue with exactly
+// 128 threads (thread f owns feature f of the tile).  The fused work is what
+// follows the matrix product in the decoder layer: rotary embedding at the
+// tree-depth position and the KV-cache write (QKV), the residual add (O,
+// down), SiLU(gate)*up (gate/up) and per-row argmax / Top-K' / max+sum-exp
+// over the vocabulary tile (LM head).
+#pragma once
+
+#include "esp_common.cuh"
+
+namespace esp {
+
+constexpr int ACC_LD = TILE_N + 1;  // padded row stride of s_acc (floats)
+
+__device__ __forceinline__ void epi_bar(int bar_id) {
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+}
+
+// s_acc: [RT][ACC_LD] fp32.  s_aux: >= RT*4 floats of scratch.  tid in [0,128).
+template <typename T, int EPI>
+__device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, const EpiArgs& a, int tid, int bar_id) {
+    const int f = tid;
+    const int n0 = tile * TILE_N;
+    const SeqState* st = a.st ? a.st + seq : nullptr;
+    const int n_rows = st ? st->n_rows : a.rows_fixed;
+    const int grow0 = seq * RT;
+
+    if constexpr (EPI == EPI_STORE_F32) {
+        if (n0 + f < a.n_out)
+            for (int r = 0; r < n_rows; ++r) a.y_f32[(size_t)(grow0 + r) * a.n_out + n0 + f] = s_acc[r * ACC_LD + f];
+    } else if constexpr (EPI == EPI_RESID) {
+        if (n0 + f < a.n_out)
+            for (int r = 0; r < n_rows; ++r) {
+                size_t i = (size_t)(grow0 + r) * a.n_out + n0 + f;
+                a.hres[i] = a.hres[i] + s_acc[r * ACC_LD + f];
+            }
+    } else if constexpr (EPI == EPI_SWIGLU) {
+        // tile rows 0..63 hold gate features [64*tile, 64*tile+64), rows 64..127 the matching up features
+        if (f < 64 && tile * 64 + f < a.n_out) {
+            T* out = reinterpret_cast<T*>(a.act_out);
+            for (int r = 0; r < n_rows; ++r) {
+                float g = s_acc[r * ACC_LD + f], u = s_acc[r * ACC_LD + f + 64];
+                float v = (g / (1.0f + expf(-g))) * u;
+                out[(size_t)(grow0 + r) * a.n_out + tile * 64 + f] = from_f32<T>(v);
+            }
+        }
+    } else if constexpr (EPI == EPI_QKV) {
+        const int h = a.h, dq = a.Hq * h, dkv = a.Hkv * h;
+        const int feat = n0 + f;  // index in the concatenated [q | k | v] feature space
+        const int which = feat < dq ? 0 : (feat < dq + dkv ? 1 : 2);
+        const int local = which == 0 ? feat : (which == 1 ? feat - dq : feat - dq - dkv);
+        const int head = local / h, fl = local % h, half = h / 2;
+        const int L = st ? st->L : 0;
+        const int warp = f >> 5;
+        if (which != 2) {
+            if (a.qk_norm) {
+                // per-head RMSNorm: sum of squares over the head's h features, per row
+                for (int r = 0; r < n_rows; ++r) {
+                    float v = s_acc[r * ACC_LD + f];
+                    float ss = warp_sum(v * v);
+                    if ((f & 31) == 0) s_aux[r * 4 + warp] = ss;
+                }
+                epi_bar(bar_id);
+                const T* g = reinterpret_cast<const T*>(which == 0 ? a.q_norm : a.k_norm);
+                const float gain = to_f32(g[fl]);
+                const int wpw = h / 32;                    // warps per head
+                const int w0 = (f / h) * wpw;              // first warp of this thread's head
+                for (int r = 0; r < n_rows; ++r) {
+                    float ss = 0.f;
+                    for (int w = 0; w < wpw; ++w) ss += s_aux[r * 4 + w0 + w];
+                    float rinv = 1.0f / sqrtf(ss / (float)h + a.rms_eps);
+                    s_acc[r * ACC_LD + f] = s_acc[r * ACC_LD + f] * rinv * gain;
+                }
+            }
+            epi_bar(bar_id);
+            // rotary embedding at position L + depth, rotate-half pairing (i, i + h/2)
+            const int partner = fl < half ? f + half : f - half;
+            for (int r = 0; r < n_rows; ++r) {
+                const int pos = L + (st ? st->row_depth[r] : r);
+                const float cs = a.rope_cos[(size_t)pos * half + (fl % half)];
+                const float sn = a.rope_sin[(size_t)pos * half + (fl % half)];
+                const float me = s_acc[r * ACC_LD + f], other = s_acc[r * ACC_LD + partner];
+                const float v = fl < half ? me * cs - other * sn : me * cs + other * sn;
+                if (which == 0) {
+                    reinterpret_cast<T*>(a.q_out)[(size_t)(grow0 + r) * dq + head * h + fl] = from_f32<T>(v);
+                } else {
+                    reinterpret_cast<T*>(a.kcache)[(((size_t)seq * a.Hkv + head) * a.cap + (L + r)) * h + fl] = from_f32<T>(v);
+                }
+            }
+        } else {
+            if (a.qk_norm) epi_bar(bar_id);
+            epi_bar(bar_id);
+            for (int r = 0; r < n_rows; ++r)
+                reinterpret_cast<T*>(a.vcache)[(((size_t)seq * a.Hkv + head) * a.cap + (L + r)) * h + fl] =
+                    from_f32<T>(s_acc[r * ACC_LD + f]);
+        }
+    } else if constexpr (EPI == EPI_LOGITS) {
+        // warp w takes rows w, w+4, ...; a lane holds features lane, lane+32, lane+64, lane+96 of the row
+        const int warp = f >> 5, lane = f & 31;
+        const int n_nodes = st ? st->n_nodes : a.rows_fixed;
+        const int Mtot = a.batch * RT;
+        for (int r = warp; r < n_rows; r += 4) {
+            float v[4];
+            int id[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                id[i] = n0 + lane + 32 * i;
+                v[i] = id[i] < a.n_out ? s_acc[r * ACC_LD + lane + 32 * i] : -INFINITY;
+                if (a.logits_dump && id[i] < a.n_out) a.logits_dump[(size_t)(grow0 + r) * a.n_out + id[i]] = v[i];
+            }
+            const bool probe = r >= n_nodes;
+            const int kp = probe ? a.KP : 1;
+            Cand* out = a.cand + ((size_t)tile * Mtot + grow0 + r) * a.KP;
+            if (probe) {
+                float tmax = warp_max(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])));
+                float s = 0.f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) s += id[i] < a.n_out ? expf(v[i] - tmax) : 0.f;
+                s = warp_sum(s);
+                if (lane == 0) a.cand_ms[(size_t)tile * Mtot + grow0 + r] = make_float2(tmax, s);
+            }
+            unsigned used = 0;
+            for (int j = 0; j < kp; ++j) {
+                // lane-local best among unused, then warp-wide best by (value desc, id asc)
+                float bv = -INFINITY;
+                int bi = 0x7fffffff, bslot = -1;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (!(used >> i & 1) && id[i] < a.n_out && cand_before(v[i], id[i], bv, bi)) { bv = v[i]; bi = id[i]; bslot = i; }
+                float wv = bv;
+                int wi = bi;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    float ov = __shfl_xor_sync(0xffffffffu, wv, o);
+                    int oi = __shfl_xor_sync(0xffffffffu, wi, o);
+                    if (cand_before(ov, oi, wv, wi)) { wv = ov; wi = oi; }
+                }
+                if (wi == bi && bslot >= 0) used |= 1u << bslot;
+                if (lane == 0) { out[j].val = wv; out[j].id = wi == 0x7fffffff ? -1 : wi; }
+            }
+        }
+    }
+}
+
+}  // namespace esp

@@ -1,0 +1,803 @@
+// CUDA-core kernels of the ESP step: row assembly, RMSNorm, the reference
+// (CUDA-core) small-M GEMM, position-canonical tree attention (split partials,
+// tail + merge), Top-K' merge, and the single-block tree kernel (verify walk,
+// KV compaction, mask update, Algorithm 1 + pruner, next row table).
+#include "esp_epilogue.cuh"
+#include "esp_launch.h"
+
+namespace esp {
+
+// ------------------------------------------------------------------ small helpers
+__global__ void k_rope_table(float* cs, float* sn, int n_pos, int h, float base) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    int half = h / 2;
+    if (i >= n_pos * half) return;
+    int pos = i / half, j = i % half;
+    double inv = pow((double)base, -2.0 * (double)j / (double)h);
+    double ang = (double)pos * inv;
+    cs[i] = (float)cos(ang);
+    sn[i] = (float)sin(ang);
+}
+
+// m = (1/t) sum_j E[x_j]  (Eq. mask_init_mean); fp32 running sum in prompt order
+template <typename T>
+__global__ void k_mask_mean(const T* embed, const int32_t* prompt, int t, int d, float* m) {
+    int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= d) return;
+    float acc = 0.f;
+    for (int i = 0; i < t; ++i) acc = acc + to_f32(embed[(size_t)prompt[i] * d + j]);
+    m[j] = acc / (float)t;
+}
+
+// Input rows of the block: E[token] for tree nodes, the shared mask vector for probe rows.
+template <typename T>
+__global__ void k_assemble(const SeqState* states, const T* embed, const float* mvec, float* hres, int d) {
+    int seq = blockIdx.y, r = blockIdx.x;
+    const SeqState* st = states + seq;
+    if (!st->active || r >= st->n_rows) return;
+    float* out = hres + (size_t)(seq * RT + r) * d;
+    int tok = st->row_token[r];
+    if (tok >= 0)
+        for (int j = threadIdx.x; j < d; j += blockDim.x) out[j] = to_f32(embed[(size_t)tok * d + j]);
+    else
+        for (int j = threadIdx.x; j < d; j += blockDim.x) out[j] = mvec[(size_t)seq * d + j];
+}
+
+// y = x * rsqrt(mean(x^2)+eps) * g, one block per row
+template <typename T>
+__global__ void __launch_bounds__(256) k_rmsnorm(const SeqState* states, const float* x, const T* g, T* y, int d, float eps,
+                                                float* copy_out) {
+    int seq = blockIdx.y, r = blockIdx.x;
+    const SeqState* st = states + seq;
+    if (!st->active || r >= st->n_rows) return;
+    const float* xr = x + (size_t)(seq * RT + r) * d;
+    __shared__ float red[8];
+    float ss = 0.f;
+    for (int j = threadIdx.x; j < d; j += 256) { float v = xr[j]; ss += v * v; }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    float rinv = 1.0f / sqrtf(tot / (float)d + eps);
+    T* yr = y + (size_t)(seq * RT + r) * d;
+    for (int j = threadIdx.x; j < d; j += 256) yr[j] = from_f32<T>(xr[j] * rinv * to_f32(g[j]));
+    if (copy_out)
+        for (int j = threadIdx.x; j < d; j += 256) copy_out[(size_t)(seq * RT + r) * d + j] = xr[j];
+}
+
+// ------------------------------------------------------------------ CUDA-core GEMM
+// y[row][n] = sum_k x[row][k] * w[n][k], k ascending, one thread per output feature of a
+// 128-feature tile and all RT rows of one sequence.  Used for fp32 models and as the on-GPU
+// cross-check of the tcgen05 kernel.  Tile -> weight rows mapping is the same as there:
+// up to three stacked matrices (q|k|v), or gate/up halves interleaved per tile.
+struct SimtGemmArgs {
+    const void* w[3];   // stacked matrices (rows_w[i] rows each); SWIGLU: w[0]=gate, w[1]=up
+    int32_t rows_w[3];
+    const void* x;      // [batch*RT][K]
+    int32_t K;
+};
+
+template <typename T, int EPI>
+__global__ void __launch_bounds__(128) k_gemm_simt(SimtGemmArgs g, EpiArgs a) {
+    extern __shared__ float smem[];
+    float* s_acc = smem;                       // RT * ACC_LD
+    float* s_aux = s_acc + RT * ACC_LD;        // RT * 4
+    float* s_x = s_aux + RT * 4;               // RT * 32
+    float* s_w = s_x + RT * 32;                // 128 * 33
+    const int tile = blockIdx.x, seq = blockIdx.y, f = threadIdx.x;
+    if (a.st && !a.st[seq].active) return;
+    const int n_rows = a.st ? a.st[seq].n_rows : a.rows_fixed;
+    const T* x = reinterpret_cast<const T*>(g.x) + (size_t)seq * RT * g.K;
+    // weight row of feature i of this tile (nullptr if outside)
+    auto wrow = [&](int i) -> const T* {
+        if (EPI == EPI_SWIGLU) {
+            int feat = tile * 64 + (i & 63);
+            if (feat >= g.rows_w[0]) return nullptr;
+            return reinterpret_cast<const T*>(g.w[i >> 6]) + (size_t)feat * g.K;
+        }
+        int feat = tile * TILE_N + i;
+        for (int m = 0; m < 3; ++m) {
+            if (feat < g.rows_w[m]) return reinterpret_cast<const T*>(g.w[m]) + (size_t)feat * g.K;
+            feat -= g.rows_w[m];
+        }
+        return nullptr;
+    };
+    float acc[RT];
+#pragma unroll
+    for (int r = 0; r < RT; ++r) acc[r] = 0.f;
+    for (int k0 = 0; k0 < g.K; k0 += 32) {
+        for (int i = f; i < RT * 32; i += 128) {
+            int r = i >> 5, c = i & 31;
+            s_x[i] = (r < n_rows && k0 + c < g.K) ? to_f32(x[(size_t)r * g.K + k0 + c]) : 0.f;
+        }
+        for (int i = 0; i < 32; ++i) {
+            int row = (f >> 5) + 4 * i, c = f & 31;
+            const T* wr = wrow(row);
+            s_w[row * 33 + c] = (wr && k0 + c < g.K) ? to_f32(wr[k0 + c]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int c = 0; c < 32; ++c) {
+            float w = s_w[f * 33 + c];
+#pragma unroll
+            for (int r = 0; r < RT; ++r) acc[r] = fmaf(s_x[r * 32 + c], w, acc[r]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int r = 0; r < RT; ++r) s_acc[r * ACC_LD + f] = acc[r];
+    __syncthreads();
+    run_epilogue<T, EPI>(s_acc, s_aux, tile, seq, a, f, 1);
+}
+
+template <typename T>
+void launch_gemm_simt_t(int epi, int n_tiles, int batch, const SimtGemmArgs& g, const EpiArgs& a, cudaStream_t s) {
+    size_t smem = sizeof(float) * (RT * ACC_LD + RT * 4 + RT * 32 + 128 * 33);
+    dim3 grid(n_tiles, batch);
+#define ESP_SIMT_CASE(E)                                                                                  \
+    case E:                                                                                               \
+        cudaFuncSetAttribute(k_gemm_simt<T, E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+        k_gemm_simt<T, E><<<grid, 128, smem, s>>>(g, a);                                                  \
+        break;
+    switch (epi) {
+        ESP_SIMT_CASE(EPI_STORE_F32)
+        ESP_SIMT_CASE(EPI_QKV)
+        ESP_SIMT_CASE(EPI_RESID)
+        ESP_SIMT_CASE(EPI_SWIGLU)
+        ESP_SIMT_CASE(EPI_LOGITS)
+    }
+#undef ESP_SIMT_CASE
+}
+
+void launch_gemm_simt(int dtype, int epi, int n_tiles, int batch, const void* const w[3], const int32_t rows_w[3],
+                      const void* x, int K, const EpiArgs& a, cudaStream_t s) {
+    SimtGemmArgs g;
+    for (int i = 0; i < 3; ++i) { g.w[i] = w[i]; g.rows_w[i] = rows_w[i]; }
+    g.x = x;
+    g.K = K;
+    if (dtype == 0) launch_gemm_simt_t<float>(epi, n_tiles, batch, g, a, s);
+    else launch_gemm_simt_t<__nv_bfloat16>(epi, n_tiles, batch, g, a, s);
+}
+
+// ------------------------------------------------------------------ attention (position-canonical)
+// Key list of a row at position P = L + depth: positions 0..P.  Positions below
+// T0 = max(0, floor((P - dcap)/16)*16) are summed by the chunked "bulk" path in splits of
+// split_len positions aligned to position 0; positions T0..P (cache tail + the row's in-flight
+// ancestors, found through its ancestor bitmask in row order = position order) by the tail.
+// Every reduction order depends on absolute positions only, so a token verified inside a tree
+// block gets bit-identical results to the same token decoded alone.
+__device__ __forceinline__ int tail_start(int P, int dcap) {
+    int t = P - dcap;
+    return t <= 0 ? 0 : (t / 16) * 16;
+}
+
+// index of the n-th (0-based) set bit of a 128-bit mask
+__device__ __forceinline__ int nth_set_bit(unsigned long long lo, unsigned long long hi, int n) {
+    int c = __popcll(lo);
+    unsigned long long m = lo;
+    int base = 0;
+    if (n >= c) { n -= c; m = hi; base = 64; }
+    for (int i = 0; i < n; ++i) m &= m - 1;
+    return m ? base + __ffsll((long long)m) - 1 : -1;
+}
+
+
+__device__ __forceinline__ void attn_row_info(const AttnArgs& a, int seq, int r, int& n_rows, int& L, int& depth,
+                                              unsigned long long& lo, unsigned long long& hi) {
+    if (a.st) {
+        const SeqState* st = a.st + seq;
+        n_rows = st->active ? st->n_rows : 0;
+        L = st->L;
+        depth = r < RT ? st->row_depth[r] : 0;
+        lo = r < RT ? st->row_anc[r][0] : 0;
+        hi = r < RT ? st->row_anc[r][1] : 0;
+    } else {
+        n_rows = a.n_rows_fixed;
+        L = a.L_fixed;
+        depth = a.depth[seq * RT + r];
+        lo = a.anc[(size_t)(seq * RT + r) * 2];
+        hi = a.anc[(size_t)(seq * RT + r) * 2 + 1];
+    }
+}
+
+// One chunk of up to 32 keys for one (row, head) handled by one warp: lane j owns key j.
+// Returns the chunk's own (max, sum, weighted values) relative to its own max, in the log2 domain.
+template <typename T, int HD>
+__device__ __forceinline__ void warp_chunk(const float* s_q, const T* kbase, const T* vbase, int slot, bool valid,
+                                           float scale_log2, float& cm, float& cl, float (&co)[HD / 32]) {
+    const int lane = threadIdx.x & 31;
+    float s = -INFINITY;
+    if (valid) {
+        const T* kr = kbase + (size_t)slot * HD;
+        float acc = 0.f;
+#pragma unroll 8
+        for (int d = 0; d < HD; ++d) acc = fmaf(s_q[d], to_f32(kr[d]), acc);
+        s = acc * scale_log2;
+    }
+    cm = warp_max(s);
+    float p = valid ? exp2f(s - cm) : 0.f;
+    cl = warp_sum(p);
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) co[i] = 0.f;
+    for (int j = 0; j < 32; ++j) {
+        float pj = __shfl_sync(0xffffffffu, p, j);
+        int sj = __shfl_sync(0xffffffffu, slot, j);
+        if (pj != 0.f) {
+            const T* vr = vbase + (size_t)sj * HD;
+#pragma unroll
+            for (int i = 0; i < HD / 32; ++i) co[i] = fmaf(pj, to_f32(vr[lane + 32 * i]), co[i]);
+        }
+    }
+}
+
+template <int N>
+__device__ __forceinline__ void merge_partial(float& m, float& l, float (&o)[N], float cm, float cl, const float (&co)[N]) {
+    float mn = fmaxf(m, cm);
+    float a = exp2f(m - mn), b = exp2f(cm - mn);
+    l = l * a + cl * b;
+#pragma unroll
+    for (int i = 0; i < N; ++i) o[i] = o[i] * a + co[i] * b;
+    m = mn;
+}
+
+// Bulk, CUDA-core version: one warp per (row, head, split).  grid = (ceil(RT/4), Hq, n_split*batch).
+template <typename T, int HD>
+__global__ void __launch_bounds__(128) k_attn_bulk_simt(AttnArgs a, int n_split_launch) {
+    __shared__ float s_qall[4][HD];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 4 + warp, head = blockIdx.y;
+    const int split = blockIdx.z % n_split_launch, seq = blockIdx.z / n_split_launch;
+    int n_rows, L, depth;
+    unsigned long long lo, hi;
+    attn_row_info(a, seq, r < RT ? r : 0, n_rows, L, depth, lo, hi);
+    if (r >= n_rows) return;
+    const int T0 = tail_start(L + depth, a.dcap);
+    const int beg = split * a.split_len, end = min(beg + a.split_len, T0);
+    if (beg >= end) return;
+    const int kvh = head / (a.Hq / a.Hkv);
+    const T* q = reinterpret_cast<const T*>(a.q) + ((size_t)(seq * RT + r) * a.Hq + head) * HD;
+    float* s_q = s_qall[warp];
+    for (int d = lane; d < HD; d += 32) s_q[d] = to_f32(q[d]);
+    __syncwarp();
+    const T* kb = reinterpret_cast<const T*>(a.kc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
+    const T* vb = reinterpret_cast<const T*>(a.vc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
+    float m = -INFINITY, l = 0.f, o[HD / 32];
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) o[i] = 0.f;
+    for (int p0 = beg; p0 < end; p0 += 32) {
+        float cm, cl, co[HD / 32];
+        int pos = p0 + lane;
+        warp_chunk<T, HD>(s_q, kb, vb, pos, pos < end, a.scale_log2, cm, cl, co);
+        merge_partial(m, l, o, cm, cl, co);
+    }
+    size_t idx = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max + split;
+    if (lane == 0) a.part_ml[idx] = make_float2(m, l);
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) a.part_o[idx * HD + lane + 32 * i] = o[i];
+}
+
+// Tail + merge: one warp per (row, head).  grid = (ceil(RT/4), Hq, batch).
+template <typename T, int HD>
+__global__ void __launch_bounds__(128) k_attn_tail_merge(AttnArgs a) {
+    __shared__ float s_qall[4][HD];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 4 + warp, head = blockIdx.y, seq = blockIdx.z;
+    int n_rows, L, depth;
+    unsigned long long lo, hi;
+    attn_row_info(a, seq, r < RT ? r : 0, n_rows, L, depth, lo, hi);
+    if (r >= n_rows) return;
+    const int P = L + depth;
+    const int T0 = tail_start(P, a.dcap);
+    const int kvh = head / (a.Hq / a.Hkv);
+    const T* q = reinterpret_cast<const T*>(a.q) + ((size_t)(seq * RT + r) * a.Hq + head) * HD;
+    float* s_q = s_qall[warp];
+    for (int d = lane; d < HD; d += 32) s_q[d] = to_f32(q[d]);
+    __syncwarp();
+    const T* kb = reinterpret_cast<const T*>(a.kc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
+    const T* vb = reinterpret_cast<const T*>(a.vc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
+    float m = -INFINITY, l = 0.f, o[HD / 32];
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) o[i] = 0.f;
+    // bulk partials in split order
+    const int n_sp = (T0 + a.split_len - 1) / a.split_len;
+    const size_t base = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max;
+    for (int s = 0; s < n_sp; ++s) {
+        float2 ml = a.part_ml[base + s];
+        float co[HD / 32];
+#pragma unroll
+        for (int i = 0; i < HD / 32; ++i) co[i] = a.part_o[(base + s) * HD + lane + 32 * i];
+        merge_partial(m, l, o, ml.x, ml.y, co);
+    }
+    // tail: positions T0..P in order
+    const int n_tail = P - T0 + 1;
+    for (int t0 = 0; t0 < n_tail; t0 += 32) {
+        int t = t0 + lane;
+        bool valid = t < n_tail;
+        int slot = 0;
+        if (valid) {
+            int pos = T0 + t;
+            if (pos < L) slot = pos;
+            else {
+                int b = nth_set_bit(lo, hi, pos - L);
+                if (b < 0) { set_error(a.err, DEV_E_INDEX); valid = false; }
+                else slot = L + b;
+            }
+        }
+        float cm, cl, co[HD / 32];
+        warp_chunk<T, HD>(s_q, kb, vb, slot, valid, a.scale_log2, cm, cl, co);
+        merge_partial(m, l, o, cm, cl, co);
+    }
+    T* out = reinterpret_cast<T*>(a.out) + ((size_t)(seq * RT + r) * a.Hq + head) * HD;
+    const float inv = 1.0f / l;
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) out[lane + 32 * i] = from_f32<T>(o[i] * inv);
+}
+
+template <typename T, int HD>
+static void launch_attn_simt_t(const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s) {
+    dim3 g1((RT + 3) / 4, a.Hq, n_split_launch * batch);
+    if (bulk_too && n_split_launch > 0) k_attn_bulk_simt<T, HD><<<g1, 128, 0, s>>>(a, n_split_launch);
+    dim3 g2((RT + 3) / 4, a.Hq, batch);
+    k_attn_tail_merge<T, HD><<<g2, 128, 0, s>>>(a);
+}
+
+int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s) {
+#define ESP_ATTN_CASE(TT, H) launch_attn_simt_t<TT, H>(a, batch, n_split_launch, bulk_too, s); return 0;
+    if (dtype == 0) {
+        if (a.h == 32) { ESP_ATTN_CASE(float, 32) }
+        if (a.h == 64) { ESP_ATTN_CASE(float, 64) }
+        if (a.h == 128) { ESP_ATTN_CASE(float, 128) }
+    } else {
+        if (a.h == 32) { ESP_ATTN_CASE(__nv_bfloat16, 32) }
+        if (a.h == 64) { ESP_ATTN_CASE(__nv_bfloat16, 64) }
+        if (a.h == 128) { ESP_ATTN_CASE(__nv_bfloat16, 128) }
+    }
+#undef ESP_ATTN_CASE
+    return -1;
+}
+
+// ------------------------------------------------------------------ Top-K' merge over vocabulary tiles
+// One block per row: global Top-K' (value desc, id asc) of the per-tile lists, plus
+// lse = max + log(sum exp) merged over tiles in a fixed order.
+__global__ void __launch_bounds__(128) k_topk_merge(const SeqState* states, const Cand* cand, const float2* cand_ms,
+                                                    int n_tiles, int KP, int batch, Cand* topk, float* lse) {
+    const int seq = blockIdx.y, r = blockIdx.x, tid = threadIdx.x;
+    const SeqState* st = states + seq;
+    if (!st->active || r >= st->n_rows) return;
+    const int Mtot = batch * RT, grow = seq * RT + r;
+    const bool probe = r >= st->n_nodes;
+    const int kp = probe ? KP : 1;
+    __shared__ float s_v[128];
+    __shared__ int s_i[128];
+    __shared__ int s_owner;
+    // each thread keeps a cursor per tile it owns; lists are sorted, so its best remaining
+    // entry is the best head among its tiles
+    constexpr int MAXT = 16;  // tiles per thread (n_tiles <= 2048)
+    unsigned char cur[MAXT];
+#pragma unroll
+    for (int i = 0; i < MAXT; ++i) cur[i] = 0;
+    for (int j = 0; j < kp; ++j) {
+        float bv = -INFINITY;
+        int bi = 0x7fffffff, bt = -1;
+#pragma unroll
+        for (int i = 0; i < MAXT; ++i) {
+            int t = tid + 128 * i;
+            if (t < n_tiles && cur[i] < kp) {
+                Cand c = cand[((size_t)t * Mtot + grow) * KP + cur[i]];
+                if (c.id >= 0 && cand_before(c.val, c.id, bv, bi)) { bv = c.val; bi = c.id; bt = i; }
+            }
+        }
+        s_v[tid] = bv;
+        s_i[tid] = bi;
+        __syncthreads();
+        for (int o = 64; o > 0; o >>= 1) {
+            if (tid < o && cand_before(s_v[tid + o], s_i[tid + o], s_v[tid], s_i[tid])) {
+                s_v[tid] = s_v[tid + o];
+                s_i[tid] = s_i[tid + o];
+            }
+            __syncthreads();
+        }
+        float wv = s_v[0];
+        int wi = s_i[0];
+        if (bt >= 0 && wi == bi) {
+#pragma unroll
+            for (int i = 0; i < MAXT; ++i) if (i == bt) cur[i]++;
+        }
+        if (tid == 0) { topk[(size_t)grow * KP_MAX + j].val = wv; topk[(size_t)grow * KP_MAX + j].id = wi == 0x7fffffff ? -1 : wi; }
+        __syncthreads();
+    }
+    if (probe) {
+        // thread-strided partial merges in tile order, then a fixed tree over threads
+        float m = -INFINITY, s = 0.f;
+        for (int t = tid; t < n_tiles; t += 128) {
+            float2 ms = cand_ms[(size_t)t * Mtot + grow];
+            float mn = fmaxf(m, ms.x);
+            s = s * expf(m - mn) + ms.y * expf(ms.x - mn);
+            m = mn;
+        }
+        s_v[tid] = m;
+        reinterpret_cast<float*>(s_i)[tid] = s;
+        __syncthreads();
+        for (int o = 64; o > 0; o >>= 1) {
+            if (tid < o) {
+                float m1 = s_v[tid], m2 = s_v[tid + o];
+                float s1 = reinterpret_cast<float*>(s_i)[tid], s2 = reinterpret_cast<float*>(s_i)[tid + o];
+                float mn = fmaxf(m1, m2);
+                float sn = (m1 == -INFINITY ? 0.f : s1 * expf(m1 - mn)) + (m2 == -INFINITY ? 0.f : s2 * expf(m2 - mn));
+                s_v[tid] = mn;
+                reinterpret_cast<float*>(s_i)[tid] = sn;
+            }
+            __syncthreads();
+        }
+        if (tid == 0) lse[grow] = s_v[0] + logf(reinterpret_cast<float*>(s_i)[0]);
+    }
+    (void)s_owner;
+}
+
+void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
+                       Cand* topk, float* lse, cudaStream_t s) {
+    dim3 grid(RT, batch);
+    k_topk_merge<<<grid, 128, 0, s>>>(st, cand, cand_ms, n_tiles, KP, batch, topk, lse);
+}
+
+// ------------------------------------------------------------------ row-table builders
+__device__ void write_probe_rows(SeqState* st, int N, int k, int first_anchor, int n_anchor_rows) {
+    // probe j (1-based) of the a-th anchored node sits at row N + a*k + (j-1)
+    for (int i = threadIdx.x; i < n_anchor_rows * k; i += blockDim.x) {
+        int aidx = i / k, j = i % k + 1;
+        int u = first_anchor + aidx;
+        int row = N + aidx * k + (j - 1);
+        st->row_token[row] = -1;
+        st->row_parent[row] = j == 1 ? u : row - 1;
+        st->row_depth[row] = st->row_depth[u] + j;
+        unsigned long long lo = st->row_anc[u][0], hi = st->row_anc[u][1];
+        for (int jj = 0; jj < j; ++jj) {
+            int b = N + aidx * k + jj;
+            if (b < 64) lo |= 1ull << b; else hi |= 1ull << (b - 64);
+        }
+        st->row_anc[row][0] = lo;
+        st->row_anc[row][1] = hi;
+        st->row_logp[row] = 0.f;
+    }
+}
+
+// Prefill chunk: rows are n consecutive prompt tokens (a chain); the last chunk appends k probes
+// behind the last prompt token (Figure 1 middle).
+__global__ void k_setup_chain(SeqState* states, int seq, const int32_t* prompt_dev, int off, int n, int last, int k) {
+    SeqState* st = states + seq;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        st->row_token[i] = prompt_dev[off + i];
+        st->row_parent[i] = i - 1;
+        st->row_depth[i] = i;
+        unsigned long long lo = i >= 63 ? ~0ull : ((1ull << (i + 1)) - 1);
+        unsigned long long hi = i < 64 ? 0ull : ((1ull << (i - 63)) - 1);
+        st->row_anc[i][0] = lo;
+        st->row_anc[i][1] = hi;
+        st->row_logp[i] = 0.f;
+    }
+    __syncthreads();
+    if (last && k > 0) write_probe_rows(st, n, k, n - 1, 1);
+    if (threadIdx.x == 0) {
+        st->n_nodes = n;
+        st->n_rows = n + (last ? k : 0);
+        st->mode = last ? 2 : 1;
+        st->active = 1;
+        if (off == 0) st->L = 0;
+    }
+}
+
+// Caller-provided tree (test hook): tokens/parents in breadth-first order.
+__global__ void k_set_tree(SeqState* states, int seq, const int32_t* tokens, const int32_t* parents, int n, int k,
+                           int n_anchor, int* err) {
+    SeqState* st = states + seq;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < n; ++i) {
+            int p = parents[i];
+            if (i == 0 ? p != -1 : (p < 0 || p >= i)) { set_error(err, DEV_E_INDEX); p = i == 0 ? -1 : 0; }
+            st->row_token[i] = tokens[i];
+            st->row_parent[i] = p;
+            st->row_depth[i] = i == 0 ? 0 : st->row_depth[p] + 1;
+            unsigned long long lo = i == 0 ? 0 : st->row_anc[p][0], hi = i == 0 ? 0 : st->row_anc[p][1];
+            if (i < 64) lo |= 1ull << i; else hi |= 1ull << (i - 64);
+            st->row_anc[i][0] = lo;
+            st->row_anc[i][1] = hi;
+            st->row_logp[i] = 0.f;
+        }
+        st->n_nodes = n;
+    }
+    __syncthreads();
+    int nA = k > 0 ? (n_anchor == 0 ? n : min(n_anchor, n)) : 0;
+    write_probe_rows(st, n, k, 0, nA);
+    if (threadIdx.x == 0) { st->n_rows = n + nA * k; st->mode = 0; st->forced = 1; }
+}
+
+// ------------------------------------------------------------------ the single-block tree kernel
+// verify walk -> KV compaction -> mask update -> Algorithm 1 + pruner -> next row table.
+
+__device__ __forceinline__ bool node_before(float lpa, int da, int ia, float lpb, int db, int ib) {
+    if (lpa != lpb) return lpa > lpb;
+    if (da != db) return da < db;
+    return ia < ib;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
+    extern __shared__ unsigned char smem_raw[];
+    int* c_tok = reinterpret_cast<int*>(smem_raw);
+    int* c_par = c_tok + MAX_CAND;
+    int* c_dep = c_par + MAX_CAND;
+    float* c_lp = reinterpret_cast<float*>(c_dep + MAX_CAND);
+    int* c_rank = reinterpret_cast<int*>(c_lp + MAX_CAND);
+    __shared__ int s_path[PROBES_MAX + 2], s_out[PROBES_MAX + 2];
+    __shared__ int s_na, s_ustar, s_delta, s_nexp, s_ncreated, s_abort;
+    __shared__ int s_exp[RT], s_sel[RT], s_new[RT];
+
+    const Dims& D = A.D;
+    const int seq = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+    SeqState* st = A.states + seq;
+    if (!st->active) return;
+    const int mode = st->mode;
+    const int N0 = st->n_nodes, L0 = st->L;
+    const int grow0 = seq * RT;
+
+    if (mode == 1) {  // prefill chunk: every row is a prompt token and is already in place
+        if (tid == 0) st->L = L0 + N0;
+        return;
+    }
+
+    // ---- verification (Section 2): follow the model's own next token through the tree
+    if (tid == 0) {
+        int a = 0, cur, n_emit = 0;
+        s_abort = 0;
+        if (mode == 2) {
+            cur = N0 - 1;  // last prompt token; nothing to verify, its argmax is the first generated token
+            s_path[0] = cur;
+            s_out[n_emit++] = A.topk[(size_t)(grow0 + cur) * KP_MAX].id;
+            s_ustar = cur;
+            s_delta = 0;
+        } else {
+            cur = 0;
+            s_path[0] = 0;
+            for (;;) {
+                int y = A.topk[(size_t)(grow0 + cur) * KP_MAX].id;
+                s_out[n_emit++] = y;
+                int nxt = -1;
+                for (int c = cur + 1; c < N0; ++c)
+                    if (st->row_parent[c] == cur && st->row_token[c] == y) { nxt = c; break; }
+                if (nxt < 0 || n_emit > PROBES_MAX) break;
+                cur = nxt;
+                s_path[++a] = cur;
+            }
+            // deepest anchored node on the accepted path
+            int nA = D.k > 0 ? (D.n_anchor == 0 ? N0 : min(D.n_anchor, N0)) : 0;
+            int us = 0;
+            for (int j = 0; j <= a; ++j) if (s_path[j] < nA) us = s_path[j];
+            s_ustar = us;
+            s_delta = a - st->row_depth[us];
+        }
+        s_na = a;
+        st->n_out = n_emit;
+        for (int j = 0; j < n_emit; ++j) st->out_tokens[j] = s_out[j];
+        A.out_ring[seq * RING] = n_emit;
+        A.out_ring[seq * RING + 1] = mode == 2 ? L0 + N0 : L0 + a + 1;
+        for (int j = 0; j < n_emit; ++j) A.out_ring[seq * RING + 2 + j] = s_out[j];
+        if (mode == 0) {
+            st->steps += 1;
+            st->emitted += n_emit;
+            st->accept_hist[a < PROBES_MAX ? a : PROBES_MAX] += 1;
+        }
+    }
+    __syncthreads();
+    const int a_acc = s_na;
+    const int n_emit = mode == 2 ? 1 : a_acc + 1;
+
+    // ---- KV compaction: cache slot L+j <- row p_j for the accepted path (row 0 is already at slot L).
+    // Sources sit at or above their destination, so increasing j with a barrier in between is safe.
+    if (mode == 0) {
+        const int vec_per_row = D.h * (int)sizeof(T) / 16;
+        const size_t layer_stride = (size_t)D.batch * D.Hkv * D.cap * D.h;
+        const int per_j = D.n_layers * D.Hkv * 2 * vec_per_row;
+        for (int j = 1; j <= a_acc; ++j) {
+            const int src = L0 + s_path[j], dst = L0 + j;
+            if (src != dst) {
+                for (int i = tid; i < per_j; i += nt) {
+                    int v = i % vec_per_row, rest = i / vec_per_row;
+                    int kv = rest & 1;
+                    rest >>= 1;
+                    int hh = rest % D.Hkv, l = rest / D.Hkv;
+                    T* basep = reinterpret_cast<T*>(kv ? A.vcache : A.kcache) + (size_t)l * layer_stride +
+                               ((size_t)seq * D.Hkv + hh) * D.cap * D.h;
+                    const uint4* s4 = reinterpret_cast<const uint4*>(basep + (size_t)src * D.h) + v;
+                    uint4* d4 = reinterpret_cast<uint4*>(basep + (size_t)dst * D.h) + v;
+                    *d4 = *s4;
+                }
+            }
+            __syncthreads();
+        }
+    }
+    const int Lnew = mode == 2 ? L0 + N0 : L0 + a_acc + 1;
+
+    // ---- mask update, Eq. (mask_update_mean): m <- m + lambda (e - m)
+    {
+        const T* E = reinterpret_cast<const T*>(A.embed);
+        float* m = A.mvec + (size_t)seq * D.d;
+        for (int j = tid; j < D.d; j += nt) {
+            float mv = m[j];
+            for (int e = D.ema_per_token ? 0 : n_emit - 1; e < n_emit; ++e) {
+                float ev = to_f32(E[(size_t)s_out[e] * D.d + j]);
+                mv = __fadd_rn(mv, __fmul_rn(D.lambda, __fsub_rn(ev, mv)));
+            }
+            m[j] = mv;
+        }
+    }
+
+    // ---- next tree (Algorithm 1 with the pruner).  Depth i draws from probe delta+i of u*.
+    const int root_tok = s_out[n_emit - 1];
+    const int ustar = s_ustar, delta = s_delta;
+    const int Dd = D.k - delta > 0 ? D.k - delta : 0;
+    if (tid == 0) {
+        c_tok[0] = root_tok; c_par[0] = -1; c_dep[0] = 0; c_lp[0] = 0.f;
+        s_exp[0] = 0; s_nexp = 1; s_ncreated = 1;
+    }
+    __syncthreads();
+    for (int i = 1; i <= Dd; ++i) {
+        const int pool = min(D.K, D.B - i);
+        if (pool <= 0) break;
+        const int prow = mode == 2 ? N0 + (i - 1) : N0 + ustar * D.k + (delta + i - 1);
+        const Cand* list = A.topk + (size_t)(grow0 + prow) * KP_MAX;
+        const float lse_i = A.lse[grow0 + prow];
+        const int base = s_ncreated, n_exp = s_nexp;
+        const int n_new = n_exp * pool;
+        if (base + n_new > MAX_CAND) { if (tid == 0) { set_error(A.err, DEV_E_TREE_OVERFLOW); s_abort = 1; } }
+        __syncthreads();
+        if (s_abort) break;
+        for (int w = tid; w < n_new; w += nt) {
+            const int e = w / pool, j = w % pool;
+            const int p = s_exp[e];
+            const int ptok = c_tok[p];
+            int seen = 0, q = 0;
+            for (; q < D.KP; ++q) {
+                int t = list[q].id;
+                if (D.prune_parent && t == ptok) continue;
+                if (D.prune_root && t == root_tok) continue;
+                if (seen == j) break;
+                ++seen;
+            }
+            const int c = base + w;
+            if (q < D.KP && list[q].id >= 0) {
+                c_tok[c] = list[q].id;
+                c_lp[c] = __fadd_rn(c_lp[p], __fsub_rn(list[q].val, lse_i));
+            } else {  // list exhausted (cannot happen when K' = K + pruner flags): never selectable
+                c_tok[c] = -1;
+                c_lp[c] = -INFINITY;
+            }
+            c_par[c] = p;
+            c_dep[c] = i;
+        }
+        __syncthreads();
+        const int width = D.W == 0 ? D.B - i : min(D.W, D.B - i);
+        for (int w = tid; w < n_new; w += nt) {
+            const int c = base + w;
+            const float lp = c_lp[c];
+            int rank = 0;
+            for (int o = 0; o < n_new; ++o) {
+                const int c2 = base + o;
+                const float lp2 = c_lp[c2];
+                rank += (lp2 > lp || (lp2 == lp && c2 < c)) ? 1 : 0;
+            }
+            if (rank < width && c_tok[c] >= 0) s_exp[rank] = c;
+        }
+        if (tid == 0) { s_ncreated = base + n_new; s_nexp = min(width, n_new); }
+        __syncthreads();
+    }
+    // final selection: root + the B-1 best created nodes by (logP desc, depth asc, creation asc)
+    const int n_created = s_ncreated;
+    for (int r = tid; r < RT; r += nt) s_sel[r] = -1;
+    __syncthreads();
+    for (int c = 1 + tid; c < n_created; c += nt) {
+        const float lp = c_lp[c];
+        const int dp = c_dep[c];
+        int rank = 0;
+        for (int o = 1; o < n_created; ++o) rank += node_before(c_lp[o], c_dep[o], o, lp, dp, c) ? 1 : 0;
+        c_rank[c] = rank;
+        if (rank < D.B - 1 && c_tok[c] >= 0 && rank < RT) s_sel[rank] = c;
+    }
+    __syncthreads();
+    int n_sel = min(D.B - 1, n_created - 1);
+    // (entries with token -1 rank last because their logP is -inf; drop them)
+    if (tid == 0) {
+        int n = 0;
+        while (n < n_sel && s_sel[n] >= 0) ++n;
+        s_nexp = n;
+    }
+    __syncthreads();
+    n_sel = s_nexp;
+    // breadth-first row order: by depth, ties by selection rank
+    for (int r = tid; r < n_sel; r += nt) {
+        const int c = s_sel[r], dp = c_dep[c];
+        int idx = 1;
+        for (int o = 0; o < n_sel; ++o) {
+            const int d2 = c_dep[s_sel[o]];
+            idx += (d2 < dp || (d2 == dp && o < r)) ? 1 : 0;
+        }
+        s_new[r] = idx;
+        c_rank[c] = idx;  // creation index -> new row index
+    }
+    if (tid == 0) c_rank[0] = 0;
+    __syncthreads();
+    const int N = n_sel + 1;
+    for (int r = tid; r < n_sel; r += nt) {
+        const int c = s_sel[r], row = s_new[r];
+        st->row_token[row] = c_tok[c];
+        st->row_parent[row] = c_rank[c_par[c]];
+        st->row_depth[row] = c_dep[c];
+        st->row_logp[row] = c_lp[c];
+        // ancestor-or-self mask by walking up the creation-time parents
+        unsigned long long lo = 0, hi = 0;
+        for (int x = c; x >= 0; x = c_par[x]) {
+            int b = c_rank[x];
+            if (b < 64) lo |= 1ull << b; else hi |= 1ull << (b - 64);
+        }
+        st->row_anc[row][0] = lo;
+        st->row_anc[row][1] = hi;
+    }
+    if (tid == 0) {
+        st->row_token[0] = root_tok; st->row_parent[0] = -1; st->row_depth[0] = 0; st->row_logp[0] = 0.f;
+        st->row_anc[0][0] = 1ull; st->row_anc[0][1] = 0ull;
+    }
+    __syncthreads();
+    const int nA = D.k > 0 ? (D.n_anchor == 0 ? N : min(D.n_anchor, N)) : 0;
+    write_probe_rows(st, N, D.k, 0, nA);
+    if (tid == 0) {
+        st->n_nodes = N;
+        st->n_rows = N + nA * D.k;
+        st->L = Lnew;
+        st->mode = 0;
+        st->forced = 0;
+        if (Lnew + RT > D.cap) set_error(A.err, DEV_E_CAPACITY);
+    }
+}
+
+void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s) {
+    size_t smem = (size_t)MAX_CAND * 20;
+    if (dtype == 0) {
+        cudaFuncSetAttribute(k_tree_step<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        k_tree_step<float><<<A.D.batch, 1024, smem, s>>>(A);
+    } else {
+        cudaFuncSetAttribute(k_tree_step<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        k_tree_step<__nv_bfloat16><<<A.D.batch, 1024, smem, s>>>(A);
+    }
+}
+
+// ------------------------------------------------------------------ thin launch wrappers
+void launch_rope_table(float* cs, float* sn, int n_pos, int h, float base, cudaStream_t s) {
+    int n = n_pos * (h / 2);
+    k_rope_table<<<(n + 255) / 256, 256, 0, s>>>(cs, sn, n_pos, h, base);
+}
+void launch_mask_mean(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, cudaStream_t s) {
+    if (dtype == 0) k_mask_mean<float><<<(d + 127) / 128, 128, 0, s>>>((const float*)embed, prompt, t, d, m);
+    else k_mask_mean<__nv_bfloat16><<<(d + 127) / 128, 128, 0, s>>>((const __nv_bfloat16*)embed, prompt, t, d, m);
+}
+void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int batch,
+                     cudaStream_t s) {
+    dim3 grid(RT, batch);
+    if (dtype == 0) k_assemble<float><<<grid, 128, 0, s>>>(st, (const float*)embed, mvec, hres, d);
+    else k_assemble<__nv_bfloat16><<<grid, 128, 0, s>>>(st, (const __nv_bfloat16*)embed, mvec, hres, d);
+}
+void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
+                    float* copy_out, cudaStream_t s) {
+    dim3 grid(RT, batch);
+    if (dtype == 0) k_rmsnorm<float><<<grid, 256, 0, s>>>(st, x, (const float*)g, (float*)y, d, eps, copy_out);
+    else k_rmsnorm<__nv_bfloat16><<<grid, 256, 0, s>>>(st, x, (const __nv_bfloat16*)g, (__nv_bfloat16*)y, d, eps, copy_out);
+}
+void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int off, int n, int last, int k, cudaStream_t s) {
+    k_setup_chain<<<1, 128, 0, s>>>(st, seq, prompt_dev, off, n, last, k);
+}
+void launch_set_tree(SeqState* st, int seq, const int32_t* tokens, const int32_t* parents, int n, int k, int n_anchor,
+                     int* err, cudaStream_t s) {
+    k_set_tree<<<1, 128, 0, s>>>(st, seq, tokens, parents, n, k, n_anchor, err);
+}
+
+}  // namespace esp

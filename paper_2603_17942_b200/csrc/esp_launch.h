@@ -1,0 +1,71 @@
+// Host-side launch interface between the translation units of the library.
+#pragma once
+
+#include "esp_common.cuh"
+
+namespace esp {
+
+struct AttnArgs {
+    const void* q;        // [batch][RT][Hq][h]
+    const void* kc;       // [batch][Hkv][cap][h]
+    const void* vc;
+    void* out;            // [batch][RT][Hq][h]
+    float* part_o;        // [batch*RT][Hq][n_split_max][h]
+    float2* part_ml;      // [batch*RT][Hq][n_split_max]
+    const SeqState* st;   // NULL -> use the explicit fields below
+    const unsigned long long* anc;  // [batch][RT][2]
+    const int32_t* depth;           // [batch][RT]
+    int32_t n_rows_fixed, L_fixed;
+    int32_t Hq, Hkv, h, cap, split_len, n_split_max, dcap;
+    float scale_log2;     // log2(e)/sqrt(h)
+    int* err;
+};
+
+struct TreeArgs {
+    Dims D;
+    SeqState* states;
+    const Cand* topk;   // [batch*RT][KP_MAX]
+    const float* lse;   // [batch*RT]
+    float* mvec;        // [batch][d]
+    const void* embed;
+    void* kcache;       // [n_layers][batch][Hkv][cap][h]
+    void* vcache;
+    int* err;
+    int32_t* out_ring;  // [batch][RING]: n_out, new L, tokens  (copied to the host by esp_read)
+};
+
+
+void launch_rope_table(float* cs, float* sn, int n_pos, int h, float base, cudaStream_t s);
+void launch_mask_mean(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, cudaStream_t s);
+void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int batch,
+                     cudaStream_t s);
+void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
+                    float* copy_out, cudaStream_t s);
+void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int off, int n, int last, int k, cudaStream_t s);
+void launch_set_tree(SeqState* st, int seq, const int32_t* tokens, const int32_t* parents, int n, int k, int n_anchor,
+                     int* err, cudaStream_t s);
+void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
+                       Cand* topk, float* lse, cudaStream_t s);
+void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s);
+
+// CUDA-core GEMM (fp32 models; on-GPU cross-check for bf16)
+void launch_gemm_simt(int dtype, int epi, int n_tiles, int batch, const void* const w[3], const int32_t rows_w[3],
+                      const void* x, int K, const EpiArgs& a, cudaStream_t s);
+
+// position-canonical attention: CUDA-core bulk (+ tail/merge), or tail/merge only when the
+// tensor-core bulk kernel already produced the split partials
+int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s);
+// tensor-core bulk for bf16, head_dim 128
+int launch_attn_bulk_mma(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s);
+
+// tcgen05 GEMM: a plan holds the TMA descriptors and the stream-K partition of one weight shape
+struct TcGemm;
+int tc_gemm_create(TcGemm** out, int epi, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
+                   int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err);
+void tc_gemm_destroy(TcGemm* g);
+int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s);
+int tc_gemm_tiles(const TcGemm* g);
+size_t tc_gemm_partial_bytes(int n_sm);
+int tc_gemm_counter_ints();
+
+}  // namespace esp
