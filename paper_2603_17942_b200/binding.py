@@ -24,11 +24,11 @@ ERRORS = {0: "ESP_OK", -1: "ESP_E_BADCFG", -2: "ESP_E_WORKSPACE", -3: "ESP_E_PRO
           -5: "ESP_E_DEVICE", -6: "ESP_E_CUDA", -7: "ESP_E_STATE", -8: "ESP_E_ARG"}
 
 EXPORTS = ["esp_workspace_bytes", "esp_init", "esp_prefill", "esp_step", "esp_step_async", "esp_read", "esp_set_tree",
-           "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_get_stats", "esp_free",
+           "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_step_profiled", "esp_get_stats", "esp_free",
            "esp_tree_attention_scratch_bytes", "esp_tree_attention", "esp_gemm_scratch_bytes", "esp_gemm_bf16"]
 
 __all__ = ["EspError", "esp_model_cfg", "esp_spec_cfg", "esp_weights", "esp_stats", "load_library", "model_cfg",
-           "spec_cfg", "Handle", "ESP_MAX_ROWS", "ESP_MAX_PROBES", "ESP_MAX_KPRIME", "EXPORTS", "LIB_PATH"] + EXPORTS
+           "spec_cfg", "Handle", "ESP_MAX_ROWS", "ESP_MAX_PROBES", "ESP_MAX_KPRIME", "EXPORTS", "LIB_PATH", "KINDS"] + EXPORTS
 
 
 class EspError(RuntimeError):
@@ -170,6 +170,15 @@ def esp_debug_capture(h, logits=None, hidden=None):
 
 def esp_debug_set_gemm(h, impl: int):
     _check(load_library().esp_debug_set_gemm(h, ctypes.c_int32(impl)), "esp_debug_set_gemm")
+
+
+KINDS = ("norm_assemble", "qkv_gemm", "tree_attention", "o_gemm", "gateup_gemm", "down_gemm", "lmhead_topk", "select_tree")
+
+
+def esp_step_profiled(h, tokens_out: np.ndarray, n_out: np.ndarray) -> Dict[str, float]:
+    ms = np.zeros(8, np.float32)
+    _check(load_library().esp_step_profiled(h, _vp(ms), _vp(tokens_out), _vp(n_out)), "esp_step_profiled")
+    return {k: float(v) for k, v in zip(KINDS, ms)}
 
 
 def esp_get_stats(h) -> esp_stats:

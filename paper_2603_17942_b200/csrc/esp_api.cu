@@ -149,11 +149,29 @@ struct esp_handle {
     float *dbg_logits = nullptr, *dbg_hidden = nullptr;
     int launches = 0, kernels_per_step = 0;
     size_t layer_kv_stride = 0;  // bytes
+    bool prof = false;           // record an event after every kernel group
+    std::vector<cudaEvent_t> ev;
+    std::vector<int> ev_kind;
+    size_t ev_used = 0;
 };
 
 namespace {
 
 int cuda_ok(cudaError_t e) { return e == cudaSuccess ? ESP_OK : ESP_E_CUDA; }
+
+enum { KIND_MISC = 0, KIND_QKV, KIND_ATTN, KIND_O, KIND_GATEUP, KIND_DOWN, KIND_LMHEAD, KIND_SELECT, KIND_N };
+
+void mark(esp_handle* h, int kind) {
+    if (!h->prof) return;
+    if (h->ev_used == h->ev.size()) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return;
+        h->ev.push_back(e);
+        h->ev_kind.push_back(0);
+    }
+    h->ev_kind[h->ev_used] = kind;
+    cudaEventRecord(h->ev[h->ev_used++], h->stream);
+}
 
 void* layer_ptr(void* base, size_t stride_bytes, int l) { return reinterpret_cast<char*>(base) + stride_bytes * l; }
 
@@ -186,11 +204,13 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
     int Lmax = 0;
     for (int i = 0; i < D.batch; ++i) Lmax = h->L_host[i] > Lmax ? h->L_host[i] : Lmax;
     const int n_split_launch = (Lmax + D.split_len - 1) / D.split_len;
+    mark(h, -1);
     launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.batch, s);
     h->launches++;
     for (int l = 0; l < D.n_layers; ++l) {
         launch_rmsnorm(h->dtype, b.states, b.hres, h->na[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s);
         h->launches++;
+        mark(h, KIND_MISC);
         {
             EpiArgs a = base_epi(h, dq + 2 * dkv);
             a.q_out = b.qbuf;
@@ -202,6 +222,7 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             const int32_t rows[3] = {dq, dkv, dkv};
             int rc = run_gemm(h, h->p_qkv.empty() ? nullptr : h->p_qkv[l], EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a);
             if (rc) return rc;
+            mark(h, KIND_QKV);
         }
         {
             AttnArgs a;
@@ -223,6 +244,7 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             }
             if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, !mma, s)) return ESP_E_BADCFG;
             h->launches += (!mma && n_split_launch > 0) ? 2 : 1;
+            mark(h, KIND_ATTN);
         }
         {
             EpiArgs a = base_epi(h, D.d);
@@ -231,9 +253,11 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             const int32_t rows[3] = {D.d, 0, 0};
             int rc = run_gemm(h, h->p_o.empty() ? nullptr : h->p_o[l], EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.attn_out, dq, a);
             if (rc) return rc;
+            mark(h, KIND_O);
         }
         launch_rmsnorm(h->dtype, b.states, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s);
         h->launches++;
+        mark(h, KIND_MISC);
         {
             EpiArgs a = base_epi(h, D.F);
             a.act_out = b.act;
@@ -241,6 +265,7 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             const int32_t rows[3] = {D.F, D.F, 0};
             int rc = run_gemm(h, h->p_gu.empty() ? nullptr : h->p_gu[l], EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a);
             if (rc) return rc;
+            mark(h, KIND_GATEUP);
         }
         {
             EpiArgs a = base_epi(h, D.d);
@@ -249,11 +274,13 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             const int32_t rows[3] = {D.d, 0, 0};
             int rc = run_gemm(h, h->p_down.empty() ? nullptr : h->p_down[l], EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.act, D.F, a);
             if (rc) return rc;
+            mark(h, KIND_DOWN);
         }
     }
     if (with_lm) {
         launch_rmsnorm(h->dtype, b.states, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, D.batch, h->dbg_hidden, s);
         h->launches++;
+        mark(h, KIND_MISC);
         const int n_tiles = (D.V + TILE_N - 1) / TILE_N;
         EpiArgs a = base_epi(h, D.V);
         a.cand = b.cand; a.cand_ms = b.cand_ms; a.n_tiles = n_tiles; a.logits_dump = h->dbg_logits;
@@ -261,8 +288,10 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
         const int32_t rows[3] = {D.V, 0, 0};
         int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a);
         if (rc) return rc;
+        mark(h, KIND_LMHEAD);
         launch_topk_merge(b.states, b.cand, b.cand_ms, n_tiles, D.KP, D.batch, b.topk, b.lse, s);
         h->launches++;
+        mark(h, KIND_SELECT);
     }
     return cuda_ok(cudaGetLastError());
 }
@@ -281,6 +310,7 @@ int tree_step(esp_handle* h) {
     A.out_ring = h->b.out_ring;
     launch_tree_step(h->dtype, A, h->stream);
     h->launches++;
+    mark(h, KIND_SELECT);
     return cuda_ok(cudaGetLastError());
 }
 
@@ -523,6 +553,24 @@ int esp_debug_set_gemm(esp_handle* h, int32_t impl) {
     return ESP_OK;
 }
 
+int esp_step_profiled(esp_handle* h, float* ms_by_kind, int32_t* tokens_out, int32_t* n_out) {
+    if (!h || !ms_by_kind) return ESP_E_ARG;
+    h->prof = true;
+    h->ev_used = 0;
+    int rc = esp_step_async(h);
+    h->prof = false;
+    if (rc) return rc;
+    rc = esp_read(h, tokens_out, n_out);
+    for (int i = 0; i < KIND_N; ++i) ms_by_kind[i] = 0.f;
+    for (size_t i = 1; i < h->ev_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, h->ev[i - 1], h->ev[i]) != cudaSuccess) return ESP_E_CUDA;
+        const int kind = h->ev_kind[i];
+        if (kind >= 0 && kind < KIND_N) ms_by_kind[kind] += ms;
+    }
+    return rc;
+}
+
 int esp_get_stats(esp_handle* h, esp_stats* out) {
     if (!h || !out) return ESP_E_ARG;
     if (cudaStreamSynchronize(h->stream) != cudaSuccess) return ESP_E_CUDA;
@@ -549,6 +597,7 @@ void esp_free(esp_handle* h) {
     for (auto* p : h->p_down) tc_gemm_destroy(p);
     tc_gemm_destroy(h->p_lm);
     if (h->pinned) cudaFreeHost(h->pinned);
+    for (auto e : h->ev) cudaEventDestroy(e);
     delete h;
 }
 

@@ -1,0 +1,205 @@
+"""GPU parity tests (need a B200): the CUDA library, called through its C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import esp as O
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pu():
+    from tests import parity_util
+    return parity_util
+
+
+TOL_FP32 = 1e-4   # of the logit range, fp32 model
+TOL_BF16 = 2e-2   # of the logit range, bf16 model
+
+
+# ------------------------------------------------------------------ config 1: tiny fp32 model, full length
+@pytest.mark.parametrize("W,n_anchor,prune", [(0, 1, True), (0, 1, False), (1, 0, False), (0, 0, False)])
+def test_tiny_fp32_full_parity(pu, W, n_anchor, prune):
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=0)
+    prompt = synth.make_prompt(shape.vocab, 64, 0)
+    B = 32 if n_anchor == 1 else 20
+    spec = O.SpecCfg(n_probes=3, topk=4, max_nodes=B, expand_width=W, n_anchor=n_anchor, prune_parent=prune)
+    run = pu.ParityRun(shape, w, spec, prompt, 64, TOL_FP32)
+    out = run.run()
+    model = O.OracleModel(shape, w)
+    assert out == O.greedy_generate(model, prompt, 64, 256)           # lossless, and equal to the oracle stream
+    dec = O.EspOracle(model, spec, 512)
+    assert out == dec.generate(prompt, 64)
+    assert run.accepts == dec.accept_hist[:len(run.accepts)]          # same accepted lengths, step by step
+    g, _ = pu.gpu_generate(shape, run.wd, pu.GREEDY, prompt, 64)
+    assert g == out                                                   # GPU ESP == GPU greedy
+    if not prune:
+        assert max(run.accepts) >= 1                                  # drafts really get accepted here
+    run.close()
+
+
+def test_tiny_fp32_nontrivial_stream(pu):
+    """Same model family with wider weights and jittered norm gains, so the stream is not one repeated token."""
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=3, gain_jitter=True, std=0.3)
+    prompt = synth.make_prompt(shape.vocab, 97, 5)       # ragged last prefill chunk (97 = 64 + 33)
+    spec = O.SpecCfg(n_probes=3, topk=4, max_nodes=20, expand_width=1, n_anchor=0)
+    run = pu.ParityRun(shape, w, spec, prompt, 40, TOL_FP32)
+    out = run.run()
+    assert len(set(out)) > 10
+    assert out == O.greedy_generate(O.OracleModel(shape, w), prompt, 40, 256)
+    g, _ = pu.gpu_generate(shape, run.wd, pu.GREEDY, prompt, 40)
+    assert g == out
+    run.close()
+
+
+def test_forced_drafts_are_accepted_and_compacted(pu):
+    """Drive acceptance lengths random-init models never reach: the tree is set to contain the true
+    continuation (found by GPU greedy decoding), so several nodes are accepted and their KV rows move."""
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=3, gain_jitter=True, std=0.3)
+    prompt = synth.make_prompt(shape.vocab, 40, 6)
+    spec = O.SpecCfg(n_probes=2, topk=4, max_nodes=16, expand_width=0, n_anchor=1)
+    run = pu.ParityRun(shape, w, spec, prompt, 48, TOL_FP32)
+    truth, _ = pu.gpu_generate(shape, run.wd, pu.GREEDY, prompt, 48)
+    st = run.prefill()
+    rng = np.random.default_rng(0)
+    while len(run.emitted) < 40:
+        n = len(run.emitted)
+        depth = int(rng.integers(0, 4))
+        # a bushy tree: distractor siblings first, the true chain woven in at varying row indices
+        toks, pars = [run.emitted[-1]], [-1]
+        cur = 0
+        for dpt in range(depth):
+            sib = [int(t) for t in rng.integers(0, shape.vocab, size=int(rng.integers(0, 3))) if int(t) != truth[n + dpt]]
+            for t in sib:
+                toks.append(t); pars.append(cur)
+            toks.append(truth[n + dpt]); pars.append(cur)
+            nxt = len(toks) - 1
+            cur = nxt
+        order = sorted(range(len(toks)), key=lambda i: (0 if i == 0 else _depth(pars, i), i))
+        remap = {o: i for i, o in enumerate(order)}
+        forced = O.Tree(np.array([toks[o] for o in order], np.int32),
+                        np.array([-1 if pars[o] < 0 else remap[pars[o]] for o in order], np.int32),
+                        np.zeros(len(order), np.int32), np.zeros(len(order), np.float32))
+        st = run.step(st, forced=forced)
+        assert run.accepts[-1] >= depth
+    assert run.emitted[:40] == truth[:40]
+    assert max(run.accepts) >= 3
+    s = run.h.stats()
+    assert s.emitted == len(run.emitted) - 1 and s.steps == len(run.accepts) and s.device_error == 0
+    assert list(s.accept_hist)[:5] == [run.accepts.count(a) for a in range(5)]
+    run.close()
+
+
+def _depth(pars, i):
+    d = 0
+    while pars[i] >= 0:
+        i = pars[i]
+        d += 1
+    return d
+
+
+# ------------------------------------------------------------------ bf16 models on the tensor-core path
+BF16_SMALL = synth.TINY.replace(name="bf16-small", dtype="bf16", tied=False, n_layers=3, d_model=512, n_q_heads=4,
+                                n_kv_heads=2, head_dim=128, d_ffn=688, vocab=5000)
+
+
+@pytest.mark.parametrize("qk_norm,W,n_anchor,plen", [(True, 0, 1, 150), (False, 1, 0, 700)])
+def test_bf16_small_parity(pu, qk_norm, W, n_anchor, plen):
+    shape = BF16_SMALL.replace(qk_norm=qk_norm, rms_eps=1e-6 if qk_norm else 1e-5)
+    w = synth.make_weights(shape, seed=1, gain_jitter=True, std=0.05)
+    prompt = synth.make_prompt(shape.vocab, plen, 2)
+    spec = O.SpecCfg(n_probes=3, topk=5, max_nodes=16 if n_anchor else 12, expand_width=W, n_anchor=n_anchor)
+    run = pu.ParityRun(shape, w, spec, prompt, 32, TOL_BF16)
+    out = run.run()
+    assert len(set(out)) > 8
+    g, _ = pu.gpu_generate(shape, run.wd, pu.GREEDY, prompt, 32)
+    assert g == out                                      # bit-exact GPU ESP == GPU greedy
+    # the CUDA-core GEMM path must agree with the tensor-core path to bf16 accuracy as well
+    run2 = pu.ParityRun(shape, w, spec, prompt, 8, TOL_BF16, gemm_impl=1, w_dev=run.wd)
+    run2.run()
+    run.close(); run2.close()
+
+
+def test_bf16_forced_acceptance_bitwise_equals_greedy(pu):
+    """Accepted draft nodes must carry exactly the bits that plain decoding produces: force long accepted
+    paths and compare the ESP stream, token for token, with GPU greedy decoding."""
+    shape = BF16_SMALL
+    w = synth.make_weights(shape, seed=4, gain_jitter=True, std=0.05)
+    wd = pu.to_device(w)
+    prompt = synth.make_prompt(shape.vocab, 333, 3)
+    n_new = 96
+    truth, _ = pu.gpu_generate(shape, wd, pu.GREEDY, prompt, n_new, max_seq_len=600)
+    import paper_2603_17942_b200 as P
+    spec = O.SpecCfg(n_probes=3, topk=5, max_nodes=24, expand_width=0, n_anchor=1)
+    h = P.Handle(shape, pu.c_spec(spec), wd, max_seq_len=600)
+    out = [h.prefill(prompt)]
+    rng = np.random.default_rng(1)
+    accepted = []
+    while len(out) < n_new - 8:
+        depth = int(rng.integers(0, 6))
+        n = len(out)
+        toks = [out[-1]] + [truth[n + i] for i in range(depth)]
+        h.set_tree(np.array(toks, np.int32), np.arange(-1, depth, dtype=np.int32))
+        new = h.step()
+        accepted.append(len(new) - 1)
+        out.extend(new)
+    assert out == truth[:len(out)]
+    assert max(accepted) >= 4 and sum(accepted) > len(accepted)
+    assert h.stats().device_error == 0
+    h.close()
+
+
+# ------------------------------------------------------------------ config 3 / 4 kernel shapes (full width, few layers)
+@pytest.mark.parametrize("base,topk,B", [(synth.LLAMA3_8B, 10, 64), (synth.QWEN3_8B, 8, 48)])
+def test_full_width_shapes_parity(pu, base, topk, B):
+    """Every GEMM, attention and LM-head launch has the shape it has in the full model (d_model 4096, 32/8
+    heads of 128, the real FFN and vocabulary sizes, 4 probes, <= 64-node trees); only the layer count is cut
+    so the CPU oracle finishes in seconds."""
+    shape = base.replace(n_layers=2)
+    w = synth.make_weights(shape, seed=0, device="cuda")
+    wh = synth.weights_to_host(w)
+    prompt = synth.make_prompt(shape.vocab, 200, 0)
+    spec = O.SpecCfg(n_probes=4, topk=topk, max_nodes=B, expand_width=0, n_anchor=1)
+    run = pu.ParityRun(shape, wh, spec, prompt, 4, TOL_BF16, w_dev=w)
+    out = run.run()
+    g, _ = pu.gpu_generate(shape, w, pu.GREEDY, prompt, 4)
+    assert g == out
+    assert run.h.stats().device_error == 0
+    run.close()
+
+
+# ------------------------------------------------------------------ errors are reported, not raised from the device
+def test_host_side_errors(pu):
+    import paper_2603_17942_b200 as P
+    shape = synth.TINY
+    w = pu.to_device(synth.make_weights(shape, seed=0))
+    with pytest.raises(P.EspError) as e:
+        P.Handle(shape, P.spec_cfg(n_probes=4, topk=4, max_nodes=70, n_anchor=0), w, 128)   # (k+1)*70 rows
+    assert e.value.code == -1
+    with pytest.raises(P.EspError):
+        P.Handle(shape.replace(head_dim=48), P.spec_cfg(), w, 128)
+    h = P.Handle(shape, P.spec_cfg(n_probes=2, topk=4, max_nodes=8), w, 96)
+    with pytest.raises(P.EspError) as e:
+        h.step()
+    assert e.value.code == -7                                   # step before prefill
+    with pytest.raises(P.EspError) as e:
+        h.prefill(np.array([1, 2, shape.vocab], np.int32))
+    assert e.value.code == -3
+    with pytest.raises(P.EspError) as e:
+        h.prefill(np.zeros(97, np.int32))
+    assert e.value.code == -3                                   # longer than max_seq_len
+    h.prefill(synth.make_prompt(shape.vocab, 80, 1))
+    with pytest.raises(P.EspError) as e:
+        h.set_tree(np.array([1, 2], np.int32), np.array([-1, 1], np.int32))   # parent not before child
+    assert e.value.code == -8
+    with pytest.raises(P.EspError) as e:
+        for _ in range(40):
+            h.step()
+    assert e.value.code == -4                                   # sequence full
+    assert h.stats().device_error == 0
+    h.close()
