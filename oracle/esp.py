@@ -50,6 +50,7 @@ def _load():
         _lib = ctypes.CDLL(_build.build())
         _lib.orc_block_forward.restype = ctypes.c_int
         _lib.orc_tree_attention.restype = ctypes.c_int
+        _lib.orc_linear.restype = ctypes.c_int
         _lib.orc_num_threads.restype = ctypes.c_int
     return _lib
 
@@ -145,6 +146,20 @@ def tree_attention(q, kc, vc, kb, vb, vis):
     if rc != 0:
         raise RuntimeError("orc_tree_attention failed")
     return out
+
+
+def linear(x, w) -> np.ndarray:
+    """y = x W^T with the oracle's matrix product (fp32 running sums over k): x [M,K] fp32, w [N,K] fp32 or bf16."""
+    x = _np(x, _F32)
+    M, K = x.shape
+    N = w.shape[0]
+    is_bf16 = hasattr(w, "dtype") and str(w.dtype).endswith("bfloat16")
+    y = np.zeros((M, N), dtype=_F32)
+    rc = _load().orc_linear(ctypes.c_int32(M), ctypes.c_int32(K), ctypes.c_int32(N), ctypes.c_void_p(x.ctypes.data),
+                            ctypes.c_void_p(_ptr(w)), ctypes.c_int32(1 if is_bf16 else 0), ctypes.c_void_p(y.ctypes.data))
+    if rc != 0:
+        raise RuntimeError("orc_linear failed")
+    return y
 
 
 # --------------------------------------------------------------------------- ESP pieces

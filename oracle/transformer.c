@@ -114,6 +114,17 @@ static void linear_T(const float* xT, int M, int K, const void* W, int wdtype, i
     }
 }
 
+/* Stand-alone entry to the matrix product above, for operator-level checks: y[M][N] = x[M][K] * W[N][K]^T. */
+int orc_linear(int32_t M, int32_t K, int32_t N, const float* x, const void* W, int32_t wdtype, float* y) {
+    float* xT = (float*)malloc(sizeof(float) * (size_t)M * K);
+    if (!xT) return -1;
+    for (int m = 0; m < M; ++m)
+        for (int k = 0; k < K; ++k) xT[(size_t)k * M + m] = x[(size_t)m * K + k];
+    linear_T(xT, M, K, W, wdtype, N, y);
+    free(xT);
+    return 0;
+}
+
 static void transpose(const float* x, int M, int K, float* xT) {
     for (int m = 0; m < M; ++m)
         for (int k = 0; k < K; ++k) xT[(size_t)k * M + m] = x[(size_t)m * K + k];

@@ -214,3 +214,17 @@ def test_tree_attention_operator_against_softmax_definition():
         s[~allow] = -np.inf
         p = torch.softmax(torch.from_numpy(s), dim=-1).numpy()
         np.testing.assert_allclose(out[:, hh], p @ V[:, hh // 2], rtol=0, atol=2e-6)
+
+
+def test_linear_operator_against_library_matmul():
+    """The stand-alone matrix product against numpy's fp64 matmul, fp32 and bf16 weights, ragged sizes; a
+    transposed operand or a dropped k term would show as an O(1) error."""
+    rng = np.random.default_rng(3)
+    for M, K, N in ((1, 8, 5), (7, 72, 131), (80, 200, 9)):
+        x = rng.standard_normal((M, K)).astype(np.float32)
+        w = torch.from_numpy(rng.standard_normal((N, K)).astype(np.float32))
+        ref = x.astype(np.float64) @ w.double().numpy().T
+        assert np.abs(esp.linear(x, w) - ref).max() <= 1e-5 * np.abs(ref).max()
+        wb = w.bfloat16()
+        refb = x.astype(np.float64) @ wb.double().numpy().T
+        assert np.abs(esp.linear(x, wb) - refb).max() <= 1e-5 * np.abs(refb).max()
