@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the ESP decode-and-verify step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config llama3-8b|qwen3-8b]
+
+One "step" is one esp_step: a decoder forward over [last accepted token, draft-tree nodes, mask probes]
+against the KV cache, Top-K' at the probe rows, verification, KV compaction, mask update and the next tree.
+Workload (default): the Llama-3-8B-shape bf16 decoder with seeded random-init weights, a 1024-token random
+prompt, 4 mask probes, Top-10 per probe, trees of at most 64 nodes, batch 1.  Weights (15 GB) are streamed
+from HBM every step, far more than the L2 holds, so no cache flush is needed between steps.
+
+Prints ONE JSON line.  `value` is accepted tokens per second with everything resident on the device
+(K esp_step_async calls between two CUDA events on the library's stream); `e2e` is the same metric through
+the synchronous esp_step call that returns the tokens in host memory every step.  With N > 1 every rank runs
+an independent replica of the whole job (the method has no cross-GPU exchange); `value` sums the replicas'
+tokens over the slowest rank's time.
+
+`--impl reference` times the CPU oracle (oracle/) on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "esp_accepted_tokens_per_s"
+UNIT = "tok/s"
+
+WORKLOADS = {
+    # name: (shape attr in synth, prompt length, probes, topk, max_nodes)
+    "llama3-8b": ("LLAMA3_8B", 1024, 4, 10, 64),
+    "qwen3-8b": ("QWEN3_8B", 2048, 4, 8, 48),
+}
+
+
+def measured_peaks():
+    """HBM copy bandwidth (GB/s) measured on this machine, else the fallback figure; returns (value, source)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ts, line in self.lines:
+            if ts < t0 or ts > t1 + 0.1:
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def random_block(n_nodes, k, seed):
+    """Row layout of a 64-node random tree with a k-probe chain under the root, for the oracle sample."""
+    import synth
+    parents = synth.random_tree_parents(n_nodes, 4, seed)
+    M = n_nodes + k
+    vis = np.zeros((M, M), np.uint8)
+    pos = np.zeros(M, np.int32)
+    for i in range(n_nodes):
+        a = i
+        while a >= 0:
+            vis[i, a] = 1
+            a = int(parents[a])
+        pos[i] = vis[i].sum() - 1
+    for j in range(k):
+        r = n_nodes + j
+        vis[r, 0] = 1
+        vis[r, n_nodes:r + 1] = 1
+        pos[r] = j + 1
+    return vis, pos
+
+
+class OracleSample:
+    """One bounded sample of the workload for the CPU oracle: a full-width block (all tree and probe rows)
+    through ONE decoder layer and the LM head against a random KV cache of the prompt's length.  The oracle's
+    time for a whole step is 32 (n_layers) x the layer time + the LM-head time; accepted tokens per step are
+    taken as 1 (random-init models accept no drafts)."""
+
+    def __init__(self, shape, plen, k, B, host_weights):
+        from oracle import esp as O
+        self.O = O
+        self.shape1 = shape.replace(n_layers=1)
+        self.n_layers = shape.n_layers
+        self.model = O.OracleModel(self.shape1, host_weights)
+        rng = np.random.default_rng(0)
+        self.L = plen
+        self.kc, self.vc = self.model.new_cache(plen + 8)
+        self.kc[:, :plen] = rng.standard_normal(self.kc[:, :plen].shape, dtype=np.float32)
+        self.vc[:, :plen] = rng.standard_normal(self.vc[:, :plen].shape, dtype=np.float32)
+        self.vis, pos = random_block(B, k, 0)
+        self.pos = plen + pos
+        self.M = B + k
+        self.x = (rng.standard_normal((self.M, shape.d_model), dtype=np.float32) * 0.02).astype(np.float32)
+        self.cores = O.num_threads()
+
+    def step_seconds(self):
+        none = np.zeros(self.M, np.uint8)
+        t0 = time.perf_counter()
+        self.model.block_forward(self.kc, self.vc, self.L, self.x, self.pos, self.vis, want=none)
+        t1 = time.perf_counter()
+        self.model.block_forward(self.kc, self.vc, self.L, self.x, self.pos, self.vis)
+        t2 = time.perf_counter()
+        t_layer, t_both = t1 - t0, t2 - t1
+        return self.n_layers * t_layer + max(t_both - t_layer, 0.0)
+
+    def describe(self):
+        return (f"one {self.M}-row block through 1 of {self.n_layers} layers + LM head, KV length {self.L}; "
+                f"step time = {self.n_layers} x layer + head, 1 token per step")
+
+
+def host_slice(shape, w_dev=None, seed=0):
+    """Host copies of what the one-layer oracle sample needs (embed, lm_head, final norm, layer 0)."""
+    import synth
+    import torch
+    if w_dev is None:
+        s1 = shape.replace(n_layers=1)
+        return synth.make_weights(s1, seed=seed, device="cpu")
+    out = {}
+    for k, v in w_dev.items():
+        out[k] = [v[0].cpu()] if isinstance(v, list) else v.cpu()
+    if w_dev["lm_head"] is w_dev["embed"]:
+        out["lm_head"] = out["embed"]
+    return out
+
+
+def run_reference(args, shape, plen, k, K, B):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleSample(shape, plen, k, B, host_slice(shape))
+    for _ in range(min(args.warmup, 1)):
+        smp.step_seconds()
+    steps = max(1, args.steps)
+    budget_s = 180.0
+    times = []
+    t_start = time.perf_counter()
+    for i in range(steps):
+        times.append(smp.step_seconds())
+        if time.perf_counter() - t_start > budget_s and i + 1 < steps:
+            break
+    sec = float(np.mean(times))
+    val = 1.0 / sec
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
+            "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.config + "-shape bf16 weights, b=1", "prompt_len": plen, "n_probes": k, "topk": K,
+                       "max_nodes": B},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": smp.describe()},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def algorithmic_bytes(shape, L_mean, rows):
+    """Bytes one step must move: every layer matrix and the LM head once, the KV cache of L positions once,
+    the K/V rows of the block written once."""
+    es = 2 if shape.dtype == "bf16" else 4
+    w = shape.n_params_streamed() * es
+    kv_per_pos = shape.n_layers * 2 * shape.n_kv_heads * shape.head_dim * es
+    return w, kv_per_pos * L_mean + kv_per_pos * rows
+
+
+def run_ours(args, shape, plen, k, K, B):
+    import torch
+    import synth
+    import paper_2603_17942_b200 as P
+    from paper_2603_17942_b200 import build as esp_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        esp_build.build()
+    if dist is not None:
+        dist.barrier()
+    P.load_library()
+
+    steps, warm = args.steps, max(args.warmup, 3)
+    w = synth.make_weights(shape, seed=rank, device="cuda")
+    prompt = synth.make_prompt(shape.vocab, plen, rank)
+    spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1)
+    max_seq = plen + (k + 1) * (2 * steps + 2 * warm + 16) + 64
+    stream = torch.cuda.Stream()
+    h = P.Handle(shape, spec, w, max_seq_len=max_seq, stream=stream)
+    h.prefill(prompt)
+
+    def emitted_steps():
+        st = h.stats()
+        return int(st.emitted), int(st.steps), st
+
+    # ---- device-resident throughput: K asynchronous steps between two events on the library's stream
+    for _ in range(warm):
+        h.step()
+    e0, s0, _ = emitted_steps()
+    L0 = h.state()["L"]
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    with torch.cuda.stream(stream):
+        ev0.record()
+        for _ in range(steps):
+            h.step_async()
+        ev1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    h.read()
+    ms = ev0.elapsed_time(ev1)
+    e1, s1, st = emitted_steps()
+    L1 = h.state()["L"]
+    tokens = e1 - e0
+    launches = int(st.kernels_per_step) * steps
+    rows = h.state()["n_rows"]
+
+    # ---- end to end: the synchronous call, tokens land in host memory every step
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    te0 = time.perf_counter()
+    e2e_tokens = 0
+    for _ in range(steps):
+        e2e_tokens += len(h.step())
+    torch.cuda.synchronize()
+    te1 = time.perf_counter()
+    e2e_ms = (te1 - te0) * 1e3
+    d2h = (P.ESP_MAX_PROBES + 4) * 4 + 4
+
+    # ---- per-kernel-group device times (events between groups), for the roofline of the dominant kernel
+    n_prof = min(steps, 20)
+    kinds = {kname: 0.0 for kname in P.KINDS}
+    for _ in range(n_prof):
+        for kname, v in P.esp_step_profiled(h.h, h.tokens_out, h.n_out).items():
+            kinds[kname] += v / n_prof
+    if h.stats().device_error != 0:
+        raise SystemExit("device error word set during the benchmark")
+
+    # ---- greedy decoding with the same kernels (one row per step), for context
+    greedy_tok_s = None
+    if rank == 0 and not args.no_greedy:
+        hg = P.Handle(shape, P.spec_cfg(), w, max_seq_len=plen + 2 * steps + 64, stream=stream)
+        hg.prefill(prompt)
+        for _ in range(warm):
+            hg.step()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            g0.record()
+            for _ in range(steps):
+                hg.step_async()
+            g1.record()
+        torch.cuda.synchronize()
+        hg.read()
+        greedy_tok_s = steps / (g0.elapsed_time(g1) * 1e-3)
+        hg.close()
+
+    # ---- aggregate over ranks: slowest rank's time, all ranks' tokens
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        c = torch.tensor([tokens, e2e_tokens, launches], device="cuda", dtype=torch.float64)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+        ms, e2e_ms = float(t[0]), float(t[1])
+        tokens, e2e_tokens, launches = int(c[0]), int(c[1]), int(c[2])
+
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        es = 2
+        F, d = shape.d_ffn, shape.d_model
+        gu_bytes = 2 * F * d * es + rows * d * es + rows * F * es   # gate+up weights, activations in, SwiGLU out
+        gu_ms = kinds["gateup_gemm"] / shape.n_layers
+        gu_ach = gu_bytes / (gu_ms * 1e-3) / 1e9 if gu_ms > 0 else None
+        wbytes, kvbytes = algorithmic_bytes(shape, 0.5 * (L0 + L1), rows)
+        step_ms = ms / steps
+        step_ach = (wbytes + kvbytes) / (step_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+            "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"{args.config}-shape bf16 decoder, random-init seeded weights, b=1",
+                       "prompt_len": plen, "n_probes": k, "topk": K, "max_nodes": B, "rows_per_step": rows,
+                       "replicas": world, "l2": "inputs exceed L2 (weights are re-streamed every step)"},
+            "mean_accepted_len": tokens / (steps * world),
+            "clocks": clocks,
+            "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": d2h,
+                    "note": "synchronous esp_step; a step's inputs are the device state left by the previous step"},
+            "gpu_launches": launches,
+            "roofline": {"bound": "hbm", "kernel": "k_gemm_tc<EPI_SWIGLU> (gate/up GEMM + SiLU*up)",
+                         "achieved": gu_ach, "peak": peak, "unit": "GB/s", "frac": gu_ach / peak if gu_ach else None,
+                         "traffic": None, "peak_source": peak_src, "bytes_per_launch": gu_bytes,
+                         "us_per_launch": gu_ms * 1e3},
+            "step_roofline": {"bound": "hbm", "bytes_per_step": wbytes + kvbytes, "weight_bytes": wbytes,
+                              "kv_bytes": kvbytes, "achieved": step_ach, "peak": peak, "unit": "GB/s",
+                              "frac": step_ach / peak, "frac_of_8TBs_nominal": step_ach / 8000.0,
+                              "peak_source": peak_src},
+            "kernel_group_ms_per_step": kinds,
+            "greedy_tok_s": greedy_tok_s,
+        }
+        if not args.no_cpu and world == 1:
+            smp = OracleSample(shape, plen, k, B, host_slice(shape, w))
+            sec = smp.step_seconds()
+            line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+                                    "sample": smp.describe(), "ms_per_step": sec * 1e3}
+        else:
+            line["cpu_baseline"] = None
+        print(json.dumps(line), flush=True)
+    h.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="llama3-8b", choices=sorted(WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="cut the layer count (smaller captures under a profiler)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--no-greedy", action="store_true", help="skip the greedy-decoding leg")
+    args = ap.parse_args()
+    import synth
+    name, plen, k, K, B = WORKLOADS[args.config]
+    shape = getattr(synth, name)
+    if args.layers > 0:
+        shape = shape.replace(n_layers=args.layers)
+    if args.impl == "reference":
+        run_reference(args, shape, plen, k, K, B)
+    else:
+        run_ours(args, shape, plen, k, K, B)
+
+
+if __name__ == "__main__":
+    main()
