@@ -150,6 +150,10 @@ struct esp_handle {
     int launches = 0, kernels_per_step = 0;
     size_t layer_kv_stride = 0;  // bytes
     bool prof = false;           // record an event after every kernel group
+    bool use_pdl = true;         // programmatic dependent launch between the kernels of a step
+    bool use_graph = true;       // replay the step's launch sequence as a CUDA graph
+    struct StepGraph { int n_split; cudaGraphExec_t exec; int kernels; };
+    std::vector<StepGraph> graphs;
     std::vector<cudaEvent_t> ev;
     std::vector<int> ev_kind;
     size_t ev_used = 0;
@@ -189,13 +193,17 @@ EpiArgs base_epi(esp_handle* h, int n_out) {
 }
 
 int run_gemm(esp_handle* h, TcGemm* plan, int epi, int n_tiles, const void* const w[3], const int32_t rows_w[3],
-             const void* x, int K, const EpiArgs& a) {
+             const void* x, int K, const EpiArgs& a, bool tc, bool pdl) {
     h->launches++;
-    if (h->dtype == 1 && h->gemm_impl == 0 && plan) return tc_gemm_launch(plan, a, h->stream);
-    launch_gemm_simt(h->dtype, epi, n_tiles, h->D.batch, w, rows_w, x, K, a, h->stream);
+    if (tc) return tc_gemm_launch(plan, a, h->stream, pdl);
+    launch_gemm_simt(h->dtype, epi, n_tiles, h->D.batch, w, rows_w, x, K, a, h->stream, pdl);
     return ESP_OK;
 }
 
+// One decoder forward over the block every active sequence has in its row table.
+// Tensor-core path (bf16, one sequence): the QKV, O and down GEMMs store stream-K partials that the next
+// kernel sums (k_qkv_finish; k_resid_norm = residual add + RMSNorm), gate/up and the LM head finish in-kernel.
+// CUDA-core path (fp32 models, batched bf16): the same layer with every epilogue fused in the GEMM.
 int forward(esp_handle* h, bool with_lm, int dcap) {
     const Dims& D = h->D;
     Buffers& b = h->b;
@@ -204,11 +212,16 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
     int Lmax = 0;
     for (int i = 0; i < D.batch; ++i) Lmax = h->L_host[i] > Lmax ? h->L_host[i] : Lmax;
     const int n_split_launch = (Lmax + D.split_len - 1) / D.split_len;
+    const bool tc = h->dtype == 1 && h->gemm_impl == 0 && h->p_lm != nullptr;
+    const bool pdl = h->use_pdl && !h->prof;
+    StreamK pending;   // partials of the last down projection, summed by the next norm
+    pending.partials = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1;
     mark(h, -1);
-    launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.batch, s);
+    launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.batch, s, false);
     h->launches++;
     for (int l = 0; l < D.n_layers; ++l) {
-        launch_rmsnorm(h->dtype, b.states, b.hres, h->na[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s);
+        if (tc) launch_resid_norm(b.states, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
+        else launch_rmsnorm(h->dtype, b.states, b.hres, h->na[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
         {
@@ -220,8 +233,12 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             a.k_norm = D.qk_norm ? h->kn[l] : nullptr;
             const void* w[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t rows[3] = {dq, dkv, dkv};
-            int rc = run_gemm(h, h->p_qkv.empty() ? nullptr : h->p_qkv[l], EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a);
+            int rc = run_gemm(h, tc ? h->p_qkv[l] : nullptr, EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a, tc, pdl);
             if (rc) return rc;
+            if (tc) {
+                if (launch_qkv_finish(a, tc_gemm_streamk(h->p_qkv[l]), s, pdl)) return ESP_E_BADCFG;
+                h->launches++;
+            }
             mark(h, KIND_QKV);
         }
         {
@@ -239,10 +256,10 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             a.err = b.err;
             const bool mma = h->dtype == 1 && D.h == 128 && h->gemm_impl == 0;
             if (mma && n_split_launch > 0) {
-                if (launch_attn_bulk_mma(a, D.batch, n_split_launch, s)) return ESP_E_BADCFG;
+                if (launch_attn_bulk_mma(a, D.batch, n_split_launch, s, pdl)) return ESP_E_BADCFG;
                 h->launches++;
             }
-            if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, !mma, s)) return ESP_E_BADCFG;
+            if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, !mma, s, pdl)) return ESP_E_BADCFG;
             h->launches += (!mma && n_split_launch > 0) ? 2 : 1;
             mark(h, KIND_ATTN);
         }
@@ -251,11 +268,12 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             a.hres = b.hres;
             const void* w[3] = {h->wo[l], nullptr, nullptr};
             const int32_t rows[3] = {D.d, 0, 0};
-            int rc = run_gemm(h, h->p_o.empty() ? nullptr : h->p_o[l], EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.attn_out, dq, a);
+            int rc = run_gemm(h, tc ? h->p_o[l] : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.attn_out, dq, a, tc, pdl);
             if (rc) return rc;
             mark(h, KIND_O);
         }
-        launch_rmsnorm(h->dtype, b.states, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s);
+        if (tc) launch_resid_norm(b.states, b.hres, tc_gemm_streamk(h->p_o[l]), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
+        else launch_rmsnorm(h->dtype, b.states, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
         {
@@ -263,7 +281,7 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             a.act_out = b.act;
             const void* w[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t rows[3] = {D.F, D.F, 0};
-            int rc = run_gemm(h, h->p_gu.empty() ? nullptr : h->p_gu[l], EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a);
+            int rc = run_gemm(h, tc ? h->p_gu[l] : nullptr, EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a, tc, pdl);
             if (rc) return rc;
             mark(h, KIND_GATEUP);
         }
@@ -272,13 +290,15 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             a.hres = b.hres;
             const void* w[3] = {h->wd[l], nullptr, nullptr};
             const int32_t rows[3] = {D.d, 0, 0};
-            int rc = run_gemm(h, h->p_down.empty() ? nullptr : h->p_down[l], EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.act, D.F, a);
+            int rc = run_gemm(h, tc ? h->p_down[l] : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.act, D.F, a, tc, pdl);
             if (rc) return rc;
+            if (tc) pending = tc_gemm_streamk(h->p_down[l]);
             mark(h, KIND_DOWN);
         }
     }
     if (with_lm) {
-        launch_rmsnorm(h->dtype, b.states, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, D.batch, h->dbg_hidden, s);
+        if (tc) launch_resid_norm(b.states, b.hres, pending, h->final_norm, b.xn, D.d, D.rms_eps, h->dbg_hidden, s, pdl);
+        else launch_rmsnorm(h->dtype, b.states, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, D.batch, h->dbg_hidden, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
         const int n_tiles = (D.V + TILE_N - 1) / TILE_N;
@@ -286,10 +306,10 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
         a.cand = b.cand; a.cand_ms = b.cand_ms; a.n_tiles = n_tiles; a.logits_dump = h->dbg_logits;
         const void* w[3] = {h->lm_head, nullptr, nullptr};
         const int32_t rows[3] = {D.V, 0, 0};
-        int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a);
+        int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl);
         if (rc) return rc;
         mark(h, KIND_LMHEAD);
-        launch_topk_merge(b.states, b.cand, b.cand_ms, n_tiles, D.KP, D.batch, b.topk, b.lse, s);
+        launch_topk_merge(b.states, b.cand, b.cand_ms, n_tiles, D.KP, D.batch, b.topk, b.lse, s, pdl);
         h->launches++;
         mark(h, KIND_SELECT);
     }
@@ -308,10 +328,15 @@ int tree_step(esp_handle* h) {
     A.vcache = h->b.vcache;
     A.err = h->b.err;
     A.out_ring = h->b.out_ring;
-    launch_tree_step(h->dtype, A, h->stream);
+    launch_tree_step(h->dtype, A, h->stream, h->use_pdl && !h->prof);
     h->launches++;
     mark(h, KIND_SELECT);
     return cuda_ok(cudaGetLastError());
+}
+
+void drop_graphs(esp_handle* h) {
+    for (auto& g : h->graphs) cudaGraphExecDestroy(g.exec);
+    h->graphs.clear();
 }
 
 __global__ void k_select(SeqState* st, int batch, int seq_only) {
@@ -389,12 +414,12 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
             TcGemm* p = nullptr;
             const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t r1[3] = {dq, dkv, dkv};
-            ok = ok && !tc_gemm_create(&p, EPI_QKV, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
             h->p_qkv.push_back(p);
             const void* w2[3] = {h->wo[l], nullptr, nullptr};
             const int32_t r2[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_RESID, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
             h->p_o.push_back(p);
             const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t r3[3] = {D.F, D.F, 0};
@@ -404,7 +429,7 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
             const void* w4[3] = {h->wd[l], nullptr, nullptr};
             const int32_t r4[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_RESID, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
             h->p_down.push_back(p);
         }
         const void* w5[3] = {h->lm_head, nullptr, nullptr};
@@ -455,17 +480,56 @@ int esp_prefill(esp_handle* h, int32_t seq, const int32_t* prompt, int32_t n_pro
 int esp_step_async(esp_handle* h) {
     if (!h) return ESP_E_ARG;
     bool any = false;
+    int Lmax = 0;
     for (int i = 0; i < h->D.batch; ++i) {
         if (!h->ready[i]) continue;
         any = true;
         if (h->L_host[i] + h->D.k + 1 + RT > h->D.cap) return ESP_E_FULL;
+        Lmax = h->L_host[i] > Lmax ? h->L_host[i] : Lmax;
     }
     if (!any) return ESP_E_STATE;
-    const int before = h->launches;
-    int rc = forward(h, true, DCAP_STEP);
-    if (rc) return rc;
-    rc = tree_step(h);
-    h->kernels_per_step = h->launches - before;
+    int rc = ESP_OK;
+    bool done = false;
+    if (h->use_graph && !h->prof) {
+        // The launch sequence of a step depends on the host only through the number of attention splits;
+        // every other quantity (L, row counts, the tree) is read from device state by the kernels.
+        const int n_split = (Lmax + h->D.split_len - 1) / h->D.split_len;
+        esp_handle::StepGraph* g = nullptr;
+        for (auto& e : h->graphs)
+            if (e.n_split == n_split) g = &e;
+        if (!g) {
+            cudaGraph_t graph = nullptr;
+            cudaGraphExec_t exec = nullptr;
+            const int before = h->launches;
+            bool ok = cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+            if (ok) {
+                int r1 = forward(h, true, DCAP_STEP);
+                int r2 = r1 ? r1 : tree_step(h);
+                ok = cudaStreamEndCapture(h->stream, &graph) == cudaSuccess && !r2 && graph;
+            }
+            if (ok) ok = cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess;
+            if (graph) cudaGraphDestroy(graph);
+            if (ok) {
+                h->graphs.push_back({n_split, exec, h->launches - before});
+                g = &h->graphs.back();
+            } else {
+                cudaGetLastError();      // capture is not available here: launch directly from now on
+                h->use_graph = false;
+            }
+        }
+        if (g) {
+            if (cudaGraphLaunch(g->exec, h->stream) != cudaSuccess) return ESP_E_CUDA;
+            h->kernels_per_step = g->kernels;
+            done = true;
+        }
+    }
+    if (!done) {
+        const int before = h->launches;
+        rc = forward(h, true, DCAP_STEP);
+        if (rc) return rc;
+        rc = tree_step(h);
+        h->kernels_per_step = h->launches - before;
+    }
     // until the result is read the host only knows an upper bound of each cache length
     for (int i = 0; i < h->D.batch; ++i)
         if (h->ready[i]) h->L_host[i] += h->D.k + 1;
@@ -542,6 +606,7 @@ int esp_debug_capture(esp_handle* h, float* logits, float* hidden) {
     if (!h) return ESP_E_ARG;
     h->dbg_logits = logits;
     h->dbg_hidden = hidden;
+    drop_graphs(h);
     return ESP_OK;
 }
 
@@ -550,6 +615,7 @@ int esp_debug_set_gemm(esp_handle* h, int32_t impl) {
     if (h->dtype == 0 && impl == 0) return ESP_E_BADCFG;
     if (impl == 0 && !h->p_lm) return ESP_E_BADCFG;
     h->gemm_impl = impl;
+    drop_graphs(h);
     return ESP_OK;
 }
 
@@ -597,6 +663,7 @@ void esp_free(esp_handle* h) {
     for (auto* p : h->p_down) tc_gemm_destroy(p);
     tc_gemm_destroy(h->p_lm);
     if (h->pinned) cudaFreeHost(h->pinned);
+    drop_graphs(h);
     for (auto e : h->ev) cudaEventDestroy(e);
     delete h;
 }
@@ -643,8 +710,8 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
     const int n_split_launch = (L + S - 1) / S;
     const bool mma = dtype == 1 && head_dim == 128;
-    if (mma && n_split_launch > 0 && launch_attn_bulk_mma(a, batch, n_split_launch, s)) return ESP_E_BADCFG;
-    if (launch_attn_simt(dtype, a, batch, n_split_launch, !mma, s)) return ESP_E_BADCFG;
+    if (mma && n_split_launch > 0 && launch_attn_bulk_mma(a, batch, n_split_launch, s, false)) return ESP_E_BADCFG;
+    if (launch_attn_simt(dtype, a, batch, n_split_launch, !mma, s, false)) return ESP_E_BADCFG;
     return cuda_ok(cudaGetLastError());
 }
 
@@ -669,7 +736,7 @@ int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const
     const int32_t rw[3] = {n_out, 0, 0};
     const int n_tiles = (n_out + TILE_N - 1) / TILE_N;
     if (impl == 1) {
-        launch_gemm_simt(1, EPI_STORE_F32, n_tiles, 1, wv, rw, x, k_in, a, s);
+        launch_gemm_simt(1, EPI_STORE_F32, n_tiles, 1, wv, rw, x, k_in, a, s, false);
         return cuda_ok(cudaGetLastError());
     }
     if (impl != 0) return ESP_E_ARG;
@@ -683,7 +750,7 @@ int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const
     if (cudaMemsetAsync(err, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
     TcGemm* plan = nullptr;
     if (tc_gemm_create(&plan, EPI_STORE_F32, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err)) return ESP_E_CUDA;
-    int rc = tc_gemm_launch(plan, a, s);
+    int rc = tc_gemm_launch(plan, a, s, false);
     int e = 0;
     if (!rc && cudaMemcpyAsync(&e, err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) rc = ESP_E_CUDA;
     if (!rc && cudaStreamSynchronize(s) != cudaSuccess) rc = ESP_E_CUDA;

@@ -56,6 +56,8 @@ __device__ __forceinline__ uint32_t kv_off(int key, int u) { return (uint32_t)(k
 
 __global__ void __launch_bounds__(128) k_attn_bulk_mma(AttnArgs a, int n_split_launch, int group, int rows_per_tile, int n_row_tiles) {
     extern __shared__ __align__(128) unsigned char smem[];
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x;
     const int kvh = blockIdx.y / n_row_tiles, rtile = blockIdx.y % n_row_tiles;
@@ -250,7 +252,7 @@ __global__ void __launch_bounds__(128) k_attn_bulk_mma(AttnArgs a, int n_split_l
 
 }  // namespace
 
-int launch_attn_bulk_mma(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s) {
+int launch_attn_bulk_mma(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl) {
     if (a.h != HD || a.Hq % a.Hkv) return -1;
     const int group = a.Hq / a.Hkv;
     if (group > PAIRS || PAIRS % group) return -1;
@@ -263,7 +265,7 @@ int launch_attn_bulk_mma(const AttnArgs& a, int batch, int n_split_launch, cudaS
         attr_set = true;
     }
     dim3 grid(n_split_launch, a.Hkv * n_row_tiles, batch);
-    k_attn_bulk_mma<<<grid, 128, smem, s>>>(a, n_split_launch, group, rows_per_tile, n_row_tiles);
+    launch_k(k_attn_bulk_mma, grid, dim3(128), (size_t)smem, s, pdl, a, n_split_launch, group, rows_per_tile, n_row_tiles);
     return 0;
 }
 

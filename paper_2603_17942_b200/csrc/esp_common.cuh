@@ -70,8 +70,32 @@ struct Dims {
     float lambda;
 };
 
-// epilogue selectors of the small-M GEMMs
-enum Epi : int { EPI_STORE_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, EPI_LOGITS = 4 };
+// epilogue selectors of the small-M GEMMs.  EPI_PARTIAL (tensor-core kernel only) finishes nothing: every
+// (tile, k-range) segment is stored as an fp32 partial and the kernel that consumes the result sums them.
+enum Epi : int { EPI_STORE_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, EPI_LOGITS = 4, EPI_PARTIAL = 5 };
+
+// Stream-K partition of a GEMM: the n_tiles*KB (tile, k-block) units are dealt out in equal contiguous
+// ranges to G persistent CTAs; CTA c owns units [c*U/G, (c+1)*U/G).  A CTA's range touches at most one
+// tile it does not start (slot 1) besides the tile holding its first unit (slot 0).  Partials live at
+// partials[((cta*2 + slot)*RT + row)*TILE_N + feature].
+struct StreamK {
+    const float* partials;  // NULL: nothing to sum
+    int32_t n_tiles, KB, G;
+};
+__host__ __device__ __forceinline__ long long sk_begin(long long c, long long U, long long G) { return c * U / G; }
+__host__ __device__ __forceinline__ int sk_cta_of_unit(long long u, long long U, long long G) {
+    return (int)(((u + 1) * G + U - 1) / U - 1);
+}
+// contributors of a tile, in the (fixed) order their partials are summed
+__host__ __device__ __forceinline__ void sk_contributors(const StreamK& s, int tile, int& c_first, int& c_last) {
+    const long long U = (long long)s.n_tiles * s.KB, t0 = (long long)tile * s.KB;
+    c_first = sk_cta_of_unit(t0, U, s.G);
+    c_last = sk_cta_of_unit(t0 + s.KB - 1, U, s.G);
+}
+__host__ __device__ __forceinline__ int sk_slot(const StreamK& s, int c, int tile) {
+    const long long U = (long long)s.n_tiles * s.KB;
+    return tile == (int)(sk_begin(c, U, s.G) / s.KB) ? 0 : 1;
+}
 
 // Everything an epilogue may need.  One struct for all variants keeps the
 // GEMM kernels identical across call sites.
@@ -130,7 +154,28 @@ __device__ __forceinline__ void set_error(int* err, int code) {
     if (err) atomicCAS(err, 0, code);
 }
 
-// ---- launchers implemented in the .cu files (all enqueue on `s`) ----
-struct GemmPlan;  // tcgen05 launch plan, see esp_gemm_tc.cu
+// Programmatic dependent launch.  A kernel launched with the attribute may start while its predecessor in
+// the stream still runs; pdl_wait() returns once the predecessor has completed and its writes are visible.
+// Rule used throughout: before pdl_wait() a kernel touches only immutable inputs (weights) and its own
+// shared/tensor memory.  Both calls are no-ops for a plain launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Launch with or without the programmatic-dependent-launch attribute.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
+                            Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
 
 }  // namespace esp

@@ -11,13 +11,22 @@
 // The step is bound by streaming the weights once from HBM, so the work is
 // cut stream-K style: the (tile, k-block) units of one GEMM are dealt out in
 // equal contiguous ranges to one persistent CTA per SM.  A tile whose k-range
-// is split over several CTAs is finished by whichever of them arrives last:
-// every CTA stores its partial tile, bumps the tile's counter, and the last
-// one sums the partials in CTA order (a fixed order, independent of arrival
-// order and of the number of rows) and runs the fused epilogue.  No CTA ever
-// waits for another.  Every mbarrier wait is bounded; on a timeout the
-// kernel records DEV_E_WAIT_TIMEOUT, lets its copies drain, frees its tensor
-// memory and returns.
+// is split over several CTAs is summed from fp32 partials in CTA order (a
+// fixed order, independent of arrival order and of the number of rows):
+//   * EPI_PARTIAL (QKV, O, down: every tile is split): the kernel only stores
+//     partials; the kernel that consumes the result (RoPE/cache write,
+//     residual add + RMSNorm) sums them, fully parallel and off this kernel's
+//     critical path;
+//   * fused epilogues (gate/up with SiLU*up, LM head with Top-K'): whichever
+//     contributor of a split tile arrives last sums and finishes it.  Each CTA
+//     does its split pieces first and its whole tiles after, so this happens
+//     while the weight stream of the whole tiles is running.
+// No CTA ever waits for another.  The kernel is launched with programmatic
+// dependent launch: the weight tiles of the first ring stages are requested
+// before waiting for the preceding kernel, the activation tiles after.
+// Every mbarrier wait is bounded; on a timeout the kernel records
+// DEV_E_WAIT_TIMEOUT, lets its copies drain, frees its tensor memory and
+// returns.
 #include <cuda.h>
 #include <new>
 #include <string.h>
@@ -111,21 +120,52 @@ __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t da, uint64_t db, 
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[16];
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// stream-K bookkeeping (all 64-bit so lm-head sized problems do not overflow)
-__device__ __forceinline__ long long unit_begin(long long c, long long U, long long G) { return c * U / G; }
-__device__ __forceinline__ int cta_of_unit(long long u, long long U, long long G) { return (int)(((u + 1) * G + U - 1) / U - 1); }
+// One (tile, k-range) piece of a CTA's stream-K range.
+struct Seg {
+    int tile, kb0, kb1, slot;
+    bool whole;
+};
+
+// A CTA's unit range [u0, u1) cut at tile boundaries.  Segments are handed out with the partial ones first
+// (tail piece, then head piece), whole tiles after them: partial tiles are then complete early in every
+// CTA's timeline and the CTA that finishes one does so while the weight stream of its whole tiles is running.
+struct Range {
+    int first_tile, last_tile, head_kb0, tail_kb1, KB, n_seg;
+    bool tail_partial;
+};
+__device__ __forceinline__ Range make_range(long long u0, long long u1, int KB) {
+    Range r;
+    r.KB = KB;
+    r.first_tile = (int)(u0 / KB);
+    r.head_kb0 = (int)(u0 % KB);
+    r.last_tile = (int)((u1 - 1) / KB);
+    r.tail_kb1 = (int)((u1 - 1) % KB) + 1;
+    r.n_seg = r.last_tile - r.first_tile + 1;
+    r.tail_partial = r.n_seg > 1 && r.tail_kb1 < KB;
+    return r;
+}
+__device__ __forceinline__ Seg get_seg(const Range& r, int i) {
+    Seg s;
+    if (r.n_seg == 1) {
+        s.tile = r.first_tile; s.kb0 = r.head_kb0; s.kb1 = r.tail_kb1; s.slot = 0;
+    } else {
+        // order: [tail if partial] head, middle tiles, [tail if whole]
+        int idx = r.tail_partial ? i - 1 : i;
+        if (idx < 0 || idx == r.n_seg - 1) { s.tile = r.last_tile; s.kb0 = 0; s.kb1 = r.tail_kb1; s.slot = 1; }
+        else if (idx == 0) { s.tile = r.first_tile; s.kb0 = r.head_kb0; s.kb1 = r.KB; s.slot = 0; }
+        else { s.tile = r.first_tile + idx; s.kb0 = 0; s.kb1 = r.KB; s.slot = 1; }
+    }
+    s.whole = s.kb0 == 0 && s.kb1 == r.KB;
+    return s;
+}
 
 // which weight matrix / row the two 64-row halves of a tile come from
 template <int EPI>
@@ -154,9 +194,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long U = (long long)p.n_tiles * p.KB, G = p.grid;
-    const long long u0 = unit_begin(blockIdx.x, U, G), u1 = unit_begin(blockIdx.x + 1, U, G);
+    const long long u0 = sk_begin(blockIdx.x, U, G), u1 = sk_begin(blockIdx.x + 1, U, G);
+    const Range rng = make_range(u0, u1, p.KB);
 
     if (threadIdx.x == 0) {
+        pdl_launch_dependents();
         for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], 128); }
         *s_abort = 0;
@@ -176,126 +218,156 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
-            int stage = 0;
+            // The weights do not depend on the kernel before this one: fill the ring with weight tiles first,
+            // wait for that kernel, then add the activation tiles.
+            const int n_items = (int)(u1 - u0);
+            const int n_pre = n_items < STAGES ? n_items : STAGES;
+            for (int pass = 0; pass < 2; ++pass) {
+                int it = 0;
+                for (int i = 0; i < rng.n_seg && it < n_pre; ++i) {
+                    const Seg sg = get_seg(rng, i);
+                    int m0, r0, m1, r1;
+                    tile_source<EPI>(p, sg.tile, 0, m0, r0);
+                    tile_source<EPI>(p, sg.tile, 1, m1, r1);
+                    for (int kb = sg.kb0; kb < sg.kb1 && it < n_pre; ++kb, ++it) {
+                        unsigned char* sa = stages + it * STAGE_BYTES;
+                        if (pass == 0) {
+                            mbar_expect_tx(&full[it], STAGE_BYTES);
+                            tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[it]);
+                            tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it]);
+                        } else {
+                            tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[it]);
+                        }
+                    }
+                }
+                if (pass == 0) pdl_wait();
+            }
+            int stage = 0, it = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (long long u = u0; u < u1 && ok;) {
-                const int tile = (int)(u / p.KB), kb0 = (int)(u % p.KB);
-                const int kb1 = (int)min((long long)p.KB, kb0 + (u1 - u));
+            for (int i = 0; i < rng.n_seg && ok; ++i) {
+                const Seg sg = get_seg(rng, i);
                 int m0, r0, m1, r1;
-                tile_source<EPI>(p, tile, 0, m0, r0);
-                tile_source<EPI>(p, tile, 1, m1, r1);
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!mbar_wait(&empty[stage], phase ^ 1, s_abort)) { ok = false; break; }
-                    unsigned char* sa = stages + stage * STAGE_BYTES;
-                    mbar_expect_tx(&full[stage], STAGE_BYTES);
-                    tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[stage]);
-                    tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage]);
-                    tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[stage]);
+                tile_source<EPI>(p, sg.tile, 0, m0, r0);
+                tile_source<EPI>(p, sg.tile, 1, m1, r1);
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
+                    if (it >= n_pre) {
+                        if (!mbar_wait(&empty[stage], phase ^ 1, s_abort)) { ok = false; break; }
+                        unsigned char* sa = stages + stage * STAGE_BYTES;
+                        mbar_expect_tx(&full[stage], STAGE_BYTES);
+                        tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[stage]);
+                        tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage]);
+                        tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[stage]);
+                    }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                u += kb1 - kb0;
             }
             if (!ok) { set_error(p.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
-            int stage = 0, seg = 0;
+            int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (long long u = u0; u < u1 && ok; ++seg) {
-                const int kb0 = (int)(u % p.KB);
-                const int kb1 = (int)min((long long)p.KB, kb0 + (u1 - u));
-                const int buf = seg & 1;
-                if (!mbar_wait(&tempty[buf], ((seg >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+            for (int i = 0; i < rng.n_seg && ok; ++i) {
+                const Seg sg = get_seg(rng, i);
+                const int buf = i & 1;
+                if (!mbar_wait(&tempty[buf], ((i >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * 128;
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
                     if (!mbar_wait(&full[stage], phase, s_abort)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t sa = smem_u32(stages + stage * STAGE_BYTES);
                     const uint64_t da = smem_desc(sa), db = smem_desc(sa + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)
-                        umma(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), (kb > kb0 || k > 0) ? 1u : 0u);
+                        umma(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), (kb > sg.kb0 || k > 0) ? 1u : 0u);
                     umma_commit(&empty[stage]);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
                 umma_commit(&tfull[buf]);
-                u += kb1 - kb0;
             }
             if (!ok) { set_error(p.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
         }
     } else {
-        // ---------------- epilogue warps: TMEM -> registers -> partial or fused epilogue
+        // ---------------- epilogue warps: TMEM -> registers -> partial and/or fused epilogue
+        pdl_wait();
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         const int f = q * 32 + lane;            // feature of the tile owned by this thread
         const int et = threadIdx.x - 64;        // 0..127 index among the epilogue threads
         const int n_rows = p.a.st ? (p.a.st->active ? p.a.st->n_rows : 0) : p.a.rows_fixed;
-        int seg = 0;
+        StreamK sk;
+        sk.partials = p.partials; sk.n_tiles = p.n_tiles; sk.KB = p.KB; sk.G = p.grid;
         bool ok = true;
-        for (long long u = u0; u < u1 && ok; ++seg) {
-            const int tile = (int)(u / p.KB), kb0 = (int)(u % p.KB);
-            const int kb1 = (int)min((long long)p.KB, kb0 + (u1 - u));
-            const int buf = seg & 1;
+        for (int i = 0; i < rng.n_seg && ok; ++i) {
+            const Seg sg = get_seg(rng, i);
+            const int buf = i & 1;
             bool mine = true;
-            if (lane == 0) mine = mbar_wait(&tfull[buf], (seg >> 1) & 1, s_abort);
+            if (lane == 0) mine = mbar_wait(&tfull[buf], (i >> 1) & 1, s_abort);
             if (lane == 0 && !mine) atomicOr(&s_flag[0], 1);
             epi_bar(2);
             if (s_flag[0]) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = tmem_base + buf * 128 + ((uint32_t)(q * 32) << 16);
-            const long long t_first = (long long)tile * p.KB;
-            const int c_first = cta_of_unit(t_first, U, G), c_last = cta_of_unit(t_first + p.KB - 1, U, G);
-            const bool whole = c_first == c_last;
-            const int slot = (tile == (int)(u0 / p.KB)) ? 0 : 1;
-            float* part = p.partials + ((size_t)(blockIdx.x * 2 + slot) * RT) * TILE_N;
+            uint32_t v[RT];
 #pragma unroll
-            for (int c = 0; c < RT / 16; ++c) {
-                float v[16];
-                tmem_ld16(taddr + c * 16, v);
-                if (whole) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) s_acc[(c * 16 + i) * ACC_LD + f] = v[i];
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (c * 16 + i < n_rows) __stcg(&part[(c * 16 + i) * TILE_N + f], v[i]);
-                }
-            }
+            for (int c = 0; c < RT / 16; ++c) tmem_ld16_issue(taddr + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            // the accumulator is in registers: hand the tensor-memory buffer back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(&tempty[buf]);
-            bool finish = whole;
-            if (!whole) {
+            const bool direct = EPI != EPI_PARTIAL && sg.whole;
+            if (direct) {
+#pragma unroll
+                for (int r = 0; r < RT; ++r) s_acc[r * ACC_LD + f] = __uint_as_float(v[r]);
+            } else {
+                float* part = p.partials + ((size_t)(blockIdx.x * 2 + sg.slot) * RT) * TILE_N + f;
+#pragma unroll
+                for (int r = 0; r < RT; ++r)
+                    if (r < n_rows) __stcg(part + r * TILE_N, __uint_as_float(v[r]));
+            }
+            if (EPI == EPI_PARTIAL) continue;   // the consumer kernel sums the partials
+            bool finish = direct;
+            if (!direct) {
+                int c_first, c_last;
+                sk_contributors(sk, sg.tile, c_first, c_last);
                 __threadfence();
                 epi_bar(2);
                 if (et == 0) {
-                    const int old = atomicAdd(&p.counters[tile], 1);
+                    const int old = atomicAdd(&p.counters[sg.tile], 1);
                     s_flag[1] = (old == c_last - c_first) ? 1 : 0;
                 }
                 epi_bar(2);
                 finish = s_flag[1] != 0;
                 if (finish) {
+                    // last contributor of this tile: sum the partials in CTA order (fixed, whoever arrives last)
                     __threadfence();
-                    for (int r = 0; r < n_rows; ++r) {
-                        float acc = 0.f;
+                    for (int r0 = 0; r0 < n_rows; r0 += 8) {
+                        float acc[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
                         for (int c = c_first; c <= c_last; ++c) {
-                            const int cslot = (tile == (int)(unit_begin(c, U, G) / p.KB)) ? 0 : 1;
-                            acc += __ldcg(&p.partials[((size_t)(c * 2 + cslot) * RT + r) * TILE_N + f]);
+                            const float* src = p.partials + ((size_t)(c * 2 + sk_slot(sk, c, sg.tile)) * RT + r0) * TILE_N + f;
+                            float t[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) t[j] = r0 + j < n_rows ? __ldcg(src + j * TILE_N) : 0.f;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) acc[j] += t[j];
                         }
-                        s_acc[r * ACC_LD + f] = acc;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) s_acc[(r0 + j) * ACC_LD + f] = acc[j];
                     }
-                    if (et == 0) p.counters[tile] = 0;
+                    if (et == 0) p.counters[sg.tile] = 0;
                 }
             }
             if (finish) {
                 epi_bar(2);
-                run_epilogue<__nv_bfloat16, EPI>(s_acc, s_aux, tile, 0, p.a, f, 2);
+                run_epilogue<__nv_bfloat16, EPI>(s_acc, s_aux, sg.tile, 0, p.a, f, 2);
             }
             epi_bar(2);
-            u += kb1 - kb0;
         }
         if (!ok && lane == 0) { set_error(p.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
     }
@@ -377,6 +449,8 @@ int tc_gemm_create(TcGemm** out, int epi, const void* const w[3], const int32_t 
     const long long U = (long long)p.n_tiles * p.KB;
     p.grid = (int)(U < n_sm ? U : n_sm);
     if (p.n_tiles > tc_gemm_counter_ints() || tc_gemm_partial_bytes(p.grid) > partial_bytes) { delete g; return -1; }
+    // partial-only output keeps two slots per CTA: a CTA's range must not span more than two tiles
+    if (epi == EPI_PARTIAL && p.n_tiles > p.grid) { delete g; return -1; }
     p.partials = reinterpret_cast<float*>(partials);
     p.counters = counters;
     p.err = err;
@@ -386,10 +460,20 @@ int tc_gemm_create(TcGemm** out, int epi, const void* const w[3], const int32_t 
 
 void tc_gemm_destroy(TcGemm* g) { delete g; }
 
-int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s) {
+StreamK tc_gemm_streamk(const TcGemm* g) {
+    StreamK k;
+    k.partials = g ? g->p.partials : nullptr;
+    k.n_tiles = g ? g->p.n_tiles : 0;
+    k.KB = g ? g->p.KB : 1;
+    k.G = g ? g->p.grid : 1;
+    return k;
+}
+
+int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl) {
     if (!g) return ESP_E_ARG;
     TcParams p = g->p;
     p.a = a;
+    cudaError_t e = cudaSuccess;
 #define ESP_TC_CASE(E)                                                                                        \
     case E: {                                                                                                 \
         static bool attr_set = false;                                                                         \
@@ -397,18 +481,17 @@ int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s) {
             if (cudaFuncSetAttribute(k_gemm_tc<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return ESP_E_CUDA; \
             attr_set = true;                                                                                  \
         }                                                                                                     \
-        k_gemm_tc<E><<<p.grid, NUM_THREADS, SMEM_BYTES, s>>>(p);                                              \
+        e = launch_k(k_gemm_tc<E>, dim3(p.grid), dim3(NUM_THREADS), SMEM_BYTES, s, pdl, p);                    \
     } break;
     switch (p.epi) {
         ESP_TC_CASE(EPI_STORE_F32)
-        ESP_TC_CASE(EPI_QKV)
-        ESP_TC_CASE(EPI_RESID)
         ESP_TC_CASE(EPI_SWIGLU)
         ESP_TC_CASE(EPI_LOGITS)
+        ESP_TC_CASE(EPI_PARTIAL)
         default: return ESP_E_ARG;
     }
 #undef ESP_TC_CASE
-    return cudaGetLastError() == cudaSuccess ? ESP_OK : ESP_E_CUDA;
+    return e == cudaSuccess ? ESP_OK : ESP_E_CUDA;
 }
 
 }  // namespace esp

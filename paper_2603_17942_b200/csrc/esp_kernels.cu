@@ -32,6 +32,8 @@ __global__ void k_mask_mean(const T* embed, const int32_t* prompt, int t, int d,
 // Input rows of the block: E[token] for tree nodes, the shared mask vector for probe rows.
 template <typename T>
 __global__ void k_assemble(const SeqState* states, const T* embed, const float* mvec, float* hres, int d) {
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
     int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
     if (!st->active || r >= st->n_rows) return;
@@ -47,6 +49,8 @@ __global__ void k_assemble(const SeqState* states, const T* embed, const float* 
 template <typename T>
 __global__ void __launch_bounds__(256) k_rmsnorm(const SeqState* states, const float* x, const T* g, T* y, int d, float eps,
                                                 float* copy_out) {
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
     int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
     if (!st->active || r >= st->n_rows) return;
@@ -65,6 +69,123 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const SeqState* states, const f
     for (int j = threadIdx.x; j < d; j += 256) yr[j] = from_f32<T>(xr[j] * rinv * to_f32(g[j]));
     if (copy_out)
         for (int j = threadIdx.x; j < d; j += 256) copy_out[(size_t)(seq * RT + r) * d + j] = xr[j];
+}
+
+// Consumer of a split GEMM (O or down projection) fused with the residual add and the next RMSNorm:
+//   hres[r] += sum over the tile's contributors, in CTA order, of their fp32 partials;  y = rmsnorm(hres[r]) * g.
+// One block per row; with sk.partials == NULL it is a plain RMSNorm of hres.  The sum order depends only on
+// the GEMM's shape, never on the number of rows in the block.
+template <typename T>
+__global__ void __launch_bounds__(512) k_resid_norm(const SeqState* states, float* hres, StreamK sk, const T* g, T* y, int d,
+                                                   float eps, float* copy_out) {
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
+    const int seq = blockIdx.y, r = blockIdx.x;
+    const SeqState* st = states + seq;
+    if (!st->active || r >= st->n_rows) return;
+    float* xr = hres + (size_t)(seq * RT + r) * d;
+    __shared__ float red[16];
+    float ss = 0.f;
+    for (int j = threadIdx.x * 4; j < d; j += 512 * 4) {
+        float4 x = *reinterpret_cast<const float4*>(xr + j);
+        if (sk.partials) {
+            const int tile = j / TILE_N, f = j % TILE_N;
+            int c_first, c_last;
+            sk_contributors(sk, tile, c_first, c_last);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c = c_first; c <= c_last; ++c) {
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(
+                    sk.partials + ((size_t)(c * 2 + sk_slot(sk, c, tile)) * RT + r) * TILE_N + f));
+                acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+            }
+            x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
+            *reinterpret_cast<float4*>(xr + j) = x;
+        }
+        ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 16; ++w) tot += red[w];
+    const float rinv = 1.0f / sqrtf(tot / (float)d + eps);
+    T* yr = y + (size_t)(seq * RT + r) * d;
+    for (int j = threadIdx.x * 4; j < d; j += 512 * 4) {
+        const float4 x = *reinterpret_cast<const float4*>(xr + j);   // this thread's own writes
+        const float xv[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) yr[j + i] = from_f32<T>(xv[i] * rinv * to_f32(g[j + i]));
+        if (copy_out) *reinterpret_cast<float4*>(copy_out + (size_t)(seq * RT + r) * d + j) = x;
+    }
+}
+
+// Consumer of the split QKV GEMM: sums the partials of one (row, head) in CTA order, then what follows
+// the projection in the decoder layer -- per-head RMSNorm on q and k (Qwen3), rotary embedding at the
+// row's position L + depth, q to the query buffer, k and v to cache slot L + row.  One warp per (row, head),
+// a lane owns HD/32 consecutive features; the rotate-half partner (i, i + HD/2) sits 16 lanes away.
+template <int HD>
+__global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
+    typedef __nv_bfloat16 T;
+    constexpr int NE = HD / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int hs = blockIdx.x * 4 + warp, r = blockIdx.y;
+    const SeqState* st = a.st;
+    const int n_rows = st ? (st->active ? st->n_rows : 0) : a.rows_fixed;
+    if (r >= n_rows || hs >= a.Hq + 2 * a.Hkv) return;
+    const int j0 = hs * HD + lane * NE;          // feature in the concatenated [q | k | v] space
+    const int tile = j0 / TILE_N, f = j0 % TILE_N;
+    int c_first, c_last;
+    sk_contributors(sk, tile, c_first, c_last);
+    float v[NE];
+#pragma unroll
+    for (int i = 0; i < NE; ++i) v[i] = 0.f;
+    for (int c = c_first; c <= c_last; ++c) {
+        const float* src = sk.partials + ((size_t)(c * 2 + sk_slot(sk, c, tile)) * RT + r) * TILE_N + f;
+        if constexpr (NE == 4) {
+            const float4 t = __ldcg(reinterpret_cast<const float4*>(src));
+            v[0] += t.x; v[1] += t.y; v[2] += t.z; v[3] += t.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < NE; ++i) v[i] += __ldcg(src + i);
+        }
+    }
+    const int which = hs < a.Hq ? 0 : (hs < a.Hq + a.Hkv ? 1 : 2);
+    const int head = which == 0 ? hs : (which == 1 ? hs - a.Hq : hs - a.Hq - a.Hkv);
+    const int L = st ? st->L : 0;
+    if (which != 2) {
+        if (a.qk_norm) {
+            float ss = 0.f;
+#pragma unroll
+            for (int i = 0; i < NE; ++i) ss += v[i] * v[i];
+            ss = warp_sum(ss);
+            const float rinv = 1.0f / sqrtf(ss / (float)HD + a.rms_eps);
+            const T* g = reinterpret_cast<const T*>(which == 0 ? a.q_norm : a.k_norm);
+#pragma unroll
+            for (int i = 0; i < NE; ++i) v[i] = v[i] * rinv * to_f32(g[lane * NE + i]);
+        }
+        constexpr int half = HD / 2;
+        const int pos = L + (st ? st->row_depth[r] : r);
+        const bool low = lane < 16;
+#pragma unroll
+        for (int i = 0; i < NE; ++i) {
+            const float other = __shfl_xor_sync(0xffffffffu, v[i], 16);
+            const int idx = (lane * NE + i) % half;
+            const float cs = a.rope_cos[(size_t)pos * half + idx], sn = a.rope_sin[(size_t)pos * half + idx];
+            v[i] = low ? v[i] * cs - other * sn : v[i] * cs + other * sn;
+        }
+    }
+    T* dst;
+    if (which == 0) dst = reinterpret_cast<T*>(a.q_out) + (size_t)r * a.Hq * HD + head * HD + lane * NE;
+    else dst = reinterpret_cast<T*>(which == 1 ? a.kcache : a.vcache) + ((size_t)head * a.cap + (L + r)) * HD + lane * NE;
+    T o[NE];
+#pragma unroll
+    for (int i = 0; i < NE; ++i) o[i] = from_f32<T>(v[i]);
+    if constexpr (NE == 4) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(o);
+    else if constexpr (NE == 2) *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(o);
+    else dst[0] = o[0];
 }
 
 // ------------------------------------------------------------------ CUDA-core GEMM
@@ -86,6 +207,7 @@ __global__ void __launch_bounds__(128) k_gemm_simt(SimtGemmArgs g, EpiArgs a) {
     float* s_aux = s_acc + RT * ACC_LD;        // RT * 4
     float* s_x = s_aux + RT * 4;               // RT * 32
     float* s_w = s_x + RT * 32;                // 128 * 33
+    pdl_wait();
     const int tile = blockIdx.x, seq = blockIdx.y, f = threadIdx.x;
     if (a.st && !a.st[seq].active) return;
     const int n_rows = a.st ? a.st[seq].n_rows : a.rows_fixed;
@@ -133,13 +255,13 @@ __global__ void __launch_bounds__(128) k_gemm_simt(SimtGemmArgs g, EpiArgs a) {
 }
 
 template <typename T>
-void launch_gemm_simt_t(int epi, int n_tiles, int batch, const SimtGemmArgs& g, const EpiArgs& a, cudaStream_t s) {
+void launch_gemm_simt_t(int epi, int n_tiles, int batch, const SimtGemmArgs& g, const EpiArgs& a, cudaStream_t s, bool pdl) {
     size_t smem = sizeof(float) * (RT * ACC_LD + RT * 4 + RT * 32 + 128 * 33);
     dim3 grid(n_tiles, batch);
 #define ESP_SIMT_CASE(E)                                                                                  \
     case E:                                                                                               \
         cudaFuncSetAttribute(k_gemm_simt<T, E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-        k_gemm_simt<T, E><<<grid, 128, smem, s>>>(g, a);                                                  \
+        launch_k(k_gemm_simt<T, E>, grid, dim3(128), smem, s, pdl, g, a);                                 \
         break;
     switch (epi) {
         ESP_SIMT_CASE(EPI_STORE_F32)
@@ -152,13 +274,13 @@ void launch_gemm_simt_t(int epi, int n_tiles, int batch, const SimtGemmArgs& g, 
 }
 
 void launch_gemm_simt(int dtype, int epi, int n_tiles, int batch, const void* const w[3], const int32_t rows_w[3],
-                      const void* x, int K, const EpiArgs& a, cudaStream_t s) {
+                      const void* x, int K, const EpiArgs& a, cudaStream_t s, bool pdl) {
     SimtGemmArgs g;
     for (int i = 0; i < 3; ++i) { g.w[i] = w[i]; g.rows_w[i] = rows_w[i]; }
     g.x = x;
     g.K = K;
-    if (dtype == 0) launch_gemm_simt_t<float>(epi, n_tiles, batch, g, a, s);
-    else launch_gemm_simt_t<__nv_bfloat16>(epi, n_tiles, batch, g, a, s);
+    if (dtype == 0) launch_gemm_simt_t<float>(epi, n_tiles, batch, g, a, s, pdl);
+    else launch_gemm_simt_t<__nv_bfloat16>(epi, n_tiles, batch, g, a, s, pdl);
 }
 
 // ------------------------------------------------------------------ attention (position-canonical)
@@ -246,6 +368,7 @@ __device__ __forceinline__ void merge_partial(float& m, float& l, float (&o)[N],
 template <typename T, int HD>
 __global__ void __launch_bounds__(128) k_attn_bulk_simt(AttnArgs a, int n_split_launch) {
     __shared__ float s_qall[4][HD];
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * 4 + warp, head = blockIdx.y;
     const int split = blockIdx.z % n_split_launch, seq = blockIdx.z / n_split_launch;
@@ -282,6 +405,8 @@ __global__ void __launch_bounds__(128) k_attn_bulk_simt(AttnArgs a, int n_split_
 template <typename T, int HD>
 __global__ void __launch_bounds__(128) k_attn_tail_merge(AttnArgs a) {
     __shared__ float s_qall[4][HD];
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * 4 + warp, head = blockIdx.y, seq = blockIdx.z;
     int n_rows, L, depth;
@@ -336,15 +461,15 @@ __global__ void __launch_bounds__(128) k_attn_tail_merge(AttnArgs a) {
 }
 
 template <typename T, int HD>
-static void launch_attn_simt_t(const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s) {
+static void launch_attn_simt_t(const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s, bool pdl) {
     dim3 g1((RT + 3) / 4, a.Hq, n_split_launch * batch);
-    if (bulk_too && n_split_launch > 0) k_attn_bulk_simt<T, HD><<<g1, 128, 0, s>>>(a, n_split_launch);
+    if (bulk_too && n_split_launch > 0) launch_k(k_attn_bulk_simt<T, HD>, g1, dim3(128), 0, s, pdl, a, n_split_launch);
     dim3 g2((RT + 3) / 4, a.Hq, batch);
-    k_attn_tail_merge<T, HD><<<g2, 128, 0, s>>>(a);
+    launch_k(k_attn_tail_merge<T, HD>, g2, dim3(128), 0, s, pdl, a);
 }
 
-int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s) {
-#define ESP_ATTN_CASE(TT, H) launch_attn_simt_t<TT, H>(a, batch, n_split_launch, bulk_too, s); return 0;
+int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s, bool pdl) {
+#define ESP_ATTN_CASE(TT, H) launch_attn_simt_t<TT, H>(a, batch, n_split_launch, bulk_too, s, pdl); return 0;
     if (dtype == 0) {
         if (a.h == 32) { ESP_ATTN_CASE(float, 32) }
         if (a.h == 64) { ESP_ATTN_CASE(float, 64) }
@@ -363,6 +488,7 @@ int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch
 // lse = max + log(sum exp) merged over tiles in a fixed order.
 __global__ void __launch_bounds__(128) k_topk_merge(const SeqState* states, const Cand* cand, const float2* cand_ms,
                                                     int n_tiles, int KP, int batch, Cand* topk, float* lse) {
+    pdl_wait();
     const int seq = blockIdx.y, r = blockIdx.x, tid = threadIdx.x;
     const SeqState* st = states + seq;
     if (!st->active || r >= st->n_rows) return;
@@ -437,9 +563,9 @@ __global__ void __launch_bounds__(128) k_topk_merge(const SeqState* states, cons
 }
 
 void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
-                       Cand* topk, float* lse, cudaStream_t s) {
+                       Cand* topk, float* lse, cudaStream_t s, bool pdl) {
     dim3 grid(RT, batch);
-    k_topk_merge<<<grid, 128, 0, s>>>(st, cand, cand_ms, n_tiles, KP, batch, topk, lse);
+    launch_k(k_topk_merge, grid, dim3(128), 0, s, pdl, st, cand, cand_ms, n_tiles, KP, batch, topk, lse);
 }
 
 // ------------------------------------------------------------------ row-table builders
@@ -534,6 +660,7 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     __shared__ int s_na, s_ustar, s_delta, s_nexp, s_ncreated, s_abort;
     __shared__ int s_exp[RT], s_sel[RT], s_new[RT];
 
+    pdl_wait();
     const Dims& D = A.D;
     const int seq = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     SeqState* st = A.states + seq;
@@ -760,14 +887,14 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     }
 }
 
-void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s) {
+void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s, bool pdl) {
     size_t smem = (size_t)MAX_CAND * 20;
     if (dtype == 0) {
         cudaFuncSetAttribute(k_tree_step<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        k_tree_step<float><<<A.D.batch, 1024, smem, s>>>(A);
+        launch_k(k_tree_step<float>, dim3(A.D.batch), dim3(1024), smem, s, pdl, A);
     } else {
         cudaFuncSetAttribute(k_tree_step<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        k_tree_step<__nv_bfloat16><<<A.D.batch, 1024, smem, s>>>(A);
+        launch_k(k_tree_step<__nv_bfloat16>, dim3(A.D.batch), dim3(1024), smem, s, pdl, A);
     }
 }
 
@@ -781,16 +908,30 @@ void launch_mask_mean(int dtype, const void* embed, const int32_t* prompt, int t
     else k_mask_mean<__nv_bfloat16><<<(d + 127) / 128, 128, 0, s>>>((const __nv_bfloat16*)embed, prompt, t, d, m);
 }
 void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int batch,
-                     cudaStream_t s) {
+                     cudaStream_t s, bool pdl) {
     dim3 grid(RT, batch);
-    if (dtype == 0) k_assemble<float><<<grid, 128, 0, s>>>(st, (const float*)embed, mvec, hres, d);
-    else k_assemble<__nv_bfloat16><<<grid, 128, 0, s>>>(st, (const __nv_bfloat16*)embed, mvec, hres, d);
+    if (dtype == 0) launch_k(k_assemble<float>, grid, dim3(128), 0, s, pdl, st, (const float*)embed, mvec, hres, d);
+    else launch_k(k_assemble<__nv_bfloat16>, grid, dim3(128), 0, s, pdl, st, (const __nv_bfloat16*)embed, mvec, hres, d);
 }
 void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
-                    float* copy_out, cudaStream_t s) {
+                    float* copy_out, cudaStream_t s, bool pdl) {
     dim3 grid(RT, batch);
-    if (dtype == 0) k_rmsnorm<float><<<grid, 256, 0, s>>>(st, x, (const float*)g, (float*)y, d, eps, copy_out);
-    else k_rmsnorm<__nv_bfloat16><<<grid, 256, 0, s>>>(st, x, (const __nv_bfloat16*)g, (__nv_bfloat16*)y, d, eps, copy_out);
+    if (dtype == 0) launch_k(k_rmsnorm<float>, grid, dim3(256), 0, s, pdl, st, x, (const float*)g, (float*)y, d, eps, copy_out);
+    else launch_k(k_rmsnorm<__nv_bfloat16>, grid, dim3(256), 0, s, pdl, st, x, (const __nv_bfloat16*)g, (__nv_bfloat16*)y, d, eps, copy_out);
+}
+void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
+                       float* copy_out, cudaStream_t s, bool pdl) {
+    launch_k(k_resid_norm<__nv_bfloat16>, dim3(RT, 1), dim3(512), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
+             (__nv_bfloat16*)y, d, eps, copy_out);
+}
+int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, cudaStream_t s, bool pdl) {
+    const int n_heads = a.Hq + 2 * a.Hkv;
+    dim3 grid((n_heads + 3) / 4, RT);
+    if (a.h == 128) launch_k(k_qkv_finish<128>, grid, dim3(128), 0, s, pdl, a, sk);
+    else if (a.h == 64) launch_k(k_qkv_finish<64>, grid, dim3(128), 0, s, pdl, a, sk);
+    else if (a.h == 32) launch_k(k_qkv_finish<32>, grid, dim3(128), 0, s, pdl, a, sk);
+    else return -1;
+    return 0;
 }
 void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int off, int n, int last, int k, cudaStream_t s) {
     k_setup_chain<<<1, 128, 0, s>>>(st, seq, prompt_dev, off, n, last, k);

@@ -38,32 +38,37 @@ struct TreeArgs {
 void launch_rope_table(float* cs, float* sn, int n_pos, int h, float base, cudaStream_t s);
 void launch_mask_mean(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, cudaStream_t s);
 void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int batch,
-                     cudaStream_t s);
+                     cudaStream_t s, bool pdl);
 void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
-                    float* copy_out, cudaStream_t s);
+                    float* copy_out, cudaStream_t s, bool pdl);
+// consumers of the split (EPI_PARTIAL) tensor-core GEMMs, bf16 models, one sequence
+void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
+                       float* copy_out, cudaStream_t s, bool pdl);
+int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, cudaStream_t s, bool pdl);
 void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int off, int n, int last, int k, cudaStream_t s);
 void launch_set_tree(SeqState* st, int seq, const int32_t* tokens, const int32_t* parents, int n, int k, int n_anchor,
                      int* err, cudaStream_t s);
 void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
-                       Cand* topk, float* lse, cudaStream_t s);
-void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s);
+                       Cand* topk, float* lse, cudaStream_t s, bool pdl);
+void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s, bool pdl);
 
 // CUDA-core GEMM (fp32 models; on-GPU cross-check for bf16)
 void launch_gemm_simt(int dtype, int epi, int n_tiles, int batch, const void* const w[3], const int32_t rows_w[3],
-                      const void* x, int K, const EpiArgs& a, cudaStream_t s);
+                      const void* x, int K, const EpiArgs& a, cudaStream_t s, bool pdl);
 
 // position-canonical attention: CUDA-core bulk (+ tail/merge), or tail/merge only when the
 // tensor-core bulk kernel already produced the split partials
-int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s);
+int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s, bool pdl);
 // tensor-core bulk for bf16, head_dim 128
-int launch_attn_bulk_mma(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s);
+int launch_attn_bulk_mma(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl);
 
 // tcgen05 GEMM: a plan holds the TMA descriptors and the stream-K partition of one weight shape
 struct TcGemm;
 int tc_gemm_create(TcGemm** out, int epi, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
                    int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err);
 void tc_gemm_destroy(TcGemm* g);
-int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s);
+int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl);
+StreamK tc_gemm_streamk(const TcGemm* g);
 int tc_gemm_tiles(const TcGemm* g);
 size_t tc_gemm_partial_bytes(int n_sm);
 int tc_gemm_counter_ints();
