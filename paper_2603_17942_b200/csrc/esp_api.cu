@@ -43,6 +43,7 @@ struct Buffers {
     float *rope_cos, *rope_sin;
     void* gemm_partials;
     int* gemm_counters;
+    int* attn_counters;
 };
 
 
@@ -128,6 +129,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.rope_sin = c.take<float>((size_t)D.cap * (D.h / 2));
     o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm));
     o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
+    o.attn_counters = c.take<int>(attn_tree_counter_ints(D.batch));
     return align_up(c.off, 256);
 }
 
@@ -255,12 +257,13 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
             a.err = b.err;
             const bool mma = h->dtype == 1 && D.h == 128 && h->gemm_impl == 0;
-            if (mma && n_split_launch > 0) {
-                if (launch_attn_bulk_mma(a, D.batch, n_split_launch, s, pdl)) return ESP_E_BADCFG;
+            if (mma) {
+                if (launch_attn_tree(a, D.batch, n_split_launch, b.attn_counters, s, pdl)) return ESP_E_BADCFG;
                 h->launches++;
+            } else {
+                if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, true, s, pdl)) return ESP_E_BADCFG;
+                h->launches += n_split_launch > 0 ? 2 : 1;
             }
-            if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, !mma, s, pdl)) return ESP_E_BADCFG;
-            h->launches += (!mma && n_split_launch > 0) ? 2 : 1;
             mark(h, KIND_ATTN);
         }
         {
@@ -675,7 +678,8 @@ int esp_tree_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t h
     while ((cap + S - 1) / S > 64) S *= 2;
     const size_t ns = (cap + S - 1) / S + 1;
     const size_t rows = (size_t)batch * RT * n_q_heads * ns;
-    *bytes_out = align_up(rows * head_dim * sizeof(float), 256) + align_up(rows * sizeof(float2), 256) + 256;
+    *bytes_out = align_up(rows * head_dim * sizeof(float), 256) + align_up(rows * sizeof(float2), 256) +
+                 align_up(sizeof(int) * attn_tree_counter_ints(batch), 256) + 256;
     return ESP_OK;
 }
 
@@ -710,8 +714,14 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
     const int n_split_launch = (L + S - 1) / S;
     const bool mma = dtype == 1 && head_dim == 128;
-    if (mma && n_split_launch > 0 && launch_attn_bulk_mma(a, batch, n_split_launch, s, false)) return ESP_E_BADCFG;
-    if (launch_attn_simt(dtype, a, batch, n_split_launch, !mma, s, false)) return ESP_E_BADCFG;
+    if (mma) {
+        int* counters = reinterpret_cast<int*>(reinterpret_cast<char*>(scratch) + align_up(rows * head_dim * sizeof(float), 256) +
+                                               align_up(rows * sizeof(float2), 256));
+        if (cudaMemsetAsync(counters, 0, sizeof(int) * attn_tree_counter_ints(batch), s) != cudaSuccess) return ESP_E_CUDA;
+        if (launch_attn_tree(a, batch, n_split_launch, counters, s, false)) return ESP_E_BADCFG;
+    } else if (launch_attn_simt(dtype, a, batch, n_split_launch, true, s, false)) {
+        return ESP_E_BADCFG;
+    }
     return cuda_ok(cudaGetLastError());
 }
 

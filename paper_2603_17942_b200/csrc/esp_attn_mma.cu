@@ -1,13 +1,17 @@
-// Tensor-core "bulk" part of the tree attention for bf16, head_dim 128.
+// Tree attention for bf16, head_dim 128, in one kernel.
 //
-// A row at position P attends to cache positions 0..T0-1 here (T0 as in
-// tail_start(): the 16-aligned position below which keys are always cache
-// resident); the remaining positions, including the row's in-flight tree
-// ancestors, are summed by the tail kernel.  The KV cache of one KV head is
-// streamed once per split through shared memory (16-byte cp.async, XOR
-// swizzle) and shared by all query heads of the group and all block rows:
-// a CTA holds 64 (row, head) pairs, a warp 16 of them, Q.K^T and P.V run on
-// mma.sync m16n8k16 with fp32 online softmax in registers.
+// A row at position P attends to cache positions 0..T0-1 through the "bulk"
+// CTAs (T0 as in tail_start(): the 16-aligned position below which keys are
+// always cache resident): the KV cache of one KV head is streamed once per
+// split through shared memory (16-byte cp.async, XOR swizzle) and shared by
+// all query heads of the group and all block rows: a CTA holds 64 (row, head)
+// pairs, a warp 16 of them, Q.K^T and P.V run on mma.sync m16n8k16 with fp32
+// online softmax in registers.  The remaining positions T0..P -- the end of
+// the cache plus the row's in-flight tree ancestors, found through its
+// ancestor bitmask -- are summed by one more "tail" CTA per group of pairs,
+// key by key in position order.  Every CTA stores (max, sum, weighted values)
+// partials; whichever CTA of a group finishes last merges them in split order
+// (tail last) and writes the output.  No CTA waits for another.
 //
 // Everything that decides a row's arithmetic -- the 64-key chunk grid, the
 // split grid, the per-position mask -- is a function of absolute positions
@@ -23,6 +27,7 @@ constexpr int HD = 128;
 constexpr int CHUNK = 64;
 constexpr int PAIRS = 64;  // (row, head) pairs per CTA
 constexpr int KV_TILE_BYTES = CHUNK * HD * 2;
+constexpr int TAIL_CTAS = 8;   // tail CTAs per group of 64 pairs: 8 pairs each, 2 per warp
 
 __device__ __forceinline__ int tail_start_mma(int P, int dcap) {
     int t = P - dcap;
@@ -54,30 +59,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // byte offset of 16-byte unit `u` (0..15) of key row `key` (0..63) inside a swizzled KV tile
 __device__ __forceinline__ uint32_t kv_off(int key, int u) { return (uint32_t)(key * 256 + ((u ^ (key & 7)) << 4)); }
 
-__global__ void __launch_bounds__(128) k_attn_bulk_mma(AttnArgs a, int n_split_launch, int group, int rows_per_tile, int n_row_tiles) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    pdl_wait();
-    if (threadIdx.x == 0) pdl_launch_dependents();
+// ---- bulk: one split of the cache for the 64 (row, head) pairs of a group
+__device__ __forceinline__ void attn_bulk_chunks(const AttnArgs& a, unsigned char* smem, int seq, int kvh, int row0, int split,
+                                                 int group, int n_rows, int L, int T0max, const __nv_bfloat16* kbase,
+                                                 const __nv_bfloat16* vbase) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int split = blockIdx.x;
-    const int kvh = blockIdx.y / n_row_tiles, rtile = blockIdx.y % n_row_tiles;
-    const int seq = blockIdx.z;
-
-    int n_rows, L;
-    if (a.st) {
-        const SeqState* st = a.st + seq;
-        n_rows = st->active ? st->n_rows : 0;
-        L = st->L;
-    } else {
-        n_rows = a.n_rows_fixed;
-        L = a.L_fixed;
-    }
-    const int row0 = rtile * rows_per_tile;
-    if (row0 >= n_rows) return;
     // per-thread pairs: A = warp*16 + lane/4, B = A + 8
     int pr[2], ph[2], pT0[2];
     bool pv[2];
-    int T0max = 0;
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int pidx = warp * 16 + (lane >> 2) + i * 8;
@@ -88,17 +77,8 @@ __global__ void __launch_bounds__(128) k_attn_bulk_mma(AttnArgs a, int n_split_l
         if (pv[i]) depth = a.st ? a.st[seq].row_depth[pr[i]] : a.depth[seq * RT + pr[i]];
         pT0[i] = pv[i] ? tail_start_mma(L + depth, a.dcap) : 0;
     }
-    // the CTA needs keys up to the largest T0 of its rows (block-uniform: computed from all rows of the tile)
-    for (int r = row0; r < min(row0 + rows_per_tile, n_rows); ++r) {
-        const int depth = a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r];
-        T0max = max(T0max, tail_start_mma(L + depth, a.dcap));
-    }
     const int beg = split * a.split_len;
     const int end = min(beg + a.split_len, T0max);
-    if (beg >= end) return;
-
-    const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.kc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
-    const __nv_bfloat16* vbase = reinterpret_cast<const __nv_bfloat16*>(a.vc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
     const uint32_t s_base = smem_u32(smem);
 
     auto load_chunk = [&](int c, int stage) {
@@ -250,22 +230,238 @@ __global__ void __launch_bounds__(128) k_attn_bulk_mma(AttnArgs a, int n_split_l
     }
 }
 
+
+// ---- tail: positions T0..P of one (row, head) pair, one warp, lane j owns key j of a 32-key chunk
+__device__ __forceinline__ int nth_set_bit128(unsigned long long lo, unsigned long long hi, int n) {
+    int c = __popcll(lo);
+    unsigned long long m = lo;
+    int base = 0;
+    if (n >= c) { n -= c; m = hi; base = 64; }
+    for (int i = 0; i < n; ++i) m &= m - 1;
+    return m ? base + __ffsll((long long)m) - 1 : -1;
+}
+
+__device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], float cm, float cl, const float (&co)[4]) {
+    const float mn = fmaxf(m, cm);
+    const float a = exp2f(m - mn), b = exp2f(cm - mn);
+    l = l * a + cl * b;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) o[i] = o[i] * a + co[i] * b;
+    m = mn;
+}
+
+__global__ void __launch_bounds__(128) k_attn_tree(AttnArgs a, int n_split_launch, int group, int rows_per_tile, int n_row_tiles,
+                                                  int* counters) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ int s_T0max, s_last;
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int split = blockIdx.x;                    // >= n_split_launch: the tail CTAs of the group
+    const int kvh = blockIdx.y / n_row_tiles, rtile = blockIdx.y % n_row_tiles;
+    const int seq = blockIdx.z;
+
+    int n_rows, L;
+    if (a.st) {
+        const SeqState* st = a.st + seq;
+        n_rows = st->active ? st->n_rows : 0;
+        L = st->L;
+    } else {
+        n_rows = a.n_rows_fixed;
+        L = a.L_fixed;
+    }
+    const int row0 = rtile * rows_per_tile;
+    if (row0 >= n_rows) return;
+    // the group needs keys up to the largest T0 of its rows (one round trip: a lane per row, then a warp max)
+    if (warp == 0) {
+        int t0 = 0;
+        for (int r = row0 + lane; r < row0 + rows_per_tile && r < n_rows; r += 32) {
+            const int depth = a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r];
+            t0 = max(t0, tail_start_mma(L + depth, a.dcap));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t0 = max(t0, __shfl_xor_sync(0xffffffffu, t0, o));
+        if (lane == 0) s_T0max = t0;
+    }
+    __syncthreads();
+    const int T0max = s_T0max;
+    const int n_bulk = (T0max + a.split_len - 1) / a.split_len;     // bulk CTAs of this group that have keys
+    const bool is_tail = split >= n_split_launch;
+    if (!is_tail && split >= n_bulk) return;
+
+    const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.kc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
+    const __nv_bfloat16* vbase = reinterpret_cast<const __nv_bfloat16*>(a.vc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
+
+    if (is_tail) {
+        // ---------------- tail CTA t of the group: warp w takes pairs t*8 + w*2 + {0, 1}
+        float* s_q = reinterpret_cast<float*>(smem) + warp * HD;
+        const int tail_cta = split - n_split_launch;
+        for (int pi = 0; pi < PAIRS / TAIL_CTAS / 4; ++pi) {
+            const int pidx = tail_cta * (PAIRS / TAIL_CTAS) + warp * (PAIRS / TAIL_CTAS / 4) + pi;
+            const int r = row0 + pidx / group, head = kvh * group + pidx % group;
+            if (r >= n_rows) break;
+            int depth;
+            unsigned long long lo, hi;
+            if (a.st) {
+                depth = a.st[seq].row_depth[r]; lo = a.st[seq].row_anc[r][0]; hi = a.st[seq].row_anc[r][1];
+            } else {
+                depth = a.depth[seq * RT + r]; lo = a.anc[(size_t)(seq * RT + r) * 2]; hi = a.anc[(size_t)(seq * RT + r) * 2 + 1];
+            }
+            const int P = L + depth, T0 = tail_start_mma(P, a.dcap);
+            const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((size_t)(seq * RT + r) * a.Hq + head) * HD;
+            __syncwarp();
+            {
+                const uint2 qq = *reinterpret_cast<const uint2*>(q + lane * 4);
+                const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qq.x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qq.y);
+                s_q[lane * 4 + 0] = __low2float(q01); s_q[lane * 4 + 1] = __high2float(q01);
+                s_q[lane * 4 + 2] = __low2float(q23); s_q[lane * 4 + 3] = __high2float(q23);
+            }
+            __syncwarp();
+            float m = -INFINITY, l = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
+            const int n_tail = P - T0 + 1;
+            for (int t0 = 0; t0 < n_tail; t0 += 32) {
+                const int t = t0 + lane;
+                bool valid = t < n_tail;
+                int slot = 0;
+                if (valid) {
+                    const int pos = T0 + t;
+                    if (pos < L) slot = pos;
+                    else {
+                        const int b = nth_set_bit128(lo, hi, pos - L);
+                        if (b < 0) { set_error(a.err, DEV_E_INDEX); valid = false; }
+                        else slot = L + b;
+                    }
+                }
+                float sc = -INFINITY;
+                if (valid) {
+                    const uint4* kr = reinterpret_cast<const uint4*>(kbase + (size_t)slot * HD);
+                    uint4 kreg[HD / 8];
+#pragma unroll
+                    for (int d8 = 0; d8 < HD / 8; ++d8) kreg[d8] = kr[d8];
+                    float acc = 0.f;
+#pragma unroll
+                    for (int d8 = 0; d8 < HD / 8; ++d8) {
+                        const uint4 kk = kreg[d8];
+                        const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kk);
+                        const float4 qa = *reinterpret_cast<const float4*>(s_q + d8 * 8), qb = *reinterpret_cast<const float4*>(s_q + d8 * 8 + 4);
+                        acc = fmaf(qa.x, __low2float(k2[0]), acc); acc = fmaf(qa.y, __high2float(k2[0]), acc);
+                        acc = fmaf(qa.z, __low2float(k2[1]), acc); acc = fmaf(qa.w, __high2float(k2[1]), acc);
+                        acc = fmaf(qb.x, __low2float(k2[2]), acc); acc = fmaf(qb.y, __high2float(k2[2]), acc);
+                        acc = fmaf(qb.z, __low2float(k2[3]), acc); acc = fmaf(qb.w, __high2float(k2[3]), acc);
+                    }
+                    sc = acc * a.scale_log2;
+                }
+                float cm = sc;
+#pragma unroll
+                for (int of = 16; of > 0; of >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, of));
+                const float pe = valid ? exp2f(sc - cm) : 0.f;
+                float cl = pe;
+#pragma unroll
+                for (int of = 16; of > 0; of >>= 1) cl += __shfl_xor_sync(0xffffffffu, cl, of);
+                float co[4] = {0.f, 0.f, 0.f, 0.f};
+                // weighted values, keys in position order; the loads of 8 keys are issued before their sums
+                // (a key that is not in the chunk reads slot 0 with weight 0 and is skipped)
+                for (int j0 = 0; j0 < 32; j0 += 8) {
+                    float pj[8];
+                    uint2 vv[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        pj[u] = __shfl_sync(0xffffffffu, pe, j0 + u);
+                        const int sj = __shfl_sync(0xffffffffu, slot, j0 + u);
+                        vv[u] = *reinterpret_cast<const uint2*>(vbase + (size_t)sj * HD + lane * 4);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (pj[u] != 0.f) {
+                            const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vv[u].x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vv[u].y);
+                            co[0] = fmaf(pj[u], __low2float(v01), co[0]); co[1] = fmaf(pj[u], __high2float(v01), co[1]);
+                            co[2] = fmaf(pj[u], __low2float(v23), co[2]); co[3] = fmaf(pj[u], __high2float(v23), co[3]);
+                        }
+                    }
+                }
+                merge_ml(m, l, o, cm, cl, co);
+            }
+            const size_t idx = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max + (a.n_split_max - 1);
+            if (lane == 0) a.part_ml[idx] = make_float2(m, l);
+            *reinterpret_cast<float4*>(a.part_o + idx * HD + lane * 4) = make_float4(o[0], o[1], o[2], o[3]);
+        }
+    } else {
+        // ---------------- bulk CTA
+        attn_bulk_chunks(a, smem, seq, kvh, row0, split, group, n_rows, L, T0max, kbase, vbase);
+    }
+
+    // ---------------- whichever CTA of the group arrives last merges the partials (fixed order: splits, then tail)
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int* ctr = counters + (size_t)seq * gridDim.y + blockIdx.y;
+        const int old = atomicAdd(ctr, 1);
+        s_last = old == n_bulk + TAIL_CTAS - 1;
+        if (s_last) *ctr = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int pi = 0; pi < 16; ++pi) {
+        const int pidx = warp * 16 + pi;
+        const int r = row0 + pidx / group, head = kvh * group + pidx % group;
+        if (r >= n_rows) break;
+        const int depth = a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r];
+        const int T0 = tail_start_mma(L + depth, a.dcap);
+        const int n_sp = (T0 + a.split_len - 1) / a.split_len;
+        const size_t base = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max;
+        float m = -INFINITY, l = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int s0 = 0; s0 <= n_sp; s0 += 8) {
+            float2 ml[8];
+            float4 c4[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int sp = s0 + u;
+                const size_t idx = base + (sp < n_sp ? sp : a.n_split_max - 1);
+                if (sp <= n_sp) {
+                    ml[u] = __ldcg(a.part_ml + idx);
+                    c4[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + idx * HD + lane * 4));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (s0 + u <= n_sp) {
+                    const float co[4] = {c4[u].x, c4[u].y, c4[u].z, c4[u].w};
+                    merge_ml(m, l, o, ml[u].x, ml[u].y, co);
+                }
+            }
+        }
+        const float inv = 1.0f / l;
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out) + ((size_t)(seq * RT + r) * a.Hq + head) * HD + lane * 4;
+        const __nv_bfloat162 o01 = __floats2bfloat162_rn(o[0] * inv, o[1] * inv), o23 = __floats2bfloat162_rn(o[2] * inv, o[3] * inv);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t*>(&o01);
+        pk.y = *reinterpret_cast<const uint32_t*>(&o23);
+        *reinterpret_cast<uint2*>(out) = pk;
+    }
+}
+
 }  // namespace
 
-int launch_attn_bulk_mma(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl) {
+int attn_tree_counter_ints(int batch) { return batch * 1024; }
+
+// One launch: grid.x = bulk splits + TAIL_CTAS tail CTAs per (KV head, row tile) group.  `counters` (attn_tree_counter_ints
+// ints, zero before the first launch; the kernel leaves them zero) count the finished CTAs of each group.
+int launch_attn_tree(const AttnArgs& a, int batch, int n_split_launch, int* counters, cudaStream_t s, bool pdl) {
     if (a.h != HD || a.Hq % a.Hkv) return -1;
     const int group = a.Hq / a.Hkv;
     if (group > PAIRS || PAIRS % group) return -1;
     const int rows_per_tile = PAIRS / group;
     const int n_row_tiles = (RT + rows_per_tile - 1) / rows_per_tile;
+    if (a.Hkv * n_row_tiles > 1024 || n_split_launch + 1 > a.n_split_max) return -1;
     static bool attr_set = false;
     const int smem = 4 * KV_TILE_BYTES;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(k_attn_bulk_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
+        if (cudaFuncSetAttribute(k_attn_tree, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
         attr_set = true;
     }
-    dim3 grid(n_split_launch, a.Hkv * n_row_tiles, batch);
-    launch_k(k_attn_bulk_mma, grid, dim3(128), (size_t)smem, s, pdl, a, n_split_launch, group, rows_per_tile, n_row_tiles);
+    dim3 grid(n_split_launch + TAIL_CTAS, a.Hkv * n_row_tiles, batch);
+    launch_k(k_attn_tree, grid, dim3(128), (size_t)smem, s, pdl, a, n_split_launch, group, rows_per_tile, n_row_tiles, counters);
     return 0;
 }
 

@@ -87,10 +87,22 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return false;
 }
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+// L2 eviction policies: weights are read once per step and never again before the whole model has streamed
+// through (evict first); activations are re-read by every CTA (evict last).
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
         : "memory");
 }
 
@@ -220,6 +232,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
         if (lane == 0) {
             // The weights do not depend on the kernel before this one: fill the ring with weight tiles first,
             // wait for that kernel, then add the activation tiles.
+            const uint64_t pol_w = l2_policy_evict_first(), pol_x = l2_policy_evict_last();
             const int n_items = (int)(u1 - u0);
             const int n_pre = n_items < STAGES ? n_items : STAGES;
             for (int pass = 0; pass < 2; ++pass) {
@@ -233,10 +246,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                         unsigned char* sa = stages + it * STAGE_BYTES;
                         if (pass == 0) {
                             mbar_expect_tx(&full[it], STAGE_BYTES);
-                            tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[it]);
-                            tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it]);
+                            tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[it], pol_w);
+                            tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it], pol_w);
                         } else {
-                            tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[it]);
+                            tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[it], pol_x);
                         }
                     }
                 }
@@ -255,9 +268,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                         if (!mbar_wait(&empty[stage], phase ^ 1, s_abort)) { ok = false; break; }
                         unsigned char* sa = stages + stage * STAGE_BYTES;
                         mbar_expect_tx(&full[stage], STAGE_BYTES);
-                        tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[stage]);
-                        tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage]);
-                        tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[stage]);
+                        tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[stage], pol_w);
+                        tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage], pol_w);
+                        tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[stage], pol_x);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -345,20 +358,43 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                 if (finish) {
                     // last contributor of this tile: sum the partials in CTA order (fixed, whoever arrives last)
                     __threadfence();
-                    for (int r0 = 0; r0 < n_rows; r0 += 8) {
-                        float acc[8];
+                    // thread et: features 4*(et%32)..+3, rows et/32 + 4*i; every load of a batch is issued before the sums
+                    const int f4 = (et & 31) * 4, rg = et >> 5;
+                    for (int i0 = 0; i0 < RT / 4; i0 += 4) {
+                        if (rg + 4 * i0 >= n_rows) break;
+                        float4 acc[4];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-                        for (int c = c_first; c <= c_last; ++c) {
-                            const float* src = p.partials + ((size_t)(c * 2 + sk_slot(sk, c, sg.tile)) * RT + r0) * TILE_N + f;
-                            float t[8];
+                        for (int ii = 0; ii < 4; ++ii) acc[ii] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int cb = c_first; cb <= c_last; cb += 4) {
+                            float4 t[4][4];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) t[j] = r0 + j < n_rows ? __ldcg(src + j * TILE_N) : 0.f;
+                            for (int cc = 0; cc < 4; ++cc) {
+                                const int c = cb + cc;
+                                const bool cv = c <= c_last;
+                                const float* src = p.partials + ((size_t)((cv ? c : c_first) * 2 + sk_slot(sk, cv ? c : c_first, sg.tile)) * RT) * TILE_N + f4;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) acc[j] += t[j];
+                                for (int ii = 0; ii < 4; ++ii) {
+                                    const int r = rg + 4 * (i0 + ii);
+                                    t[cc][ii] = (cv && r < n_rows) ? __ldcg(reinterpret_cast<const float4*>(src + (size_t)r * TILE_N))
+                                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+                                }
+                            }
+#pragma unroll
+                            for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                                for (int ii = 0; ii < 4; ++ii) {
+                                    acc[ii].x += t[cc][ii].x; acc[ii].y += t[cc][ii].y;
+                                    acc[ii].z += t[cc][ii].z; acc[ii].w += t[cc][ii].w;
+                                }
                         }
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) s_acc[(r0 + j) * ACC_LD + f] = acc[j];
+                        for (int ii = 0; ii < 4; ++ii) {
+                            const int r = rg + 4 * (i0 + ii);
+                            if (r < RT) {
+                                float* d = s_acc + r * ACC_LD + f4;
+                                d[0] = acc[ii].x; d[1] = acc[ii].y; d[2] = acc[ii].z; d[3] = acc[ii].w;
+                            }
+                        }
                     }
                     if (et == 0) p.counters[sg.tile] = 0;
                 }

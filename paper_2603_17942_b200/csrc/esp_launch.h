@@ -59,8 +59,9 @@ void launch_gemm_simt(int dtype, int epi, int n_tiles, int batch, const void* co
 // position-canonical attention: CUDA-core bulk (+ tail/merge), or tail/merge only when the
 // tensor-core bulk kernel already produced the split partials
 int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s, bool pdl);
-// tensor-core bulk for bf16, head_dim 128
-int launch_attn_bulk_mma(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl);
+// bf16, head_dim 128: the whole operator in one launch (tensor-core bulk CTAs + tail CTAs + last-arriver merge)
+int launch_attn_tree(const AttnArgs& a, int batch, int n_split_launch, int* counters, cudaStream_t s, bool pdl);
+int attn_tree_counter_ints(int batch);
 
 // tcgen05 GEMM: a plan holds the TMA descriptors and the stream-K partition of one weight shape
 struct TcGemm;
