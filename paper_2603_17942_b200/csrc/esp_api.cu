@@ -43,7 +43,6 @@ struct Buffers {
     float *rope_cos, *rope_sin;
     void* gemm_partials;
     int* gemm_counters;
-    int* attn_counters;
 };
 
 
@@ -129,7 +128,6 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.rope_sin = c.take<float>((size_t)D.cap * (D.h / 2));
     o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm));
     o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
-    o.attn_counters = c.take<int>(attn_tree_counter_ints(D.batch));
     return align_up(c.off, 256);
 }
 
@@ -217,7 +215,7 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
     const bool tc = h->dtype == 1 && h->gemm_impl == 0 && h->p_lm != nullptr;
     const bool pdl = h->use_pdl && !h->prof;
     StreamK pending;   // partials of the last down projection, summed by the next norm
-    pending.partials = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1;
+    pending.partials = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2;
     mark(h, -1);
     launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.batch, s, false);
     h->launches++;
@@ -258,8 +256,8 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             a.err = b.err;
             const bool mma = h->dtype == 1 && D.h == 128 && h->gemm_impl == 0;
             if (mma) {
-                if (launch_attn_tree(a, D.batch, n_split_launch, b.attn_counters, s, pdl)) return ESP_E_BADCFG;
-                h->launches++;
+                if (launch_attn_tree(a, D.batch, n_split_launch, s, pdl)) return ESP_E_BADCFG;
+                h->launches += 2;
             } else {
                 if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, true, s, pdl)) return ESP_E_BADCFG;
                 h->launches += n_split_launch > 0 ? 2 : 1;
@@ -286,6 +284,10 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             const int32_t rows[3] = {D.F, D.F, 0};
             int rc = run_gemm(h, tc ? h->p_gu[l] : nullptr, EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a, tc, pdl);
             if (rc) return rc;
+            if (tc) {
+                launch_swiglu_finish(b.states, tc_gemm_streamk(h->p_gu[l]), b.act, D.F, s, pdl);
+                h->launches++;
+            }
             mark(h, KIND_GATEUP);
         }
         {
@@ -417,27 +419,27 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
             TcGemm* p = nullptr;
             const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t r1[3] = {dq, dkv, dkv};
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
             h->p_qkv.push_back(p);
             const void* w2[3] = {h->wo[l], nullptr, nullptr};
             const int32_t r2[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
             h->p_o.push_back(p);
             const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t r3[3] = {D.F, D.F, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, w3, r3, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
             h->p_gu.push_back(p);
             const void* w4[3] = {h->wd[l], nullptr, nullptr};
             const int32_t r4[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
             h->p_down.push_back(p);
         }
         const void* w5[3] = {h->lm_head, nullptr, nullptr};
         const int32_t r5[3] = {D.V, 0, 0};
-        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
         if (!ok) { esp_free(h); return ESP_E_CUDA; }
     } else if (model->dtype == 1) {
         h->gemm_impl = 1;  // batched rows: CUDA-core path until the tensor-core kernel tiles over sequences
@@ -678,8 +680,7 @@ int esp_tree_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t h
     while ((cap + S - 1) / S > 64) S *= 2;
     const size_t ns = (cap + S - 1) / S + 1;
     const size_t rows = (size_t)batch * RT * n_q_heads * ns;
-    *bytes_out = align_up(rows * head_dim * sizeof(float), 256) + align_up(rows * sizeof(float2), 256) +
-                 align_up(sizeof(int) * attn_tree_counter_ints(batch), 256) + 256;
+    *bytes_out = align_up(rows * head_dim * sizeof(float), 256) + align_up(rows * sizeof(float2), 256) + 256;
     return ESP_OK;
 }
 
@@ -715,10 +716,7 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     const int n_split_launch = (L + S - 1) / S;
     const bool mma = dtype == 1 && head_dim == 128;
     if (mma) {
-        int* counters = reinterpret_cast<int*>(reinterpret_cast<char*>(scratch) + align_up(rows * head_dim * sizeof(float), 256) +
-                                               align_up(rows * sizeof(float2), 256));
-        if (cudaMemsetAsync(counters, 0, sizeof(int) * attn_tree_counter_ints(batch), s) != cudaSuccess) return ESP_E_CUDA;
-        if (launch_attn_tree(a, batch, n_split_launch, counters, s, false)) return ESP_E_BADCFG;
+        if (launch_attn_tree(a, batch, n_split_launch, s, false)) return ESP_E_BADCFG;
     } else if (launch_attn_simt(dtype, a, batch, n_split_launch, true, s, false)) {
         return ESP_E_BADCFG;
     }
@@ -759,7 +757,7 @@ int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const
     if (cudaMemsetAsync(counters, 0, sizeof(int) * tc_gemm_counter_ints() , s) != cudaSuccess) return ESP_E_CUDA;
     if (cudaMemsetAsync(err, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
     TcGemm* plan = nullptr;
-    if (tc_gemm_create(&plan, EPI_STORE_F32, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err)) return ESP_E_CUDA;
+    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err)) return ESP_E_CUDA;
     int rc = tc_gemm_launch(plan, a, s, false);
     int e = 0;
     if (!rc && cudaMemcpyAsync(&e, err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) rc = ESP_E_CUDA;

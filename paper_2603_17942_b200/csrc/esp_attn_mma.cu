@@ -1,4 +1,4 @@
-// Tree attention for bf16, head_dim 128, in one kernel.
+// Tree attention for bf16, head_dim 128.
 //
 // A row at position P attends to cache positions 0..T0-1 through the "bulk"
 // CTAs (T0 as in tail_start(): the 16-aligned position below which keys are
@@ -8,10 +8,10 @@
 // pairs, a warp 16 of them, Q.K^T and P.V run on mma.sync m16n8k16 with fp32
 // online softmax in registers.  The remaining positions T0..P -- the end of
 // the cache plus the row's in-flight tree ancestors, found through its
-// ancestor bitmask -- are summed by one more "tail" CTA per group of pairs,
-// key by key in position order.  Every CTA stores (max, sum, weighted values)
-// partials; whichever CTA of a group finishes last merges them in split order
-// (tail last) and writes the output.  No CTA waits for another.
+// ancestor bitmask -- are summed by "tail" CTAs of the same launch, key by
+// key in position order.  Every CTA stores (max, sum, weighted values)
+// partials; a second small kernel (one warp per (row, head)) merges them in
+// split order, tail last, and writes the output.
 //
 // Everything that decides a row's arithmetic -- the 64-key chunk grid, the
 // split grid, the per-position mask -- is a function of absolute positions
@@ -250,10 +250,9 @@ __device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], floa
     m = mn;
 }
 
-__global__ void __launch_bounds__(128) k_attn_tree(AttnArgs a, int n_split_launch, int group, int rows_per_tile, int n_row_tiles,
-                                                  int* counters) {
+__global__ void __launch_bounds__(128) k_attn_tree(AttnArgs a, int n_split_launch, int group, int rows_per_tile, int n_row_tiles) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ int s_T0max, s_last;
+    __shared__ int s_T0max;
     pdl_wait();
     if (threadIdx.x == 0) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -390,22 +389,25 @@ __global__ void __launch_bounds__(128) k_attn_tree(AttnArgs a, int n_split_launc
         attn_bulk_chunks(a, smem, seq, kvh, row0, split, group, n_rows, L, T0max, kbase, vbase);
     }
 
-    // ---------------- whichever CTA of the group arrives last merges the partials (fixed order: splits, then tail)
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int* ctr = counters + (size_t)seq * gridDim.y + blockIdx.y;
-        const int old = atomicAdd(ctr, 1);
-        s_last = old == n_bulk + TAIL_CTAS - 1;
-        if (s_last) *ctr = 0;
+}
+
+// Merge of the partials of one (row, head) pair, one warp per pair: bulk splits in split order, the tail last.
+__global__ void __launch_bounds__(128) k_attn_merge(AttnArgs a) {
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 4 + warp, head = blockIdx.y, seq = blockIdx.z;
+    int n_rows, L;
+    if (a.st) {
+        const SeqState* st = a.st + seq;
+        n_rows = st->active ? st->n_rows : 0;
+        L = st->L;
+    } else {
+        n_rows = a.n_rows_fixed;
+        L = a.L_fixed;
     }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    for (int pi = 0; pi < 16; ++pi) {
-        const int pidx = warp * 16 + pi;
-        const int r = row0 + pidx / group, head = kvh * group + pidx % group;
-        if (r >= n_rows) break;
+    if (r >= n_rows) return;
+    {
         const int depth = a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r];
         const int T0 = tail_start_mma(L + depth, a.dcap);
         const int n_sp = (T0 + a.split_len - 1) / a.split_len;
@@ -443,17 +445,15 @@ __global__ void __launch_bounds__(128) k_attn_tree(AttnArgs a, int n_split_launc
 
 }  // namespace
 
-int attn_tree_counter_ints(int batch) { return batch * 1024; }
-
-// One launch: grid.x = bulk splits + TAIL_CTAS tail CTAs per (KV head, row tile) group.  `counters` (attn_tree_counter_ints
-// ints, zero before the first launch; the kernel leaves them zero) count the finished CTAs of each group.
-int launch_attn_tree(const AttnArgs& a, int batch, int n_split_launch, int* counters, cudaStream_t s, bool pdl) {
+// Two launches: k_attn_tree with grid.x = bulk splits + TAIL_CTAS tail CTAs per (KV head, row tile) group, each
+// storing (max, sum, weighted values) partials, then k_attn_merge with one warp per (row, head).
+int launch_attn_tree(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl) {
     if (a.h != HD || a.Hq % a.Hkv) return -1;
     const int group = a.Hq / a.Hkv;
     if (group > PAIRS || PAIRS % group) return -1;
     const int rows_per_tile = PAIRS / group;
     const int n_row_tiles = (RT + rows_per_tile - 1) / rows_per_tile;
-    if (a.Hkv * n_row_tiles > 1024 || n_split_launch + 1 > a.n_split_max) return -1;
+    if (n_split_launch + 1 > a.n_split_max) return -1;
     static bool attr_set = false;
     const int smem = 4 * KV_TILE_BYTES;
     if (!attr_set) {
@@ -461,7 +461,8 @@ int launch_attn_tree(const AttnArgs& a, int batch, int n_split_launch, int* coun
         attr_set = true;
     }
     dim3 grid(n_split_launch + TAIL_CTAS, a.Hkv * n_row_tiles, batch);
-    launch_k(k_attn_tree, grid, dim3(128), (size_t)smem, s, pdl, a, n_split_launch, group, rows_per_tile, n_row_tiles, counters);
+    launch_k(k_attn_tree, grid, dim3(128), (size_t)smem, s, pdl, a, n_split_launch, group, rows_per_tile, n_row_tiles);
+    launch_k(k_attn_merge, dim3((RT + 3) / 4, a.Hq, batch), dim3(128), 0, s, pdl, a);
     return 0;
 }
 

@@ -75,12 +75,12 @@ struct Dims {
 enum Epi : int { EPI_STORE_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, EPI_LOGITS = 4, EPI_PARTIAL = 5 };
 
 // Stream-K partition of a GEMM: the n_tiles*KB (tile, k-block) units are dealt out in equal contiguous
-// ranges to G persistent CTAs; CTA c owns units [c*U/G, (c+1)*U/G).  A CTA's range touches at most one
-// tile it does not start (slot 1) besides the tile holding its first unit (slot 0).  Partials live at
-// partials[((cta*2 + slot)*RT + row)*TILE_N + feature].
+// ranges to G persistent CTAs; CTA c owns units [c*U/G, (c+1)*U/G).  The piece of tile t a CTA computed is
+// kept in slot min(t - first tile of the CTA, slots - 1) of that CTA:
+// partials[((cta*slots + slot)*RT + row)*TILE_N + feature].
 struct StreamK {
     const float* partials;  // NULL: nothing to sum
-    int32_t n_tiles, KB, G;
+    int32_t n_tiles, KB, G, slots;
 };
 __host__ __device__ __forceinline__ long long sk_begin(long long c, long long U, long long G) { return c * U / G; }
 __host__ __device__ __forceinline__ int sk_cta_of_unit(long long u, long long U, long long G) {
@@ -94,7 +94,12 @@ __host__ __device__ __forceinline__ void sk_contributors(const StreamK& s, int t
 }
 __host__ __device__ __forceinline__ int sk_slot(const StreamK& s, int c, int tile) {
     const long long U = (long long)s.n_tiles * s.KB;
-    return tile == (int)(sk_begin(c, U, s.G) / s.KB) ? 0 : 1;
+    const int d = tile - (int)(sk_begin(c, U, s.G) / s.KB);
+    return d < s.slots - 1 ? d : s.slots - 1;
+}
+// address of contributor c's partial row of a tile
+__device__ __forceinline__ const float* sk_partial(const StreamK& s, int c, int tile, int row) {
+    return s.partials + ((size_t)(c * s.slots + sk_slot(s, c, tile)) * RT + row) * TILE_N;
 }
 
 // Everything an epilogue may need.  One struct for all variants keeps the

@@ -52,7 +52,9 @@ struct TcParams {
     CUtensorMap map_b;
     int32_t rows_w[3];
     int32_t n_tiles, KB, grid, epi;
-    float* partials;   // [grid][2][RT][TILE_N]
+    int32_t map_swiglu;  // tile = 64 rows of w[0] (gate) + the matching 64 rows of w[1] (up)
+    int32_t slots;       // partial slots per CTA
+    float* partials;   // [grid][slots][RT][TILE_N]
     int* counters;     // [n_tiles], zero between launches
     int* err;
     EpiArgs a;
@@ -150,12 +152,13 @@ struct Seg {
 // (tail piece, then head piece), whole tiles after them: partial tiles are then complete early in every
 // CTA's timeline and the CTA that finishes one does so while the weight stream of its whole tiles is running.
 struct Range {
-    int first_tile, last_tile, head_kb0, tail_kb1, KB, n_seg;
+    int first_tile, last_tile, head_kb0, tail_kb1, KB, n_seg, slots;
     bool tail_partial;
 };
-__device__ __forceinline__ Range make_range(long long u0, long long u1, int KB) {
+__device__ __forceinline__ Range make_range(long long u0, long long u1, int KB, int slots) {
     Range r;
     r.KB = KB;
+    r.slots = slots;
     r.first_tile = (int)(u0 / KB);
     r.head_kb0 = (int)(u0 % KB);
     r.last_tile = (int)((u1 - 1) / KB);
@@ -175,14 +178,14 @@ __device__ __forceinline__ Seg get_seg(const Range& r, int i) {
         else if (idx == 0) { s.tile = r.first_tile; s.kb0 = r.head_kb0; s.kb1 = r.KB; s.slot = 0; }
         else { s.tile = r.first_tile + idx; s.kb0 = 0; s.kb1 = r.KB; s.slot = 1; }
     }
+    s.slot = s.tile - r.first_tile < r.slots - 1 ? s.tile - r.first_tile : r.slots - 1;
     s.whole = s.kb0 == 0 && s.kb1 == r.KB;
     return s;
 }
 
 // which weight matrix / row the two 64-row halves of a tile come from
-template <int EPI>
 __device__ __forceinline__ void tile_source(const TcParams& p, int tile, int half, int& m, int& row) {
-    if (EPI == EPI_SWIGLU) { m = half; row = tile * 64; return; }
+    if (p.map_swiglu) { m = half; row = tile * 64; return; }
     int feat = tile * TILE_N;
     m = 0;
     while (m < 2 && feat >= p.rows_w[m]) { feat -= p.rows_w[m]; ++m; }
@@ -207,7 +210,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long U = (long long)p.n_tiles * p.KB, G = p.grid;
     const long long u0 = sk_begin(blockIdx.x, U, G), u1 = sk_begin(blockIdx.x + 1, U, G);
-    const Range rng = make_range(u0, u1, p.KB);
+    const Range rng = make_range(u0, u1, p.KB, p.slots);
 
     if (threadIdx.x == 0) {
         pdl_launch_dependents();
@@ -240,8 +243,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                 for (int i = 0; i < rng.n_seg && it < n_pre; ++i) {
                     const Seg sg = get_seg(rng, i);
                     int m0, r0, m1, r1;
-                    tile_source<EPI>(p, sg.tile, 0, m0, r0);
-                    tile_source<EPI>(p, sg.tile, 1, m1, r1);
+                    tile_source(p, sg.tile, 0, m0, r0);
+                    tile_source(p, sg.tile, 1, m1, r1);
                     for (int kb = sg.kb0; kb < sg.kb1 && it < n_pre; ++kb, ++it) {
                         unsigned char* sa = stages + it * STAGE_BYTES;
                         if (pass == 0) {
@@ -261,8 +264,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
             for (int i = 0; i < rng.n_seg && ok; ++i) {
                 const Seg sg = get_seg(rng, i);
                 int m0, r0, m1, r1;
-                tile_source<EPI>(p, sg.tile, 0, m0, r0);
-                tile_source<EPI>(p, sg.tile, 1, m1, r1);
+                tile_source(p, sg.tile, 0, m0, r0);
+                tile_source(p, sg.tile, 1, m1, r1);
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
                     if (it >= n_pre) {
                         if (!mbar_wait(&empty[stage], phase ^ 1, s_abort)) { ok = false; break; }
@@ -313,7 +316,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
         const int et = threadIdx.x - 64;        // 0..127 index among the epilogue threads
         const int n_rows = p.a.st ? (p.a.st->active ? p.a.st->n_rows : 0) : p.a.rows_fixed;
         StreamK sk;
-        sk.partials = p.partials; sk.n_tiles = p.n_tiles; sk.KB = p.KB; sk.G = p.grid;
+        sk.partials = p.partials; sk.n_tiles = p.n_tiles; sk.KB = p.KB; sk.G = p.grid; sk.slots = p.slots;
         bool ok = true;
         for (int i = 0; i < rng.n_seg && ok; ++i) {
             const Seg sg = get_seg(rng, i);
@@ -337,7 +340,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
 #pragma unroll
                 for (int r = 0; r < RT; ++r) s_acc[r * ACC_LD + f] = __uint_as_float(v[r]);
             } else {
-                float* part = p.partials + ((size_t)(blockIdx.x * 2 + sg.slot) * RT) * TILE_N + f;
+                float* part = p.partials + ((size_t)(blockIdx.x * p.slots + sg.slot) * RT) * TILE_N + f;
 #pragma unroll
                 for (int r = 0; r < RT; ++r)
                     if (r < n_rows) __stcg(part + r * TILE_N, __uint_as_float(v[r]));
@@ -371,7 +374,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                             for (int cc = 0; cc < 4; ++cc) {
                                 const int c = cb + cc;
                                 const bool cv = c <= c_last;
-                                const float* src = p.partials + ((size_t)((cv ? c : c_first) * 2 + sk_slot(sk, cv ? c : c_first, sg.tile)) * RT) * TILE_N + f4;
+                                const float* src = sk_partial(sk, cv ? c : c_first, sg.tile, 0) + f4;
 #pragma unroll
                                 for (int ii = 0; ii < 4; ++ii) {
                                     const int r = rg + 4 * (i0 + ii);
@@ -456,12 +459,13 @@ struct TcGemm {
     TcParams p;
 };
 
-size_t tc_gemm_partial_bytes(int n_sm) { return (size_t)n_sm * 2 * RT * TILE_N * sizeof(float); }
+constexpr int MAX_SLOTS = 4;
+size_t tc_gemm_partial_bytes(int n_sm) { return (size_t)n_sm * MAX_SLOTS * RT * TILE_N * sizeof(float); }
 int tc_gemm_counter_ints() { return 4096; }
 int tc_gemm_tiles(const TcGemm* g) { return g ? g->p.n_tiles : 0; }
 
-int tc_gemm_create(TcGemm** out, int epi, const void* const w[3], const int32_t rows_w[3], int K, const void* x, int batch,
-                   void* partials, size_t partial_bytes, int* counters, int n_sm, int* err) {
+int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
+                   int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err) {
     if (!out || batch != 1 || K % 8 || n_sm < 1) return -1;
     if (reinterpret_cast<uintptr_t>(x) % 16) return -1;
     TcGemm* g = new (std::nothrow) TcGemm();
@@ -479,14 +483,26 @@ int tc_gemm_create(TcGemm** out, int epi, const void* const w[3], const int32_t 
         }
     }
     if (make_map(&p.map_b, x, RT, K, RT)) { delete g; return -1; }
-    p.epi = epi;
+    p.map_swiglu = epi == EPI_SWIGLU;
+    p.epi = defer ? (int)EPI_PARTIAL : epi;
     p.n_tiles = epi == EPI_SWIGLU ? (rows_w[0] + 63) / 64 : (total_rows + TILE_N - 1) / TILE_N;
     p.KB = (K + BK - 1) / BK;
     const long long U = (long long)p.n_tiles * p.KB;
     p.grid = (int)(U < n_sm ? U : n_sm);
     if (p.n_tiles > tc_gemm_counter_ints() || tc_gemm_partial_bytes(p.grid) > partial_bytes) { delete g; return -1; }
-    // partial-only output keeps two slots per CTA: a CTA's range must not span more than two tiles
-    if (epi == EPI_PARTIAL && p.n_tiles > p.grid) { delete g; return -1; }
+    // fused epilogues store only the head and tail pieces of a range (2 slots); partial-only output stores every
+    // piece, one slot per tile the range touches
+    p.slots = 2;
+    if (p.epi == EPI_PARTIAL) {
+        int most = 1;
+        for (int c = 0; c < p.grid; ++c) {
+            const long long a0 = sk_begin(c, U, p.grid), a1 = sk_begin(c + 1, U, p.grid);
+            const int n = (int)((a1 - 1) / p.KB - a0 / p.KB) + 1;
+            most = n > most ? n : most;
+        }
+        if (most > MAX_SLOTS) { delete g; return -1; }
+        p.slots = most < 2 ? 2 : most;
+    }
     p.partials = reinterpret_cast<float*>(partials);
     p.counters = counters;
     p.err = err;
@@ -502,6 +518,7 @@ StreamK tc_gemm_streamk(const TcGemm* g) {
     k.n_tiles = g ? g->p.n_tiles : 0;
     k.KB = g ? g->p.KB : 1;
     k.G = g ? g->p.grid : 1;
+    k.slots = g ? g->p.slots : 2;
     return k;
 }
 
@@ -521,7 +538,6 @@ int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl) 
     } break;
     switch (p.epi) {
         ESP_TC_CASE(EPI_STORE_F32)
-        ESP_TC_CASE(EPI_SWIGLU)
         ESP_TC_CASE(EPI_LOGITS)
         ESP_TC_CASE(EPI_PARTIAL)
         default: return ESP_E_ARG;

@@ -94,8 +94,7 @@ __global__ void __launch_bounds__(512) k_resid_norm(const SeqState* states, floa
             sk_contributors(sk, tile, c_first, c_last);
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int c = c_first; c <= c_last; ++c) {
-                const float4 t = __ldcg(reinterpret_cast<const float4*>(
-                    sk.partials + ((size_t)(c * 2 + sk_slot(sk, c, tile)) * RT + r) * TILE_N + f));
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(sk_partial(sk, c, tile, r) + f));
                 acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
             }
             x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
@@ -143,7 +142,7 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
 #pragma unroll
     for (int i = 0; i < NE; ++i) v[i] = 0.f;
     for (int c = c_first; c <= c_last; ++c) {
-        const float* src = sk.partials + ((size_t)(c * 2 + sk_slot(sk, c, tile)) * RT + r) * TILE_N + f;
+        const float* src = sk_partial(sk, c, tile, r) + f;
         if constexpr (NE == 4) {
             const float4 t = __ldcg(reinterpret_cast<const float4*>(src));
             v[0] += t.x; v[1] += t.y; v[2] += t.z; v[3] += t.w;
@@ -186,6 +185,33 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
     if constexpr (NE == 4) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(o);
     else if constexpr (NE == 2) *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(o);
     else dst[0] = o[0];
+}
+
+// Consumer of the split gate/up GEMM: a tile holds 64 gate features (columns 0..63) and the matching 64 up
+// features (columns 64..127); sums both over the tile's contributors in CTA order and stores silu(gate) * up.
+__global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, int rows_fixed, StreamK sk, __nv_bfloat16* act, int F) {
+    pdl_wait();
+    if (threadIdx.x == 0) pdl_launch_dependents();
+    const int r = blockIdx.y;
+    const int n_rows = states ? (states->active ? states->n_rows : 0) : rows_fixed;
+    const int j = (blockIdx.x * 256 + threadIdx.x) * 4;
+    if (r >= n_rows || j >= F) return;
+    const int tile = j / 64, f = j % 64;
+    int c_first, c_last;
+    sk_contributors(sk, tile, c_first, c_last);
+    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+    for (int c = c_first; c <= c_last; ++c) {
+        const float* src = sk_partial(sk, c, tile, r);
+        const float4 tg = __ldcg(reinterpret_cast<const float4*>(src + f));
+        const float4 tu = __ldcg(reinterpret_cast<const float4*>(src + 64 + f));
+        g.x += tg.x; g.y += tg.y; g.z += tg.z; g.w += tg.w;
+        u.x += tu.x; u.y += tu.y; u.z += tu.z; u.w += tu.w;
+    }
+    const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+    __nv_bfloat16 o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) o[i] = __float2bfloat16_rn((gv[i] / (1.0f + expf(-gv[i]))) * uv[i]);
+    *reinterpret_cast<uint2*>(act + (size_t)r * F + j) = *reinterpret_cast<const uint2*>(o);
 }
 
 // ------------------------------------------------------------------ CUDA-core GEMM
@@ -923,6 +949,9 @@ void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const
                        float* copy_out, cudaStream_t s, bool pdl) {
     launch_k(k_resid_norm<__nv_bfloat16>, dim3(RT, 1), dim3(512), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
              (__nv_bfloat16*)y, d, eps, copy_out);
+}
+void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, cudaStream_t s, bool pdl) {
+    launch_k(k_swiglu_finish, dim3((F / 4 + 255) / 256, RT), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act, F);
 }
 int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, cudaStream_t s, bool pdl) {
     const int n_heads = a.Hq + 2 * a.Hkv;

@@ -45,6 +45,7 @@ void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g
 void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
                        float* copy_out, cudaStream_t s, bool pdl);
 int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, cudaStream_t s, bool pdl);
+void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, cudaStream_t s, bool pdl);
 void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int off, int n, int last, int k, cudaStream_t s);
 void launch_set_tree(SeqState* st, int seq, const int32_t* tokens, const int32_t* parents, int n, int k, int n_anchor,
                      int* err, cudaStream_t s);
@@ -59,13 +60,14 @@ void launch_gemm_simt(int dtype, int epi, int n_tiles, int batch, const void* co
 // position-canonical attention: CUDA-core bulk (+ tail/merge), or tail/merge only when the
 // tensor-core bulk kernel already produced the split partials
 int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s, bool pdl);
-// bf16, head_dim 128: the whole operator in one launch (tensor-core bulk CTAs + tail CTAs + last-arriver merge)
-int launch_attn_tree(const AttnArgs& a, int batch, int n_split_launch, int* counters, cudaStream_t s, bool pdl);
-int attn_tree_counter_ints(int batch);
+// bf16, head_dim 128: tensor-core bulk CTAs + tail CTAs in one launch, then the merge of their partials
+int launch_attn_tree(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl);
 
 // tcgen05 GEMM: a plan holds the TMA descriptors and the stream-K partition of one weight shape
 struct TcGemm;
-int tc_gemm_create(TcGemm** out, int epi, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
+// epi selects the tile -> weight-row mapping and the fused epilogue; with defer the kernel only stores partials
+// (EPI_PARTIAL) and the caller runs the matching consumer kernel
+int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
                    int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err);
 void tc_gemm_destroy(TcGemm* g);
 int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl);
