@@ -43,7 +43,9 @@ struct Buffers {
     float *rope_cos, *rope_sin;
     void* gemm_partials;
     int* gemm_counters;
+    TileSrc* sk_tables;   // [4][SK_TABLE_TILES]: QKV, O, gate/up, down (every layer has the same partition)
 };
+constexpr int SK_TABLE_TILES = 2048;
 
 
 int spec_rows(const esp_spec_cfg& s) {
@@ -128,6 +130,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.rope_sin = c.take<float>((size_t)D.cap * (D.h / 2));
     o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm));
     o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
+    o.sk_tables = c.take<TileSrc>(4 * SK_TABLE_TILES);
     return align_up(c.off, 256);
 }
 
@@ -215,7 +218,7 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
     const bool tc = h->dtype == 1 && h->gemm_impl == 0 && h->p_lm != nullptr;
     const bool pdl = h->use_pdl && !h->prof;
     StreamK pending;   // partials of the last down projection, summed by the next norm
-    pending.partials = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2;
+    pending.partials = nullptr; pending.table = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2;
     mark(h, -1);
     launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.batch, s, false);
     h->launches++;
@@ -419,27 +422,27 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
             TcGemm* p = nullptr;
             const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t r1[3] = {dq, dkv, dkv};
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, h->stream);
             h->p_qkv.push_back(p);
             const void* w2[3] = {h->wo[l], nullptr, nullptr};
             const int32_t r2[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, h->stream);
             h->p_o.push_back(p);
             const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t r3[3] = {D.F, D.F, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, h->stream);
             h->p_gu.push_back(p);
             const void* w4[3] = {h->wd[l], nullptr, nullptr};
             const int32_t r4[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, h->stream);
             h->p_down.push_back(p);
         }
         const void* w5[3] = {h->lm_head, nullptr, nullptr};
         const int32_t r5[3] = {D.V, 0, 0};
-        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err);
+        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->stream);
         if (!ok) { esp_free(h); return ESP_E_CUDA; }
     } else if (model->dtype == 1) {
         h->gemm_impl = 1;  // batched rows: CUDA-core path until the tensor-core kernel tiles over sequences
@@ -757,7 +760,7 @@ int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const
     if (cudaMemsetAsync(counters, 0, sizeof(int) * tc_gemm_counter_ints() , s) != cudaSuccess) return ESP_E_CUDA;
     if (cudaMemsetAsync(err, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
     TcGemm* plan = nullptr;
-    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err)) return ESP_E_CUDA;
+    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err, nullptr, 0, s)) return ESP_E_CUDA;
     int rc = tc_gemm_launch(plan, a, s, false);
     int e = 0;
     if (!rc && cudaMemcpyAsync(&e, err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) rc = ESP_E_CUDA;

@@ -250,7 +250,7 @@ __device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], floa
     m = mn;
 }
 
-__global__ void __launch_bounds__(128) k_attn_tree(AttnArgs a, int n_split_launch, int group, int rows_per_tile, int n_row_tiles) {
+__global__ void __launch_bounds__(128, 3) k_attn_tree(AttnArgs a, int n_split_launch, int group, int rows_per_tile, int n_row_tiles) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_T0max;
     pdl_wait();

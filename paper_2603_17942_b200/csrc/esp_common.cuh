@@ -78,8 +78,15 @@ enum Epi : int { EPI_STORE_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, 
 // ranges to G persistent CTAs; CTA c owns units [c*U/G, (c+1)*U/G).  The piece of tile t a CTA computed is
 // kept in slot min(t - first tile of the CTA, slots - 1) of that CTA:
 // partials[((cta*slots + slot)*RT + row)*TILE_N + feature].
+// `table` (device memory, one entry per tile, written once when the GEMM plan is made) lists, in CTA order,
+// the cta*slots+slot index of every piece of the tile, so consumer kernels need no partition arithmetic.
+struct TileSrc {
+    uint16_t n;        // contributors of the tile
+    uint16_t idx[15];  // their cta*slots + slot, ascending CTA
+};
 struct StreamK {
     const float* partials;  // NULL: nothing to sum
+    const TileSrc* table;
     int32_t n_tiles, KB, G, slots;
 };
 __host__ __device__ __forceinline__ long long sk_begin(long long c, long long U, long long G) { return c * U / G; }
@@ -100,6 +107,34 @@ __host__ __device__ __forceinline__ int sk_slot(const StreamK& s, int c, int til
 // address of contributor c's partial row of a tile
 __device__ __forceinline__ const float* sk_partial(const StreamK& s, int c, int tile, int row) {
     return s.partials + ((size_t)(c * s.slots + sk_slot(s, c, tile)) * RT + row) * TILE_N;
+}
+// Sum over the contributors of `tile`, in CTA order, of the four floats at column f of row r.  The loads of up
+// to eight contributors are issued before the first addition (adding the zeros of absent ones changes nothing).
+__device__ __forceinline__ float4 sk_sum4(const StreamK& s, int tile, int r, int f) {
+    const uint4* e = reinterpret_cast<const uint4*>(s.table + tile);
+    const uint4 e0 = __ldg(e), e1 = __ldg(e + 1);
+    const uint32_t w[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
+    const int n = (int)(w[0] & 0xffffu);
+    const float* base = s.partials + (size_t)r * TILE_N + f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int cb = 0; cb < 16; cb += 8) {
+        if (cb < n) {
+            float4 t[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int hw = cb + u + 1;   // halfword holding idx[cb + u]
+                t[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (hw < 16 && cb + u < n) {
+                    const uint32_t idx = (w[hw >> 1] >> ((hw & 1) * 16)) & 0xffffu;
+                    t[u] = __ldcg(reinterpret_cast<const float4*>(base + (size_t)idx * (RT * TILE_N)));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
+        }
+    }
+    return acc;
 }
 
 // Everything an epilogue may need.  One struct for all variants keeps the

@@ -316,7 +316,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
         const int et = threadIdx.x - 64;        // 0..127 index among the epilogue threads
         const int n_rows = p.a.st ? (p.a.st->active ? p.a.st->n_rows : 0) : p.a.rows_fixed;
         StreamK sk;
-        sk.partials = p.partials; sk.n_tiles = p.n_tiles; sk.KB = p.KB; sk.G = p.grid; sk.slots = p.slots;
+        sk.partials = p.partials; sk.table = nullptr; sk.n_tiles = p.n_tiles; sk.KB = p.KB; sk.G = p.grid; sk.slots = p.slots;
         bool ok = true;
         for (int i = 0; i < rng.n_seg && ok; ++i) {
             const Seg sg = get_seg(rng, i);
@@ -457,6 +457,7 @@ int make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
 
 struct TcGemm {
     TcParams p;
+    const TileSrc* table = nullptr;
 };
 
 constexpr int MAX_SLOTS = 4;
@@ -465,7 +466,8 @@ int tc_gemm_counter_ints() { return 4096; }
 int tc_gemm_tiles(const TcGemm* g) { return g ? g->p.n_tiles : 0; }
 
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
-                   int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err) {
+                   int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
+                   int table_entries, cudaStream_t stream) {
     if (!out || batch != 1 || K % 8 || n_sm < 1) return -1;
     if (reinterpret_cast<uintptr_t>(x) % 16) return -1;
     TcGemm* g = new (std::nothrow) TcGemm();
@@ -502,6 +504,27 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
         }
         if (most > MAX_SLOTS) { delete g; return -1; }
         p.slots = most < 2 ? 2 : most;
+        // contributor table for the consumer kernels
+        if (!table_dev || p.n_tiles > table_entries) { delete g; return -1; }
+        StreamK k;
+        k.partials = nullptr; k.table = nullptr; k.n_tiles = p.n_tiles; k.KB = p.KB; k.G = p.grid; k.slots = p.slots;
+        TileSrc* tab = new (std::nothrow) TileSrc[p.n_tiles];
+        if (!tab) { delete g; return -1; }
+        bool fits = true;
+        for (int t = 0; t < p.n_tiles && fits; ++t) {
+            int c0, c1;
+            sk_contributors(k, t, c0, c1);
+            if (c1 - c0 + 1 > 15 || (c1 * p.slots + p.slots) > 65535) { fits = false; break; }
+            memset(&tab[t], 0, sizeof(TileSrc));
+            tab[t].n = (uint16_t)(c1 - c0 + 1);
+            for (int c = c0; c <= c1; ++c) tab[t].idx[c - c0] = (uint16_t)(c * p.slots + sk_slot(k, c, t));
+        }
+        // stream-ordered after the caller's clearing of the workspace; pageable source: staged before the call returns
+        if (fits && cudaMemcpyAsync(table_dev, tab, sizeof(TileSrc) * p.n_tiles, cudaMemcpyHostToDevice, stream) != cudaSuccess) fits = false;
+        if (fits && cudaStreamSynchronize(stream) != cudaSuccess) fits = false;
+        delete[] tab;
+        if (!fits) { delete g; return -1; }
+        g->table = table_dev;
     }
     p.partials = reinterpret_cast<float*>(partials);
     p.counters = counters;
@@ -515,6 +538,7 @@ void tc_gemm_destroy(TcGemm* g) { delete g; }
 StreamK tc_gemm_streamk(const TcGemm* g) {
     StreamK k;
     k.partials = g ? g->p.partials : nullptr;
+    k.table = g ? g->table : nullptr;
     k.n_tiles = g ? g->p.n_tiles : 0;
     k.KB = g ? g->p.KB : 1;
     k.G = g ? g->p.grid : 1;

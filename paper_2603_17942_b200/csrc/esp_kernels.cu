@@ -76,30 +76,27 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const SeqState* states, const f
 // One block per row; with sk.partials == NULL it is a plain RMSNorm of hres.  The sum order depends only on
 // the GEMM's shape, never on the number of rows in the block.
 template <typename T>
-__global__ void __launch_bounds__(512) k_resid_norm(const SeqState* states, float* hres, StreamK sk, const T* g, T* y, int d,
-                                                   float eps, float* copy_out) {
+__global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, float* hres, StreamK sk, const T* g, T* y, int d,
+                                                    float eps, float* copy_out) {
     pdl_wait();
     if (threadIdx.x == 0) pdl_launch_dependents();
     const int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
     if (!st->active || r >= st->n_rows) return;
     float* xr = hres + (size_t)(seq * RT + r) * d;
-    __shared__ float red[16];
+    __shared__ float red[32];
+    constexpr int STRIDE = 1024 * 4;
+    float4 keep[2];
     float ss = 0.f;
-    for (int j = threadIdx.x * 4; j < d; j += 512 * 4) {
+    int it = 0;
+    for (int j = threadIdx.x * 4; j < d; j += STRIDE, ++it) {
         float4 x = *reinterpret_cast<const float4*>(xr + j);
         if (sk.partials) {
-            const int tile = j / TILE_N, f = j % TILE_N;
-            int c_first, c_last;
-            sk_contributors(sk, tile, c_first, c_last);
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int c = c_first; c <= c_last; ++c) {
-                const float4 t = __ldcg(reinterpret_cast<const float4*>(sk_partial(sk, c, tile, r) + f));
-                acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
-            }
+            const float4 acc = sk_sum4(sk, j / TILE_N, r, j % TILE_N);
             x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
             *reinterpret_cast<float4*>(xr + j) = x;
         }
+        if (it < 2) keep[it] = x;
         ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
     }
     ss = warp_sum(ss);
@@ -107,14 +104,18 @@ __global__ void __launch_bounds__(512) k_resid_norm(const SeqState* states, floa
     __syncthreads();
     float tot = 0.f;
 #pragma unroll
-    for (int w = 0; w < 16; ++w) tot += red[w];
+    for (int w = 0; w < 32; ++w) tot += red[w];
     const float rinv = 1.0f / sqrtf(tot / (float)d + eps);
     T* yr = y + (size_t)(seq * RT + r) * d;
-    for (int j = threadIdx.x * 4; j < d; j += 512 * 4) {
-        const float4 x = *reinterpret_cast<const float4*>(xr + j);   // this thread's own writes
+    it = 0;
+    for (int j = threadIdx.x * 4; j < d; j += STRIDE, ++it) {
+        const float4 x = it < 2 ? keep[it] : *reinterpret_cast<const float4*>(xr + j);   // beyond: this thread's own writes
         const float xv[4] = {x.x, x.y, x.z, x.w};
+        T o[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) yr[j + i] = from_f32<T>(xv[i] * rinv * to_f32(g[j + i]));
+        for (int i = 0; i < 4; ++i) o[i] = from_f32<T>(xv[i] * rinv * to_f32(g[j + i]));
+        if constexpr (sizeof(T) == 2) *reinterpret_cast<uint2*>(yr + j) = *reinterpret_cast<const uint2*>(o);
+        else *reinterpret_cast<float4*>(yr + j) = *reinterpret_cast<const float4*>(o);
         if (copy_out) *reinterpret_cast<float4*>(copy_out + (size_t)(seq * RT + r) * d + j) = x;
     }
 }
@@ -136,20 +137,16 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
     if (r >= n_rows || hs >= a.Hq + 2 * a.Hkv) return;
     const int j0 = hs * HD + lane * NE;          // feature in the concatenated [q | k | v] space
     const int tile = j0 / TILE_N, f = j0 % TILE_N;
-    int c_first, c_last;
-    sk_contributors(sk, tile, c_first, c_last);
     float v[NE];
+    if constexpr (NE == 4) {
+        const float4 t = sk_sum4(sk, tile, r, f);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else {
+        // narrower heads: the same sum through the four-float helper on the enclosing aligned group
+        const float4 t = sk_sum4(sk, tile, r, f & ~3);
+        const float tv[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
-    for (int i = 0; i < NE; ++i) v[i] = 0.f;
-    for (int c = c_first; c <= c_last; ++c) {
-        const float* src = sk_partial(sk, c, tile, r) + f;
-        if constexpr (NE == 4) {
-            const float4 t = __ldcg(reinterpret_cast<const float4*>(src));
-            v[0] += t.x; v[1] += t.y; v[2] += t.z; v[3] += t.w;
-        } else {
-#pragma unroll
-            for (int i = 0; i < NE; ++i) v[i] += __ldcg(src + i);
-        }
+        for (int i = 0; i < NE; ++i) v[i] = tv[(f & 3) + i];
     }
     const int which = hs < a.Hq ? 0 : (hs < a.Hq + a.Hkv ? 1 : 2);
     const int head = which == 0 ? hs : (which == 1 ? hs - a.Hq : hs - a.Hq - a.Hkv);
@@ -197,16 +194,7 @@ __global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, i
     const int j = (blockIdx.x * 256 + threadIdx.x) * 4;
     if (r >= n_rows || j >= F) return;
     const int tile = j / 64, f = j % 64;
-    int c_first, c_last;
-    sk_contributors(sk, tile, c_first, c_last);
-    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
-    for (int c = c_first; c <= c_last; ++c) {
-        const float* src = sk_partial(sk, c, tile, r);
-        const float4 tg = __ldcg(reinterpret_cast<const float4*>(src + f));
-        const float4 tu = __ldcg(reinterpret_cast<const float4*>(src + 64 + f));
-        g.x += tg.x; g.y += tg.y; g.z += tg.z; g.w += tg.w;
-        u.x += tu.x; u.y += tu.y; u.z += tu.z; u.w += tu.w;
-    }
+    const float4 g = sk_sum4(sk, tile, r, f), u = sk_sum4(sk, tile, r, 64 + f);
     const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
     __nv_bfloat16 o[4];
 #pragma unroll
@@ -511,87 +499,108 @@ int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch
 
 // ------------------------------------------------------------------ Top-K' merge over vocabulary tiles
 // One block per row: global Top-K' (value desc, id asc) of the per-tile lists, plus
-// lse = max + log(sum exp) merged over tiles in a fixed order.
-__global__ void __launch_bounds__(128) k_topk_merge(const SeqState* states, const Cand* cand, const float2* cand_ms,
-                                                    int n_tiles, int KP, int batch, Cand* topk, float* lse) {
+// lse = max + log(sum exp) merged over tiles in a fixed order.  The row's per-tile lists are staged in
+// shared memory (when they fit) so the K' selection rounds touch no global memory.
+constexpr int TOPK_THREADS = 256;
+constexpr int TOPK_MAXT = 8;   // tiles per thread (n_tiles <= 2048)
+__global__ void __launch_bounds__(TOPK_THREADS) k_topk_merge(const SeqState* states, const Cand* cand, const float2* cand_ms,
+                                                             int n_tiles, int KP, int batch, Cand* topk, float* lse, int stage) {
+    extern __shared__ __align__(16) unsigned char tk_smem[];
+    Cand* s_c = reinterpret_cast<Cand*>(tk_smem);
+    __shared__ float s_v[TOPK_THREADS];
+    __shared__ int s_i[TOPK_THREADS];
     pdl_wait();
-    const int seq = blockIdx.y, r = blockIdx.x, tid = threadIdx.x;
+    const int seq = blockIdx.y, r = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const SeqState* st = states + seq;
     if (!st->active || r >= st->n_rows) return;
     const int Mtot = batch * RT, grow = seq * RT + r;
     const bool probe = r >= st->n_nodes;
     const int kp = probe ? KP : 1;
-    __shared__ float s_v[128];
-    __shared__ int s_i[128];
-    __shared__ int s_owner;
-    // each thread keeps a cursor per tile it owns; lists are sorted, so its best remaining
-    // entry is the best head among its tiles
-    constexpr int MAXT = 16;  // tiles per thread (n_tiles <= 2048)
-    unsigned char cur[MAXT];
+    if (stage) {
+        for (int i = tid; i < n_tiles * kp; i += TOPK_THREADS) {
+            const int t = i / kp, q = i - t * kp;
+            s_c[i] = cand[((size_t)t * Mtot + grow) * KP + q];
+        }
+        __syncthreads();
+    }
+    auto entry = [&](int t, int q) -> Cand { return stage ? s_c[t * kp + q] : cand[((size_t)t * Mtot + grow) * KP + q]; };
+    unsigned char cur[TOPK_MAXT];
 #pragma unroll
-    for (int i = 0; i < MAXT; ++i) cur[i] = 0;
+    for (int i = 0; i < TOPK_MAXT; ++i) cur[i] = 0;
     for (int j = 0; j < kp; ++j) {
+        // this thread's best remaining entry: lists are sorted, so it is the best head among its tiles
         float bv = -INFINITY;
         int bi = 0x7fffffff, bt = -1;
 #pragma unroll
-        for (int i = 0; i < MAXT; ++i) {
-            int t = tid + 128 * i;
+        for (int i = 0; i < TOPK_MAXT; ++i) {
+            const int t = tid + TOPK_THREADS * i;
             if (t < n_tiles && cur[i] < kp) {
-                Cand c = cand[((size_t)t * Mtot + grow) * KP + cur[i]];
+                const Cand c = entry(t, cur[i]);
                 if (c.id >= 0 && cand_before(c.val, c.id, bv, bi)) { bv = c.val; bi = c.id; bt = i; }
             }
         }
-        s_v[tid] = bv;
-        s_i[tid] = bi;
-        __syncthreads();
-        for (int o = 64; o > 0; o >>= 1) {
-            if (tid < o && cand_before(s_v[tid + o], s_i[tid + o], s_v[tid], s_i[tid])) {
-                s_v[tid] = s_v[tid + o];
-                s_i[tid] = s_i[tid + o];
-            }
-            __syncthreads();
-        }
-        float wv = s_v[0];
-        int wi = s_i[0];
-        if (bt >= 0 && wi == bi) {
+        float wv = bv;
+        int wi = bi;
 #pragma unroll
-            for (int i = 0; i < MAXT; ++i) if (i == bt) cur[i]++;
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, wv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, wi, o);
+            if (cand_before(ov, oi, wv, wi)) { wv = ov; wi = oi; }
+        }
+        if (lane == 0) { s_v[warp] = wv; s_i[warp] = wi; }
+        __syncthreads();
+        wv = s_v[0];
+        wi = s_i[0];
+#pragma unroll
+        for (int w = 1; w < TOPK_THREADS / 32; ++w)
+            if (cand_before(s_v[w], s_i[w], wv, wi)) { wv = s_v[w]; wi = s_i[w]; }
+        if (bt >= 0 && wi == bi) {     // token ids are unique across tiles: exactly one thread owns the winner
+#pragma unroll
+            for (int i = 0; i < TOPK_MAXT; ++i) if (i == bt) cur[i]++;
         }
         if (tid == 0) { topk[(size_t)grow * KP_MAX + j].val = wv; topk[(size_t)grow * KP_MAX + j].id = wi == 0x7fffffff ? -1 : wi; }
         __syncthreads();
     }
     if (probe) {
         // thread-strided partial merges in tile order, then a fixed tree over threads
-        float m = -INFINITY, s = 0.f;
-        for (int t = tid; t < n_tiles; t += 128) {
-            float2 ms = cand_ms[(size_t)t * Mtot + grow];
-            float mn = fmaxf(m, ms.x);
-            s = s * expf(m - mn) + ms.y * expf(ms.x - mn);
+        float m = -INFINITY, sm = 0.f;
+        for (int t = tid; t < n_tiles; t += TOPK_THREADS) {
+            const float2 ms = cand_ms[(size_t)t * Mtot + grow];
+            const float mn = fmaxf(m, ms.x);
+            sm = sm * expf(m - mn) + ms.y * expf(ms.x - mn);
             m = mn;
         }
+        float* s_s = reinterpret_cast<float*>(s_i);
         s_v[tid] = m;
-        reinterpret_cast<float*>(s_i)[tid] = s;
+        s_s[tid] = sm;
         __syncthreads();
-        for (int o = 64; o > 0; o >>= 1) {
+        for (int o = TOPK_THREADS / 2; o > 0; o >>= 1) {
             if (tid < o) {
-                float m1 = s_v[tid], m2 = s_v[tid + o];
-                float s1 = reinterpret_cast<float*>(s_i)[tid], s2 = reinterpret_cast<float*>(s_i)[tid + o];
-                float mn = fmaxf(m1, m2);
-                float sn = (m1 == -INFINITY ? 0.f : s1 * expf(m1 - mn)) + (m2 == -INFINITY ? 0.f : s2 * expf(m2 - mn));
+                const float m1 = s_v[tid], m2 = s_v[tid + o];
+                const float s1 = s_s[tid], s2 = s_s[tid + o];
+                const float mn = fmaxf(m1, m2);
+                const float sn = (m1 == -INFINITY ? 0.f : s1 * expf(m1 - mn)) + (m2 == -INFINITY ? 0.f : s2 * expf(m2 - mn));
                 s_v[tid] = mn;
-                reinterpret_cast<float*>(s_i)[tid] = sn;
+                s_s[tid] = sn;
             }
             __syncthreads();
         }
-        if (tid == 0) lse[grow] = s_v[0] + logf(reinterpret_cast<float*>(s_i)[0]);
+        if (tid == 0) lse[grow] = s_v[0] + logf(s_s[0]);
     }
-    (void)s_owner;
 }
 
 void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
                        Cand* topk, float* lse, cudaStream_t s, bool pdl) {
     dim3 grid(RT, batch);
-    launch_k(k_topk_merge, grid, dim3(128), 0, s, pdl, st, cand, cand_ms, n_tiles, KP, batch, topk, lse);
+    size_t smem = (size_t)n_tiles * KP * sizeof(Cand);
+    int stage = smem <= 160 * 1024 ? 1 : 0;
+    if (!stage) smem = 0;
+    static size_t attr_bytes = 0;
+    if (smem > attr_bytes) {
+        cudaFuncSetAttribute(k_topk_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_bytes = smem;
+    }
+    launch_k(k_topk_merge, grid, dim3(TOPK_THREADS), smem, s, pdl, st, cand, cand_ms, n_tiles, KP, batch, topk, lse, stage);
 }
 
 // ------------------------------------------------------------------ row-table builders
@@ -668,10 +677,12 @@ __global__ void k_set_tree(SeqState* states, int seq, const int32_t* tokens, con
 // ------------------------------------------------------------------ the single-block tree kernel
 // verify walk -> KV compaction -> mask update -> Algorithm 1 + pruner -> next row table.
 
-__device__ __forceinline__ bool node_before(float lpa, int da, int ia, float lpb, int db, int ib) {
-    if (lpa != lpb) return lpa > lpb;
-    if (da != db) return da < db;
-    return ia < ib;
+// Total order of created nodes as one integer: (logP descending, depth ascending, creation index ascending);
+// a smaller key comes first.  -0.0 and +0.0 compare equal as floats, so both map to the key of +0.0.
+__device__ __forceinline__ unsigned long long node_key(float lp, int depth, int idx) {
+    unsigned u = __float_as_uint(lp == 0.f ? 0.f : lp);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);   // monotone: larger float -> larger u
+    return ((unsigned long long)(~u) << 32) | ((unsigned long long)depth << 16) | (unsigned long long)idx;
 }
 
 template <typename T>
@@ -685,6 +696,10 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     __shared__ int s_path[PROBES_MAX + 2], s_out[PROBES_MAX + 2];
     __shared__ int s_na, s_ustar, s_delta, s_nexp, s_ncreated, s_abort;
     __shared__ int s_exp[RT], s_sel[RT], s_new[RT];
+    __shared__ int s_rtok[RT], s_rpar[RT], s_rdep[RT], s_arg[RT];   // this step's row table and per-row argmax
+    __shared__ Cand s_list[PROBES_MAX][KP_MAX];                       // Top-K' lists of the probes the next tree uses
+    __shared__ float s_lse[PROBES_MAX];
+    unsigned long long* c_key = reinterpret_cast<unsigned long long*>(c_rank + MAX_CAND);   // total-order keys
 
     pdl_wait();
     const Dims& D = A.D;
@@ -699,6 +714,13 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
         if (tid == 0) st->L = L0 + N0;
         return;
     }
+    for (int r = tid; r < N0; r += nt) {
+        s_rtok[r] = st->row_token[r];
+        s_rpar[r] = st->row_parent[r];
+        s_rdep[r] = st->row_depth[r];
+        s_arg[r] = A.topk[(size_t)(grow0 + r) * KP_MAX].id;
+    }
+    __syncthreads();
 
     // ---- verification (Section 2): follow the model's own next token through the tree
     if (tid == 0) {
@@ -707,18 +729,18 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
         if (mode == 2) {
             cur = N0 - 1;  // last prompt token; nothing to verify, its argmax is the first generated token
             s_path[0] = cur;
-            s_out[n_emit++] = A.topk[(size_t)(grow0 + cur) * KP_MAX].id;
+            s_out[n_emit++] = s_arg[cur];
             s_ustar = cur;
             s_delta = 0;
         } else {
             cur = 0;
             s_path[0] = 0;
             for (;;) {
-                int y = A.topk[(size_t)(grow0 + cur) * KP_MAX].id;
+                int y = s_arg[cur];
                 s_out[n_emit++] = y;
                 int nxt = -1;
                 for (int c = cur + 1; c < N0; ++c)
-                    if (st->row_parent[c] == cur && st->row_token[c] == y) { nxt = c; break; }
+                    if (s_rpar[c] == cur && s_rtok[c] == y) { nxt = c; break; }
                 if (nxt < 0 || n_emit > PROBES_MAX) break;
                 cur = nxt;
                 s_path[++a] = cur;
@@ -728,7 +750,7 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
             int us = 0;
             for (int j = 0; j <= a; ++j) if (s_path[j] < nA) us = s_path[j];
             s_ustar = us;
-            s_delta = a - st->row_depth[us];
+            s_delta = a - s_rdep[us];
         }
         s_na = a;
         st->n_out = n_emit;
@@ -794,13 +816,19 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
         c_tok[0] = root_tok; c_par[0] = -1; c_dep[0] = 0; c_lp[0] = 0.f;
         s_exp[0] = 0; s_nexp = 1; s_ncreated = 1;
     }
+    // the probe lists the tree draws from, staged once
+    for (int w = tid; w < Dd * KP_MAX; w += nt) {
+        const int i = w / KP_MAX + 1, q = w % KP_MAX;
+        const int prow = mode == 2 ? N0 + (i - 1) : N0 + ustar * D.k + (delta + i - 1);
+        s_list[i - 1][q] = A.topk[(size_t)(grow0 + prow) * KP_MAX + q];
+        if (q == 0) s_lse[i - 1] = A.lse[grow0 + prow];
+    }
     __syncthreads();
     for (int i = 1; i <= Dd; ++i) {
         const int pool = min(D.K, D.B - i);
         if (pool <= 0) break;
-        const int prow = mode == 2 ? N0 + (i - 1) : N0 + ustar * D.k + (delta + i - 1);
-        const Cand* list = A.topk + (size_t)(grow0 + prow) * KP_MAX;
-        const float lse_i = A.lse[grow0 + prow];
+        const Cand* list = s_list[i - 1];
+        const float lse_i = s_lse[i - 1];
         const int base = s_ncreated, n_exp = s_nexp;
         const int n_new = n_exp * pool;
         if (base + n_new > MAX_CAND) { if (tid == 0) { set_error(A.err, DEV_E_TREE_OVERFLOW); s_abort = 1; } }
@@ -828,18 +856,15 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
             }
             c_par[c] = p;
             c_dep[c] = i;
+            c_key[c] = node_key(c_lp[c], i, c);
         }
         __syncthreads();
         const int width = D.W == 0 ? D.B - i : min(D.W, D.B - i);
         for (int w = tid; w < n_new; w += nt) {
             const int c = base + w;
-            const float lp = c_lp[c];
+            const unsigned long long key = c_key[c];   // same depth: (logP desc, creation asc)
             int rank = 0;
-            for (int o = 0; o < n_new; ++o) {
-                const int c2 = base + o;
-                const float lp2 = c_lp[c2];
-                rank += (lp2 > lp || (lp2 == lp && c2 < c)) ? 1 : 0;
-            }
+            for (int o = 0; o < n_new; ++o) rank += c_key[base + o] < key ? 1 : 0;
             if (rank < width && c_tok[c] >= 0) s_exp[rank] = c;
         }
         if (tid == 0) { s_ncreated = base + n_new; s_nexp = min(width, n_new); }
@@ -850,10 +875,9 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     for (int r = tid; r < RT; r += nt) s_sel[r] = -1;
     __syncthreads();
     for (int c = 1 + tid; c < n_created; c += nt) {
-        const float lp = c_lp[c];
-        const int dp = c_dep[c];
+        const unsigned long long key = c_key[c];
         int rank = 0;
-        for (int o = 1; o < n_created; ++o) rank += node_before(c_lp[o], c_dep[o], o, lp, dp, c) ? 1 : 0;
+        for (int o = 1; o < n_created; ++o) rank += c_key[o] < key ? 1 : 0;
         c_rank[c] = rank;
         if (rank < D.B - 1 && c_tok[c] >= 0 && rank < RT) s_sel[rank] = c;
     }
@@ -914,7 +938,7 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
 }
 
 void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s, bool pdl) {
-    size_t smem = (size_t)MAX_CAND * 20;
+    size_t smem = (size_t)MAX_CAND * 28;
     if (dtype == 0) {
         cudaFuncSetAttribute(k_tree_step<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         launch_k(k_tree_step<float>, dim3(A.D.batch), dim3(1024), smem, s, pdl, A);
@@ -947,7 +971,7 @@ void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g
 }
 void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
                        float* copy_out, cudaStream_t s, bool pdl) {
-    launch_k(k_resid_norm<__nv_bfloat16>, dim3(RT, 1), dim3(512), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
+    launch_k(k_resid_norm<__nv_bfloat16>, dim3(RT, 1), dim3(1024), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
              (__nv_bfloat16*)y, d, eps, copy_out);
 }
 void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, cudaStream_t s, bool pdl) {

@@ -68,7 +68,8 @@ struct TcGemm;
 // epi selects the tile -> weight-row mapping and the fused epilogue; with defer the kernel only stores partials
 // (EPI_PARTIAL) and the caller runs the matching consumer kernel
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
-                   int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err);
+                   int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
+                   int table_entries, cudaStream_t stream);
 void tc_gemm_destroy(TcGemm* g);
 int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl);
 StreamK tc_gemm_streamk(const TcGemm* g);
