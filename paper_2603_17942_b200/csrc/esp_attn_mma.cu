@@ -97,6 +97,11 @@ __device__ __forceinline__ void attn_bulk_chunks(const AttnArgs& a, unsigned cha
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
+    // The cache below T0 was written by earlier steps: request the first chunk before waiting for the kernel
+    // that produces this block's queries.
+    const int n_chunks = (end - beg + CHUNK - 1) / CHUNK;
+    load_chunk(0, 0);
+    pdl_wait();
     // Q fragments (A operand), straight from global memory
     uint32_t qf[HD / 16][4];
     {
@@ -123,8 +128,6 @@ __device__ __forceinline__ void attn_bulk_chunks(const AttnArgs& a, unsigned cha
     for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 
-    const int n_chunks = (end - beg + CHUNK - 1) / CHUNK;
-    load_chunk(0, 0);
     for (int c = 0; c < n_chunks; ++c) {
         const int stage = c & 1;
         if (c + 1 < n_chunks) {
@@ -253,7 +256,8 @@ __device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], floa
 __global__ void __launch_bounds__(128, 3) k_attn_tree(AttnArgs a, int n_split_launch, int group, int rows_per_tile, int n_row_tiles) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_T0max;
-    pdl_wait();
+    // Everything read before pdl_wait() -- the sequence state and the cache below T0 -- was written by earlier
+    // steps; the queries and the block's own keys/values (written by the preceding kernel) are read after it.
     if (threadIdx.x == 0) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x;                    // >= n_split_launch: the tail CTAs of the group
@@ -270,7 +274,7 @@ __global__ void __launch_bounds__(128, 3) k_attn_tree(AttnArgs a, int n_split_la
         L = a.L_fixed;
     }
     const int row0 = rtile * rows_per_tile;
-    if (row0 >= n_rows) return;
+    if (row0 >= n_rows) { pdl_wait(); return; }
     // the group needs keys up to the largest T0 of its rows (one round trip: a lane per row, then a warp max)
     if (warp == 0) {
         int t0 = 0;
@@ -286,7 +290,7 @@ __global__ void __launch_bounds__(128, 3) k_attn_tree(AttnArgs a, int n_split_la
     const int T0max = s_T0max;
     const int n_bulk = (T0max + a.split_len - 1) / a.split_len;     // bulk CTAs of this group that have keys
     const bool is_tail = split >= n_split_launch;
-    if (!is_tail && split >= n_bulk) return;
+    if (!is_tail && split >= n_bulk) { pdl_wait(); return; }
 
     const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.kc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
     const __nv_bfloat16* vbase = reinterpret_cast<const __nv_bfloat16*>(a.vc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
@@ -295,6 +299,7 @@ __global__ void __launch_bounds__(128, 3) k_attn_tree(AttnArgs a, int n_split_la
         // ---------------- tail CTA t of the group: warp w takes pairs t*8 + w*2 + {0, 1}
         float* s_q = reinterpret_cast<float*>(smem) + warp * HD;
         const int tail_cta = split - n_split_launch;
+        pdl_wait();
         for (int pi = 0; pi < PAIRS / TAIL_CTAS / 4; ++pi) {
             const int pidx = tail_cta * (PAIRS / TAIL_CTAS) + warp * (PAIRS / TAIL_CTAS / 4) + pi;
             const int r = row0 + pidx / group, head = kvh * group + pidx % group;
