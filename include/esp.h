@@ -183,6 +183,27 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
                        const void* vcache, const uint64_t* anc, const int32_t* depth, void* out, void* scratch,
                        size_t scratch_bytes, void* cuda_stream);
 
+/* esp_tree_attention for callers that cannot hand over scratch memory (the paper has no counterpart; this is
+ * a packaging variant of the operator above).  Meant for hosts that may not allocate device memory at the
+ * point of the call: a serving loop whose device memory was budgeted up front and handed to other owners, a
+ * plug-in running inside somebody else's process that must not touch the allocator, code between the
+ * begin and end of work where an allocation would stall the whole device.  The split partials live in a
+ * fixed array inside the library instead (ESP_STATIC_SCRATCH_BYTES, 16 MiB, held on every GPU that loads
+ * the library until the process exits).  Same arguments, layouts and results as esp_tree_attention, minus
+ * the scratch pair.  Returns ESP_E_WORKSPACE when the shape needs more than the array holds
+ * (esp_tree_attention_scratch_bytes(batch, n_q_heads, head_dim, cap) > ESP_STATIC_SCRATCH_BYTES; e.g. 32
+ * query heads of 128 with cap <= 2128 at batch 1 fit).  It allocates and frees nothing, on the host or the
+ * device.  The first call on each device looks up the array's device address (a one-time query, no
+ * allocation); make that first call outside any stream capture.  All calls share the one array and it keeps
+ * the previous call's contents: the entry point re-zeroes the error word it reads, everything else is
+ * overwritten before it is read.  Two calls whose kernels can overlap on the GPU (different streams, no
+ * dependency between them) would write the same partials and race: keep them ordered. */
+#define ESP_STATIC_SCRATCH_BYTES (16u << 20)
+int esp_tree_attention_static(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, int32_t cap, int32_t n_q_heads,
+                              int32_t n_kv_heads, int32_t head_dim, int32_t dcap, const void* q, const void* kcache,
+                              const void* vcache, const uint64_t* anc, const int32_t* depth, void* out,
+                              void* cuda_stream);
+
 /* y[rows][n_out] (fp32) = x[rows][k_in] (bf16) * w[n_out][k_in]^T (bf16) on the tcgen05 path
  * (impl 0) or the CUDA-core path (impl 1).  All pointers [device]; x must hold ESP_MAX_ROWS
  * rows (rows beyond `rows` are ignored); scratch as esp_gemm_scratch_bytes says. */

@@ -25,10 +25,11 @@ ERRORS = {0: "ESP_OK", -1: "ESP_E_BADCFG", -2: "ESP_E_WORKSPACE", -3: "ESP_E_PRO
 
 EXPORTS = ["esp_workspace_bytes", "esp_init", "esp_prefill", "esp_step", "esp_step_async", "esp_read", "esp_set_tree",
            "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_step_profiled", "esp_get_stats", "esp_free",
-           "esp_tree_attention_scratch_bytes", "esp_tree_attention", "esp_gemm_scratch_bytes", "esp_gemm_bf16"]
+           "esp_tree_attention_scratch_bytes", "esp_tree_attention", "esp_tree_attention_static", "esp_gemm_scratch_bytes",
+           "esp_gemm_bf16"]
 
 __all__ = ["EspError", "esp_model_cfg", "esp_spec_cfg", "esp_weights", "esp_stats", "load_library", "model_cfg",
-           "spec_cfg", "Handle", "ESP_MAX_ROWS", "ESP_MAX_PROBES", "ESP_MAX_KPRIME", "EXPORTS", "LIB_PATH", "KINDS"] + EXPORTS
+           "spec_cfg", "Handle", "ESP_MAX_ROWS", "ESP_MAX_PROBES", "ESP_MAX_KPRIME", "ESP_STATIC_SCRATCH_BYTES", "EXPORTS", "LIB_PATH", "KINDS"] + EXPORTS
 
 
 class EspError(RuntimeError):
@@ -206,6 +207,18 @@ def esp_tree_attention(dtype: int, batch: int, n_rows: int, L: int, cap: int, n_
         ctypes.c_int32(n_q_heads), ctypes.c_int32(n_kv_heads), ctypes.c_int32(head_dim), ctypes.c_int32(dcap), _vp(q),
         _vp(kcache), _vp(vcache), _vp(anc), _vp(depth), _vp(out), _vp(scratch), ctypes.c_size_t(scratch_bytes), _vp(stream)),
         "esp_tree_attention")
+
+
+ESP_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def esp_tree_attention_static(dtype: int, batch: int, n_rows: int, L: int, cap: int, n_q_heads: int, n_kv_heads: int,
+                              head_dim: int, dcap: int, q, kcache, vcache, anc, depth, out, stream=None):
+    """esp_tree_attention with the library's built-in 16 MiB scratch array: no scratch argument, no allocation."""
+    _check(load_library().esp_tree_attention_static(
+        ctypes.c_int32(dtype), ctypes.c_int32(batch), ctypes.c_int32(n_rows), ctypes.c_int32(L), ctypes.c_int32(cap),
+        ctypes.c_int32(n_q_heads), ctypes.c_int32(n_kv_heads), ctypes.c_int32(head_dim), ctypes.c_int32(dcap), _vp(q),
+        _vp(kcache), _vp(vcache), _vp(anc), _vp(depth), _vp(out), _vp(stream)), "esp_tree_attention_static")
 
 
 def esp_gemm_scratch_bytes() -> int:

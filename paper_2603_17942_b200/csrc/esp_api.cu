@@ -1,6 +1,7 @@
 // C ABI of the ESP B200 library: configuration checks, workspace carving,
 // prefill, the decode-and-verify step and the stand-alone operators.
 #include <math.h>
+#include <mutex>
 #include <new>
 #include <string.h>
 #include <vector>
@@ -724,6 +725,51 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
         return ESP_E_BADCFG;
     }
     return cuda_ok(cudaGetLastError());
+}
+
+// ---- the same operator with its scratch inside the library: nothing is allocated by anyone
+// File-scope device array; every GPU that loads the library keeps one copy until the process ends.  In host
+// code the name below is only a handle for cudaGetSymbolAddress, never a pointer a kernel may be given.
+static __device__ __align__(256) unsigned char g_static_scratch[ESP_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int STATIC_MAX_DEVICES = 64;
+void* g_static_ptr[STATIC_MAX_DEVICES];   // device address of g_static_scratch, per device, 0 until looked up
+std::mutex g_static_mutex;
+
+// Device address of the array on the current device (looked up once per device, with that device current).
+int static_scratch_ptr(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ESP_E_CUDA;
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return ESP_E_BADCFG;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return ESP_E_CUDA;
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return ESP_OK;
+}
+}  // namespace
+
+int esp_tree_attention_static(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, int32_t cap, int32_t n_q_heads,
+                              int32_t n_kv_heads, int32_t head_dim, int32_t dcap, const void* q, const void* kcache,
+                              const void* vcache, const uint64_t* anc, const int32_t* depth, void* out,
+                              void* cuda_stream) {
+    size_t need = 0;
+    int rc = esp_tree_attention_scratch_bytes(batch, n_q_heads, head_dim, cap, &need);
+    if (rc) return rc;
+    if (need > (size_t)ESP_STATIC_SCRATCH_BYTES) return ESP_E_WORKSPACE;   // shape beyond the built-in array
+    void* scratch = nullptr;
+    rc = static_scratch_ptr(&scratch);
+    if (rc) return rc;
+    // the array still holds the previous call's bytes: the error word (last 256 bytes of the used part) must
+    // start at zero; the partials are written by this call before they are read
+    if (cudaMemsetAsync(reinterpret_cast<char*>(scratch) + need - 256, 0, 256, reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return ESP_E_CUDA;
+    return esp_tree_attention(dtype, batch, n_rows, L, cap, n_q_heads, n_kv_heads, head_dim, dcap, q, kcache, vcache, anc,
+                              depth, out, scratch, need, cuda_stream);
 }
 
 int esp_gemm_scratch_bytes(size_t* bytes_out) {
