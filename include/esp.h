@@ -152,8 +152,10 @@ int esp_debug_set_gemm(esp_handle* h, int32_t impl);
 
 /* Measurement hook (no counterpart in the paper): one esp_step with a CUDA event recorded on the handle's
  * stream after every kernel group; ms_by_kind [host] [8] receives the device time per group in this order:
- * 0 row assembly + RMSNorm, 1 QKV GEMM, 2 tree attention, 3 O GEMM, 4 gate/up GEMM, 5 down GEMM,
- * 6 LM-head GEMM with fused selection, 7 Top-K' merge + tree kernel.  tokens_out / n_out as esp_step. */
+ * 0 row assembly, RMSNorm and the kernels that sum GEMM partials (residual add + norm, RoPE + cache write,
+ * SiLU*up), 1 QKV GEMM, 2 tree attention, 3 O GEMM, 4 gate/up GEMM, 5 down GEMM, 6 LM-head GEMM with fused
+ * selection, 7 Top-K' merge + tree kernel.  The kernels run back to back without overlap in this mode, so the
+ * groups add up to more than an unprofiled step.  tokens_out / n_out as esp_step. */
 int esp_step_profiled(esp_handle* h, float* ms_by_kind, int32_t* tokens_out, int32_t* n_out);
 
 int esp_get_stats(esp_handle* h, esp_stats* out);

@@ -173,7 +173,7 @@ def esp_debug_set_gemm(h, impl: int):
     _check(load_library().esp_debug_set_gemm(h, ctypes.c_int32(impl)), "esp_debug_set_gemm")
 
 
-KINDS = ("norm_assemble", "qkv_gemm", "tree_attention", "o_gemm", "gateup_gemm", "down_gemm", "lmhead_topk", "select_tree")
+KINDS = ("norm_and_partial_consumers", "qkv_gemm", "tree_attention", "o_gemm", "gateup_gemm", "down_gemm", "lmhead_topk", "select_tree")
 
 
 def esp_step_profiled(h, tokens_out: np.ndarray, n_out: np.ndarray) -> Dict[str, float]:

@@ -239,11 +239,12 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             const int32_t rows[3] = {dq, dkv, dkv};
             int rc = run_gemm(h, tc ? h->p_qkv[l] : nullptr, EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a, tc, pdl);
             if (rc) return rc;
+            mark(h, KIND_QKV);
             if (tc) {
                 if (launch_qkv_finish(a, tc_gemm_streamk(h->p_qkv[l]), s, pdl)) return ESP_E_BADCFG;
                 h->launches++;
+                mark(h, KIND_MISC);
             }
-            mark(h, KIND_QKV);
         }
         {
             AttnArgs a;
@@ -288,11 +289,12 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             const int32_t rows[3] = {D.F, D.F, 0};
             int rc = run_gemm(h, tc ? h->p_gu[l] : nullptr, EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a, tc, pdl);
             if (rc) return rc;
+            mark(h, KIND_GATEUP);
             if (tc) {
                 launch_swiglu_finish(b.states, tc_gemm_streamk(h->p_gu[l]), b.act, D.F, s, pdl);
                 h->launches++;
+                mark(h, KIND_MISC);
             }
-            mark(h, KIND_GATEUP);
         }
         {
             EpiArgs a = base_epi(h, D.d);
