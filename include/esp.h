@@ -98,12 +98,17 @@ typedef struct esp_handle esp_handle;
 
 /* Bytes of [device] workspace esp_init needs (KV cache for max_batch sequences of
  * max_seq_len + ESP_MAX_ROWS positions, activations, split-K and attention
- * partials, per-sequence state).  ESP_E_BADCFG if the configuration is unsupported. */
+ * partials, per-sequence state and -- for bf16 models with max_batch 1 -- a copy of
+ * every layer matrix and of the LM head repacked into the 16 KB blocks the GEMM
+ * main loop streams, i.e. about the size of the model again).
+ * ESP_E_BADCFG if the configuration is unsupported. */
 int esp_workspace_bytes(const esp_model_cfg* model, const esp_spec_cfg* spec, size_t* bytes_out);
 
 /* Create a handle.  `workspace` [device] must be 256-byte aligned and at least
  * esp_workspace_bytes large; it is zeroed here.  `cuda_stream` is a cudaStream_t
- * (NULL = default stream).  Builds the rotary table and TMA descriptors.
+ * (NULL = default stream).  Builds the rotary table, the TMA descriptors and the repacked
+ * weight copy (the caller's matrices are still read by the CUDA-core path and the embedding
+ * gather, so they must stay alive).
  * The frozen model is the f_theta of Section 2. */
 int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_weights* weights, void* workspace,
              size_t workspace_bytes, void* cuda_stream, esp_handle** handle_out);

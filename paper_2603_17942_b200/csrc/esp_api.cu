@@ -45,6 +45,9 @@ struct Buffers {
     void* gemm_partials;
     int* gemm_counters;
     TileSrc* sk_tables;   // [4][SK_TABLE_TILES]: QKV, O, gate/up, down (every layer has the same partition)
+    // weights repacked for streaming (bf16 models, one sequence): per layer [qkv | o | gate/up | down], then the LM head
+    char* packed;
+    size_t pk_qkv, pk_o, pk_gu, pk_down, pk_lm, pk_layer;
 };
 constexpr int SK_TABLE_TILES = 2048;
 
@@ -132,6 +135,19 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm));
     o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
     o.sk_tables = c.take<TileSrc>(4 * SK_TABLE_TILES);
+    o.packed = nullptr;
+    o.pk_qkv = o.pk_o = o.pk_gu = o.pk_down = o.pk_lm = o.pk_layer = 0;
+    if (dtype == 1 && D.batch == 1) {
+        const int32_t dq = D.Hq * D.h, dkv = D.Hkv * D.h;
+        const int32_t r1[3] = {dq, dkv, dkv}, r2[3] = {D.d, 0, 0}, r3[3] = {D.F, D.F, 0}, r5[3] = {D.V, 0, 0};
+        o.pk_qkv = tc_gemm_packed_bytes(EPI_PARTIAL, r1, D.d);
+        o.pk_o = tc_gemm_packed_bytes(EPI_PARTIAL, r2, dq);
+        o.pk_gu = tc_gemm_packed_bytes(EPI_SWIGLU, r3, D.d);
+        o.pk_down = tc_gemm_packed_bytes(EPI_PARTIAL, r2, D.F);
+        o.pk_lm = tc_gemm_packed_bytes(EPI_LOGITS, r5, D.d);
+        o.pk_layer = o.pk_qkv + o.pk_o + o.pk_gu + o.pk_down;
+        o.packed = c.take<char>(o.pk_layer * D.n_layers + o.pk_lm);
+    }
     return align_up(c.off, 256);
 }
 
@@ -423,29 +439,30 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
         bool ok = true;
         for (int l = 0; l < D.n_layers && ok; ++l) {
             TcGemm* p = nullptr;
+            char* pk = h->b.packed + h->b.pk_layer * l;
             const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t r1[3] = {dq, dkv, dkv};
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream);
             h->p_qkv.push_back(p);
             const void* w2[3] = {h->wo[l], nullptr, nullptr};
             const int32_t r2[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream);
             h->p_o.push_back(p);
             const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t r3[3] = {D.F, D.F, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream);
             h->p_gu.push_back(p);
             const void* w4[3] = {h->wd[l], nullptr, nullptr};
             const int32_t r4[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream);
             h->p_down.push_back(p);
         }
         const void* w5[3] = {h->lm_head, nullptr, nullptr};
         const int32_t r5[3] = {D.V, 0, 0};
-        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->stream);
+        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
         if (!ok) { esp_free(h); return ESP_E_CUDA; }
     } else if (model->dtype == 1) {
         h->gemm_impl = 1;  // batched rows: CUDA-core path until the tensor-core kernel tiles over sequences
@@ -808,7 +825,7 @@ int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const
     if (cudaMemsetAsync(counters, 0, sizeof(int) * tc_gemm_counter_ints() , s) != cudaSuccess) return ESP_E_CUDA;
     if (cudaMemsetAsync(err, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
     TcGemm* plan = nullptr;
-    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err, nullptr, 0, s)) return ESP_E_CUDA;
+    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err, nullptr, 0, nullptr, s)) return ESP_E_CUDA;
     int rc = tc_gemm_launch(plan, a, s, false);
     int e = 0;
     if (!rc && cudaMemcpyAsync(&e, err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) rc = ESP_E_CUDA;

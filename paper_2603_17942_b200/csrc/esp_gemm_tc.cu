@@ -54,6 +54,7 @@ struct TcParams {
     int32_t n_tiles, KB, grid, epi;
     int32_t map_swiglu;  // tile = 64 rows of w[0] (gate) + the matching 64 rows of w[1] (up)
     int32_t slots;       // partial slots per CTA
+    const unsigned char* a_packed;  // weights repacked per (tile, k-block) unit, or NULL: read w[] through map_a
     float* partials;   // [grid][slots][RT][TILE_N]
     int* counters;     // [n_tiles], zero between launches
     int* err;
@@ -105,6 +106,14 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
+
+// one contiguous 16 KB unit of repacked weights (already in the swizzled shared-memory layout)
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
 
@@ -249,8 +258,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                         unsigned char* sa = stages + it * STAGE_BYTES;
                         if (pass == 0) {
                             mbar_expect_tx(&full[it], STAGE_BYTES);
-                            tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[it], pol_w);
-                            tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it], pol_w);
+                            if (p.a_packed) {
+                                bulk_load(sa, p.a_packed + ((size_t)sg.tile * p.KB + kb) * A_BYTES, A_BYTES, &full[it], pol_w);
+                            } else {
+                                tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[it], pol_w);
+                                tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it], pol_w);
+                            }
                         } else {
                             tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[it], pol_x);
                         }
@@ -271,8 +284,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                         if (!mbar_wait(&empty[stage], phase ^ 1, s_abort)) { ok = false; break; }
                         unsigned char* sa = stages + stage * STAGE_BYTES;
                         mbar_expect_tx(&full[stage], STAGE_BYTES);
-                        tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[stage], pol_w);
-                        tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage], pol_w);
+                        if (p.a_packed) {
+                            bulk_load(sa, p.a_packed + ((size_t)sg.tile * p.KB + kb) * A_BYTES, A_BYTES, &full[stage], pol_w);
+                        } else {
+                            tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[stage], pol_w);
+                            tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage], pol_w);
+                        }
                         tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[stage], pol_x);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -422,6 +439,35 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
     }
 }
 
+// Repack of the weights for streaming: unit (tile, k-block) = the 128 x 64 bf16 block the main loop consumes per
+// stage, stored contiguously (16 KB) in the 128-byte-swizzled layout the MMA descriptor expects, rows and columns
+// outside the matrices zero.  One block per unit, thread r copies row r.
+struct PackArgs {
+    const __nv_bfloat16* w[3];
+    int32_t rows_w[3];
+    int32_t K, KB, map_swiglu;
+};
+__global__ void __launch_bounds__(128) k_pack_weights(PackArgs g, unsigned char* out) {
+    const long long unit = blockIdx.x;
+    const int tile = (int)(unit / g.KB), kb = (int)(unit % g.KB), r = threadIdx.x;
+    int m, row;
+    if (g.map_swiglu) { m = r >> 6; row = tile * 64 + (r & 63); }
+    else {
+        row = tile * TILE_N + r;
+        m = 0;
+        while (m < 2 && row >= g.rows_w[m]) { row -= g.rows_w[m]; ++m; }
+    }
+    const bool row_ok = g.w[m] != nullptr && row < g.rows_w[m];
+    unsigned char* dst = out + (size_t)unit * A_BYTES + r * 128;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int k0 = kb * BK + j * 8;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (row_ok && k0 < g.K) v = *reinterpret_cast<const uint4*>(g.w[m] + (size_t)row * g.K + k0);
+        *reinterpret_cast<uint4*>(dst + ((j ^ (r & 7)) << 4)) = v;
+    }
+}
+
 constexpr size_t SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + sizeof(float) * (RT * ACC_LD + RT * 4) + 256;
 
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -463,11 +509,16 @@ struct TcGemm {
 constexpr int MAX_SLOTS = 4;
 size_t tc_gemm_partial_bytes(int n_sm) { return (size_t)n_sm * MAX_SLOTS * RT * TILE_N * sizeof(float); }
 int tc_gemm_counter_ints() { return 4096; }
+size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K) {
+    const long long total = (long long)rows_w[0] + rows_w[1] + rows_w[2];
+    const long long n_tiles = epi == EPI_SWIGLU ? (rows_w[0] + 63) / 64 : (total + TILE_N - 1) / TILE_N;
+    return (size_t)(n_tiles * ((K + BK - 1) / BK)) * A_BYTES;
+}
 int tc_gemm_tiles(const TcGemm* g) { return g ? g->p.n_tiles : 0; }
 
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
                    int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
-                   int table_entries, cudaStream_t stream) {
+                   int table_entries, void* packed, cudaStream_t stream) {
     if (!out || batch != 1 || K % 8 || n_sm < 1) return -1;
     if (reinterpret_cast<uintptr_t>(x) % 16) return -1;
     TcGemm* g = new (std::nothrow) TcGemm();
@@ -525,6 +576,14 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
         delete[] tab;
         if (!fits) { delete g; return -1; }
         g->table = table_dev;
+    }
+    if (packed) {
+        PackArgs pa;
+        for (int i = 0; i < 3; ++i) { pa.w[i] = reinterpret_cast<const __nv_bfloat16*>(w[i]); pa.rows_w[i] = rows_w[i]; }
+        pa.K = K; pa.KB = p.KB; pa.map_swiglu = p.map_swiglu;
+        k_pack_weights<<<(unsigned)U, 128, 0, stream>>>(pa, reinterpret_cast<unsigned char*>(packed));
+        if (cudaGetLastError() != cudaSuccess) { delete g; return -1; }
+        p.a_packed = reinterpret_cast<const unsigned char*>(packed);
     }
     p.partials = reinterpret_cast<float*>(partials);
     p.counters = counters;

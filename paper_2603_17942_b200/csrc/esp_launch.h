@@ -69,7 +69,9 @@ struct TcGemm;
 // (EPI_PARTIAL) and the caller runs the matching consumer kernel
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
                    int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
-                   int table_entries, cudaStream_t stream);
+                   int table_entries, void* packed, cudaStream_t stream);
+// bytes of the repacked copy of a weight set (tc_gemm_create's `packed`; NULL there = stream the caller's matrices)
+size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K);
 void tc_gemm_destroy(TcGemm* g);
 int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl);
 StreamK tc_gemm_streamk(const TcGemm* g);

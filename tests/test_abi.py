@@ -37,7 +37,8 @@ def test_workspace_bytes_and_config_checks(lib):
     s = P.spec_cfg(n_probes=4, topk=10, max_nodes=64, expand_width=0, n_anchor=1)
     nbytes = P.esp_workspace_bytes(m, s)
     kv = 2 * 32 * 8 * (1296 + P.ESP_MAX_ROWS) * 128 * 2
-    assert kv < nbytes < kv + (1 << 30)
+    packed = synth.LLAMA3_8B.n_params_streamed() * 2       # the streaming copy of every layer matrix and the LM head
+    assert kv + packed <= nbytes < kv + packed + (1 << 30)
     # the paper's operating points fit: k=1 with a 30-node tree, k=2 with a 20-node tree (60 rows each)
     for k, B in ((1, 30), (2, 20)):
         P.esp_workspace_bytes(m, P.spec_cfg(n_probes=k, topk=14, max_nodes=B, n_anchor=0))
