@@ -385,19 +385,84 @@ def run_ours(args, shape, plen, k, K, B):
         dist.destroy_process_group()
 
 
+def run_attention_op(args):
+    """Tree-attention operator alone (32 query / 8 KV heads of 128, KV length 4096, a 64-node random tree of
+    depth <= 5 plus 4 mask-probe rows, N(0,1) bf16 cache), batch 1 and batch 16: device time per call, achieved
+    KV bytes/s and FLOP/s.  Between timed calls a 512 MB buffer is rewritten so the cache is read from HBM."""
+    import torch
+    import synth
+    import paper_2603_17942_b200 as P
+    from paper_2603_17942_b200 import build as esp_build
+    esp_build.build()
+    torch.cuda.set_device(0)
+    R, Hq, Hkv, h, L, n_nodes, n_probes = P.ESP_MAX_ROWS, 32, 8, 128, args.prompt_len or 4096, 64, 4
+    M = n_nodes + n_probes
+    peak, peak_src = measured_peaks()
+    flush = torch.zeros(512 << 20, dtype=torch.uint8, device="cuda")
+    results = {}
+    for batch in (1, 16):
+        cap = L + R
+        q, kc, vc, kb, vb = synth.random_qkv((batch, R, Hq, h), (batch, Hkv, cap, h), (batch, Hkv, M, h), seed=batch, device="cuda")
+        kc[:, :, L:L + M] = kb
+        vc[:, :, L:L + M] = vb
+        anc = np.zeros((batch, R, 2), np.uint64)
+        depth = np.zeros((batch, R), np.int32)
+        for s in range(batch):
+            vis, pos = random_block(n_nodes, n_probes, 10 * batch + s)
+            depth[s, :M] = pos
+            for r in range(M):
+                for i in np.nonzero(vis[r])[0]:
+                    anc[s, r, i // 64] |= np.uint64(1) << np.uint64(i % 64)
+            for r in range(M, R):
+                anc[s, r, r // 64] = np.uint64(1) << np.uint64(r % 64)
+        anc_d, depth_d = torch.from_numpy(anc.view(np.int64)).cuda(), torch.from_numpy(depth).cuda()
+        out = torch.zeros_like(q)
+        nb = P.esp_tree_attention_scratch_bytes(batch, Hq, h, cap)
+        scratch = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+        times = []
+        for it in range(args.warmup + args.steps):
+            flush.add_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            P.esp_tree_attention(1, batch, M, L, cap, Hq, Hkv, h, 16, q, kc, vc, anc_d, depth_d, out, scratch, nb,
+                                 torch.cuda.current_stream().cuda_stream)
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                times.append(e0.elapsed_time(e1) * 1e3)
+        us = float(np.median(times))
+        kv_bytes = batch * Hkv * (L + M) * h * 2 * 2
+        flops = 4.0 * batch * M * Hq * (L + 6) * h          # QK^T and PV over the cache and a row's own path
+        results[f"b{batch}"] = {"us": us, "kv_bytes": kv_bytes, "achieved_GBs": kv_bytes / us / 1e3,
+                                "frac_of_hbm_peak": kv_bytes / us / 1e3 / peak, "achieved_TFLOPs": flops / us / 1e6}
+    line = {"metric": "tree_attention_us", "value": results["b16"]["us"], "unit": "us", "n_gpus": 1, "steps": args.steps,
+            "warmup": args.warmup, "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"tree-attention operator, 32/8 heads x 128, KV {L}, 64-node tree + 4 probes, batch 1 and 16",
+                       "l2": "512 MB buffer rewritten between calls"},
+            "results": results, "peak_GBs": peak, "peak_source": peak_src, "gpu_launches": 2 * args.steps}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="llama3-8b", choices=sorted(WORKLOADS))
+    ap.add_argument("--config", default="llama3-8b", choices=sorted(WORKLOADS) + ["attention-op"])
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt / KV length")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer count (smaller captures under a profiler)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-greedy", action="store_true", help="skip the greedy-decoding leg")
     args = ap.parse_args()
     import synth
+    if args.config == "attention-op":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_attention_op(args)
+        return
     name, plen, k, K, B = WORKLOADS[args.config]
+    if args.prompt_len > 0:
+        plen = args.prompt_len
     shape = getattr(synth, name)
     if args.layers > 0:
         shape = shape.replace(n_layers=args.layers)

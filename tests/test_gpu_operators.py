@@ -163,3 +163,24 @@ def test_tree_attention_rows_equal_decoding_each_path_alone():
             anc1[0, i, i // 64] = np.uint64(1) << np.uint64(i % 64)
         alone = _run_attention(1, q1, kc1, vc1, anc1, np.zeros((1, R), np.int32), 1, L + d, Hq, Hkv, h)
         assert torch.equal(alone[0, 0], tree_out[0, r]), f"row {r} (depth {d})"
+
+
+def test_tree_attention_long_context_against_oracle():
+    """KV length 32768 (the longest context of the batch sweep): 128 splits of 256... become 64 of 512; every
+    row and head against the oracle."""
+    Hq, Hkv, h, n_nodes, n_probes, L = 32, 8, 128, 64, 4, 32768
+    M = n_nodes + n_probes
+    cap = L + R
+    q, kc, vc, kb, vb = synth.random_qkv((1, R, Hq, h), (1, Hkv, cap, h), (1, Hkv, M, h), seed=3, device="cuda")
+    kc[:, :, L:L + M] = kb
+    vc[:, :, L:L + M] = vb
+    _, d, vis = _tree_block(n_nodes, n_probes, 5, seed=5)
+    depth = np.zeros((1, R), np.int32)
+    depth[0, :M] = d
+    out = _run_attention(1, q, kc, vc, _anc_words(vis)[None], depth, M, L, Hq, Hkv, h)
+    ref = O.tree_attention(q[0, :M].float().cpu().numpy(), kc[0, :, :L].float().permute(1, 0, 2).cpu().numpy(),
+                           vc[0, :, :L].float().permute(1, 0, 2).cpu().numpy(), kb[0].float().permute(1, 0, 2).cpu().numpy(),
+                           vb[0].float().permute(1, 0, 2).cpu().numpy(), vis)
+    got = out[0, :M].float().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= 2e-2
