@@ -91,7 +91,7 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
         D->cap = m->max_seq_len + RT;
         D->batch = m->max_batch;
         int S = 256;
-        while ((m->max_seq_len + S - 1) / S > 64) S *= 2;
+        while ((m->max_seq_len + S - 1) / S > 32) S *= 2;   // at most 32 splits: the partials stay small next to the cache
         D->split_len = S;
         D->n_split_max = (m->max_seq_len + S - 1) / S + 1;
         D->rms_eps = m->rms_eps;
@@ -163,6 +163,7 @@ struct esp_handle {
     const void *embed, *lm_head, *final_norm;
     std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, na, nf, qn, kn;
     std::vector<TcGemm*> p_qkv, p_o, p_gu, p_down;
+    std::vector<AttnTc*> p_attn;   // per layer, bf16 models with head_dim 128
     TcGemm* p_lm = nullptr;
     std::vector<int> L_host, ready;
     int32_t* pinned = nullptr;  // [batch][RING] + 4 ints (error words)
@@ -275,10 +276,10 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             a.dcap = dcap;
             a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
             a.err = b.err;
-            const bool mma = h->dtype == 1 && D.h == 128 && h->gemm_impl == 0;
+            const bool mma = h->gemm_impl == 0 && !h->p_attn.empty();
             if (mma) {
-                if (launch_attn_tree(a, D.batch, n_split_launch, s, pdl)) return ESP_E_BADCFG;
-                h->launches += 2;
+                if (attn_tc_launch(h->p_attn[l], a, D.batch, n_split_launch, s, pdl)) return ESP_E_BADCFG;
+                h->launches += n_split_launch > 0 ? 2 : 1;
             } else {
                 if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, true, s, pdl)) return ESP_E_BADCFG;
                 h->launches += n_split_launch > 0 ? 2 : 1;
@@ -434,6 +435,14 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
         return ESP_E_CUDA;
     }
     launch_rope_table(h->b.rope_cos, h->b.rope_sin, D.cap, D.h, model->rope_base, h->stream);
+    if (model->dtype == 1 && attn_tc_supported(D.h, D.Hq, D.Hkv)) {
+        for (int l = 0; l < D.n_layers; ++l) {
+            AttnTc* t = nullptr;
+            if (attn_tc_create(&t, h->b.qbuf, layer_ptr(h->b.kcache, h->layer_kv_stride, l), layer_ptr(h->b.vcache, h->layer_kv_stride, l),
+                               D.batch, D.Hq, D.Hkv, D.cap)) { esp_free(h); return ESP_E_CUDA; }
+            h->p_attn.push_back(t);
+        }
+    }
     if (model->dtype == 1 && D.batch == 1) {
         const int dq = D.Hq * D.h, dkv = D.Hkv * D.h;
         bool ok = true;
@@ -690,6 +699,7 @@ void esp_free(esp_handle* h) {
     for (auto* p : h->p_gu) tc_gemm_destroy(p);
     for (auto* p : h->p_down) tc_gemm_destroy(p);
     tc_gemm_destroy(h->p_lm);
+    for (auto* t : h->p_attn) attn_tc_destroy(t);
     if (h->pinned) cudaFreeHost(h->pinned);
     drop_graphs(h);
     for (auto e : h->ev) cudaEventDestroy(e);
@@ -700,7 +710,7 @@ void esp_free(esp_handle* h) {
 int esp_tree_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t cap, size_t* bytes_out) {
     if (!bytes_out || batch < 1 || n_q_heads < 1 || cap < RT) return ESP_E_ARG;
     int S = 256;
-    while ((cap + S - 1) / S > 64) S *= 2;
+    while ((cap + S - 1) / S > 32) S *= 2;
     const size_t ns = (cap + S - 1) / S + 1;
     const size_t rows = (size_t)batch * RT * n_q_heads * ns;
     *bytes_out = align_up(rows * head_dim * sizeof(float), 256) + align_up(rows * sizeof(float2), 256) + 256;
@@ -720,7 +730,7 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     esp_tree_attention_scratch_bytes(batch, n_q_heads, head_dim, cap, &need);
     if (scratch_bytes < need || reinterpret_cast<uintptr_t>(scratch) % 256) return ESP_E_WORKSPACE;
     int S = 256;
-    while ((cap + S - 1) / S > 64) S *= 2;
+    while ((cap + S - 1) / S > 32) S *= 2;
     const size_t ns = (cap + S - 1) / S + 1;
     const size_t rows = (size_t)batch * RT * n_q_heads * ns;
     AttnArgs a;
@@ -737,9 +747,13 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     a.err = reinterpret_cast<int*>(reinterpret_cast<char*>(scratch) + need - 256);
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
     const int n_split_launch = (L + S - 1) / S;
-    const bool mma = dtype == 1 && head_dim == 128;
+    const bool mma = dtype == 1 && attn_tc_supported(head_dim, n_q_heads, n_kv_heads);
     if (mma) {
-        if (launch_attn_tree(a, batch, n_split_launch, s, false)) return ESP_E_BADCFG;
+        AttnTc* t = nullptr;
+        if (attn_tc_create(&t, q, kcache, vcache, batch, n_q_heads, n_kv_heads, cap)) return ESP_E_CUDA;
+        const int rc = attn_tc_launch(t, a, batch, n_split_launch, s, false);   // the descriptors travel by value
+        attn_tc_destroy(t);
+        if (rc) return ESP_E_BADCFG;
     } else if (launch_attn_simt(dtype, a, batch, n_split_launch, true, s, false)) {
         return ESP_E_BADCFG;
     }

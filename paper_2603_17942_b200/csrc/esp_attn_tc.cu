@@ -1,0 +1,676 @@
+// Tree attention for bf16, head_dim 128, on the Blackwell tensor cores.
+//
+// A row at position P = L + depth attends to cache positions 0..P.  Positions
+// below T0 = floor((P - dcap)/16)*16 are always cache resident, whatever the
+// tree looks like; they are summed by the "bulk" kernel here.  The remaining
+// <= dcap+16 positions -- the end of the cache and the row's in-flight tree
+// ancestors, found through its ancestor bitmask -- are summed key by key in
+// position order by the tail+merge kernel, which also merges the bulk
+// partials (split order, tail last) and writes the output.  Every reduction
+// order is a function of absolute positions only, so a token verified inside a
+// tree block gets the bits it would get decoded alone.
+//
+// Bulk kernel (k_attn_bulk_tc): one CTA per (split of the cache, KV head, tile
+// of 128 (row, query head) pairs).  The KV cache of the split is streamed once
+// through shared memory by TMA in chunks of 128 keys and shared by all pairs:
+//   S = Q K^T   tcgen05.mma, Q (128 pairs x 128 dims) and the K chunk both
+//               K-major in shared memory, S (128 x 128 fp32) in tensor memory;
+//   softmax     128 threads, one per pair (= tensor-memory lane): mask by the
+//               row's T0, running max / sum in the log2 domain, P as bf16 into
+//               shared memory in the A-operand layout;
+//   O += P V    tcgen05.mma with V as the MN-major B operand (the cache keeps
+//               values as [key][dim]); O (128 x 128 fp32) stays in tensor
+//               memory and is rescaled there when the running max moves.
+// Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 softmax.  S and the
+// K/V stages are double buffered, so Q K^T of chunk c+1 overlaps the softmax of
+// chunk c.  Every mbarrier wait is bounded; on a timeout the kernel records
+// DEV_E_WAIT_TIMEOUT, frees its tensor memory and returns.
+#include <cuda.h>
+#include <new>
+#include <string.h>
+
+#include "esp_launch.h"
+
+namespace esp {
+
+namespace {
+
+constexpr int HD = 128;
+constexpr int CK = 128;                   // keys per chunk
+constexpr int MP = 128;                   // (row, head) pairs per CTA
+constexpr int HALF_BYTES = 128 * 128;     // one 128-row x 64-element (128-byte) swizzled tile
+constexpr int Q_BYTES = 2 * HALF_BYTES, K_BYTES = 2 * HALF_BYTES, V_BYTES = 2 * HALF_BYTES, P_BYTES = 2 * HALF_BYTES;
+constexpr int KV_STAGE = K_BYTES + V_BYTES;
+constexpr int OFF_Q = 0, OFF_KV = Q_BYTES, OFF_P = OFF_KV + 2 * KV_STAGE, OFF_BAR = OFF_P + P_BYTES;
+constexpr size_t SMEM_BYTES = 1024 + OFF_BAR + 256;
+constexpr int TMEM_COLS = 512;            // S0 at 0, S1 at 128, O at 256
+constexpr int NUM_THREADS = 192;
+constexpr unsigned long long WAIT_LIMIT_NS = 50ull * 1000 * 1000;   // 50 ms
+
+struct BulkParams {
+    CUtensorMap map_q;   // [batch*RT][Hq][128], box 64 x group x rows_per_tile
+    CUtensorMap map_k;   // [batch*Hkv*cap][128], box 64 x 128 keys
+    CUtensorMap map_v;
+    AttnArgs a;
+    int32_t group, rows_per_tile, n_row_tiles;
+};
+
+__device__ __forceinline__ int tail_start_tc(int P, int dcap) {
+    int t = P - dcap;
+    return t <= 0 ? 0 : (t / 16) * 16;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait: gives up after WAIT_LIMIT_NS of wall time (a try_wait may itself block for a while, so the
+// bound is on the clock, not on the number of polls) or as soon as another role has given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    const uint32_t addr = smem_u32(bar);
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((it & 15u) == 15u) {
+            if (*abort_flag) return false;
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024 bytes apart.
+// K-major operands use lbo = 1 (ignored); the MN-major operand (V) gives the distance between its two
+// 64-element column blocks as lbo.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)(lbo_bytes >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// kind::f16 instruction descriptors: D = f32, A = B = bf16, M = 128, N = 128; PV takes B (V) MN-major
+constexpr uint32_t IDESC_QK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+constexpr uint32_t IDESC_PV = IDESC_QK | (1u << 16);
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+// a whole 128-column row of this lane: four loads in flight, one wait
+__device__ __forceinline__ void tmem_ld128(uint32_t taddr, uint32_t (&r)[128]) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b) tmem_ld32_issue(taddr + b * 32, &r[b * 32]);
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_constant__ BulkParams p) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ int s_T0max;
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);   // [2]
+    uint64_t* kv_empty = kv_full + 2;                                  // [2]
+    uint64_t* s_full = kv_empty + 2;                                   // [2]
+    uint64_t* q_full = s_full + 2;
+    uint64_t* p_ready = q_full + 1;
+    uint64_t* pv_done = p_ready + 1;
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(pv_done + 1);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+    const AttnArgs& a = p.a;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int split = blockIdx.x;
+    const int kvh = blockIdx.y / p.n_row_tiles, rtile = blockIdx.y % p.n_row_tiles;
+    const int seq = blockIdx.z;
+
+    // Read before pdl_wait(): the sequence state and the cache below T0, both written by earlier steps.
+    if (threadIdx.x == 0) pdl_launch_dependents();
+    int n_rows, L;
+    if (a.st) {
+        const SeqState* st = a.st + seq;
+        n_rows = st->active ? st->n_rows : 0;
+        L = st->L;
+    } else {
+        n_rows = a.n_rows_fixed;
+        L = a.L_fixed;
+    }
+    const int row0 = rtile * p.rows_per_tile;
+    if (row0 >= n_rows) { pdl_wait(); return; }
+    if (warp == 2) {
+        int t0 = 0;
+        for (int r = row0 + lane; r < row0 + p.rows_per_tile && r < n_rows; r += 32) {
+            const int depth = a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r];
+            t0 = max(t0, tail_start_tc(L + depth, a.dcap));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t0 = max(t0, __shfl_xor_sync(0xffffffffu, t0, o));
+        if (lane == 0) s_T0max = t0;
+    }
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); mbar_init(&s_full[i], 1); }
+        mbar_init(q_full, 1);
+        mbar_init(p_ready, 128);
+        mbar_init(pv_done, 1);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int T0max = s_T0max;
+    const int n_bulk = (T0max + a.split_len - 1) / a.split_len;
+    if (split >= n_bulk) { pdl_wait(); return; }     // block-uniform: nobody holds tensor memory yet
+    const int beg = split * a.split_len;
+    const int end = min(beg + a.split_len, T0max);
+    const int n_chunks = (end - beg + CK - 1) / CK;
+
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *s_tmem;
+    unsigned char* sQ = smem + OFF_Q;
+    unsigned char* sP = smem + OFF_P;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            const int kvrow0 = (seq * a.Hkv + kvh) * a.cap + beg;
+            bool ok = true;
+            auto load_chunk = [&](int c) {
+                unsigned char* st = smem + OFF_KV + (c & 1) * KV_STAGE;
+                mbar_expect_tx(&kv_full[c & 1], KV_STAGE);
+                tma_load_2d(st, &p.map_k, 0, kvrow0 + c * CK, &kv_full[c & 1]);
+                tma_load_2d(st + HALF_BYTES, &p.map_k, 64, kvrow0 + c * CK, &kv_full[c & 1]);
+                tma_load_2d(st + K_BYTES, &p.map_v, 0, kvrow0 + c * CK, &kv_full[c & 1]);
+                tma_load_2d(st + K_BYTES + HALF_BYTES, &p.map_v, 64, kvrow0 + c * CK, &kv_full[c & 1]);
+            };
+            for (int c = 0; c < n_chunks && c < 2; ++c) load_chunk(c);
+            pdl_wait();     // the queries come from the kernel before this one
+            mbar_expect_tx(q_full, Q_BYTES);
+            tma_load_3d(sQ, &p.map_q, 0, kvh * p.group, seq * RT + row0, q_full);
+            tma_load_3d(sQ + HALF_BYTES, &p.map_q, 64, kvh * p.group, seq * RT + row0, q_full);
+            for (int c = 2; c < n_chunks && ok; ++c) {
+                if (!mbar_wait(&kv_empty[c & 1], ((c >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                load_chunk(c);
+            }
+            if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
+            auto issue_qk = [&](int c) {
+                const uint32_t k_addr = smem_u32(smem + OFF_KV + (c & 1) * KV_STAGE);
+                const uint32_t tmem_s = tmem_base + (c & 1) * 128;
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+                    umma(tmem_s, smem_desc(q_addr + off, 16), smem_desc(k_addr + off, 16), IDESC_QK, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(&s_full[c & 1]);
+            };
+            ok = mbar_wait(q_full, 0, s_abort) && mbar_wait(&kv_full[0], 0, s_abort);
+            if (ok) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                issue_qk(0);
+            }
+            for (int c = 0; c < n_chunks && ok; ++c) {
+                if (c + 1 < n_chunks) {     // S of the next chunk while the softmax of this one runs
+                    if (!mbar_wait(&kv_full[(c + 1) & 1], ((c + 1) >> 1) & 1, s_abort)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    issue_qk(c + 1);
+                }
+                if (!mbar_wait(p_ready, c & 1, s_abort)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t v_addr = smem_u32(smem + OFF_KV + (c & 1) * KV_STAGE + K_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < CK / 16; ++kk) {
+                    const uint32_t p_off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;     // P: K-major over keys
+                    const uint32_t v_off = kk * 16 * 128;                              // V: 16 key rows of 128 bytes further
+                    umma(tmem_base + 256, smem_desc(p_addr + p_off, 16), smem_desc(v_addr + v_off, HALF_BYTES), IDESC_PV,
+                         (c > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(pv_done);
+                umma_commit(&kv_empty[c & 1]);
+            }
+            if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
+        }
+    } else {
+        // ---------------- softmax warps: thread = pair = tensor-memory lane
+        const int q4 = warp & 3;
+        const int pair = q4 * 32 + lane;
+        const int r = row0 + pair / p.group, head = kvh * p.group + pair % p.group;
+        const bool pv = pair / p.group < p.rows_per_tile && r < n_rows && r < RT;
+        int T0row = 0;
+        if (pv) T0row = tail_start_tc(L + (a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r]), a.dcap);
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int c = 0; c < n_chunks && ok; ++c) {
+            // (a wait that fails must take the whole warp out: the tensor-memory accesses below are warp-wide)
+            if (!__all_sync(0xffffffffu, mbar_wait(&s_full[c & 1], (c >> 1) & 1, s_abort))) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t s_addr = lane_addr + (c & 1) * 128;
+            const int cbase = beg + c * CK;
+            // the row's 128 scores, masked to its visible keys and scaled to the log2 domain
+            uint32_t sv[128];
+            tmem_ld128(s_addr, sv);
+            float cmax = -INFINITY;
+            if (__all_sync(0xffffffffu, cbase + CK <= T0row)) {     // the whole chunk is visible to every row of the warp
+#pragma unroll
+                for (int i = 0; i < 128; ++i) {
+                    const float s = __uint_as_float(sv[i]) * a.scale_log2;
+                    sv[i] = __float_as_uint(s);
+                    cmax = fmaxf(cmax, s);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 128; ++i) {
+                    const float s = cbase + i < T0row ? __uint_as_float(sv[i]) * a.scale_log2 : -INFINITY;
+                    sv[i] = __float_as_uint(s);
+                    cmax = fmaxf(cmax, s);
+                }
+            }
+            const float m_new = fmaxf(m_run, cmax);
+            const float m_use = m_new == -INFINITY ? 0.f : m_new;
+            const float alpha = exp2f(m_run - m_use);
+            // P of the previous chunk must have been consumed before it is overwritten, and O must be final
+            // before it is rescaled
+            if (c > 0 && !__all_sync(0xffffffffu, mbar_wait(pv_done, (c - 1) & 1, s_abort))) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // probabilities, their sum (key order), P as bf16 in the A-operand layout
+            float csum = 0.f;
+#pragma unroll
+            for (int blk = 0; blk < 4; ++blk) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float p0 = exp2f(__uint_as_float(sv[blk * 32 + i]) - m_use), p1 = exp2f(__uint_as_float(sv[blk * 32 + i + 1]) - m_use);
+                    csum += p0;
+                    csum += p1;
+                    const __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&b);
+                }
+                unsigned char* prow = sP + (blk >> 1) * HALF_BYTES + pair * 128;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int chunk16 = (blk & 1) * 4 + j;
+                    *reinterpret_cast<uint4*>(prow + ((chunk16 ^ (pair & 7)) << 4)) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                }
+            }
+            if (c > 0) {
+                // O <- alpha * O (in tensor memory)
+                if (__any_sync(0xffffffffu, alpha != 1.0f)) {   // warp-uniform: skip when no lane's maximum moved
+                    tmem_ld128(lane_addr + 256, sv);
+#pragma unroll
+                    for (int blk = 0; blk < 4; ++blk) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) sv[blk * 32 + i] = __float_as_uint(__uint_as_float(sv[blk * 32 + i]) * alpha);
+                        tmem_st32(lane_addr + 256 + blk * 32, *reinterpret_cast<const uint32_t(*)[32]>(&sv[blk * 32]));
+                    }
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                }
+            }
+            l_run = l_run * alpha + csum;
+            m_run = m_new;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes -> tensor-core reads
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(p_ready);
+        }
+        if (ok && !__all_sync(0xffffffffu, mbar_wait(pv_done, (n_chunks - 1) & 1, s_abort))) ok = false;
+        if (ok) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // O row -> shared memory (the K/V stages are free now) -> one 512-byte bulk copy per pair.  The
+            // tensor-memory load is warp-wide: every lane takes part, lanes without a pair copy nothing.
+            uint32_t ov[128];
+            tmem_ld128(lane_addr + 256, ov);
+            float* orow = reinterpret_cast<float*>(smem + OFF_KV) + pair * (HD + 4);   // rows padded by 16 bytes: no bank conflicts
+#pragma unroll
+            for (int i = 0; i < 128; i += 4)
+                *reinterpret_cast<uint4*>(orow + i) = make_uint4(ov[i], ov[i + 1], ov[i + 2], ov[i + 3]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (pv) {
+                const size_t idx = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max + split;
+                a.part_ml[idx] = make_float2(m_run, l_run);
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                             ::"l"(a.part_o + idx * HD), "r"(smem_u32(orow)), "r"(HD * 4) : "memory");
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");        // copies complete: shared memory may be released
+        } else if (lane == 0) {
+            set_error(a.err, DEV_E_WAIT_TIMEOUT);
+            *s_abort = 1;
+        }
+    }
+    // ---------------- teardown (every thread arrives here)
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (*s_abort) {
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);   // let copies in flight land before shared memory goes away
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- tail + merge: one warp per (row, head) pair
+__device__ __forceinline__ int nth_set_bit128(unsigned long long lo, unsigned long long hi, int n) {
+    int c = __popcll(lo);
+    unsigned long long m = lo;
+    int base = 0;
+    if (n >= c) { n -= c; m = hi; base = 64; }
+    for (int i = 0; i < n; ++i) m &= m - 1;
+    return m ? base + __ffsll((long long)m) - 1 : -1;
+}
+__device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], float cm, float cl, const float (&co)[4]) {
+    const float mn = fmaxf(m, cm);
+    const float a = exp2f(m - mn), b = exp2f(cm - mn);
+    l = l * a + cl * b;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) o[i] = o[i] * a + co[i] * b;
+    m = mn;
+}
+
+// The tail: positions T0..P in position order, lane j owns key j of a 32-key chunk (chunk grid anchored at T0).
+// Then the merge: bulk partials in split order, the tail last; a lane owns 4 of the 128 output dims.
+__global__ void __launch_bounds__(128) k_attn_tail_merge_tc(AttnArgs a) {
+    __shared__ float s_qall[4][HD];
+    if (threadIdx.x == 0) pdl_launch_dependents();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 4 + warp, head = blockIdx.y, seq = blockIdx.z;
+    // the sequence state was written by an earlier step; everything else is read after the wait
+    int n_rows, L, depth = 0;
+    unsigned long long lo = 0, hi = 0;
+    if (a.st) {
+        const SeqState* st = a.st + seq;
+        n_rows = st->active ? st->n_rows : 0;
+        L = st->L;
+        if (r < n_rows) { depth = st->row_depth[r]; lo = st->row_anc[r][0]; hi = st->row_anc[r][1]; }
+    } else {
+        n_rows = a.n_rows_fixed;
+        L = a.L_fixed;
+        if (r < n_rows) { depth = a.depth[seq * RT + r]; lo = a.anc[(size_t)(seq * RT + r) * 2]; hi = a.anc[(size_t)(seq * RT + r) * 2 + 1]; }
+    }
+    pdl_wait();
+    if (r >= n_rows) return;
+    const int kvh = head / (a.Hq / a.Hkv);
+    const int P = L + depth, T0 = tail_start_tc(P, a.dcap);
+    const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.kc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
+    const __nv_bfloat16* vbase = reinterpret_cast<const __nv_bfloat16*>(a.vc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
+    const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((size_t)(seq * RT + r) * a.Hq + head) * HD;
+    float* s_q = s_qall[warp];
+    {
+        const uint2 qq = *reinterpret_cast<const uint2*>(q + lane * 4);
+        const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qq.x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qq.y);
+        s_q[lane * 4 + 0] = __low2float(q01); s_q[lane * 4 + 1] = __high2float(q01);
+        s_q[lane * 4 + 2] = __low2float(q23); s_q[lane * 4 + 3] = __high2float(q23);
+    }
+    __syncwarp();
+    // bulk partials: request the first eight now, they are summed after the tail is done
+    const int n_sp = (T0 + a.split_len - 1) / a.split_len;
+    const size_t base = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max;
+    float2 ml0[8];
+    float4 c40[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        if (u < n_sp) {
+            ml0[u] = __ldcg(a.part_ml + base + u);
+            c40[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (base + u) * HD + lane * 4));
+        }
+    }
+    // ---- tail
+    float tm = -INFINITY, tl = 0.f, to[4] = {0.f, 0.f, 0.f, 0.f};
+    const int n_tail = P - T0 + 1;
+    for (int t0 = 0; t0 < n_tail; t0 += 32) {
+        const int t = t0 + lane;
+        bool valid = t < n_tail;
+        int slot = 0;
+        if (valid) {
+            const int pos = T0 + t;
+            if (pos < L) slot = pos;
+            else {
+                const int b = nth_set_bit128(lo, hi, pos - L);
+                if (b < 0) { set_error(a.err, DEV_E_INDEX); valid = false; }
+                else slot = L + b;
+            }
+        }
+        float sc = -INFINITY;
+        if (valid) {
+            const uint4* kr = reinterpret_cast<const uint4*>(kbase + (size_t)slot * HD);
+            uint4 kreg[HD / 8];
+#pragma unroll
+            for (int d8 = 0; d8 < HD / 8; ++d8) kreg[d8] = kr[d8];
+            float acc = 0.f;
+#pragma unroll
+            for (int d8 = 0; d8 < HD / 8; ++d8) {
+                const uint4 kk = kreg[d8];
+                const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kk);
+                const float4 qa = *reinterpret_cast<const float4*>(s_q + d8 * 8), qb = *reinterpret_cast<const float4*>(s_q + d8 * 8 + 4);
+                acc = fmaf(qa.x, __low2float(k2[0]), acc); acc = fmaf(qa.y, __high2float(k2[0]), acc);
+                acc = fmaf(qa.z, __low2float(k2[1]), acc); acc = fmaf(qa.w, __high2float(k2[1]), acc);
+                acc = fmaf(qb.x, __low2float(k2[2]), acc); acc = fmaf(qb.y, __high2float(k2[2]), acc);
+                acc = fmaf(qb.z, __low2float(k2[3]), acc); acc = fmaf(qb.w, __high2float(k2[3]), acc);
+            }
+            sc = acc * a.scale_log2;
+        }
+        float cm = sc;
+#pragma unroll
+        for (int of = 16; of > 0; of >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, of));
+        const float pe = valid ? exp2f(sc - cm) : 0.f;
+        float cl = pe;
+#pragma unroll
+        for (int of = 16; of > 0; of >>= 1) cl += __shfl_xor_sync(0xffffffffu, cl, of);
+        float co[4] = {0.f, 0.f, 0.f, 0.f};
+        // weighted values, keys in position order; the loads of 16 keys are issued before their sums
+        // (a key that is not in the chunk reads slot 0 with weight 0 and is skipped)
+        for (int j0 = 0; j0 < 32; j0 += 16) {
+            float pj[16];
+            uint2 vv[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                pj[u] = __shfl_sync(0xffffffffu, pe, j0 + u);
+                const int sj = __shfl_sync(0xffffffffu, slot, j0 + u);
+                vv[u] = *reinterpret_cast<const uint2*>(vbase + (size_t)sj * HD + lane * 4);
+            }
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                if (pj[u] != 0.f) {
+                    const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vv[u].x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vv[u].y);
+                    co[0] = fmaf(pj[u], __low2float(v01), co[0]); co[1] = fmaf(pj[u], __high2float(v01), co[1]);
+                    co[2] = fmaf(pj[u], __low2float(v23), co[2]); co[3] = fmaf(pj[u], __high2float(v23), co[3]);
+                }
+            }
+        }
+        merge_ml(tm, tl, to, cm, cl, co);
+    }
+    // ---- merge: splits in order, then the tail
+    float m = -INFINITY, l = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        if (u < n_sp) {
+            const float co[4] = {c40[u].x, c40[u].y, c40[u].z, c40[u].w};
+            merge_ml(m, l, o, ml0[u].x, ml0[u].y, co);
+        }
+    }
+    for (int s0 = 8; s0 < n_sp; s0 += 8) {
+        float2 ml[8];
+        float4 c4[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (s0 + u < n_sp) {
+                ml[u] = __ldcg(a.part_ml + base + s0 + u);
+                c4[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (base + s0 + u) * HD + lane * 4));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (s0 + u < n_sp) {
+                const float co[4] = {c4[u].x, c4[u].y, c4[u].z, c4[u].w};
+                merge_ml(m, l, o, ml[u].x, ml[u].y, co);
+            }
+        }
+    }
+    merge_ml(m, l, o, tm, tl, to);
+    const float inv = 1.0f / l;
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out) + ((size_t)(seq * RT + r) * a.Hq + head) * HD + lane * 4;
+    const __nv_bfloat162 o01 = __floats2bfloat162_rn(o[0] * inv, o[1] * inv), o23 = __floats2bfloat162_rn(o[2] * inv, o[3] * inv);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&o01);
+    pk.y = *reinterpret_cast<const uint32_t*>(&o23);
+    *reinterpret_cast<uint2*>(out) = pk;
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn get_encode() {
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) return nullptr;
+        fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+}  // namespace
+
+struct AttnTc {
+    BulkParams p;
+};
+
+bool attn_tc_supported(int h, int Hq, int Hkv) {
+    if (h != HD || Hkv < 1 || Hq % Hkv) return false;
+    const int group = Hq / Hkv;
+    return group <= MP && MP % group == 0 && group <= 256;
+}
+
+// TMA descriptors of one layer's query buffer [batch*RT][Hq][128] and KV cache [batch*Hkv*cap][128] (bf16).
+int attn_tc_create(AttnTc** out, const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap) {
+    if (!out || !attn_tc_supported(HD, Hq, Hkv)) return -1;
+    EncodeFn enc = get_encode();
+    if (!enc) return -1;
+    AttnTc* t = new (std::nothrow) AttnTc();
+    if (!t) return -1;
+    memset(&t->p, 0, sizeof(t->p));
+    const int group = Hq / Hkv, rows_per_tile = MP / group;
+    t->p.group = group;
+    t->p.rows_per_tile = rows_per_tile;
+    t->p.n_row_tiles = (RT + rows_per_tile - 1) / rows_per_tile;
+    const cuuint32_t estr3[3] = {1, 1, 1};
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)HD, (cuuint64_t)Hq, (cuuint64_t)batch * RT};
+        cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)Hq * HD * 2};
+        cuuint32_t box[3] = {64, (cuuint32_t)group, (cuuint32_t)rows_per_tile};
+        if (enc(&t->p.map_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, estr3,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) { delete t; return -1; }
+    }
+    for (int i = 0; i < 2; ++i) {
+        cuuint64_t dims[2] = {(cuuint64_t)HD, (cuuint64_t)batch * Hkv * cap};
+        cuuint64_t strides[1] = {(cuuint64_t)HD * 2};
+        cuuint32_t box[2] = {64, (cuuint32_t)CK};
+        if (enc(i ? &t->p.map_v : &t->p.map_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(i ? vcache : kcache), dims,
+                strides, box, estr3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) { delete t; return -1; }
+    }
+    *out = t;
+    return 0;
+}
+
+void attn_tc_destroy(AttnTc* t) { delete t; }
+
+// Two launches: the bulk kernel (grid = splits x (KV heads x row tiles) x sequences), then tail + merge.
+int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl) {
+    if (!t || n_split_launch + 1 > a.n_split_max || a.split_len % CK) return -1;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(k_attn_bulk_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return -1;
+        attr_set = true;
+    }
+    BulkParams p = t->p;
+    p.a = a;
+    if (n_split_launch > 0) {
+        dim3 grid(n_split_launch, a.Hkv * p.n_row_tiles, batch);
+        if (launch_k(k_attn_bulk_tc, grid, dim3(NUM_THREADS), SMEM_BYTES, s, pdl, p) != cudaSuccess) return -1;
+    }
+    if (launch_k(k_attn_tail_merge_tc, dim3((RT + 3) / 4, a.Hq, batch), dim3(128), 0, s, pdl, a) != cudaSuccess) return -1;
+    return 0;
+}
+
+}  // namespace esp

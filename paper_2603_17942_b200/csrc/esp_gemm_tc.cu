@@ -45,7 +45,7 @@ constexpr int B_BYTES = RT * BK * 2;         // 10240
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 256;               // two accumulator buffers of 128 columns
 constexpr int NUM_THREADS = 192;
-constexpr uint32_t WAIT_LIMIT = 1u << 20;
+constexpr unsigned long long WAIT_LIMIT_NS = 50ull * 1000 * 1000;   // 50 ms
 
 struct TcParams {
     CUtensorMap map_a[3];
@@ -72,10 +72,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Bounded wait; false if it ran out (or another role already gave up).
+// Bounded wait: gives up after WAIT_LIMIT_NS of wall time (a try_wait may itself block for a while, so the
+// bound is on the clock, not on the number of polls) or as soon as another role has given up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -85,9 +87,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             : "r"(addr), "r"(parity)
             : "memory");
         if (done) return true;
-        if ((it & 1023u) == 1023u && *abort_flag) return false;
+        if ((it & 15u) == 15u) {
+            if (*abort_flag) return false;
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) return false;
+        }
     }
-    return false;
 }
 
 // L2 eviction policies: weights are read once per step and never again before the whole model has streamed

@@ -60,8 +60,13 @@ void launch_gemm_simt(int dtype, int epi, int n_tiles, int batch, const void* co
 // position-canonical attention: CUDA-core bulk (+ tail/merge), or tail/merge only when the
 // tensor-core bulk kernel already produced the split partials
 int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch, bool bulk_too, cudaStream_t s, bool pdl);
-// bf16, head_dim 128: tensor-core bulk CTAs + tail CTAs in one launch, then the merge of their partials
-int launch_attn_tree(const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl);
+// bf16, head_dim 128: tcgen05 bulk kernel over the cache below each row's T0, then tail + merge (esp_attn_tc.cu).
+// A plan holds the TMA descriptors of one query buffer and one layer's KV cache.
+struct AttnTc;
+bool attn_tc_supported(int h, int Hq, int Hkv);
+int attn_tc_create(AttnTc** out, const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap);
+void attn_tc_destroy(AttnTc* t);
+int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl);
 
 // tcgen05 GEMM: a plan holds the TMA descriptors and the stream-K partition of one weight shape
 struct TcGemm;

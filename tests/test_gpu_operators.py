@@ -166,7 +166,7 @@ def test_tree_attention_rows_equal_decoding_each_path_alone():
 
 
 def test_tree_attention_long_context_against_oracle():
-    """KV length 32768 (the longest context of the batch sweep): 128 splits of 256... become 64 of 512; every
+    """KV length 32768 (the longest context of the batch sweep): the cache is cut in 32 splits of 1024; every
     row and head against the oracle."""
     Hq, Hkv, h, n_nodes, n_probes, L = 32, 8, 128, 64, 4, 32768
     M = n_nodes + n_probes
