@@ -697,6 +697,7 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     __shared__ int s_na, s_ustar, s_delta, s_nexp, s_ncreated, s_abort;
     __shared__ int s_exp[RT], s_sel[RT], s_new[RT];
     __shared__ int s_rtok[RT], s_rpar[RT], s_rdep[RT], s_arg[RT];   // this step's row table and per-row argmax
+    __shared__ int s_keep[PROBES_MAX * RT], s_nkeep;                  // per depth, the B-1 best nodes: the only ones the final pick can take
     __shared__ Cand s_list[PROBES_MAX][KP_MAX];                       // Top-K' lists of the probes the next tree uses
     __shared__ float s_lse[PROBES_MAX];
     unsigned long long* c_key = reinterpret_cast<unsigned long long*>(c_rank + MAX_CAND);   // total-order keys
@@ -814,7 +815,7 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     const int Dd = D.k - delta > 0 ? D.k - delta : 0;
     if (tid == 0) {
         c_tok[0] = root_tok; c_par[0] = -1; c_dep[0] = 0; c_lp[0] = 0.f;
-        s_exp[0] = 0; s_nexp = 1; s_ncreated = 1;
+        s_exp[0] = 0; s_nexp = 1; s_ncreated = 1; s_nkeep = 0;
     }
     // the probe lists the tree draws from, staged once
     for (int w = tid; w < Dd * KP_MAX; w += nt) {
@@ -866,23 +867,27 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
             int rank = 0;
             for (int o = 0; o < n_new; ++o) rank += c_key[base + o] < key ? 1 : 0;
             if (rank < width && c_tok[c] >= 0) s_exp[rank] = c;
+            // a node with B-1 or more nodes of its own depth before it cannot be among the B-1 best overall
+            if (rank < D.B - 1 && rank < RT) s_keep[atomicAdd(&s_nkeep, 1)] = c;
         }
         if (tid == 0) { s_ncreated = base + n_new; s_nexp = min(width, n_new); }
         __syncthreads();
     }
     // final selection: root + the B-1 best created nodes by (logP desc, depth asc, creation asc)
-    const int n_created = s_ncreated;
+    // (ranked among the kept nodes only: every node that precedes one of the B-1 best is itself kept)
+    const int n_keep = s_nkeep;
     for (int r = tid; r < RT; r += nt) s_sel[r] = -1;
     __syncthreads();
-    for (int c = 1 + tid; c < n_created; c += nt) {
+    for (int w = tid; w < n_keep; w += nt) {
+        const int c = s_keep[w];
         const unsigned long long key = c_key[c];
         int rank = 0;
-        for (int o = 1; o < n_created; ++o) rank += c_key[o] < key ? 1 : 0;
+        for (int o = 0; o < n_keep; ++o) rank += c_key[s_keep[o]] < key ? 1 : 0;
         c_rank[c] = rank;
         if (rank < D.B - 1 && c_tok[c] >= 0 && rank < RT) s_sel[rank] = c;
     }
     __syncthreads();
-    int n_sel = min(D.B - 1, n_created - 1);
+    int n_sel = min(D.B - 1, n_keep);
     // (entries with token -1 rank last because their logP is -inf; drop them)
     if (tid == 0) {
         int n = 0;
