@@ -65,6 +65,11 @@ typedef struct {
     int32_t prune_root;    /* also drop a candidate equal to the last generated token */
     int32_t ema_per_token; /* mask update per emitted token (1) or once per step (0) */
     float lambda;          /* mask update rate, Eq. (mask_update_mean); 0.1 in the paper */
+    /* Static tree (Section 4.2, "[K_1, .., K_k]"): when static_widths[0] > 0 the tree is not grown by
+     * Algorithm 1; instead the Top-1 node of depth i-1 gets the first static_widths[i-1] candidates of
+     * probe i (after the pruner), for as many depths as there are non-zero widths.  topk, max_nodes and
+     * expand_width are then ignored (the tree has 1 + sum of widths nodes). */
+    int32_t static_widths[ESP_MAX_PROBES];
 } esp_spec_cfg;
 
 /* Model weights. [device] matrices; the per-layer members are [host] arrays of

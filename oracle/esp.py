@@ -189,11 +189,13 @@ class SpecCfg:
     prune_root: bool = False
     ema_per_token: bool = True
     lam: float = 0.1
+    static_widths: Tuple[int, ...] = ()   # fixed branch widths [K_1..K_k] (Section 4.2); empty = dynamic tree
 
     @property
     def k_prime(self) -> int:
         """Entries kept per probe so the list refills to K after pruning ("next best candidate")."""
-        return self.topk + int(self.prune_parent) + int(self.prune_root)
+        k = max(self.static_widths) if self.static_widths else self.topk
+        return k + int(self.prune_parent) + int(self.prune_root)
 
 
 def mask_init_mean(E_rows: np.ndarray) -> np.ndarray:
@@ -425,6 +427,13 @@ def call_reduction_percent(tau: float) -> float:
     return 100.0 * (1.0 - 1.0 / tau)
 
 
+def next_tree(root_token: int, cand_ids, cand_logits, lses, spec: SpecCfg) -> Tree:
+    """The tree the next step verifies: Algorithm 1, or the fixed-width tree when spec.static_widths is set."""
+    if spec.static_widths:
+        return build_static_tree(root_token, cand_ids, spec.static_widths, spec)
+    return build_tree(root_token, cand_ids, cand_logits, lses, spec)
+
+
 def block_complexity(k: int, widths: Sequence[int]) -> int:
     """BC = (k+1) (1 + sum_i K_i) (Section 3.3)."""
     return (k + 1) * (1 + int(sum(widths)))
@@ -490,7 +499,7 @@ class EspOracle:
         if not sp.ema_per_token:
             self.m = mask_update(self.m, self.model.embed(y), sp.lam)
         ids, vals, lses = self._probe_lists(logits, range(t, t + k))
-        self.tree = build_tree(y, ids, vals, lses, sp) if k else root_only(y)
+        self.tree = next_tree(y, ids, vals, lses, sp) if k else root_only(y)
         if self.keep_logits:
             self.log.append({"kind": "prefill", "logits": logits[t - 1:].copy(), "first": y})
         return y
@@ -529,7 +538,7 @@ class EspOracle:
         if self.keep_logits:
             rec["logits"] = logits
         self.log.append(rec)
-        self.tree = build_tree(out[-1], ids, vals, lses, sp) if k else root_only(out[-1])
+        self.tree = next_tree(out[-1], ids, vals, lses, sp) if k else root_only(out[-1])
         self.steps += 1
         self.accept_hist.append(a)
         return out

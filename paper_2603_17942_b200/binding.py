@@ -47,7 +47,8 @@ class esp_model_cfg(ctypes.Structure):
 
 class esp_spec_cfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("n_probes", "topk", "max_nodes", "expand_width", "n_anchor",
-                                              "prune_parent", "prune_root", "ema_per_token")] + [("lam", ctypes.c_float)]
+                                              "prune_parent", "prune_root", "ema_per_token")] + [("lam", ctypes.c_float)] + \
+               [("static_widths", ctypes.c_int32 * ESP_MAX_PROBES)]
 
 
 _PP = ctypes.POINTER(ctypes.c_void_p)
@@ -107,9 +108,10 @@ def model_cfg(shape, max_seq_len: int, max_batch: int = 1) -> esp_model_cfg:
 
 
 def spec_cfg(n_probes=0, topk=1, max_nodes=1, expand_width=1, n_anchor=0, prune_parent=True, prune_root=False,
-             ema_per_token=True, lam=0.1) -> esp_spec_cfg:
+             ema_per_token=True, lam=0.1, static_widths=()) -> esp_spec_cfg:
+    widths = (ctypes.c_int32 * ESP_MAX_PROBES)(*[int(w) for w in static_widths])
     return esp_spec_cfg(n_probes, topk, max_nodes, expand_width, n_anchor, int(prune_parent), int(prune_root),
-                        int(ema_per_token), float(lam))
+                        int(ema_per_token), float(lam), widths)
 
 
 # ---------------------------------------------------------------- raw calls (same names as the header)

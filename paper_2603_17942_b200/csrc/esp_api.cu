@@ -52,9 +52,27 @@ struct Buffers {
 constexpr int SK_TABLE_TILES = 2048;
 
 
+// tree nodes including the root: max_nodes, or 1 + the fixed widths of a static tree
+int spec_nodes(const esp_spec_cfg& s) {
+    if (s.n_probes > 0 && s.static_widths[0] > 0) {
+        int n = 1;
+        for (int i = 0; i < s.n_probes && i < PROBES_MAX && s.static_widths[i] > 0; ++i) n += s.static_widths[i];
+        return n;
+    }
+    return s.max_nodes;
+}
+int spec_topk(const esp_spec_cfg& s) {
+    if (s.n_probes > 0 && s.static_widths[0] > 0) {
+        int m = 0;
+        for (int i = 0; i < s.n_probes && i < PROBES_MAX && s.static_widths[i] > 0; ++i) m = s.static_widths[i] > m ? s.static_widths[i] : m;
+        return m;
+    }
+    return s.topk;
+}
 int spec_rows(const esp_spec_cfg& s) {
-    int nA = s.n_probes > 0 ? (s.n_anchor == 0 ? s.max_nodes : (s.n_anchor < s.max_nodes ? s.n_anchor : s.max_nodes)) : 0;
-    return s.max_nodes + s.n_probes * nA;
+    const int B = spec_nodes(s);
+    int nA = s.n_probes > 0 ? (s.n_anchor == 0 ? B : (s.n_anchor < B ? s.n_anchor : B)) : 0;
+    return B + s.n_probes * nA;
 }
 
 int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
@@ -69,14 +87,18 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
     if (m->max_batch < 1 || m->max_seq_len < 1) return ESP_E_BADCFG;
     if (s->n_probes < 0 || s->n_probes > PROBES_MAX) return ESP_E_BADCFG;
     if (s->max_nodes < 1) return ESP_E_BADCFG;
-    const int KP = s->topk + (s->prune_parent ? 1 : 0) + (s->prune_root ? 1 : 0);
-    if (s->n_probes > 0 && (s->topk < 1 || KP > KP_MAX || KP > m->vocab)) return ESP_E_BADCFG;
+    const bool is_static = s->n_probes > 0 && s->static_widths[0] > 0;
+    for (int i = 0; i < PROBES_MAX; ++i)
+        if (s->static_widths[i] < 0 || (i > 0 && s->static_widths[i] > 0 && s->static_widths[i - 1] == 0)) return ESP_E_BADCFG;
+    const int topk = spec_topk(*s), n_nodes = spec_nodes(*s);
+    const int KP = topk + (s->prune_parent ? 1 : 0) + (s->prune_root ? 1 : 0);
+    if (s->n_probes > 0 && (topk < 1 || KP > KP_MAX || KP > m->vocab)) return ESP_E_BADCFG;
     if (spec_rows(*s) > RT) return ESP_E_BADCFG;
     if (2 * s->n_probes > DCAP_STEP) return ESP_E_BADCFG;
     if (s->expand_width < 0 || s->n_anchor < 0) return ESP_E_BADCFG;
     // Algorithm 1 must not create more than MAX_CAND nodes
     long created = 1, n_exp = 1;
-    for (int i = 1; i <= s->n_probes; ++i) {
+    for (int i = 1; i <= s->n_probes && !is_static; ++i) {
         long pool = s->topk < s->max_nodes - i ? s->topk : s->max_nodes - i;
         if (pool <= 0) break;
         long n_new = n_exp * pool;
@@ -95,7 +117,8 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
         D->split_len = S;
         D->n_split_max = (m->max_seq_len + S - 1) / S + 1;
         D->rms_eps = m->rms_eps;
-        D->k = s->n_probes; D->K = s->topk; D->KP = s->n_probes > 0 ? KP : 1; D->B = s->max_nodes; D->W = s->expand_width;
+        D->k = s->n_probes; D->K = topk; D->KP = s->n_probes > 0 ? KP : 1; D->B = n_nodes; D->W = is_static ? 1 : s->expand_width;
+        for (int i = 0; i < PROBES_MAX; ++i) D->static_w[i] = is_static && i < s->n_probes ? s->static_widths[i] : 0;
         D->n_anchor = s->n_anchor; D->prune_parent = s->prune_parent; D->prune_root = s->prune_root;
         D->ema_per_token = s->ema_per_token; D->lambda = s->lambda;
     }

@@ -826,7 +826,8 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     }
     __syncthreads();
     for (int i = 1; i <= Dd; ++i) {
-        const int pool = min(D.K, D.B - i);
+        // Algorithm 1 draws min(K, B-i) candidates per expanded node; a static tree its fixed width for this depth
+        const int pool = D.static_w[0] > 0 ? D.static_w[i - 1] : min(D.K, D.B - i);
         if (pool <= 0) break;
         const Cand* list = s_list[i - 1];
         const float lse_i = s_lse[i - 1];

@@ -33,7 +33,7 @@ def to_device(w, device="cuda"):
 def c_spec(o: O.SpecCfg):
     return P.spec_cfg(n_probes=o.n_probes, topk=o.topk, max_nodes=o.max_nodes, expand_width=o.expand_width,
                       n_anchor=o.n_anchor, prune_parent=o.prune_parent, prune_root=o.prune_root,
-                      ema_per_token=o.ema_per_token, lam=o.lam)
+                      ema_per_token=o.ema_per_token, lam=o.lam, static_widths=o.static_widths)
 
 
 class ParityRun:
@@ -87,7 +87,7 @@ class ParityRun:
         return O.Tree(st["row_token"][:N].copy(), st["row_parent"][:N].copy(), st["row_depth"][:N].copy(), np.zeros(N, np.float32))
 
     def _check_next_tree(self, st_after, root, ids, vals, lses):
-        tree = O.build_tree(root, ids, vals, lses, self.spec) if self.spec.n_probes else O.root_only(root)
+        tree = O.next_tree(root, ids, vals, lses, self.spec) if self.spec.n_probes else O.root_only(root)
         N = st_after["n_nodes"]
         assert N == tree.n, f"next tree size {N} vs oracle {tree.n}"
         assert list(st_after["row_token"][:N]) == list(tree.tokens)

@@ -41,6 +41,21 @@ def test_tiny_fp32_full_parity(pu, W, n_anchor, prune):
     run.close()
 
 
+@pytest.mark.parametrize("widths,n_anchor", [((7, 2), 0), ((15, 4), 0), ((7, 5, 3), 1)])
+def test_tiny_fp32_static_tree_parity(pu, widths, n_anchor):
+    """Static trees with the paper's branch widths ([7,2] = BC 30, [15,4] = BC 60 with two masks per node)."""
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=3, gain_jitter=True, std=0.3)
+    prompt = synth.make_prompt(shape.vocab, 50, 7)
+    spec = O.SpecCfg(n_probes=len(widths), topk=1, max_nodes=1, n_anchor=n_anchor, static_widths=widths)
+    run = pu.ParityRun(shape, w, spec, prompt, 24, TOL_FP32)
+    out = run.run()
+    assert out == O.greedy_generate(O.OracleModel(shape, w), prompt, 24, 256)
+    if n_anchor == 0:
+        assert run.h.state()["n_rows"] <= (len(widths) + 1) * (1 + sum(widths))
+    run.close()
+
+
 def test_tiny_fp32_nontrivial_stream(pu):
     """Same model family with wider weights and jittered norm gains, so the stream is not one repeated token."""
     shape = synth.TINY

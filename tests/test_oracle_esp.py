@@ -273,3 +273,38 @@ def test_forced_perfect_draft_is_fully_accepted():
     while len(dec.emitted) < 12:
         dec.step()
     assert dec.emitted[:12] == ref
+
+
+# ---------------------------------------------------------------- static trees (Section 4.2)
+@pytest.mark.parametrize("widths,n_anchor", [((7, 2), 0), ((5, 4), 0), ((4,), 0), ((7, 5, 3), 1)])
+def test_static_tree_generation_is_lossless_and_has_the_papers_block_size(widths, n_anchor):
+    """Fixed branch widths [K_1..K_k]: the tree has 1 + sum K_i nodes whenever the probes offer enough
+    candidates, every node carries k masks in the paper's layout (BC = (k+1)(1 + sum K_i): [7,2] -> 30,
+    [4] -> 10), the Top-1 node of each depth is the only one with children, and decoding stays lossless."""
+    k = len(widths)
+    shape = synth.TINY.replace(n_layers=2, d_model=64, n_q_heads=4, n_kv_heads=2, head_dim=16, d_ffn=160, vocab=97)
+    w = synth.make_weights(shape, seed=22, gain_jitter=True, std=0.3)
+    model = esp.OracleModel(shape, w)
+    prompt = synth.make_prompt(shape.vocab, 15, 4)
+    ref = esp.greedy_generate(model, prompt, 30, 128)
+    spec = esp.SpecCfg(n_probes=k, topk=1, max_nodes=1, n_anchor=n_anchor, static_widths=widths)
+    dec = esp.EspOracle(model, spec, 256)
+    assert dec.generate(prompt, 30) == ref
+    full = 0
+    for rec in dec.log:
+        if rec["kind"] != "step":
+            continue
+        t = rec["tree"]
+        assert t.n <= 1 + sum(widths)
+        for d in range(1, k + 1):
+            nodes = [i for i in range(t.n) if t.depths[i] == d]
+            assert len(nodes) <= widths[d - 1]
+            assert len({int(t.parents[i]) for i in nodes}) <= 1          # one parent per depth
+            if nodes and d > 1:
+                prev = [i for i in range(t.n) if t.depths[i] == d - 1]
+                assert int(t.parents[nodes[0]]) == prev[0]               # ... the first (Top-1) node of the depth above
+        if n_anchor == 0 and t.n == 1 + sum(widths):
+            full += 1
+            assert rec["block"].m == esp.block_complexity(k, widths)
+    if n_anchor == 0:
+        assert full > 0
