@@ -27,16 +27,18 @@
 // Every mbarrier wait is bounded; on a timeout the kernel records
 // DEV_E_WAIT_TIMEOUT, lets its copies drain, frees its tensor memory and
 // returns.
-#include <cuda.h>
 #include <new>
 #include <string.h>
 
 #include "esp_epilogue.cuh"
 #include "esp_launch.h"
+#include "esp_tc.cuh"
 
 namespace esp {
 
 namespace {
+
+using namespace tc;
 
 constexpr int BK = 64;                       // k elements per stage (128 bytes of bf16)
 constexpr int STAGES = 6;
@@ -45,7 +47,6 @@ constexpr int B_BYTES = RT * BK * 2;         // 10240
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 256;               // two accumulator buffers of 128 columns
 constexpr int NUM_THREADS = 192;
-constexpr unsigned long long WAIT_LIMIT_NS = 50ull * 1000 * 1000;   // 50 ms
 
 struct TcParams {
     CUtensorMap map_a[3];
@@ -61,102 +62,8 @@ struct TcParams {
     EpiArgs a;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Bounded wait: gives up after WAIT_LIMIT_NS of wall time (a try_wait may itself block for a while, so the
-// bound is on the clock, not on the number of polls) or as soon as another role has given up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    const uint32_t addr = smem_u32(bar);
-    unsigned long long t0 = 0;
-    for (uint32_t it = 0;; ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(addr), "r"(parity)
-            : "memory");
-        if (done) return true;
-        if ((it & 15u) == 15u) {
-            if (*abort_flag) return false;
-            unsigned long long now;
-            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) return false;
-        }
-    }
-}
-
-// L2 eviction policies: weights are read once per step and never again before the whole model has streamed
-// through (evict first); activations are re-read by every CTA (evict last).
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_last() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
-        : "memory");
-}
-
-// one contiguous 16 KB unit of repacked weights (already in the swizzled shared-memory layout)
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
-        : "memory");
-}
-
-// K-major operand tile in shared memory, rows of 128 bytes, 128-byte swizzle:
-// 8-row groups are 1024 bytes apart (stride byte offset), descriptor version 1.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFF) >> 4);       // start address
-    d |= (uint64_t)1 << 16;                       // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;             // stride byte offset
-    d |= (uint64_t)1 << 46;                       // descriptor version (Blackwell)
-    d |= (uint64_t)2 << 61;                       // 128-byte swizzle
-    return d;
-}
-
 // kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = 80
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RT >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
-
-__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-}
 
 // One (tile, k-range) piece of a CTA's stream-K range.
 struct Seg {
@@ -268,11 +175,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                             if (p.a_packed) {
                                 bulk_load(sa, p.a_packed + ((size_t)sg.tile * p.KB + kb) * A_BYTES, A_BYTES, &full[it], pol_w);
                             } else {
-                                tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[it], pol_w);
-                                tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it], pol_w);
+                                tma_load_2d_hint(sa, &p.map_a[m0], kb * BK, r0, &full[it], pol_w);
+                                tma_load_2d_hint(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it], pol_w);
                             }
                         } else {
-                            tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[it], pol_x);
+                            tma_load_2d_hint(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[it], pol_x);
                         }
                     }
                 }
@@ -294,10 +201,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                         if (p.a_packed) {
                             bulk_load(sa, p.a_packed + ((size_t)sg.tile * p.KB + kb) * A_BYTES, A_BYTES, &full[stage], pol_w);
                         } else {
-                            tma_load_2d(sa, &p.map_a[m0], kb * BK, r0, &full[stage], pol_w);
-                            tma_load_2d(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage], pol_w);
+                            tma_load_2d_hint(sa, &p.map_a[m0], kb * BK, r0, &full[stage], pol_w);
+                            tma_load_2d_hint(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage], pol_w);
                         }
-                        tma_load_2d(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[stage], pol_x);
+                        tma_load_2d_hint(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[stage], pol_x);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -320,10 +227,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                     if (!mbar_wait(&full[stage], phase, s_abort)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t sa = smem_u32(stages + stage * STAGE_BYTES);
-                    const uint64_t da = smem_desc(sa), db = smem_desc(sa + A_BYTES);
+                    const uint64_t da = smem_desc(sa, 16), db = smem_desc(sa + A_BYTES, 16);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)
-                        umma(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), (kb > sg.kb0 || k > 0) ? 1u : 0u);
+                        umma(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), IDESC, (kb > sg.kb0 || k > 0) ? 1u : 0u);
                     umma_commit(&empty[stage]);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -476,21 +383,6 @@ __global__ void __launch_bounds__(128) k_pack_weights(PackArgs g, unsigned char*
 }
 
 constexpr size_t SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + sizeof(float) * (RT * ACC_LD + RT * 4) + 256;
-
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn get_encode() {
-    static EncodeFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) return nullptr;
-        fn = reinterpret_cast<EncodeFn>(p);
-    }
-    return fn;
-}
 
 // [rows][K] bf16 row-major, box = 64 k-elements x box_rows rows, 128-byte swizzle, out-of-range reads give zero
 int make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
