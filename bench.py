@@ -217,6 +217,60 @@ def algorithmic_bytes(shape, L_mean, rows):
     return w, kv_per_pos * L_mean + kv_per_pos * rows
 
 
+def replay_leg(P, shape, w, prompt, stream, k, B, n_tokens, seed=0):
+    """Throughput under a synthetic acceptance schedule.  Random-init models accept no drafts, so the draft trees
+    of this leg are set from outside (esp_set_tree): each holds the true continuation (taken from a greedy run of
+    the same kernels) down to a depth drawn per step -- 0, 1, 2, 3 drafts with probability .55/.30/.12/.03, mean
+    0.63, i.e. the paper's tau = 1.63 -- inside a full tree of B nodes of wrong siblings.  The emitted stream must
+    equal the greedy stream token for token.  Says nothing about model quality; it shows what a step costs when
+    drafts are accepted, their KV rows compacted and the host is in the loop (set_tree + step, synchronous)."""
+    import torch
+    plen = len(prompt)
+    max_seq = plen + n_tokens + 64
+    hg = P.Handle(shape, P.spec_cfg(), w, max_seq_len=max_seq, stream=stream)
+    truth = hg.generate(prompt, n_tokens + 8)
+    hg.close()
+    h = P.Handle(shape, P.spec_cfg(n_probes=k, topk=10, max_nodes=B, expand_width=0, n_anchor=1), w, max_seq_len=max_seq, stream=stream)
+    out = [h.prefill(prompt)]
+    rng = np.random.default_rng(seed)
+    per_level = (B - 1) // k
+    steps = 0
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    while len(out) < n_tokens:
+        n = len(out)
+        a = int(min(rng.choice(4, p=[0.55, 0.30, 0.12, 0.03]), k))
+        toks, pars, main = [out[-1]], [-1], 0
+        for d in range(1, k + 1):
+            level = []
+            if d <= a:
+                level.append(truth[n + d - 1])
+            wrong = rng.integers(0, shape.vocab - 1, size=per_level - len(level))
+            wrong = [int(t) + (int(t) >= truth[n + d - 1]) for t in wrong]      # never the true token
+            first = len(toks)
+            for t in level + wrong:
+                toks.append(t)
+                pars.append(main)
+            main = first                                                        # the true node while d <= a
+        h.set_tree(np.array(toks, np.int32), np.array(pars, np.int32))
+        new = h.step()
+        steps += 1
+        if len(new) != a + 1:
+            raise SystemExit(f"replay: accepted {len(new) - 1} drafts, schedule said {a}")
+        out.extend(new)
+    torch.cuda.synchronize()
+    sec = time.perf_counter() - t0
+    if out[:n_tokens] != truth[:n_tokens]:
+        raise SystemExit("replay: ESP stream differs from the greedy stream")
+    err = h.stats().device_error
+    h.close()
+    if err:
+        raise SystemExit("replay: device error word set")
+    return {"tau": (len(out) - 1) / steps, "tok_s": (len(out) - 1) / sec, "steps": steps, "ms_per_step": sec / steps * 1e3,
+            "note": "synthetic acceptance schedule (forced drafts, mean 0.63 accepted per step), not model quality; "
+                    "includes the host round trip of esp_set_tree every step; stream checked equal to greedy"}
+
+
 def aggregate_over_ranks(dist, times_ms, counts, device):
     """Replicas share nothing: the job's time is the slowest rank's (MAX), its work the sum over ranks (SUM)."""
     import torch
@@ -332,6 +386,10 @@ def run_ours(args, shape, plen, k, K, B):
         greedy_tok_s = steps / (g0.elapsed_time(g1) * 1e-3)
         hg.close()
 
+    replay = None
+    if rank == 0 and not args.no_greedy:
+        replay = replay_leg(P, shape, w, prompt, stream, k, B, min(256, steps))
+
     # ---- aggregate over ranks: slowest rank's time, all ranks' tokens
     if dist is not None:
         (ms, e2e_ms), (tokens, e2e_tokens, launches) = aggregate_over_ranks(dist, [ms, e2e_ms], [tokens, e2e_tokens, launches], "cuda")
@@ -370,6 +428,7 @@ def run_ours(args, shape, plen, k, K, B):
                               "peak_source": peak_src},
             "kernel_group_ms_per_step": kinds,
             "greedy_tok_s": greedy_tok_s,
+            "replay_tau_1_63": replay,
         }
         if not args.no_cpu and world == 1:
             smp = OracleSample(shape, plen, k, B, host_slice(shape, w))
