@@ -15,13 +15,13 @@
 // through shared memory by TMA in chunks of 128 keys and shared by all pairs:
 //   S = Q K^T   tcgen05.mma, Q (128 pairs x 128 dims) and the K chunk both
 //               K-major in shared memory, S (128 x 128 fp32) in tensor memory;
-//   softmax     128 threads, one per pair (= tensor-memory lane): mask by the
+//   softmax     256 threads, two per pair (= tensor-memory lane): mask by the
 //               row's T0, running max / sum in the log2 domain, P as bf16 into
 //               shared memory in the A-operand layout;
 //   O += P V    tcgen05.mma with V as the MN-major B operand (the cache keeps
 //               values as [key][dim]); O (128 x 128 fp32) stays in tensor
 //               memory and is rescaled there when the running max moves.
-// Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 softmax.  S and the
+// Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 softmax (two threads per pair, 64 keys each).  S and the
 // K/V stages are double buffered, so Q K^T of chunk c+1 overlaps the softmax of
 // chunk c.  Every mbarrier wait is bounded; on a timeout the kernel records
 // DEV_E_WAIT_TIMEOUT, frees its tensor memory and returns.
@@ -46,7 +46,7 @@ constexpr int KV_STAGE = K_BYTES + V_BYTES;
 constexpr int OFF_Q = 0, OFF_KV = Q_BYTES, OFF_P = OFF_KV + 2 * KV_STAGE, OFF_BAR = OFF_P + P_BYTES;
 constexpr size_t SMEM_BYTES = 1024 + OFF_BAR + 256;
 constexpr int TMEM_COLS = 512;            // S0 at 0, S1 at 128, O at 256
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;           // producer warp, MMA warp, 8 softmax warps
 
 struct BulkParams {
     CUtensorMap map_q;   // [batch*RT][Hq][128], box 64 x group x rows_per_tile
@@ -65,9 +65,17 @@ __device__ __forceinline__ int tail_start_tc(int P, int dcap) {
 constexpr uint32_t IDESC_QK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 constexpr uint32_t IDESC_PV = IDESC_QK | (1u << 16);
 
+// 64 consecutive columns of this lane: two loads in flight, one wait
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
+    tmem_ld32_issue(taddr, &r[0]);
+    tmem_ld32_issue(taddr + 32, &r[32]);
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_constant__ BulkParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ int s_T0max;
+    __shared__ float s_xchg[2][2 * MP];   // [exchange parity][half][pair]
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);   // [2]
     uint64_t* kv_empty = kv_full + 2;                                  // [2]
@@ -75,7 +83,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
     uint64_t* q_full = s_full + 2;
     uint64_t* p_ready = q_full + 1;
     uint64_t* pv_done = p_ready + 1;
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(pv_done + 1);
+    uint64_t* xchg = pv_done + 1;                                      // the two threads of a pair exchanged a value
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(xchg + 1);
     volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
     const AttnArgs& a = p.a;
@@ -110,8 +119,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); mbar_init(&s_full[i], 1); }
         mbar_init(q_full, 1);
-        mbar_init(p_ready, 128);
+        mbar_init(p_ready, 256);
         mbar_init(pv_done, 1);
+        mbar_init(xchg, 256);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -200,14 +210,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
             if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
         }
     } else {
-        // ---------------- softmax warps: thread = pair = tensor-memory lane
+        // ---------------- softmax warps 2..9: a thread owns one pair (= tensor-memory lane) and one half of the
+        // chunk's 128 keys (warps 2-5 keys 0..63, warps 6-9 keys 64..127); the two threads of a pair exchange
+        // their maxima (per chunk) and their sums (at the end) through shared memory
         const int q4 = warp & 3;
+        const int hf = (warp - 2) >> 2;
         const int pair = q4 * 32 + lane;
         const int r = row0 + pair / p.group, head = kvh * p.group + pair % p.group;
         const bool pv = pair / p.group < p.rows_per_tile && r < n_rows && r < RT;
         int T0row = 0;
         if (pv) T0row = tail_start_tc(L + (a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r]), a.dcap);
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16) + hf * 64;   // this thread's 64 columns of S / O
         float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;
         for (int c = 0; c < n_chunks && ok; ++c) {
@@ -215,26 +228,32 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
             if (!__all_sync(0xffffffffu, mbar_wait(&s_full[c & 1], (c >> 1) & 1, s_abort))) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t s_addr = lane_addr + (c & 1) * 128;
-            const int cbase = beg + c * CK;
-            // the row's 128 scores, masked to its visible keys and scaled to the log2 domain
-            uint32_t sv[128];
-            tmem_ld128(s_addr, sv);
+            const int cbase = beg + c * CK + hf * 64;
+            // the row's scores for this half, masked to its visible keys and scaled to the log2 domain
+            uint32_t sv[64];
+            tmem_ld64(s_addr, sv);
             float cmax = -INFINITY;
-            if (__all_sync(0xffffffffu, cbase + CK <= T0row)) {     // the whole chunk is visible to every row of the warp
+            if (__all_sync(0xffffffffu, cbase + 64 <= T0row)) {     // every key of the half is visible to every row of the warp
 #pragma unroll
-                for (int i = 0; i < 128; ++i) {
-                    const float s = __uint_as_float(sv[i]) * a.scale_log2;
-                    sv[i] = __float_as_uint(s);
-                    cmax = fmaxf(cmax, s);
+                for (int i = 0; i < 64; ++i) {
+                    const float sc = __uint_as_float(sv[i]) * a.scale_log2;
+                    sv[i] = __float_as_uint(sc);
+                    cmax = fmaxf(cmax, sc);
                 }
             } else {
 #pragma unroll
-                for (int i = 0; i < 128; ++i) {
-                    const float s = cbase + i < T0row ? __uint_as_float(sv[i]) * a.scale_log2 : -INFINITY;
-                    sv[i] = __float_as_uint(s);
-                    cmax = fmaxf(cmax, s);
+                for (int i = 0; i < 64; ++i) {
+                    const float sc = cbase + i < T0row ? __uint_as_float(sv[i]) * a.scale_log2 : -INFINITY;
+                    sv[i] = __float_as_uint(sc);
+                    cmax = fmaxf(cmax, sc);
                 }
             }
+            // the chunk maximum over both halves
+            // (double buffered by exchange parity: a thread can be one exchange ahead of its partner, not two)
+            s_xchg[c & 1][hf * MP + pair] = cmax;
+            mbar_arrive(xchg);
+            if (!__all_sync(0xffffffffu, mbar_wait(xchg, c & 1, s_abort))) { ok = false; break; }
+            cmax = fmaxf(s_xchg[c & 1][pair], s_xchg[c & 1][MP + pair]);
             const float m_new = fmaxf(m_run, cmax);
             const float m_use = m_new == -INFINITY ? 0.f : m_new;
             const float alpha = exp2f(m_run - m_use);
@@ -242,32 +261,32 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
             // before it is rescaled
             if (c > 0 && !__all_sync(0xffffffffu, mbar_wait(pv_done, (c - 1) & 1, s_abort))) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // probabilities, their sum (key order), P as bf16 in the A-operand layout
+            // probabilities, their sum (key order), P as bf16 in the A-operand layout (this half = one swizzled tile)
             float csum = 0.f;
+            unsigned char* prow = sP + hf * HALF_BYTES + pair * 128;
 #pragma unroll
-            for (int blk = 0; blk < 4; ++blk) {
+            for (int blk = 0; blk < 2; ++blk) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
                     const float p0 = exp2f(__uint_as_float(sv[blk * 32 + i]) - m_use), p1 = exp2f(__uint_as_float(sv[blk * 32 + i + 1]) - m_use);
                     csum += p0;
                     csum += p1;
-                    const __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&b);
+                    const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
                 }
-                unsigned char* prow = sP + (blk >> 1) * HALF_BYTES + pair * 128;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const int chunk16 = (blk & 1) * 4 + j;
+                    const int chunk16 = blk * 4 + j;
                     *reinterpret_cast<uint4*>(prow + ((chunk16 ^ (pair & 7)) << 4)) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
                 }
             }
             if (c > 0) {
-                // O <- alpha * O (in tensor memory)
+                // O <- alpha * O (in tensor memory), this thread's 64 of the 128 columns
                 if (__any_sync(0xffffffffu, alpha != 1.0f)) {   // warp-uniform: skip when no lane's maximum moved
-                    tmem_ld128(lane_addr + 256, sv);
+                    tmem_ld64(lane_addr + 256, sv);
 #pragma unroll
-                    for (int blk = 0; blk < 4; ++blk) {
+                    for (int blk = 0; blk < 2; ++blk) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) sv[blk * 32 + i] = __float_as_uint(__uint_as_float(sv[blk * 32 + i]) * alpha);
                         tmem_st32(lane_addr + 256 + blk * 32, *reinterpret_cast<const uint32_t(*)[32]>(&sv[blk * 32]));
@@ -275,7 +294,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 }
             }
-            l_run = l_run * alpha + csum;
+            l_run = l_run * alpha + csum;     // this half's share of the row sum
             m_run = m_new;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes -> tensor-core reads
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -283,21 +302,27 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
         }
         if (ok && !__all_sync(0xffffffffu, mbar_wait(pv_done, (n_chunks - 1) & 1, s_abort))) ok = false;
         if (ok) {
+            // the row sum = first half's share + second half's share
+            s_xchg[n_chunks & 1][hf * MP + pair] = l_run;
+            mbar_arrive(xchg);
+            if (!__all_sync(0xffffffffu, mbar_wait(xchg, n_chunks & 1, s_abort))) ok = false;
+        }
+        if (ok) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // O row -> shared memory (the K/V stages are free now) -> one 512-byte bulk copy per pair.  The
+            // O half-row -> shared memory (the K/V stages are free now) -> one 256-byte bulk copy per thread.  The
             // tensor-memory load is warp-wide: every lane takes part, lanes without a pair copy nothing.
-            uint32_t ov[128];
-            tmem_ld128(lane_addr + 256, ov);
-            float* orow = reinterpret_cast<float*>(smem + OFF_KV) + pair * (HD + 4);   // rows padded by 16 bytes: no bank conflicts
+            uint32_t ov[64];
+            tmem_ld64(lane_addr + 256, ov);
+            float* orow = reinterpret_cast<float*>(smem + OFF_KV) + pair * (HD + 4) + hf * 64;   // rows padded by 16 bytes: no bank conflicts
 #pragma unroll
-            for (int i = 0; i < 128; i += 4)
+            for (int i = 0; i < 64; i += 4)
                 *reinterpret_cast<uint4*>(orow + i) = make_uint4(ov[i], ov[i + 1], ov[i + 2], ov[i + 3]);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             if (pv) {
                 const size_t idx = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max + split;
-                a.part_ml[idx] = make_float2(m_run, l_run);
+                if (hf == 0) a.part_ml[idx] = make_float2(m_run, s_xchg[n_chunks & 1][pair] + s_xchg[n_chunks & 1][MP + pair]);
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                             ::"l"(a.part_o + idx * HD), "r"(smem_u32(orow)), "r"(HD * 4) : "memory");
+                             ::"l"(a.part_o + idx * HD + hf * 64), "r"(smem_u32(orow)), "r"(64 * 4) : "memory");
             }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");        // copies complete: shared memory may be released

@@ -39,10 +39,26 @@ __global__ void k_assemble(const SeqState* states, const T* embed, const float* 
     if (!st->active || r >= st->n_rows) return;
     float* out = hres + (size_t)(seq * RT + r) * d;
     int tok = st->row_token[r];
-    if (tok >= 0)
-        for (int j = threadIdx.x; j < d; j += blockDim.x) out[j] = to_f32(embed[(size_t)tok * d + j]);
-    else
-        for (int j = threadIdx.x; j < d; j += blockDim.x) out[j] = mvec[(size_t)seq * d + j];
+    // four elements per thread and step (d is a multiple of 8), independent loads in flight
+    if (tok >= 0) {
+        const T* src = embed + (size_t)tok * d;
+#pragma unroll 4
+        for (int j = threadIdx.x * 4; j < d; j += blockDim.x * 4) {
+            float4 v;
+            if constexpr (sizeof(T) == 2) {
+                const uint2 raw = *reinterpret_cast<const uint2*>(src + j);
+                const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&raw.x), hi = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+                v = make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+            } else {
+                v = *reinterpret_cast<const float4*>(src + j);
+            }
+            *reinterpret_cast<float4*>(out + j) = v;
+        }
+    } else {
+        const float* src = mvec + (size_t)seq * d;
+#pragma unroll 4
+        for (int j = threadIdx.x * 4; j < d; j += blockDim.x * 4) *reinterpret_cast<float4*>(out + j) = *reinterpret_cast<const float4*>(src + j);
+    }
 }
 
 // y = x * rsqrt(mean(x^2)+eps) * g, one block per row
