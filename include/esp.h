@@ -70,6 +70,13 @@ typedef struct {
      * probe i (after the pruner), for as many depths as there are non-zero widths.  topk, max_nodes and
      * expand_width are then ignored (the tree has 1 + sum of widths nodes). */
     int32_t static_widths[ESP_MAX_PROBES];
+    /* How esp_prefill sets the k mask vectors (Section 3.1; Section 4 "Different mask embedding designs"):
+     * 0 = all k to the mean of the prompt embeddings (Eq. mask_init_mean, the paper's method);
+     * 1 = "Last K": mask i gets the embedding of the i-th of the last k prompt tokens;
+     * 2 = given by the caller with esp_set_mask before esp_prefill (the "Sample" N(mu, sigma^2 I) and the
+     *     mu + n*sigma initialisations: the caller draws or builds the vectors).
+     * Every mask vector then follows the same update, Eq. (mask_update_mean). */
+    int32_t mask_init;
 } esp_spec_cfg;
 
 /* Model weights. [device] matrices; the per-layer members are [host] arrays of
@@ -136,6 +143,10 @@ int esp_step(esp_handle* h, int32_t* tokens_out, int32_t* n_out);
 int esp_step_async(esp_handle* h);
 int esp_read(esp_handle* h, int32_t* tokens_out, int32_t* n_out);
 
+/* Mask vectors of sequence `seq` given by the caller (mask_init = 2): mask [host] [n_probes][d_model] fp32.
+ * Call before esp_prefill of that sequence (a later call replaces the current vectors).  Synchronises. */
+int esp_set_mask(esp_handle* h, int32_t seq, const float* mask);
+
 /* Test hook: replace the draft tree of sequence `seq` for the next step.
  * tokens/parents [host] n nodes in breadth-first order (parents[0] = -1,
  * parents[i] < i); node 0 must carry the current root token.  Has no
@@ -146,7 +157,7 @@ int esp_set_tree(esp_handle* h, int32_t seq, const int32_t* tokens, const int32_
 /* Debug/parity access to device state of sequence `seq`, copied to [host] buffers (any may be NULL):
  *   row_token/row_parent/row_depth [ESP_MAX_ROWS], n_nodes, n_rows, L of the block the NEXT step will run;
  *   topk_ids/topk_vals [ESP_MAX_ROWS][ESP_MAX_KPRIME], lse [ESP_MAX_ROWS] from the LAST forward;
- *   mask_vec [d_model].  Synchronises. */
+ *   mask_vec [max(n_probes, 1)][d_model].  Synchronises. */
 int esp_debug_state(esp_handle* h, int32_t seq, int32_t* row_token, int32_t* row_parent, int32_t* row_depth,
                     int32_t* n_nodes, int32_t* n_rows, int32_t* L, int32_t* topk_ids, float* topk_vals, float* lse,
                     float* mask_vec);
@@ -169,6 +180,13 @@ int esp_debug_set_gemm(esp_handle* h, int32_t impl);
 int esp_step_profiled(esp_handle* h, float* ms_by_kind, int32_t* tokens_out, int32_t* n_out);
 
 int esp_get_stats(esp_handle* h, esp_stats* out);
+
+/* Self-test of the bounded waits the tensor-core kernels use (no counterpart in the paper): launches one
+ * small kernel that waits on a barrier nothing ever signals; the wait must give up after its time limit
+ * (50 ms), record the wait-timeout code and return normally.  *device_status_out [host] receives the code the
+ * kernel recorded (1 = wait timed out, as expected).  The CUDA context stays usable.  `scratch` [device] >= 256
+ * bytes. */
+int esp_debug_wait_selftest(void* scratch, void* cuda_stream, int32_t* device_status_out);
 
 /* Releases host-side bookkeeping only. */
 void esp_free(esp_handle* h);

@@ -190,6 +190,7 @@ class SpecCfg:
     ema_per_token: bool = True
     lam: float = 0.1
     static_widths: Tuple[int, ...] = ()   # fixed branch widths [K_1..K_k] (Section 4.2); empty = dynamic tree
+    mask_init: str = "mean"               # "mean" (Eq. mask_init_mean) | "last_k" | "given" (Section 4, mask designs)
 
     @property
     def k_prime(self) -> int:
@@ -204,6 +205,15 @@ def mask_init_mean(E_rows: np.ndarray) -> np.ndarray:
     for j in range(E_rows.shape[0]):
         acc = (acc + E_rows[j].astype(_F32)).astype(_F32)
     return (acc / _F32(E_rows.shape[0])).astype(_F32)
+
+
+def mask_init_last_k(E_rows: np.ndarray, k: int) -> np.ndarray:
+    """"Last K (hard init)" of Section 4: the k masks take the embeddings of the last k prompt tokens.  The
+    paper's index expression (e_{t-k-i}) does not address the last k tokens it names; the words are followed:
+    mask i (1-based) = embedding of prompt token t-k+i, i.e. the last k tokens in prompt order (a prompt
+    shorter than k repeats its first token)."""
+    t = E_rows.shape[0]
+    return np.stack([E_rows[max(t - k + i, 0)].astype(_F32) for i in range(k)])
 
 
 def mask_update(m: np.ndarray, e: np.ndarray, lam: float) -> np.ndarray:
@@ -447,7 +457,8 @@ class EspOracle:
         self.model, self.spec = model, spec
         self.kc, self.vc = model.new_cache(cap)
         self.L = 0
-        self.m: Optional[np.ndarray] = None
+        self.m: Optional[np.ndarray] = None      # [max(k,1)][d]: one vector per mask position, all updated alike
+        self.given_mask: Optional[np.ndarray] = None
         self.tree: Optional[Tree] = None
         self.emitted: List[int] = []
         self.steps = 0
@@ -458,9 +469,14 @@ class EspOracle:
     # -- helpers
     def _rows_x(self, blk: Block) -> np.ndarray:
         x = np.empty((blk.m, self.model.d), dtype=_F32)
+        probe_of_row = {row: j for (_, j), row in blk.probe_row.items()}
         for r in range(blk.m):
-            x[r] = self.model.embed(int(blk.row_token[r])) if blk.row_token[r] >= 0 else self.m
+            x[r] = self.model.embed(int(blk.row_token[r])) if blk.row_token[r] >= 0 else self.m[probe_of_row[r] - 1]
         return x
+
+    def set_mask(self, m: np.ndarray):
+        """Mask vectors given from outside ("Sample" and mu + n*sigma initialisations): [k][d], used by prefill."""
+        self.given_mask = np.array(m, dtype=_F32).reshape(max(self.spec.n_probes, 1), self.model.d)
 
     def _emit(self, y: int):
         self.emitted.append(int(y))
@@ -484,9 +500,14 @@ class EspOracle:
         """
         sp, t, k = self.spec, len(prompt), self.spec.n_probes
         E = np.stack([self.model.embed(int(x)) for x in prompt])
-        self.m = mask_init_mean(E)
+        if sp.mask_init == "last_k" and k:
+            self.m = mask_init_last_k(E, k)
+        elif sp.mask_init == "given":
+            self.m = self.given_mask.copy()
+        else:
+            self.m = np.tile(mask_init_mean(E), (max(k, 1), 1))
         M = t + k
-        x = np.concatenate([E, np.tile(self.m, (k, 1))], axis=0) if k else E
+        x = np.concatenate([E, self.m[:k]], axis=0) if k else E
         vis = np.tril(np.ones((M, M), np.uint8))
         want = np.zeros(M, np.uint8)
         want[t - 1:] = 1

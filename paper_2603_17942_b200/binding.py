@@ -23,8 +23,9 @@ ESP_MAX_KPRIME = 32
 ERRORS = {0: "ESP_OK", -1: "ESP_E_BADCFG", -2: "ESP_E_WORKSPACE", -3: "ESP_E_PROMPT", -4: "ESP_E_FULL",
           -5: "ESP_E_DEVICE", -6: "ESP_E_CUDA", -7: "ESP_E_STATE", -8: "ESP_E_ARG"}
 
-EXPORTS = ["esp_workspace_bytes", "esp_init", "esp_prefill", "esp_step", "esp_step_async", "esp_read", "esp_set_tree",
-           "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_step_profiled", "esp_get_stats", "esp_free",
+EXPORTS = ["esp_workspace_bytes", "esp_init", "esp_prefill", "esp_step", "esp_step_async", "esp_read", "esp_set_mask", "esp_set_tree",
+           "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_step_profiled", "esp_get_stats",
+           "esp_debug_wait_selftest", "esp_free",
            "esp_tree_attention_scratch_bytes", "esp_tree_attention", "esp_tree_attention_static", "esp_gemm_scratch_bytes",
            "esp_gemm_bf16"]
 
@@ -48,7 +49,7 @@ class esp_model_cfg(ctypes.Structure):
 class esp_spec_cfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("n_probes", "topk", "max_nodes", "expand_width", "n_anchor",
                                               "prune_parent", "prune_root", "ema_per_token")] + [("lam", ctypes.c_float)] + \
-               [("static_widths", ctypes.c_int32 * ESP_MAX_PROBES)]
+               [("static_widths", ctypes.c_int32 * ESP_MAX_PROBES), ("mask_init", ctypes.c_int32)]
 
 
 _PP = ctypes.POINTER(ctypes.c_void_p)
@@ -108,10 +109,10 @@ def model_cfg(shape, max_seq_len: int, max_batch: int = 1) -> esp_model_cfg:
 
 
 def spec_cfg(n_probes=0, topk=1, max_nodes=1, expand_width=1, n_anchor=0, prune_parent=True, prune_root=False,
-             ema_per_token=True, lam=0.1, static_widths=()) -> esp_spec_cfg:
+             ema_per_token=True, lam=0.1, static_widths=(), mask_init=0) -> esp_spec_cfg:
     widths = (ctypes.c_int32 * ESP_MAX_PROBES)(*[int(w) for w in static_widths])
     return esp_spec_cfg(n_probes, topk, max_nodes, expand_width, n_anchor, int(prune_parent), int(prune_root),
-                        int(ema_per_token), float(lam), widths)
+                        int(ema_per_token), float(lam), widths, int(mask_init))
 
 
 # ---------------------------------------------------------------- raw calls (same names as the header)
@@ -147,17 +148,22 @@ def esp_read(h, tokens_out: np.ndarray, n_out: np.ndarray):
     _check(load_library().esp_read(h, _vp(tokens_out), _vp(n_out)), "esp_read")
 
 
+def esp_set_mask(h, seq: int, mask):
+    mask = np.ascontiguousarray(mask, dtype=np.float32)
+    _check(load_library().esp_set_mask(h, ctypes.c_int32(seq), _vp(mask)), "esp_set_mask")
+
+
 def esp_set_tree(h, seq: int, tokens, parents):
     tokens = np.ascontiguousarray(tokens, dtype=np.int32)
     parents = np.ascontiguousarray(parents, dtype=np.int32)
     _check(load_library().esp_set_tree(h, ctypes.c_int32(seq), _vp(tokens), _vp(parents), ctypes.c_int32(len(tokens))), "esp_set_tree")
 
 
-def esp_debug_state(h, seq: int, d_model: int) -> Dict[str, object]:
+def esp_debug_state(h, seq: int, d_model: int, n_probes: int = 1) -> Dict[str, object]:
     R, KP = ESP_MAX_ROWS, ESP_MAX_KPRIME
     out = {"row_token": np.zeros(R, np.int32), "row_parent": np.zeros(R, np.int32), "row_depth": np.zeros(R, np.int32),
            "topk_ids": np.zeros((R, KP), np.int32), "topk_vals": np.zeros((R, KP), np.float32),
-           "lse": np.zeros(R, np.float32), "mask_vec": np.zeros(d_model, np.float32)}
+           "lse": np.zeros(R, np.float32), "mask_vec": np.zeros((max(n_probes, 1), d_model), np.float32)}
     nn, nr, L = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
     _check(load_library().esp_debug_state(h, ctypes.c_int32(seq), _vp(out["row_token"]), _vp(out["row_parent"]),
                                           _vp(out["row_depth"]), ctypes.byref(nn), ctypes.byref(nr), ctypes.byref(L),
@@ -188,6 +194,13 @@ def esp_get_stats(h) -> esp_stats:
     st = esp_stats()
     _check(load_library().esp_get_stats(h, ctypes.byref(st)), "esp_get_stats")
     return st
+
+
+def esp_debug_wait_selftest(scratch, stream=None) -> int:
+    """Runs the bounded-wait self-test; returns the device status code the kernel recorded (1 = timed out)."""
+    st = ctypes.c_int32(-1)
+    _check(load_library().esp_debug_wait_selftest(_vp(scratch), _vp(stream), ctypes.byref(st)), "esp_debug_wait_selftest")
+    return st.value
 
 
 def esp_free(h):
@@ -284,8 +297,11 @@ class Handle:
     def set_tree(self, tokens, parents, seq: int = 0):
         esp_set_tree(self.h, seq, tokens, parents)
 
+    def set_mask(self, mask, seq: int = 0):
+        esp_set_mask(self.h, seq, mask)
+
     def state(self, seq: int = 0):
-        return esp_debug_state(self.h, seq, self.shape.d_model)
+        return esp_debug_state(self.h, seq, self.shape.d_model, self.spec.n_probes)
 
     def stats(self) -> esp_stats:
         return esp_get_stats(self.h)

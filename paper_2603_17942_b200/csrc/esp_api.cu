@@ -96,6 +96,7 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
     if (spec_rows(*s) > RT) return ESP_E_BADCFG;
     if (2 * s->n_probes > DCAP_STEP) return ESP_E_BADCFG;
     if (s->expand_width < 0 || s->n_anchor < 0) return ESP_E_BADCFG;
+    if (s->mask_init < 0 || s->mask_init > 2) return ESP_E_BADCFG;
     // Algorithm 1 must not create more than MAX_CAND nodes
     long created = 1, n_exp = 1;
     for (int i = 1; i <= s->n_probes && !is_static; ++i) {
@@ -118,6 +119,7 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
         D->n_split_max = (m->max_seq_len + S - 1) / S + 1;
         D->rms_eps = m->rms_eps;
         D->k = s->n_probes; D->K = topk; D->KP = s->n_probes > 0 ? KP : 1; D->B = n_nodes; D->W = is_static ? 1 : s->expand_width;
+        D->mask_slots = s->n_probes > 0 ? s->n_probes : 1;
         for (int i = 0; i < PROBES_MAX; ++i) D->static_w[i] = is_static && i < s->n_probes ? s->static_widths[i] : 0;
         D->n_anchor = s->n_anchor; D->prune_parent = s->prune_parent; D->prune_root = s->prune_root;
         D->ema_per_token = s->ema_per_token; D->lambda = s->lambda;
@@ -147,7 +149,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.cand_ms = c.take<float2>((size_t)n_tiles_v * Mtot);
     o.topk = c.take<Cand>(Mtot * KP_MAX);
     o.lse = c.take<float>(Mtot);
-    o.mvec = c.take<float>((size_t)D.batch * D.d);
+    o.mvec = c.take<float>((size_t)D.batch * D.mask_slots * D.d);
     o.states = c.take<SeqState>(D.batch);
     o.err = c.take<int>(4);
     o.out_ring = c.take<int32_t>((size_t)D.batch * RING);
@@ -261,7 +263,7 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
     StreamK pending;   // partials of the last down projection, summed by the next norm
     pending.partials = nullptr; pending.table = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2;
     mark(h, -1);
-    launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.batch, s, false);
+    launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.mask_slots, D.batch, s, false);
     h->launches++;
     for (int l = 0; l < D.n_layers; ++l) {
         if (tc) launch_resid_norm(b.states, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
@@ -512,7 +514,9 @@ int esp_prefill(esp_handle* h, int32_t seq, const int32_t* prompt, int32_t n_pro
         if (prompt[i] < 0 || prompt[i] >= h->D.V) return ESP_E_PROMPT;
     cudaStream_t s = h->stream;
     if (cudaMemcpyAsync(h->b.prompt_dev, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, s) != cudaSuccess) return ESP_E_CUDA;
-    launch_mask_mean(h->dtype, h->embed, h->b.prompt_dev, n_prompt, h->D.d, h->b.mvec + (size_t)seq * h->D.d, s);
+    if (h->sc.mask_init != 2)   // 2: the caller's vectors (esp_set_mask) stay
+        launch_mask_init(h->dtype, h->embed, h->b.prompt_dev, n_prompt, h->D.d, h->b.mvec + (size_t)seq * h->D.mask_slots * h->D.d,
+                         h->D.mask_slots, h->sc.mask_init, s);
     k_select<<<1, 32, 0, s>>>(h->b.states, h->D.batch, seq);
     std::vector<int> saved = h->L_host;
     for (int i = 0; i < h->D.batch; ++i) h->L_host[i] = 0;
@@ -616,6 +620,15 @@ int esp_step(esp_handle* h, int32_t* tokens_out, int32_t* n_out) {
     return esp_read(h, tokens_out, n_out);
 }
 
+int esp_set_mask(esp_handle* h, int32_t seq, const float* mask) {
+    if (!h || !mask) return ESP_E_ARG;
+    if (seq < 0 || seq >= h->D.batch) return ESP_E_ARG;
+    if (h->sc.n_probes < 1) return ESP_E_STATE;
+    const size_t n = (size_t)h->D.mask_slots * h->D.d;
+    if (cudaMemcpyAsync(h->b.mvec + (size_t)seq * n, mask, sizeof(float) * n, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return ESP_E_CUDA;
+    return cuda_ok(cudaStreamSynchronize(h->stream));
+}
+
 int esp_set_tree(esp_handle* h, int32_t seq, const int32_t* tokens, const int32_t* parents, int32_t n) {
     if (!h || !tokens || !parents) return ESP_E_ARG;
     if (seq < 0 || seq >= h->D.batch || !h->ready[seq]) return ESP_E_STATE;
@@ -658,7 +671,8 @@ int esp_debug_state(esp_handle* h, int32_t seq, int32_t* row_token, int32_t* row
         }
     }
     if (lse && cudaMemcpy(lse, h->b.lse + (size_t)seq * RT, sizeof(float) * RT, cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
-    if (mask_vec && cudaMemcpy(mask_vec, h->b.mvec + (size_t)seq * h->D.d, sizeof(float) * h->D.d, cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+    const size_t mbytes = sizeof(float) * h->D.mask_slots * h->D.d;
+    if (mask_vec && cudaMemcpy(mask_vec, h->b.mvec + (size_t)seq * h->D.mask_slots * h->D.d, mbytes, cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
     return ESP_OK;
 }
 
@@ -712,6 +726,19 @@ int esp_get_stats(esp_handle* h, esp_stats* out) {
     if (cudaMemcpy(&e, h->b.err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
     out->device_error = e;
     out->kernels_per_step = h->kernels_per_step;
+    return ESP_OK;
+}
+
+int esp_debug_wait_selftest(void* scratch, void* cuda_stream, int32_t* device_status_out) {
+    if (!scratch || !device_status_out) return ESP_E_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int* err = reinterpret_cast<int*>(scratch);
+    if (cudaMemsetAsync(err, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
+    if (tc_wait_selftest(err, s)) return ESP_E_CUDA;
+    int e = 0;
+    if (cudaMemcpyAsync(&e, err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return ESP_E_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return ESP_E_CUDA;
+    *device_status_out = e;
     return ESP_OK;
 }
 

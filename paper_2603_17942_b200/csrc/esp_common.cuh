@@ -68,6 +68,7 @@ struct Dims {
     // speculation
     int32_t k, K, KP, B, W, n_anchor, prune_parent, prune_root, ema_per_token;
     int32_t static_w[PROBES_MAX];   // fixed branch widths per depth; static_w[0] == 0: Algorithm 1
+    int32_t mask_slots;             // mask vectors per sequence: max(k, 1)
     float lambda;
 };
 

@@ -493,6 +493,22 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
 
 void tc_gemm_destroy(TcGemm* g) { delete g; }
 
+// A wait that nothing completes: exercises the time bound of mbar_wait without disturbing the device.
+__global__ void k_wait_selftest(int* err) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait(&bar, 0, &abort_flag)) set_error(err, DEV_E_WAIT_TIMEOUT);
+    }
+}
+int tc_wait_selftest(int* err_dev, cudaStream_t s) {
+    k_wait_selftest<<<1, 32, 0, s>>>(err_dev);
+    return cudaGetLastError() == cudaSuccess ? 0 : -1;
+}
+
 StreamK tc_gemm_streamk(const TcGemm* g) {
     StreamK k;
     k.partials = g ? g->p.partials : nullptr;

@@ -19,19 +19,30 @@ __global__ void k_rope_table(float* cs, float* sn, int n_pos, int h, float base)
     sn[i] = (float)sin(ang);
 }
 
-// m = (1/t) sum_j E[x_j]  (Eq. mask_init_mean); fp32 running sum in prompt order
+// Mask initialisation at prefill, m [slots][d].  mode 0: every slot = (1/t) sum_j E[x_j] (Eq. mask_init_mean; fp32
+// running sum in prompt order).  mode 1 ("Last K"): slot i = embedding of the i-th of the last `slots` prompt tokens.
 template <typename T>
-__global__ void k_mask_mean(const T* embed, const int32_t* prompt, int t, int d, float* m) {
+__global__ void k_mask_init(const T* embed, const int32_t* prompt, int t, int d, float* m, int slots, int mode) {
     int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= d) return;
+    if (mode == 1) {
+        for (int i = 0; i < slots; ++i) {
+            int src = t - slots + i;
+            if (src < 0) src = 0;
+            m[(size_t)i * d + j] = to_f32(embed[(size_t)prompt[src] * d + j]);
+        }
+        return;
+    }
     float acc = 0.f;
     for (int i = 0; i < t; ++i) acc = acc + to_f32(embed[(size_t)prompt[i] * d + j]);
-    m[j] = acc / (float)t;
+    const float mean = acc / (float)t;
+    for (int i = 0; i < slots; ++i) m[(size_t)i * d + j] = mean;
 }
 
-// Input rows of the block: E[token] for tree nodes, the shared mask vector for probe rows.
+// Input rows of the block: E[token] for tree nodes; probe j of a chain gets mask vector j (rows after the
+// tree nodes hold the chains back to back, k rows each).
 template <typename T>
-__global__ void k_assemble(const SeqState* states, const T* embed, const float* mvec, float* hres, int d) {
+__global__ void k_assemble(const SeqState* states, const T* embed, const float* mvec, float* hres, int d, int mask_slots) {
     pdl_wait();
     if (threadIdx.x == 0) pdl_launch_dependents();
     int seq = blockIdx.y, r = blockIdx.x;
@@ -55,7 +66,7 @@ __global__ void k_assemble(const SeqState* states, const T* embed, const float* 
             *reinterpret_cast<float4*>(out + j) = v;
         }
     } else {
-        const float* src = mvec + (size_t)seq * d;
+        const float* src = mvec + ((size_t)seq * mask_slots + (r - st->n_nodes) % mask_slots) * d;
 #pragma unroll 4
         for (int j = threadIdx.x * 4; j < d; j += blockDim.x * 4) *reinterpret_cast<float4*>(out + j) = *reinterpret_cast<const float4*>(src + j);
     }
@@ -814,14 +825,16 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     // ---- mask update, Eq. (mask_update_mean): m <- m + lambda (e - m)
     {
         const T* E = reinterpret_cast<const T*>(A.embed);
-        float* m = A.mvec + (size_t)seq * D.d;
+        float* m = A.mvec + (size_t)seq * D.mask_slots * D.d;
         for (int j = tid; j < D.d; j += nt) {
-            float mv = m[j];
-            for (int e = D.ema_per_token ? 0 : n_emit - 1; e < n_emit; ++e) {
-                float ev = to_f32(E[(size_t)s_out[e] * D.d + j]);
-                mv = __fadd_rn(mv, __fmul_rn(D.lambda, __fsub_rn(ev, mv)));
+            float ev[PROBES_MAX + 2];
+            const int e0 = D.ema_per_token ? 0 : n_emit - 1;
+            for (int e = e0; e < n_emit; ++e) ev[e] = to_f32(E[(size_t)s_out[e] * D.d + j]);
+            for (int slot = 0; slot < D.mask_slots; ++slot) {      // every mask vector follows the same update
+                float mv = m[(size_t)slot * D.d + j];
+                for (int e = e0; e < n_emit; ++e) mv = __fadd_rn(mv, __fmul_rn(D.lambda, __fsub_rn(ev[e], mv)));
+                m[(size_t)slot * D.d + j] = mv;
             }
-            m[j] = mv;
         }
     }
 
@@ -975,15 +988,15 @@ void launch_rope_table(float* cs, float* sn, int n_pos, int h, float base, cudaS
     int n = n_pos * (h / 2);
     k_rope_table<<<(n + 255) / 256, 256, 0, s>>>(cs, sn, n_pos, h, base);
 }
-void launch_mask_mean(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, cudaStream_t s) {
-    if (dtype == 0) k_mask_mean<float><<<(d + 127) / 128, 128, 0, s>>>((const float*)embed, prompt, t, d, m);
-    else k_mask_mean<__nv_bfloat16><<<(d + 127) / 128, 128, 0, s>>>((const __nv_bfloat16*)embed, prompt, t, d, m);
+void launch_mask_init(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, int slots, int mode, cudaStream_t s) {
+    if (dtype == 0) k_mask_init<float><<<(d + 127) / 128, 128, 0, s>>>((const float*)embed, prompt, t, d, m, slots, mode);
+    else k_mask_init<__nv_bfloat16><<<(d + 127) / 128, 128, 0, s>>>((const __nv_bfloat16*)embed, prompt, t, d, m, slots, mode);
 }
-void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int batch,
-                     cudaStream_t s, bool pdl) {
+void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int mask_slots,
+                     int batch, cudaStream_t s, bool pdl) {
     dim3 grid(RT, batch);
-    if (dtype == 0) launch_k(k_assemble<float>, grid, dim3(128), 0, s, pdl, st, (const float*)embed, mvec, hres, d);
-    else launch_k(k_assemble<__nv_bfloat16>, grid, dim3(128), 0, s, pdl, st, (const __nv_bfloat16*)embed, mvec, hres, d);
+    if (dtype == 0) launch_k(k_assemble<float>, grid, dim3(128), 0, s, pdl, st, (const float*)embed, mvec, hres, d, mask_slots);
+    else launch_k(k_assemble<__nv_bfloat16>, grid, dim3(128), 0, s, pdl, st, (const __nv_bfloat16*)embed, mvec, hres, d, mask_slots);
 }
 void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
                     float* copy_out, cudaStream_t s, bool pdl) {

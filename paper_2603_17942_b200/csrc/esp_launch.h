@@ -26,7 +26,7 @@ struct TreeArgs {
     SeqState* states;
     const Cand* topk;   // [batch*RT][KP_MAX]
     const float* lse;   // [batch*RT]
-    float* mvec;        // [batch][d]
+    float* mvec;        // [batch][mask_slots][d]
     const void* embed;
     void* kcache;       // [n_layers][batch][Hkv][cap][h]
     void* vcache;
@@ -36,9 +36,9 @@ struct TreeArgs {
 
 
 void launch_rope_table(float* cs, float* sn, int n_pos, int h, float base, cudaStream_t s);
-void launch_mask_mean(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, cudaStream_t s);
-void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int batch,
-                     cudaStream_t s, bool pdl);
+void launch_mask_init(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, int slots, int mode, cudaStream_t s);
+void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int mask_slots,
+                     int batch, cudaStream_t s, bool pdl);
 void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
                     float* copy_out, cudaStream_t s, bool pdl);
 // consumers of the split (EPI_PARTIAL) tensor-core GEMMs, bf16 models, one sequence
@@ -80,6 +80,7 @@ size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K);
 void tc_gemm_destroy(TcGemm* g);
 int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl);
 StreamK tc_gemm_streamk(const TcGemm* g);
+int tc_wait_selftest(int* err_dev, cudaStream_t s);
 int tc_gemm_tiles(const TcGemm* g);
 size_t tc_gemm_partial_bytes(int n_sm);
 int tc_gemm_counter_ints();

@@ -33,11 +33,12 @@ def to_device(w, device="cuda"):
 def c_spec(o: O.SpecCfg):
     return P.spec_cfg(n_probes=o.n_probes, topk=o.topk, max_nodes=o.max_nodes, expand_width=o.expand_width,
                       n_anchor=o.n_anchor, prune_parent=o.prune_parent, prune_root=o.prune_root,
-                      ema_per_token=o.ema_per_token, lam=o.lam, static_widths=o.static_widths)
+                      ema_per_token=o.ema_per_token, lam=o.lam, static_widths=o.static_widths,
+                      mask_init={"mean": 0, "last_k": 1, "given": 2}[o.mask_init])
 
 
 class ParityRun:
-    def __init__(self, shape, w_host, spec: O.SpecCfg, prompt, max_new, tol, gemm_impl=None, w_dev=None):
+    def __init__(self, shape, w_host, spec: O.SpecCfg, prompt, max_new, tol, gemm_impl=None, w_dev=None, given_mask=None):
         self.shape, self.spec, self.tol = shape, spec, tol
         self.model = O.OracleModel(shape, w_host)
         self.wd = w_dev if w_dev is not None else to_device(w_host)
@@ -51,6 +52,9 @@ class ParityRun:
         self.kc, self.vc = self.model.new_cache(len(prompt) + max_new + 16 + P.ESP_MAX_ROWS)
         self.L = 0
         self.m = None
+        self.given_mask = given_mask
+        if given_mask is not None:
+            self.h.set_mask(given_mask)
         self.near_ties = 0
         self.worst = 0.0
         self.emitted = []
@@ -105,9 +109,14 @@ class ParityRun:
         st = self.h.state()
         gl = self.logits.cpu().numpy()
         E = np.stack([self.model.embed(int(x)) for x in self.prompt])
-        self.m = O.mask_init_mean(E)
+        if sp.mask_init == "last_k" and k:
+            self.m = O.mask_init_last_k(E, k)
+        elif sp.mask_init == "given":
+            self.m = np.array(self.given_mask, np.float32).reshape(max(k, 1), -1)
+        else:
+            self.m = np.tile(O.mask_init_mean(E), (max(k, 1), 1))
         M = t + k
-        x = np.concatenate([E, np.tile(self.m, (k, 1))], 0) if k else E
+        x = np.concatenate([E, self.m[:k]], 0) if k else E
         want = np.zeros(M, np.uint8)
         want[t - 1:] = 1
         ref, kb, vb, _ = self.model.block_forward(self.kc, self.vc, 0, x, np.arange(M), np.tril(np.ones((M, M), np.uint8)), want)
@@ -143,7 +152,8 @@ class ParityRun:
         toks = self.h.step()
         st = self.h.state()
         gl = self.logits.cpu().numpy()
-        x = np.stack([self.model.embed(int(t)) if t >= 0 else self.m for t in blk.row_token])
+        probe_of_row = {row: j for (_, j), row in blk.probe_row.items()}
+        x = np.stack([self.model.embed(int(t)) if t >= 0 else self.m[probe_of_row[r] - 1] for r, t in enumerate(blk.row_token)])
         ref, kb, vb, _ = self.model.block_forward(self.kc, self.vc, self.L, x, self.L + blk.row_pos_off, blk.vis)
         rng = self._cmp_logits(gl[:blk.m], ref, f"step {len(self.accepts)}")
         self._check_selection(gl, st, range(blk.n_nodes), range(blk.n_nodes, blk.m))

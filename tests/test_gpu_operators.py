@@ -184,3 +184,21 @@ def test_tree_attention_long_context_against_oracle():
     got = out[0, :M].float().cpu().numpy()
     assert np.isfinite(got).all()
     assert np.abs(got - ref).max() <= 2e-2
+
+
+def test_bounded_wait_gives_up_and_leaves_the_context_usable():
+    """A barrier that nothing signals: the kernel's wait must run out (about 50 ms), report the wait-timeout
+    code through the error word and return; the next kernel on the same context works."""
+    import time
+    scratch = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    t0 = time.perf_counter()
+    status = P.esp_debug_wait_selftest(scratch)
+    dt = time.perf_counter() - t0
+    assert status == 1                      # DEV_E_WAIT_TIMEOUT
+    assert 0.03 < dt < 2.0
+    g = torch.Generator().manual_seed(1)
+    x = torch.randn(4, 64, generator=g).bfloat16()
+    w = (torch.randn(128, 64, generator=g) * 0.05).bfloat16().cuda()
+    got = _gemm(0, x, w, 4)
+    ref = O.linear(x.float().numpy(), w.cpu())
+    assert np.abs(got - ref).max() <= 2e-5 * np.abs(ref).max()

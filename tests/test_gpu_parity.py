@@ -56,6 +56,29 @@ def test_tiny_fp32_static_tree_parity(pu, widths, n_anchor):
     run.close()
 
 
+@pytest.mark.parametrize("mode", ["last_k", "sample", "mu_plus_5_sigma"])
+def test_tiny_fp32_mask_init_variants_parity(pu, mode):
+    """Mask initialisations of Section 4: the last k prompt embeddings, a draw from N(mu, sigma^2 I) with the
+    embedding table's mean and standard deviation (drawn here, handed over through esp_set_mask), mu + 5 sigma."""
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=3, gain_jitter=True, std=0.3)
+    prompt = synth.make_prompt(shape.vocab, 50, 8)
+    k = 3
+    given = None
+    if mode != "last_k":
+        emb = w["embed"].float().numpy()
+        mu, sigma = float(emb.mean()), float(emb.std())
+        rng = np.random.default_rng(4)
+        given = (mu + sigma * rng.standard_normal((k, shape.d_model))).astype(np.float32) if mode == "sample" \
+            else np.full((k, shape.d_model), mu + 5 * sigma, np.float32)
+    spec = O.SpecCfg(n_probes=k, topk=4, max_nodes=20, expand_width=0, n_anchor=1,
+                     mask_init="last_k" if mode == "last_k" else "given")
+    run = pu.ParityRun(shape, w, spec, prompt, 24, TOL_FP32, given_mask=given)
+    out = run.run()
+    assert out == O.greedy_generate(O.OracleModel(shape, w), prompt, 24, 256)
+    run.close()
+
+
 def test_tiny_fp32_nontrivial_stream(pu):
     """Same model family with wider weights and jittered norm gains, so the stream is not one repeated token."""
     shape = synth.TINY

@@ -308,3 +308,35 @@ def test_static_tree_generation_is_lossless_and_has_the_papers_block_size(widths
             assert rec["block"].m == esp.block_complexity(k, widths)
     if n_anchor == 0:
         assert full > 0
+
+
+# ---------------------------------------------------------------- mask initialisations (Section 4, mask designs)
+def test_mask_init_variants():
+    shape = synth.TINY.replace(n_layers=2, d_model=64, n_q_heads=4, n_kv_heads=2, head_dim=16, d_ffn=160, vocab=97)
+    w = synth.make_weights(shape, seed=23, gain_jitter=True, std=0.3)
+    model = esp.OracleModel(shape, w)
+    prompt = synth.make_prompt(shape.vocab, 13, 5)
+    E = np.stack([model.embed(int(x)) for x in prompt])
+    ref = esp.greedy_generate(model, prompt, 24, 128)
+    # Last K: the k masks are the embeddings of the last k prompt tokens, in prompt order
+    lk = esp.mask_init_last_k(E, 3)
+    assert np.array_equal(lk, E[-3:]) and np.array_equal(esp.mask_init_last_k(E[:2], 3), np.stack([E[0], E[0], E[1]]))
+    base = esp.SpecCfg(n_probes=3, topk=4, max_nodes=12, expand_width=0, n_anchor=1)
+    runs = {}
+    for mode in ("mean", "last_k", "given"):
+        dec = esp.EspOracle(model, esp.SpecCfg(**{**base.__dict__, "mask_init": mode}), 256)
+        if mode == "given":
+            dec.set_mask(np.tile(esp.mask_init_mean(E), (3, 1)))      # the prompt mean, given from outside
+        assert dec.generate(prompt, 24) == ref                        # lossless whatever the masks are
+        runs[mode] = dec
+    # giving the prompt mean from outside is the mean initialisation: same trees, same masks, step by step
+    a, b = runs["mean"], runs["given"]
+    assert a.accept_hist == b.accept_hist and np.array_equal(a.m, b.m)
+    assert all(np.array_equal(x["tree"].tokens, y["tree"].tokens) for x, y in zip(a.log, b.log) if x["kind"] == "step")
+    # Last K starts from different vectors per mask, and every vector follows Eq. (mask_update_mean)
+    c = runs["last_k"]
+    want = lk.copy()
+    for y in c.emitted:
+        want = esp.mask_update(want, model.embed(y), base.lam)
+    np.testing.assert_allclose(c.m, want, rtol=0, atol=1e-6)
+    assert not np.allclose(c.m[0], c.m[2])
