@@ -162,7 +162,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.sk_tables = c.take<TileSrc>(4 * SK_TABLE_TILES);
     o.packed = nullptr;
     o.pk_qkv = o.pk_o = o.pk_gu = o.pk_down = o.pk_lm = o.pk_layer = 0;
-    if (dtype == 1 && D.batch == 1) {
+    if (dtype == 1) {
         const int32_t dq = D.Hq * D.h, dkv = D.Hkv * D.h;
         const int32_t r1[3] = {dq, dkv, dkv}, r2[3] = {D.d, 0, 0}, r3[3] = {D.F, D.F, 0}, r5[3] = {D.V, 0, 0};
         o.pk_qkv = tc_gemm_packed_bytes(EPI_PARTIAL, r1, D.d);
@@ -198,7 +198,7 @@ struct esp_handle {
     bool prof = false;           // record an event after every kernel group
     bool use_pdl = true;         // programmatic dependent launch between the kernels of a step
     bool use_graph = true;       // replay the step's launch sequence as a CUDA graph
-    struct StepGraph { int n_split; cudaGraphExec_t exec; int kernels; };
+    struct StepGraph { unsigned long long key; cudaGraphExec_t exec; int kernels; };
     std::vector<StepGraph> graphs;
     std::vector<cudaEvent_t> ev;
     std::vector<int> ev_kind;
@@ -225,12 +225,15 @@ void mark(esp_handle* h, int kind) {
 
 void* layer_ptr(void* base, size_t stride_bytes, int l) { return reinterpret_cast<char*>(base) + stride_bytes * l; }
 
-EpiArgs base_epi(esp_handle* h, int n_out) {
+// One forward pass covers sequences [s0, s0 + nb): all of them on the CUDA-core path (nb = max_batch), one at a
+// time on the tensor-core path (nb = 1; the activation buffers are shared, only the sequence state, the KV
+// cache, the mask vectors and the selection results are per sequence).
+EpiArgs base_epi(esp_handle* h, int n_out, int s0, int nb) {
     EpiArgs a;
     memset(&a, 0, sizeof(a));
     a.n_out = n_out;
-    a.st = h->b.states;
-    a.batch = h->D.batch;
+    a.st = h->b.states + s0;
+    a.batch = nb;
     a.Hq = h->D.Hq; a.Hkv = h->D.Hkv; a.h = h->D.h; a.cap = h->D.cap; a.qk_norm = h->D.qk_norm;
     a.rms_eps = h->D.rms_eps;
     a.rope_cos = h->b.rope_cos; a.rope_sin = h->b.rope_sin;
@@ -250,31 +253,34 @@ int run_gemm(esp_handle* h, TcGemm* plan, int epi, int n_tiles, const void* cons
 // Tensor-core path (bf16, one sequence): the QKV, O and down GEMMs store stream-K partials that the next
 // kernel sums (k_qkv_finish; k_resid_norm = residual add + RMSNorm), gate/up and the LM head finish in-kernel.
 // CUDA-core path (fp32 models, batched bf16): the same layer with every epilogue fused in the GEMM.
-int forward(esp_handle* h, bool with_lm, int dcap) {
+int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc) {
     const Dims& D = h->D;
     Buffers& b = h->b;
     cudaStream_t s = h->stream;
     const int dq = D.Hq * D.h, dkv = D.Hkv * D.h;
+    const size_t es = h->dtype ? 2 : 4;
     int Lmax = 0;
-    for (int i = 0; i < D.batch; ++i) Lmax = h->L_host[i] > Lmax ? h->L_host[i] : Lmax;
+    for (int i = s0; i < s0 + nb; ++i) Lmax = h->L_host[i] > Lmax ? h->L_host[i] : Lmax;
     const int n_split_launch = (Lmax + D.split_len - 1) / D.split_len;
-    const bool tc = h->dtype == 1 && h->gemm_impl == 0 && h->p_lm != nullptr;
     const bool pdl = h->use_pdl && !h->prof;
+    SeqState* st0 = b.states + s0;
+    const size_t kv_seq_off = (size_t)s0 * D.Hkv * D.cap * D.h * es;   // this pass's first sequence inside a layer's cache
+    float* mvec0 = b.mvec + (size_t)s0 * D.mask_slots * D.d;
     StreamK pending;   // partials of the last down projection, summed by the next norm
     pending.partials = nullptr; pending.table = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2;
     mark(h, -1);
-    launch_assemble(h->dtype, b.states, h->embed, b.mvec, b.hres, D.d, D.mask_slots, D.batch, s, false);
+    launch_assemble(h->dtype, st0, h->embed, mvec0, b.hres, D.d, D.mask_slots, nb, s, false);
     h->launches++;
     for (int l = 0; l < D.n_layers; ++l) {
-        if (tc) launch_resid_norm(b.states, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
-        else launch_rmsnorm(h->dtype, b.states, b.hres, h->na[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s, pdl);
+        if (tc) launch_resid_norm(st0, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
+        else launch_rmsnorm(h->dtype, st0, b.hres, h->na[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
         {
-            EpiArgs a = base_epi(h, dq + 2 * dkv);
+            EpiArgs a = base_epi(h, dq + 2 * dkv, s0, nb);
             a.q_out = b.qbuf;
-            a.kcache = layer_ptr(b.kcache, h->layer_kv_stride, l);
-            a.vcache = layer_ptr(b.vcache, h->layer_kv_stride, l);
+            a.kcache = reinterpret_cast<char*>(layer_ptr(b.kcache, h->layer_kv_stride, l)) + kv_seq_off;
+            a.vcache = reinterpret_cast<char*>(layer_ptr(b.vcache, h->layer_kv_stride, l)) + kv_seq_off;
             a.q_norm = D.qk_norm ? h->qn[l] : nullptr;
             a.k_norm = D.qk_norm ? h->kn[l] : nullptr;
             const void* w[3] = {h->wq[l], h->wk[l], h->wv[l]};
@@ -292,27 +298,26 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             AttnArgs a;
             memset(&a, 0, sizeof(a));
             a.q = b.qbuf;
-            a.kc = layer_ptr(b.kcache, h->layer_kv_stride, l);
-            a.vc = layer_ptr(b.vcache, h->layer_kv_stride, l);
+            a.kc = reinterpret_cast<char*>(layer_ptr(b.kcache, h->layer_kv_stride, l)) + kv_seq_off;
+            a.vc = reinterpret_cast<char*>(layer_ptr(b.vcache, h->layer_kv_stride, l)) + kv_seq_off;
             a.out = b.attn_out;
             a.part_o = b.part_o; a.part_ml = b.part_ml;
-            a.st = b.states;
+            a.st = st0;
             a.Hq = D.Hq; a.Hkv = D.Hkv; a.h = D.h; a.cap = D.cap; a.split_len = D.split_len; a.n_split_max = D.n_split_max;
             a.dcap = dcap;
             a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
             a.err = b.err;
-            const bool mma = h->gemm_impl == 0 && !h->p_attn.empty();
-            if (mma) {
-                if (attn_tc_launch(h->p_attn[l], a, D.batch, n_split_launch, s, pdl)) return ESP_E_BADCFG;
+            if (tc) {
+                if (attn_tc_launch(h->p_attn[(size_t)l * D.batch + s0], a, 1, n_split_launch, s, pdl)) return ESP_E_BADCFG;
                 h->launches += n_split_launch > 0 ? 2 : 1;
             } else {
-                if (launch_attn_simt(h->dtype, a, D.batch, n_split_launch, true, s, pdl)) return ESP_E_BADCFG;
+                if (launch_attn_simt(h->dtype, a, nb, n_split_launch, true, s, pdl)) return ESP_E_BADCFG;
                 h->launches += n_split_launch > 0 ? 2 : 1;
             }
             mark(h, KIND_ATTN);
         }
         {
-            EpiArgs a = base_epi(h, D.d);
+            EpiArgs a = base_epi(h, D.d, s0, nb);
             a.hres = b.hres;
             const void* w[3] = {h->wo[l], nullptr, nullptr};
             const int32_t rows[3] = {D.d, 0, 0};
@@ -320,12 +325,12 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             if (rc) return rc;
             mark(h, KIND_O);
         }
-        if (tc) launch_resid_norm(b.states, b.hres, tc_gemm_streamk(h->p_o[l]), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
-        else launch_rmsnorm(h->dtype, b.states, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, D.batch, nullptr, s, pdl);
+        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(h->p_o[l]), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
+        else launch_rmsnorm(h->dtype, st0, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
         {
-            EpiArgs a = base_epi(h, D.F);
+            EpiArgs a = base_epi(h, D.F, s0, nb);
             a.act_out = b.act;
             const void* w[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t rows[3] = {D.F, D.F, 0};
@@ -333,13 +338,13 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
             if (rc) return rc;
             mark(h, KIND_GATEUP);
             if (tc) {
-                launch_swiglu_finish(b.states, tc_gemm_streamk(h->p_gu[l]), b.act, D.F, s, pdl);
+                launch_swiglu_finish(st0, tc_gemm_streamk(h->p_gu[l]), b.act, D.F, s, pdl);
                 h->launches++;
                 mark(h, KIND_MISC);
             }
         }
         {
-            EpiArgs a = base_epi(h, D.d);
+            EpiArgs a = base_epi(h, D.d, s0, nb);
             a.hres = b.hres;
             const void* w[3] = {h->wd[l], nullptr, nullptr};
             const int32_t rows[3] = {D.d, 0, 0};
@@ -350,23 +355,37 @@ int forward(esp_handle* h, bool with_lm, int dcap) {
         }
     }
     if (with_lm) {
-        if (tc) launch_resid_norm(b.states, b.hres, pending, h->final_norm, b.xn, D.d, D.rms_eps, h->dbg_hidden, s, pdl);
-        else launch_rmsnorm(h->dtype, b.states, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, D.batch, h->dbg_hidden, s, pdl);
+        float* dbg_hidden = h->dbg_hidden ? h->dbg_hidden + (size_t)s0 * RT * D.d : nullptr;
+        if (tc) launch_resid_norm(st0, b.hres, pending, h->final_norm, b.xn, D.d, D.rms_eps, dbg_hidden, s, pdl);
+        else launch_rmsnorm(h->dtype, st0, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, nb, dbg_hidden, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
         const int n_tiles = (D.V + TILE_N - 1) / TILE_N;
-        EpiArgs a = base_epi(h, D.V);
-        a.cand = b.cand; a.cand_ms = b.cand_ms; a.n_tiles = n_tiles; a.logits_dump = h->dbg_logits;
+        EpiArgs a = base_epi(h, D.V, s0, nb);
+        a.cand = b.cand; a.cand_ms = b.cand_ms; a.n_tiles = n_tiles;
+        a.logits_dump = h->dbg_logits ? h->dbg_logits + (size_t)s0 * RT * D.V : nullptr;
         const void* w[3] = {h->lm_head, nullptr, nullptr};
         const int32_t rows[3] = {D.V, 0, 0};
         int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl);
         if (rc) return rc;
         mark(h, KIND_LMHEAD);
-        launch_topk_merge(b.states, b.cand, b.cand_ms, n_tiles, D.KP, D.batch, b.topk, b.lse, s, pdl);
+        launch_topk_merge(st0, b.cand, b.cand_ms, n_tiles, D.KP, nb, b.topk + (size_t)s0 * RT * KP_MAX, b.lse + (size_t)s0 * RT, s, pdl);
         h->launches++;
         mark(h, KIND_SELECT);
     }
     return cuda_ok(cudaGetLastError());
+}
+
+// Forward over the sequences that take part: `only_seq` (prefill) or every prefilled sequence (a step).
+int forward(esp_handle* h, bool with_lm, int dcap, int only_seq) {
+    const bool tc = h->dtype == 1 && h->gemm_impl == 0 && h->p_lm != nullptr;
+    if (!tc) return forward_pass(h, with_lm, dcap, 0, h->D.batch, false);
+    for (int i = 0; i < h->D.batch; ++i) {
+        if (only_seq >= 0 ? i != only_seq : !h->ready[i]) continue;
+        const int rc = forward_pass(h, with_lm, dcap, i, 1, true);
+        if (rc) return rc;
+    }
+    return ESP_OK;
 }
 
 int tree_step(esp_handle* h) {
@@ -461,14 +480,18 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
     }
     launch_rope_table(h->b.rope_cos, h->b.rope_sin, D.cap, D.h, model->rope_base, h->stream);
     if (model->dtype == 1 && attn_tc_supported(D.h, D.Hq, D.Hkv)) {
+        const size_t seq_bytes = (size_t)D.Hkv * D.cap * D.h * 2;
         for (int l = 0; l < D.n_layers; ++l) {
-            AttnTc* t = nullptr;
-            if (attn_tc_create(&t, h->b.qbuf, layer_ptr(h->b.kcache, h->layer_kv_stride, l), layer_ptr(h->b.vcache, h->layer_kv_stride, l),
-                               D.batch, D.Hq, D.Hkv, D.cap)) { esp_free(h); return ESP_E_CUDA; }
-            h->p_attn.push_back(t);
+            for (int i = 0; i < D.batch; ++i) {      // one sequence per pass: its slice of the layer's cache, the shared q buffer
+                AttnTc* t = nullptr;
+                char* kc = reinterpret_cast<char*>(layer_ptr(h->b.kcache, h->layer_kv_stride, l)) + seq_bytes * i;
+                char* vc = reinterpret_cast<char*>(layer_ptr(h->b.vcache, h->layer_kv_stride, l)) + seq_bytes * i;
+                if (attn_tc_create(&t, h->b.qbuf, kc, vc, 1, D.Hq, D.Hkv, D.cap)) { esp_free(h); return ESP_E_CUDA; }
+                h->p_attn.push_back(t);
+            }
         }
     }
-    if (model->dtype == 1 && D.batch == 1) {
+    if (model->dtype == 1) {
         const int dq = D.Hq * D.h, dkv = D.Hkv * D.h;
         bool ok = true;
         for (int l = 0; l < D.n_layers && ok; ++l) {
@@ -498,8 +521,6 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
         const int32_t r5[3] = {D.V, 0, 0};
         ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
         if (!ok) { esp_free(h); return ESP_E_CUDA; }
-    } else if (model->dtype == 1) {
-        h->gemm_impl = 1;  // batched rows: CUDA-core path until the tensor-core kernel tiles over sequences
     }
     if (cudaStreamSynchronize(h->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) { esp_free(h); return ESP_E_CUDA; }
     *handle_out = h;
@@ -525,7 +546,7 @@ int esp_prefill(esp_handle* h, int32_t seq, const int32_t* prompt, int32_t n_pro
         const int last = off + cn == n_prompt;
         launch_setup_chain(h->b.states, seq, h->b.prompt_dev, off, cn, last, h->D.k, s);
         h->L_host[seq] = off;
-        int rc = forward(h, last, DCAP_PREFILL);
+        int rc = forward(h, last, DCAP_PREFILL, seq);
         if (rc) return rc;
         rc = tree_step(h);
         if (rc) return rc;
@@ -557,24 +578,29 @@ int esp_step_async(esp_handle* h) {
     if (h->use_graph && !h->prof) {
         // The launch sequence of a step depends on the host only through the number of attention splits;
         // every other quantity (L, row counts, the tree) is read from device state by the kernels.
-        const int n_split = (Lmax + h->D.split_len - 1) / h->D.split_len;
+        // (key: which sequences take part and how many cache splits each one's attention launches)
+        unsigned long long key = 1469598103934665603ull;
+        for (int i = 0; i < h->D.batch; ++i) {
+            const unsigned long long v = h->ready[i] ? 1ull + (unsigned long long)((h->L_host[i] + h->D.split_len - 1) / h->D.split_len) : 0ull;
+            key = (key ^ v) * 1099511628211ull;
+        }
         esp_handle::StepGraph* g = nullptr;
         for (auto& e : h->graphs)
-            if (e.n_split == n_split) g = &e;
+            if (e.key == key) g = &e;
         if (!g) {
             cudaGraph_t graph = nullptr;
             cudaGraphExec_t exec = nullptr;
             const int before = h->launches;
             bool ok = cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
             if (ok) {
-                int r1 = forward(h, true, DCAP_STEP);
+                int r1 = forward(h, true, DCAP_STEP, -1);
                 int r2 = r1 ? r1 : tree_step(h);
                 ok = cudaStreamEndCapture(h->stream, &graph) == cudaSuccess && !r2 && graph;
             }
             if (ok) ok = cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess;
             if (graph) cudaGraphDestroy(graph);
             if (ok) {
-                h->graphs.push_back({n_split, exec, h->launches - before});
+                h->graphs.push_back({key, exec, h->launches - before});
                 g = &h->graphs.back();
             } else {
                 cudaGetLastError();      // capture is not available here: launch directly from now on
@@ -589,7 +615,7 @@ int esp_step_async(esp_handle* h) {
     }
     if (!done) {
         const int before = h->launches;
-        rc = forward(h, true, DCAP_STEP);
+        rc = forward(h, true, DCAP_STEP, -1);
         if (rc) return rc;
         rc = tree_step(h);
         h->kernels_per_step = h->launches - before;

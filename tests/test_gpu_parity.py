@@ -192,6 +192,38 @@ def test_bf16_forced_acceptance_bitwise_equals_greedy(pu):
     h.close()
 
 
+def test_bf16_batch_of_sequences_equals_each_sequence_alone(pu):
+    """Sequences are independent (each has its own cache, masks and tree): a handle holding three of them,
+    prefilled with different prompts (one of them later than the others), must emit for each exactly the stream
+    a single-sequence handle emits -- on the tensor-core path, which takes the sequences one at a time."""
+    import paper_2603_17942_b200 as P
+    shape = BF16_SMALL
+    w = synth.make_weights(shape, seed=5, gain_jitter=True, std=0.05)
+    wd = pu.to_device(w)
+    spec = O.SpecCfg(n_probes=3, topk=5, max_nodes=16, expand_width=0, n_anchor=1)
+    prompts = [synth.make_prompt(shape.vocab, n, 10 + i) for i, n in enumerate((90, 300, 17))]
+    n_new, max_seq = 24, 400
+    alone = []
+    for pr in prompts:
+        h1 = P.Handle(shape, pu.c_spec(spec), wd, max_seq_len=max_seq)
+        alone.append(h1.generate(pr, n_new))
+        h1.close()
+    h = P.Handle(shape, pu.c_spec(spec), wd, max_seq_len=max_seq, max_batch=3)
+    outs = [[h.prefill(prompts[0], 0)], [h.prefill(prompts[1], 1)], []]
+    for step in range(200):
+        if step == 3:
+            outs[2].append(h.prefill(prompts[2], 2))          # a sequence joins while the others are decoding
+        if all(len(o) >= n_new for o in outs):
+            break
+        P.esp_step(h.h, h.tokens_out, h.n_out)
+        for i in range(3):
+            outs[i].extend(int(t) for t in h.tokens_out[i, :h.n_out[i]])
+    assert h.stats().device_error == 0
+    for i in range(3):
+        assert outs[i][:n_new] == alone[i], f"sequence {i}"
+    h.close()
+
+
 # ------------------------------------------------------------------ config 3 / 4 kernel shapes (full width, few layers)
 @pytest.mark.parametrize("base,topk,B", [(synth.LLAMA3_8B, 10, 64), (synth.QWEN3_8B, 8, 48)])
 def test_full_width_shapes_parity(pu, base, topk, B):
