@@ -309,8 +309,11 @@ def run_ours(args, shape, plen, k, K, B):
     spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1)
     max_seq = plen + (k + 1) * (2 * steps + 2 * warm + 16) + 64
     stream = torch.cuda.Stream()
-    h = P.Handle(shape, spec, w, max_seq_len=max_seq, stream=stream)
+    nbatch = max(1, args.batch)
+    h = P.Handle(shape, spec, w, max_seq_len=max_seq, max_batch=nbatch, stream=stream)
     h.prefill(prompt)
+    for i in range(1, nbatch):
+        h.prefill(synth.make_prompt(shape.vocab, plen, 1000 * rank + i), i)
 
     def emitted_steps():
         st = h.stats()
@@ -353,11 +356,12 @@ def run_ours(args, shape, plen, k, K, B):
     te0 = time.perf_counter()
     e2e_tokens = 0
     for _ in range(steps):
-        e2e_tokens += len(h.step())
+        h.step()
+        e2e_tokens += int(h.n_out.sum())
     torch.cuda.synchronize()
     te1 = time.perf_counter()
     e2e_ms = (te1 - te0) * 1e3
-    d2h = (P.ESP_MAX_PROBES + 4) * 4 + 4
+    d2h = nbatch * (P.ESP_MAX_PROBES + 4) * 4 + 4
 
     # ---- per-kernel-group device times (events between groups), for the roofline of the dominant kernel
     n_prof = min(steps, 20)
@@ -370,7 +374,7 @@ def run_ours(args, shape, plen, k, K, B):
 
     # ---- greedy decoding with the same kernels (one row per step), for context
     greedy_tok_s = None
-    if rank == 0 and not args.no_greedy:
+    if rank == 0 and not args.no_greedy and nbatch == 1:
         hg = P.Handle(shape, P.spec_cfg(), w, max_seq_len=plen + 2 * steps + 64, stream=stream)
         hg.prefill(prompt)
         for _ in range(warm):
@@ -387,7 +391,7 @@ def run_ours(args, shape, plen, k, K, B):
         hg.close()
 
     replay = None
-    if rank == 0 and not args.no_greedy:
+    if rank == 0 and not args.no_greedy and nbatch == 1:
         replay = replay_leg(P, shape, w, prompt, stream, k, B, min(256, steps))
 
     # ---- aggregate over ranks: slowest rank's time, all ranks' tokens
@@ -402,16 +406,17 @@ def run_ours(args, shape, plen, k, K, B):
         gu_ms = kinds["gateup_gemm"] / shape.n_layers
         gu_ach = gu_bytes / (gu_ms * 1e-3) / 1e9 if gu_ms > 0 else None
         wbytes, kvbytes = algorithmic_bytes(shape, 0.5 * (L0 + L1), rows)
+        kvbytes *= nbatch                    # weights once per step, every sequence's cache
         step_ms = ms / steps
         step_ach = (wbytes + kvbytes) / (step_ms * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
             "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": f"{args.config}-shape bf16 decoder, random-init seeded weights, b=1",
-                       "prompt_len": plen, "n_probes": k, "topk": K, "max_nodes": B, "rows_per_step": rows,
+            "config": {"workload": f"{args.config}-shape bf16 decoder, random-init seeded weights, b={nbatch}",
+                       "prompt_len": plen, "batch": nbatch, "n_probes": k, "topk": K, "max_nodes": B, "rows_per_step": rows,
                        "replicas": world, "l2": "inputs exceed L2 (weights are re-streamed every step)"},
-            "mean_accepted_len": tokens / (steps * world),
+            "mean_accepted_len": tokens / (steps * world * nbatch),
             "clocks": clocks,
             "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
                     "d2h_bytes_per_step": d2h,
@@ -510,6 +515,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="llama3-8b", choices=sorted(WORKLOADS) + ["attention-op"])
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt / KV length")
+    ap.add_argument("--batch", type=int, default=1, help="independent sequences in one handle (long-context / batch sweep)")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer count (smaller captures under a profiler)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-greedy", action="store_true", help="skip the greedy-decoding leg")
