@@ -363,7 +363,7 @@ __device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], floa
 
 // The tail: positions T0..P in position order, lane j owns key j of a 32-key chunk (chunk grid anchored at T0).
 // Then the merge: bulk partials in split order, the tail last; a lane owns 4 of the 128 output dims.
-__global__ void __launch_bounds__(128) k_attn_tail_merge_tc(AttnArgs a) {
+__global__ void __launch_bounds__(128, 4) k_attn_tail_merge_tc(AttnArgs a) {
     __shared__ float s_qall[4][HD];
     if (threadIdx.x == 0) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

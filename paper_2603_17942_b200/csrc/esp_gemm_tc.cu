@@ -41,7 +41,10 @@ namespace {
 using namespace tc;
 
 constexpr int BK = 64;                       // k elements per stage (128 bytes of bf16)
-constexpr int STAGES = 6;
+// Ring depth.  The bytes in flight per SM (depth x 16 KB of weights) over the load round trip bound the stream rate,
+// and the ring is also what is requested before the preceding kernel has finished: deeper is better.  The
+// partial-only kernel keeps no accumulator copy in shared memory and spends that room on the ring.
+__host__ __device__ constexpr int stages_of(int epi) { return epi == EPI_PARTIAL ? 8 : 6; }
 constexpr int A_BYTES = TILE_N * BK * 2;     // 16384
 constexpr int B_BYTES = RT * BK * 2;         // 10240
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -119,10 +122,11 @@ template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constant__ TcParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int STAGES = stages_of(EPI);
     unsigned char* stages = smem;
     float* s_acc = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES);
-    float* s_aux = s_acc + RT * ACC_LD;
-    uint64_t* full = reinterpret_cast<uint64_t*>(s_aux + RT * 4);
+    float* s_aux = s_acc + (EPI == EPI_PARTIAL ? 0 : RT * ACC_LD);
+    uint64_t* full = reinterpret_cast<uint64_t*>(s_aux + (EPI == EPI_PARTIAL ? 0 : RT * 4));
     uint64_t* empty = full + STAGES;
     uint64_t* tfull = empty + STAGES;
     uint64_t* tempty = tfull + 2;
@@ -382,7 +386,9 @@ __global__ void __launch_bounds__(128) k_pack_weights(PackArgs g, unsigned char*
     }
 }
 
-constexpr size_t SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + sizeof(float) * (RT * ACC_LD + RT * 4) + 256;
+constexpr size_t smem_bytes_of(int epi) {
+    return 1024 + (size_t)stages_of(epi) * STAGE_BYTES + (epi == EPI_PARTIAL ? 0 : sizeof(float) * (RT * ACC_LD + RT * 4)) + 256;
+}
 
 // [rows][K] bf16 row-major, box = 64 k-elements x box_rows rows, 128-byte swizzle, out-of-range reads give zero
 int make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
@@ -529,10 +535,10 @@ int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl) 
     case E: {                                                                                                 \
         static bool attr_set = false;                                                                         \
         if (!attr_set) {                                                                                      \
-            if (cudaFuncSetAttribute(k_gemm_tc<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return ESP_E_CUDA; \
+            if (cudaFuncSetAttribute(k_gemm_tc<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(E)) != cudaSuccess) return ESP_E_CUDA; \
             attr_set = true;                                                                                  \
         }                                                                                                     \
-        e = launch_k(k_gemm_tc<E>, dim3(p.grid), dim3(NUM_THREADS), SMEM_BYTES, s, pdl, p);                    \
+        e = launch_k(k_gemm_tc<E>, dim3(p.grid), dim3(NUM_THREADS), smem_bytes_of(E), s, pdl, p);                    \
     } break;
     switch (p.epi) {
         ESP_TC_CASE(EPI_STORE_F32)
