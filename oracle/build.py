@@ -5,7 +5,7 @@ import os
 import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-SRC = os.path.join(HERE, "transformer.c")
+SRCS = [os.path.join(HERE, "transformer.c"), os.path.join(HERE, "sampling.c")]
 LIB = os.path.join(HERE, "liboracle.so")
 
 
@@ -16,10 +16,10 @@ def build(force: bool = False) -> str:
     fp32 operation, so the oracle's results do not depend on whether the
     host CPU has fused multiply-add.
     """
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= os.path.getmtime(SRC):
+    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= max(os.path.getmtime(s) for s in SRCS):
         return LIB
     cmd = ["gcc", "-O3", "-march=x86-64-v3", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
-           "-Wall", "-o", LIB, SRC, "-lm"]
+           "-Wall", "-o", LIB] + SRCS + ["-lm"]
     subprocess.run(cmd, check=True)
     return LIB
 

@@ -52,6 +52,12 @@ def _load():
         _lib.orc_tree_attention.restype = ctypes.c_int
         _lib.orc_linear.restype = ctypes.c_int
         _lib.orc_num_threads.restype = ctypes.c_int
+        _lib.orc_det_logf.restype = ctypes.c_float
+        _lib.orc_det_logf.argtypes = [ctypes.c_float]
+        _lib.orc_gumbel_from_bits.restype = ctypes.c_float
+        _lib.orc_gumbel_from_bits.argtypes = [ctypes.c_uint32]
+        _lib.orc_uniform_from_bits.restype = ctypes.c_float
+        _lib.orc_uniform_from_bits.argtypes = [ctypes.c_uint32]
     return _lib
 
 
@@ -191,6 +197,8 @@ class SpecCfg:
     lam: float = 0.1
     static_widths: Tuple[int, ...] = ()   # fixed branch widths [K_1..K_k] (Section 4.2); empty = dynamic tree
     mask_init: str = "mean"               # "mean" (Eq. mask_init_mean) | "last_k" | "given" (Section 4, mask designs)
+    temperature: float = 0.0              # 0 = greedy matching; > 0 = sample matching at that temperature (Section 4)
+    seed: int = 0                         # 64-bit seed of the sampling noise
 
     @property
     def k_prime(self) -> int:
@@ -229,6 +237,38 @@ def topk_desc(logits: np.ndarray, kp: int) -> Tuple[np.ndarray, np.ndarray]:
     ids = np.arange(logits.shape[0])
     order = np.lexsort((ids, -logits.astype(np.float64)))[:kp]
     return order.astype(np.int32), logits[order].astype(_F32)
+
+
+def philox4x32_10(ctr: Sequence[int], key: Sequence[int]) -> List[int]:
+    """One Philox4x32-10 block (Salmon et al., SC'11): 4 counter words, 2 key words -> 4 output words."""
+    c = (ctypes.c_uint32 * 4)(*[int(x) & 0xffffffff for x in ctr])
+    k = (ctypes.c_uint32 * 2)(*[int(x) & 0xffffffff for x in key])
+    o = (ctypes.c_uint32 * 4)()
+    _load().orc_philox4x32_10(c, k, o)
+    return [int(x) for x in o]
+
+
+def gumbel_noise(seed: int, position: int, n_vocab: int) -> np.ndarray:
+    """g(seed, position, v) for every token v: standard Gumbel noise, a pure function of its arguments."""
+    out = np.empty(n_vocab, dtype=_F32)
+    _load().orc_gumbel_noise(ctypes.c_uint32(seed & 0xffffffff), ctypes.c_uint32((seed >> 32) & 0xffffffff),
+                             ctypes.c_uint32(position), ctypes.c_int32(n_vocab), ctypes.c_void_p(out.ctypes.data))
+    return out
+
+
+def sample_scores(logits: np.ndarray, position: int, temperature: float, seed: int) -> np.ndarray:
+    """logits / T + g in fp32: one rounded multiply by fl(1/T), one rounded add."""
+    inv_t = _F32(1.0) / _F32(temperature)
+    return (np.asarray(logits, dtype=_F32) * inv_t).astype(_F32) + gumbel_noise(seed, position, len(logits))
+
+
+def next_token(logits: np.ndarray, position: int, spec: "SpecCfg") -> int:
+    """The base model's token for absolute position `position` given the logits of the row before it:
+    the arg-max (temperature 0, Section 2 first equation) or the Gumbel-max draw from softmax(logits / T)
+    (Section 4 "sample matching"); ties go to the lower token id."""
+    if spec.temperature > 0.0:
+        return int(topk_desc(sample_scores(logits, position, spec.temperature, spec.seed), 1)[0][0])
+    return int(topk_desc(logits, 1)[0][0])
 
 
 def log_sum_exp(logits: np.ndarray) -> np.float32:
@@ -515,7 +555,7 @@ class EspOracle:
         self.kc[:, :t] = kb[:, :t]
         self.vc[:, :t] = vb[:, :t]
         self.L = t
-        y = int(topk_desc(logits[t - 1], 1)[0][0])
+        y = next_token(logits[t - 1], t, sp)
         self._emit(y)
         if not sp.ema_per_token:
             self.m = mask_update(self.m, self.model.embed(y), sp.lam)
@@ -533,7 +573,8 @@ class EspOracle:
         x = self._rows_x(blk)
         pos = self.L + blk.row_pos_off
         logits, kb, vb, _ = self.model.block_forward(self.kc, self.vc, self.L, x, pos, blk.vis)
-        nxt = [int(topk_desc(logits[r], 1)[0][0]) for r in range(blk.n_nodes)]
+        # node r sits at position pos[r]; its logits decide the token at pos[r] + 1
+        nxt = [next_token(logits[r], int(pos[r]) + 1, sp) for r in range(blk.n_nodes)]
         path, out = verify_walk(tree, nxt)
         a = len(path) - 1
         # the accepted nodes' keys/values become cache entries (Appendix E: the cache grows by the
@@ -577,8 +618,11 @@ class EspOracle:
         return acceptance_length(len(self.emitted) - 1, self.steps) if self.steps else float("nan")
 
 
-def greedy_generate(model: OracleModel, prompt: Sequence[int], max_new: int, cap: int, return_logits=False):
-    """Plain autoregressive greedy decoding, one token per model call (Section 2, first equation)."""
+def greedy_generate(model: OracleModel, prompt: Sequence[int], max_new: int, cap: int, return_logits=False,
+                    spec: Optional[SpecCfg] = None):
+    """Plain autoregressive decoding, one token per model call (Section 2, first equation): greedy, or sampled
+    with spec.temperature / spec.seed when a spec with temperature > 0 is given."""
+    spec = spec if spec is not None else SpecCfg()
     kc, vc = model.new_cache(cap)
     t = len(prompt)
     E = np.stack([model.embed(int(x)) for x in prompt])
@@ -587,13 +631,13 @@ def greedy_generate(model: OracleModel, prompt: Sequence[int], max_new: int, cap
     logits, kb, vb, _ = model.block_forward(kc, vc, 0, E, np.arange(t), np.tril(np.ones((t, t), np.uint8)), want)
     kc[:, :t], vc[:, :t] = kb, vb
     L = t
-    out = [int(topk_desc(logits[t - 1], 1)[0][0])]
+    out = [next_token(logits[t - 1], t, spec)]
     all_logits = [logits[t - 1].copy()]
     while len(out) < max_new:
         x = model.embed(out[-1])[None]
         logits, kb, vb, _ = model.block_forward(kc, vc, L, x, np.array([L]), np.ones((1, 1), np.uint8))
         kc[:, L], vc[:, L] = kb[:, 0], vb[:, 0]
         L += 1
-        out.append(int(topk_desc(logits[0], 1)[0][0]))
+        out.append(next_token(logits[0], L, spec))
         all_logits.append(logits[0].copy())
     return (out, np.stack(all_logits)) if return_logits else out

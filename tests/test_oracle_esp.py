@@ -340,3 +340,102 @@ def test_mask_init_variants():
         want = esp.mask_update(want, model.embed(y), base.lam)
     np.testing.assert_allclose(c.m, want, rtol=0, atol=1e-6)
     assert not np.allclose(c.m[0], c.m[2])
+
+
+# ---------------------------------------------------------------- sampling verification (temperature > 0)
+def test_philox_known_answers():
+    """The counter-based generator against the published known-answer vectors."""
+    rows = _rows("philox4x32_10_kat.txt")
+    assert len(rows) == 3
+    for r in rows:
+        w = [int(x, 16) for x in r]
+        assert esp.philox4x32_10(w[0:4], w[4:6]) == w[6:10]
+
+
+def test_uniform_mapping_and_logarithm():
+    """u = (2n+1)/2^24 with n the top 23 bits: strictly inside (0,1) and exact; the written-out fp32 logarithm
+    agrees with the fp64 library logarithm to fp32 accuracy over the whole range the noise uses."""
+    lib = esp._load()
+    assert lib.orc_uniform_from_bits(0) == 2.0 ** -24
+    assert lib.orc_uniform_from_bits(0xffffffff) == 1.0 - 2.0 ** -24
+    assert lib.orc_uniform_from_bits(0x80000000) == 0.5 + 2.0 ** -24
+    assert lib.orc_uniform_from_bits(0x000001ff) == 2.0 ** -24          # the low 9 bits are not used
+    rng = np.random.default_rng(5)
+    xs = np.concatenate([np.exp(rng.uniform(np.log(5e-8), np.log(20.0), 30000)),
+                         [2.0 ** -24, 1 - 2.0 ** -24, 1.0, 0.5, 2.0, 0.70710677, 0.7071068, 16.635532]]).astype(np.float32)
+    for x in xs:
+        ref = math.log(float(x))
+        got = lib.orc_det_logf(float(x))
+        assert abs(got - ref) <= 3e-7 * max(abs(ref), 1.0), (x, got, ref)
+    assert lib.orc_det_logf(1.0) == 0.0
+    # -log(1 - 2^-24) must not collapse to 0: the second logarithm needs a positive argument
+    assert lib.orc_det_logf(1.0 - 2.0 ** -24) < 0.0
+
+
+def test_gumbel_noise_moments_and_keys():
+    """Standard Gumbel: mean = Euler-Mascheroni constant, variance = pi^2/6; the noise is a function of
+    (seed, position, token) and of nothing else."""
+    g = np.concatenate([esp.gumbel_noise(7, p, 50000) for p in range(8)]).astype(np.float64)
+    n = g.size
+    assert abs(g.mean() - 0.5772156649) < 5 * math.sqrt(math.pi ** 2 / 6 / n)
+    assert abs(g.var() - math.pi ** 2 / 6) < 0.03
+    a = esp.gumbel_noise(7, 3, 1000)
+    assert np.array_equal(a, esp.gumbel_noise(7, 3, 1000))
+    assert np.array_equal(a[:10], esp.gumbel_noise(7, 3, 10))             # token v does not depend on the vocabulary size
+    assert not np.array_equal(a, esp.gumbel_noise(7, 4, 1000))
+    assert not np.array_equal(a, esp.gumbel_noise(8, 3, 1000))
+    assert not np.array_equal(a, esp.gumbel_noise(7 + (1 << 32), 3, 1000))  # the high seed word is used
+    # token v at position p is Philox word 0 of counter (v, p, 0, 0)
+    x = esp.philox4x32_10([5, 3, 0, 0], [7, 0])[0]
+    assert a[5] == esp._load().orc_gumbel_from_bits(x)
+
+
+@pytest.mark.parametrize("temperature", [1.0, 2.0, 0.5])
+def test_gumbel_max_draws_follow_the_softmax(temperature):
+    """argmax(logits/T + g) is a draw from softmax(logits/T): chi-square of 60000 draws against the exact
+    probabilities (5 degrees of freedom; 0.9999 quantile = 25.7)."""
+    logits = np.array([1.3, -0.2, 0.7, 2.1, -1.5, 0.0], dtype=np.float32)
+    p = np.exp(logits.astype(np.float64) / temperature)
+    p /= p.sum()
+    spec = esp.SpecCfg(temperature=temperature, seed=12345)
+    n = 60000
+    counts = np.zeros(len(logits))
+    for pos in range(n):
+        counts[esp.next_token(logits, pos, spec)] += 1
+    chi2 = float(((counts - n * p) ** 2 / (n * p)).sum())
+    assert chi2 < 25.7, (chi2, counts / n, p)
+
+
+def test_temperature_zero_is_the_argmax_and_ties_go_to_the_lower_id():
+    logits = np.array([0.5, 2.0, 2.0, -1.0], dtype=np.float32)
+    assert esp.next_token(logits, 11, esp.SpecCfg()) == 1
+    # with noise, the winner is the arg-max of the fp32 scores under the same tie rule
+    spec = esp.SpecCfg(temperature=1.0, seed=3)
+    s = esp.sample_scores(logits, 11, 1.0, 3)
+    assert s.dtype == np.float32
+    assert esp.next_token(logits, 11, spec) == int(np.flatnonzero(s == s.max())[0])
+    assert np.array_equal(s, logits + esp.gumbel_noise(3, 11, 4))
+
+
+@pytest.mark.parametrize("W,n_anchor,temperature", [(0, 0, 1.0), (1, 1, 1.0), (0, 1, 0.7)])
+def test_sample_matching_is_lossless_token_by_token(W, n_anchor, temperature):
+    """Section 4 "sample matching": with the draw at a position fixed by (seed, position), ESP emits exactly
+    the stream plain autoregressive sampling emits; another seed gives another stream."""
+    shape = synth.TINY.replace(n_layers=2, d_model=64, n_q_heads=4, n_kv_heads=2, head_dim=16, d_ffn=160, vocab=97)
+    w = synth.make_weights(shape, seed=21, gain_jitter=True, std=0.3)
+    model = esp.OracleModel(shape, w)
+    prompt = synth.make_prompt(shape.vocab, 17, 3)
+    spec = esp.SpecCfg(n_probes=3, topk=4, max_nodes=12, expand_width=W, n_anchor=n_anchor,
+                       temperature=temperature, seed=99)
+    ref = esp.greedy_generate(model, prompt, 40, 128, spec=spec)
+    dec = esp.EspOracle(model, spec, 256)
+    assert dec.generate(prompt, 40) == ref
+    assert ref != esp.greedy_generate(model, prompt, 40, 128)                       # not the greedy stream
+    other = dataclasses_replace(spec, seed=100)
+    assert ref != esp.greedy_generate(model, prompt, 40, 128, spec=other)
+    assert sum(a + 1 for a in dec.accept_hist) == len(dec.emitted) - 1
+
+
+def dataclasses_replace(spec, **kw):
+    import dataclasses
+    return dataclasses.replace(spec, **kw)
