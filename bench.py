@@ -306,7 +306,7 @@ def run_ours(args, shape, plen, k, K, B):
     steps, warm = args.steps, max(args.warmup, 3)
     w = synth.make_weights(shape, seed=rank, device="cuda")
     prompt = synth.make_prompt(shape.vocab, plen, rank)
-    spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1)
+    spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1, temperature=args.temperature, seed=1)
     max_seq = plen + (k + 1) * (2 * steps + 2 * warm + 16) + 64
     stream = torch.cuda.Stream()
     nbatch = max(1, args.batch)
@@ -414,7 +414,7 @@ def run_ours(args, shape, plen, k, K, B):
             "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": f"{args.config}-shape bf16 decoder, random-init seeded weights, b={nbatch}",
-                       "prompt_len": plen, "batch": nbatch, "n_probes": k, "topk": K, "max_nodes": B, "rows_per_step": rows,
+                       "prompt_len": plen, "batch": nbatch, "temperature": args.temperature, "n_probes": k, "topk": K, "max_nodes": B, "rows_per_step": rows,
                        "replicas": world, "l2": "inputs exceed L2 (weights are re-streamed every step)"},
             "mean_accepted_len": tokens / (steps * world * nbatch),
             "clocks": clocks,
@@ -516,6 +516,8 @@ def main():
     ap.add_argument("--config", default="llama3-8b", choices=sorted(WORKLOADS) + ["attention-op"])
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt / KV length")
     ap.add_argument("--batch", type=int, default=1, help="independent sequences in one handle (long-context / batch sweep)")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="0 = greedy matching (default); > 0 = sample matching at that temperature")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer count (smaller captures under a profiler)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-greedy", action="store_true", help="skip the greedy-decoding leg")

@@ -77,6 +77,14 @@ typedef struct {
      *     mu + n*sigma initialisations: the caller draws or builds the vectors).
      * Every mask vector then follows the same update, Eq. (mask_update_mean). */
     int32_t mask_init;
+    /* Matching rule of the verification (Section 4: greedy matching at temperature 0, "sample matching"
+     * otherwise).  temperature = 0: a node's next token is the arg-max of its logits.  temperature > 0: it is
+     * a draw from softmax(logits / temperature), taken as argmax_v(logits[v] / temperature + g(seed, t, v))
+     * with t the absolute position of the drawn token and g standard Gumbel noise from Philox4x32-10 on
+     * counter (v, t, 0, 0), key (seed_lo, seed_hi): the stream equals plain autoregressive sampling with the
+     * same seed, token by token.  Drafts (probe rows) are always the Top-K of the probe logits. */
+    float temperature;
+    uint32_t seed_lo, seed_hi;
 } esp_spec_cfg;
 
 /* Model weights. [device] matrices; the per-layer members are [host] arrays of
@@ -187,6 +195,11 @@ int esp_get_stats(esp_handle* h, esp_stats* out);
  * kernel recorded (1 = wait timed out, as expected).  The CUDA context stays usable.  `scratch` [device] >= 256
  * bytes. */
 int esp_debug_wait_selftest(void* scratch, void* cuda_stream, int32_t* device_status_out);
+
+/* The sampling noise of sample matching, for checking it bit by bit: noise_out [device] [n_tokens] fp32 receives
+ * g(seed, position, v) for v = 0..n_tokens-1 (see esp_spec_cfg.temperature).  Asynchronous on cuda_stream. */
+int esp_debug_gumbel(uint32_t seed_lo, uint32_t seed_hi, uint32_t position, int32_t n_tokens, float* noise_out,
+                     void* cuda_stream);
 
 /* Releases host-side bookkeeping only. */
 void esp_free(esp_handle* h);

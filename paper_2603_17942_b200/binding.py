@@ -25,7 +25,7 @@ ERRORS = {0: "ESP_OK", -1: "ESP_E_BADCFG", -2: "ESP_E_WORKSPACE", -3: "ESP_E_PRO
 
 EXPORTS = ["esp_workspace_bytes", "esp_init", "esp_prefill", "esp_step", "esp_step_async", "esp_read", "esp_set_mask", "esp_set_tree",
            "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_step_profiled", "esp_get_stats",
-           "esp_debug_wait_selftest", "esp_free",
+           "esp_debug_wait_selftest", "esp_debug_gumbel", "esp_free",
            "esp_tree_attention_scratch_bytes", "esp_tree_attention", "esp_tree_attention_static", "esp_gemm_scratch_bytes",
            "esp_gemm_bf16"]
 
@@ -49,7 +49,8 @@ class esp_model_cfg(ctypes.Structure):
 class esp_spec_cfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("n_probes", "topk", "max_nodes", "expand_width", "n_anchor",
                                               "prune_parent", "prune_root", "ema_per_token")] + [("lam", ctypes.c_float)] + \
-               [("static_widths", ctypes.c_int32 * ESP_MAX_PROBES), ("mask_init", ctypes.c_int32)]
+               [("static_widths", ctypes.c_int32 * ESP_MAX_PROBES), ("mask_init", ctypes.c_int32),
+                ("temperature", ctypes.c_float), ("seed_lo", ctypes.c_uint32), ("seed_hi", ctypes.c_uint32)]
 
 
 _PP = ctypes.POINTER(ctypes.c_void_p)
@@ -109,10 +110,11 @@ def model_cfg(shape, max_seq_len: int, max_batch: int = 1) -> esp_model_cfg:
 
 
 def spec_cfg(n_probes=0, topk=1, max_nodes=1, expand_width=1, n_anchor=0, prune_parent=True, prune_root=False,
-             ema_per_token=True, lam=0.1, static_widths=(), mask_init=0) -> esp_spec_cfg:
+             ema_per_token=True, lam=0.1, static_widths=(), mask_init=0, temperature=0.0, seed=0) -> esp_spec_cfg:
     widths = (ctypes.c_int32 * ESP_MAX_PROBES)(*[int(w) for w in static_widths])
     return esp_spec_cfg(n_probes, topk, max_nodes, expand_width, n_anchor, int(prune_parent), int(prune_root),
-                        int(ema_per_token), float(lam), widths, int(mask_init))
+                        int(ema_per_token), float(lam), widths, int(mask_init), float(temperature),
+                        int(seed) & 0xffffffff, (int(seed) >> 32) & 0xffffffff)
 
 
 # ---------------------------------------------------------------- raw calls (same names as the header)
@@ -201,6 +203,12 @@ def esp_debug_wait_selftest(scratch, stream=None) -> int:
     st = ctypes.c_int32(-1)
     _check(load_library().esp_debug_wait_selftest(_vp(scratch), _vp(stream), ctypes.byref(st)), "esp_debug_wait_selftest")
     return st.value
+
+
+def esp_debug_gumbel(seed: int, position: int, n_tokens: int, noise_out, stream=None):
+    _check(load_library().esp_debug_gumbel(ctypes.c_uint32(seed & 0xffffffff), ctypes.c_uint32((seed >> 32) & 0xffffffff),
+                                           ctypes.c_uint32(position), ctypes.c_int32(n_tokens), _vp(noise_out), _vp(stream)),
+           "esp_debug_gumbel")
 
 
 def esp_free(h):

@@ -97,6 +97,7 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
     if (2 * s->n_probes > DCAP_STEP) return ESP_E_BADCFG;
     if (s->expand_width < 0 || s->n_anchor < 0) return ESP_E_BADCFG;
     if (s->mask_init < 0 || s->mask_init > 2) return ESP_E_BADCFG;
+    if (!(s->temperature >= 0.f) || s->temperature > 1e6f) return ESP_E_BADCFG;
     // Algorithm 1 must not create more than MAX_CAND nodes
     long created = 1, n_exp = 1;
     for (int i = 1; i <= s->n_probes && !is_static; ++i) {
@@ -123,6 +124,8 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
         for (int i = 0; i < PROBES_MAX; ++i) D->static_w[i] = is_static && i < s->n_probes ? s->static_widths[i] : 0;
         D->n_anchor = s->n_anchor; D->prune_parent = s->prune_parent; D->prune_root = s->prune_root;
         D->ema_per_token = s->ema_per_token; D->lambda = s->lambda;
+        D->inv_temp = s->temperature > 0.f ? 1.0f / s->temperature : 0.f;
+        D->seed_lo = s->seed_lo; D->seed_hi = s->seed_hi;
     }
     return ESP_OK;
 }
@@ -238,6 +241,7 @@ EpiArgs base_epi(esp_handle* h, int n_out, int s0, int nb) {
     a.rms_eps = h->D.rms_eps;
     a.rope_cos = h->b.rope_cos; a.rope_sin = h->b.rope_sin;
     a.KP = h->D.KP;
+    a.samp_inv_temp = h->D.inv_temp; a.samp_key0 = h->D.seed_lo; a.samp_key1 = h->D.seed_hi;
     return a;
 }
 
@@ -766,6 +770,14 @@ int esp_debug_wait_selftest(void* scratch, void* cuda_stream, int32_t* device_st
     if (cudaStreamSynchronize(s) != cudaSuccess) return ESP_E_CUDA;
     *device_status_out = e;
     return ESP_OK;
+}
+
+int esp_debug_gumbel(uint32_t seed_lo, uint32_t seed_hi, uint32_t position, int32_t n_tokens, float* noise_out,
+                     void* cuda_stream) {
+    if (!noise_out || n_tokens < 0) return ESP_E_ARG;
+    if (n_tokens == 0) return ESP_OK;
+    launch_gumbel_noise(seed_lo, seed_hi, position, n_tokens, noise_out, reinterpret_cast<cudaStream_t>(cuda_stream));
+    return cuda_ok(cudaGetLastError());
 }
 
 void esp_free(esp_handle* h) {

@@ -70,6 +70,8 @@ struct Dims {
     int32_t static_w[PROBES_MAX];   // fixed branch widths per depth; static_w[0] == 0: Algorithm 1
     int32_t mask_slots;             // mask vectors per sequence: max(k, 1)
     float lambda;
+    float inv_temp;                 // 1 / temperature, 0 = greedy matching
+    uint32_t seed_lo, seed_hi;      // key of the sampling noise
 };
 
 // epilogue selectors of the small-M GEMMs.  EPI_PARTIAL (tensor-core kernel only) finishes nothing: every
@@ -168,6 +170,9 @@ struct EpiArgs {
     int32_t KP;
     int32_t n_tiles;
     float* logits_dump;       // optional [batch*RT][V]
+    // sample matching: tree rows pick argmax(logit * samp_inv_temp + Gumbel noise); 0 = greedy matching
+    float samp_inv_temp;
+    uint32_t samp_key0, samp_key1;
 };
 
 __device__ __forceinline__ float to_f32(float x) { return x; }

@@ -9,6 +9,7 @@
 #pragma once
 
 #include "esp_common.cuh"
+#include "esp_sampling.cuh"
 
 namespace esp {
 
@@ -101,6 +102,8 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
         const int warp = f >> 5, lane = f & 31;
         const int n_nodes = st ? st->n_nodes : a.rows_fixed;
         const int Mtot = a.batch * RT;
+        uint32_t noise_pos = 0xffffffffu;   // rows come in breadth-first order: equal depths are neighbours and
+        float noise[4] = {0.f, 0.f, 0.f, 0.f};   // share their noise, which is a function of (position, token)
         for (int r = warp; r < n_rows; r += 4) {
             float v[4];
             int id[4];
@@ -113,6 +116,18 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
             const bool probe = r >= n_nodes;
             const int kp = probe ? a.KP : 1;
             Cand* out = a.cand + ((size_t)tile * Mtot + grow0 + r) * a.KP;
+            if (!probe && st && a.samp_inv_temp > 0.f) {
+                // sample matching: this row's token for position L + depth + 1 is the arg-max of the noisy scores
+                const uint32_t pos = (uint32_t)(st->L + st->row_depth[r] + 1);
+                if (pos != noise_pos) {
+                    noise_pos = pos;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) noise[i] = gumbel_noise(a.samp_key0, a.samp_key1, pos, (uint32_t)id[i]);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (id[i] < a.n_out) v[i] = sample_score(v[i], a.samp_inv_temp, noise[i]);
+            }
             if (probe) {
                 float tmax = warp_max(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])));
                 float s = 0.f;

@@ -630,6 +630,15 @@ void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_
     launch_k(k_topk_merge, grid, dim3(TOPK_THREADS), smem, s, pdl, st, cand, cand_ms, n_tiles, KP, batch, topk, lse, stage);
 }
 
+// ------------------------------------------------------------------ sampling noise, stand-alone (for checking)
+__global__ void k_gumbel_noise(uint32_t key0, uint32_t key1, uint32_t position, int n, float* out) {
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;
+    if (v < n) out[v] = gumbel_noise(key0, key1, position, (uint32_t)v);
+}
+void launch_gumbel_noise(uint32_t key0, uint32_t key1, uint32_t position, int n, float* out, cudaStream_t s) {
+    k_gumbel_noise<<<(n + 255) / 256, 256, 0, s>>>(key0, key1, position, n, out);
+}
+
 // ------------------------------------------------------------------ row-table builders
 __device__ void write_probe_rows(SeqState* st, int N, int k, int first_anchor, int n_anchor_rows) {
     // probe j (1-based) of the a-th anchored node sits at row N + a*k + (j-1)

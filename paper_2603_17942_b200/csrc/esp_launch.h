@@ -36,6 +36,7 @@ struct TreeArgs {
 
 
 void launch_rope_table(float* cs, float* sn, int n_pos, int h, float base, cudaStream_t s);
+void launch_gumbel_noise(uint32_t key0, uint32_t key1, uint32_t position, int n, float* out, cudaStream_t s);
 void launch_mask_init(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, int slots, int mode, cudaStream_t s);
 void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int mask_slots,
                      int batch, cudaStream_t s, bool pdl);

@@ -8,6 +8,8 @@ Per step it checks
     rows and the oracle's own KV cache and mask vector: max |diff| <= tol * (logit range);
   * selection, bit-exact given the GPU's logits: argmax / Top-K' lists equal a full sort of the dumped
     logits, log-sum-exp agrees to fp32 rounding;
+  * sample matching (temperature > 0): a node's token is the arg-max of the oracle's noisy scores of the
+    GPU's logits at the node's position, bit for bit;
   * verification: the oracle's walk over the GPU's per-node argmax gives the GPU's emitted tokens;
   * next tree: the oracle's Algorithm 1 fed with the GPU's Top-K' lists and lse gives the GPU's next
     row table exactly;
@@ -34,7 +36,8 @@ def c_spec(o: O.SpecCfg):
     return P.spec_cfg(n_probes=o.n_probes, topk=o.topk, max_nodes=o.max_nodes, expand_width=o.expand_width,
                       n_anchor=o.n_anchor, prune_parent=o.prune_parent, prune_root=o.prune_root,
                       ema_per_token=o.ema_per_token, lam=o.lam, static_widths=o.static_widths,
-                      mask_init={"mean": 0, "last_k": 1, "given": 2}[o.mask_init])
+                      mask_init={"mean": 0, "last_k": 1, "given": 2}[o.mask_init],
+                      temperature=o.temperature, seed=o.seed)
 
 
 class ParityRun:
@@ -68,10 +71,16 @@ class ParityRun:
         assert err <= self.tol, f"{what}: logits off by {err:.3e} of the logit range (tol {self.tol})"
         return rng
 
-    def _check_selection(self, gl, st, rows_nodes, rows_probes):
+    def _scores(self, row_logits, pos):
+        """What a node row's arg-max is taken over: the logits, or the noisy scores for the token at position pos."""
+        if self.spec.temperature > 0:
+            return O.sample_scores(row_logits, pos, self.spec.temperature, self.spec.seed)
+        return row_logits
+
+    def _check_selection(self, gl, st, rows_nodes, rows_probes, node_pos):
         kp = self.spec.k_prime
         for r in rows_nodes:
-            ids, vals = O.topk_desc(gl[r], 1)
+            ids, vals = O.topk_desc(self._scores(gl[r], node_pos[r] + 1), 1)
             assert st["topk_ids"][r, 0] == ids[0] and st["topk_vals"][r, 0] == vals[0], f"argmax row {r}"
         for r in rows_probes:
             ids, vals = O.topk_desc(gl[r], kp)
@@ -79,11 +88,13 @@ class ParityRun:
             assert np.array_equal(st["topk_vals"][r, :kp], vals), f"Top-K' values row {r}"
             assert abs(float(st["lse"][r]) - float(O.log_sum_exp(gl[r]))) <= 2e-5 * max(1.0, abs(float(st["lse"][r])))
 
-    def _near_tie(self, ref_row, gpu_tok, rng, what):
+    def _near_tie(self, ref_row, gpu_tok, rng, what, pos):
+        ref_row = self._scores(ref_row, pos + 1)
         o_ids, o_vals = O.topk_desc(ref_row, 2)
         if int(o_ids[0]) != int(gpu_tok):
             gap = float(ref_row[o_ids[0]] - ref_row[gpu_tok])
-            assert gap <= 2 * self.tol * rng, f"{what}: GPU picked {gpu_tok}, oracle {o_ids[0]}, gap {gap} is not a near-tie"
+            scale = 1.0 / self.spec.temperature if self.spec.temperature > 0 else 1.0
+            assert gap <= 2 * self.tol * rng * max(1.0, scale), f"{what}: GPU picked {gpu_tok}, oracle {o_ids[0]}, gap {gap} is not a near-tie"
             self.near_ties += 1
 
     def _tree_from_state(self, st):
@@ -125,9 +136,9 @@ class ParityRun:
         # the last prefill chunk holds the final (t-1) % 64 + 1 prompt rows followed by the k mask rows
         r0 = (t - 1) % 64
         rng = self._cmp_logits(gl[r0:r0 + 1 + k], ref[t - 1:], "prefill")
-        self._check_selection(gl, st, [r0], range(r0 + 1, r0 + 1 + k))
+        self._check_selection(gl, st, [r0], range(r0 + 1, r0 + 1 + k), {r0: t - 1})
         assert first == st["topk_ids"][r0, 0]
-        self._near_tie(ref[t - 1], first, rng, "prefill")
+        self._near_tie(ref[t - 1], first, rng, "prefill", t - 1)
         self.emitted.append(first)
         self.m = O.mask_update(self.m, self.model.embed(first), sp.lam)
         assert st["L"] == t
@@ -156,12 +167,13 @@ class ParityRun:
         x = np.stack([self.model.embed(int(t)) if t >= 0 else self.m[probe_of_row[r] - 1] for r, t in enumerate(blk.row_token)])
         ref, kb, vb, _ = self.model.block_forward(self.kc, self.vc, self.L, x, self.L + blk.row_pos_off, blk.vis)
         rng = self._cmp_logits(gl[:blk.m], ref, f"step {len(self.accepts)}")
-        self._check_selection(gl, st, range(blk.n_nodes), range(blk.n_nodes, blk.m))
+        node_pos = {r: self.L + int(blk.row_pos_off[r]) for r in range(blk.n_nodes)}
+        self._check_selection(gl, st, range(blk.n_nodes), range(blk.n_nodes, blk.m), node_pos)
         gpu_next = [int(st["topk_ids"][r, 0]) for r in range(blk.n_nodes)]
         path, out = O.verify_walk(tree, gpu_next)
         assert toks == out, f"emitted {toks} vs verify walk {out}"
         for p in path:
-            self._near_tie(ref[p], gpu_next[p], rng, f"step {len(self.accepts)} node {p}")
+            self._near_tie(ref[p], gpu_next[p], rng, f"step {len(self.accepts)} node {p}", node_pos[p])
         a = len(path) - 1
         for j, p in enumerate(path):
             self.kc[:, self.L + j], self.vc[:, self.L + j] = kb[:, p], vb[:, p]

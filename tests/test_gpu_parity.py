@@ -243,6 +243,64 @@ def test_full_width_shapes_parity(pu, base, topk, B):
     run.close()
 
 
+# ------------------------------------------------------------------ sample matching (temperature > 0)
+def test_sampling_noise_bitwise_equals_oracle():
+    """The Gumbel noise of the CUDA path and of the oracle are the same fp32 numbers, bit for bit."""
+    import paper_2603_17942_b200 as P
+    n = 200_000
+    out = torch.empty(n, device="cuda")
+    for seed, pos in [(0, 0), (99, 17), ((5 << 32) | 12345, 4096), (2 ** 64 - 1, 2 ** 31 + 5)]:
+        P.esp_debug_gumbel(seed, pos, n, out)
+        torch.cuda.synchronize()
+        ref = O.gumbel_noise(seed, pos, n)
+        got = out.cpu().numpy()
+        assert np.array_equal(got.view(np.uint32), ref.view(np.uint32)), (seed, pos)
+
+
+@pytest.mark.parametrize("W,n_anchor,prune,temperature", [(0, 1, True, 1.0), (1, 0, False, 1.0), (0, 0, False, 0.6)])
+def test_tiny_fp32_sample_matching_parity(pu, W, n_anchor, prune, temperature):
+    """Section 4 "sample matching": every step against the oracle (noisy scores taken on the GPU's logits, bit for
+    bit), the stream equal to the oracle's sampled stream and to plain sampling on the GPU with the same seed."""
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=0)
+    prompt = synth.make_prompt(shape.vocab, 64, 0)
+    B = 32 if n_anchor == 1 else 20
+    spec = O.SpecCfg(n_probes=3, topk=4, max_nodes=B, expand_width=W, n_anchor=n_anchor, prune_parent=prune,
+                     temperature=temperature, seed=(7 << 32) | 2024)
+    run = pu.ParityRun(shape, w, spec, prompt, 64, TOL_FP32)
+    out = run.run()
+    model = O.OracleModel(shape, w)
+    assert out == O.greedy_generate(model, prompt, 64, 256, spec=spec)     # plain sampling in the oracle
+    dec = O.EspOracle(model, spec, 512)
+    assert out == dec.generate(prompt, 64)
+    import dataclasses
+    plain = dataclasses.replace(pu.GREEDY, temperature=temperature, seed=spec.seed)
+    g, _ = pu.gpu_generate(shape, run.wd, plain, prompt, 64)
+    assert g == out                                                        # GPU ESP == GPU plain sampling
+    assert out != O.greedy_generate(model, prompt, 64, 256)                # and it is not the greedy stream
+    assert len(set(out)) > 16
+    run.close()
+
+
+def test_bf16_sample_matching_equals_plain_sampling(pu):
+    """bf16 tensor-core path: parity per step, and the ESP stream at temperature 1 equals one-token-per-call
+    sampling with the same seed (a row in a tree block draws what it would draw alone)."""
+    import dataclasses
+    shape = BF16_SMALL
+    w = synth.make_weights(shape, seed=1, gain_jitter=True, std=0.05)
+    prompt = synth.make_prompt(shape.vocab, 300, 2)
+    spec = O.SpecCfg(n_probes=3, topk=5, max_nodes=16, expand_width=0, n_anchor=1, temperature=1.0, seed=31337)
+    run = pu.ParityRun(shape, w, spec, prompt, 32, TOL_BF16)
+    out = run.run()
+    plain = dataclasses.replace(pu.GREEDY, temperature=1.0, seed=31337)
+    g, _ = pu.gpu_generate(shape, run.wd, plain, prompt, 32)
+    assert g == out
+    g2, _ = pu.gpu_generate(shape, run.wd, dataclasses.replace(plain, seed=31338), prompt, 32)
+    assert g2 != out
+    assert run.h.stats().device_error == 0
+    run.close()
+
+
 # ------------------------------------------------------------------ errors are reported, not raised from the device
 def test_host_side_errors(pu):
     import paper_2603_17942_b200 as P
