@@ -160,7 +160,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.tree_dev = c.take<int32_t>(2 * RT);
     o.rope_cos = c.take<float>((size_t)D.cap * (D.h / 2));
     o.rope_sin = c.take<float>((size_t)D.cap * (D.h / 2));
-    o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm));
+    o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm, D.batch < tc_gemm_max_nq() ? D.batch : tc_gemm_max_nq()));
     o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
     o.sk_tables = c.take<TileSrc>(4 * SK_TABLE_TILES);
     o.packed = nullptr;
@@ -246,17 +246,18 @@ EpiArgs base_epi(esp_handle* h, int n_out, int s0, int nb) {
 }
 
 int run_gemm(esp_handle* h, TcGemm* plan, int epi, int n_tiles, const void* const w[3], const int32_t rows_w[3],
-             const void* x, int K, const EpiArgs& a, bool tc, bool pdl) {
+             const void* x, int K, const EpiArgs& a, bool tc, bool pdl, int nq = 1, int b_row0 = 0) {
     h->launches++;
-    if (tc) return tc_gemm_launch(plan, a, h->stream, pdl);
+    if (tc) return tc_gemm_launch(plan, a, h->stream, pdl, nq, b_row0);
     launch_gemm_simt(h->dtype, epi, n_tiles, h->D.batch, w, rows_w, x, K, a, h->stream, pdl);
     return ESP_OK;
 }
 
-// One decoder forward over the block every active sequence has in its row table.
-// Tensor-core path (bf16, one sequence): the QKV, O and down GEMMs store stream-K partials that the next
-// kernel sums (k_qkv_finish; k_resid_norm = residual add + RMSNorm), gate/up and the LM head finish in-kernel.
-// CUDA-core path (fp32 models, batched bf16): the same layer with every epilogue fused in the GEMM.
+// One decoder forward over the block every active sequence of [s0, s0 + nb) has in its row table.
+// Tensor-core path (bf16, nb <= 3 sequences whose activation blocks sit RT rows apart): the layer GEMMs stream
+// their weights once for all nb sequences and store stream-K partials that the next kernel sums (k_qkv_finish;
+// k_resid_norm = residual add + RMSNorm; k_swiglu_finish); the LM head runs once per sequence and finishes
+// in-kernel.  CUDA-core path (fp32 models): the same layer with every epilogue fused in the GEMM.
 int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc) {
     const Dims& D = h->D;
     Buffers& b = h->b;
@@ -271,12 +272,12 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
     const size_t kv_seq_off = (size_t)s0 * D.Hkv * D.cap * D.h * es;   // this pass's first sequence inside a layer's cache
     float* mvec0 = b.mvec + (size_t)s0 * D.mask_slots * D.d;
     StreamK pending;   // partials of the last down projection, summed by the next norm
-    pending.partials = nullptr; pending.table = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2;
+    pending.partials = nullptr; pending.table = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2; pending.rows = RT;
     mark(h, -1);
     launch_assemble(h->dtype, st0, h->embed, mvec0, b.hres, D.d, D.mask_slots, nb, s, false);
     h->launches++;
     for (int l = 0; l < D.n_layers; ++l) {
-        if (tc) launch_resid_norm(st0, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
+        if (tc) launch_resid_norm(st0, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->na[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -289,11 +290,11 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.k_norm = D.qk_norm ? h->kn[l] : nullptr;
             const void* w[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t rows[3] = {dq, dkv, dkv};
-            int rc = run_gemm(h, tc ? h->p_qkv[l] : nullptr, EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a, tc, pdl);
+            int rc = run_gemm(h, tc ? h->p_qkv[l] : nullptr, EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a, tc, pdl, tc ? nb : 1);
             if (rc) return rc;
             mark(h, KIND_QKV);
             if (tc) {
-                if (launch_qkv_finish(a, tc_gemm_streamk(h->p_qkv[l]), s, pdl)) return ESP_E_BADCFG;
+                if (launch_qkv_finish(a, tc_gemm_streamk(h->p_qkv[l], nb), nb, s, pdl)) return ESP_E_BADCFG;
                 h->launches++;
                 mark(h, KIND_MISC);
             }
@@ -312,7 +313,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
             a.err = b.err;
             if (tc) {
-                if (attn_tc_launch(h->p_attn[(size_t)l * D.batch + s0], a, 1, n_split_launch, s, pdl)) return ESP_E_BADCFG;
+                if (attn_tc_launch(h->p_attn[(size_t)l * D.batch + s0], a, nb, n_split_launch, s, pdl)) return ESP_E_BADCFG;
                 h->launches += n_split_launch > 0 ? 2 : 1;
             } else {
                 if (launch_attn_simt(h->dtype, a, nb, n_split_launch, true, s, pdl)) return ESP_E_BADCFG;
@@ -325,11 +326,11 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.hres = b.hres;
             const void* w[3] = {h->wo[l], nullptr, nullptr};
             const int32_t rows[3] = {D.d, 0, 0};
-            int rc = run_gemm(h, tc ? h->p_o[l] : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.attn_out, dq, a, tc, pdl);
+            int rc = run_gemm(h, tc ? h->p_o[l] : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.attn_out, dq, a, tc, pdl, tc ? nb : 1);
             if (rc) return rc;
             mark(h, KIND_O);
         }
-        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(h->p_o[l]), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, s, pdl);
+        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(h->p_o[l], nb), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -338,11 +339,11 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.act_out = b.act;
             const void* w[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t rows[3] = {D.F, D.F, 0};
-            int rc = run_gemm(h, tc ? h->p_gu[l] : nullptr, EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a, tc, pdl);
+            int rc = run_gemm(h, tc ? h->p_gu[l] : nullptr, EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a, tc, pdl, tc ? nb : 1);
             if (rc) return rc;
             mark(h, KIND_GATEUP);
             if (tc) {
-                launch_swiglu_finish(st0, tc_gemm_streamk(h->p_gu[l]), b.act, D.F, s, pdl);
+                launch_swiglu_finish(st0, tc_gemm_streamk(h->p_gu[l], nb), b.act, D.F, nb, s, pdl);
                 h->launches++;
                 mark(h, KIND_MISC);
             }
@@ -352,30 +353,35 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.hres = b.hres;
             const void* w[3] = {h->wd[l], nullptr, nullptr};
             const int32_t rows[3] = {D.d, 0, 0};
-            int rc = run_gemm(h, tc ? h->p_down[l] : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.act, D.F, a, tc, pdl);
+            int rc = run_gemm(h, tc ? h->p_down[l] : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.act, D.F, a, tc, pdl, tc ? nb : 1);
             if (rc) return rc;
-            if (tc) pending = tc_gemm_streamk(h->p_down[l]);
+            if (tc) pending = tc_gemm_streamk(h->p_down[l], nb);
             mark(h, KIND_DOWN);
         }
     }
     if (with_lm) {
         float* dbg_hidden = h->dbg_hidden ? h->dbg_hidden + (size_t)s0 * RT * D.d : nullptr;
-        if (tc) launch_resid_norm(st0, b.hres, pending, h->final_norm, b.xn, D.d, D.rms_eps, dbg_hidden, s, pdl);
+        if (tc) launch_resid_norm(st0, b.hres, pending, h->final_norm, b.xn, D.d, D.rms_eps, dbg_hidden, nb, s, pdl);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, nb, dbg_hidden, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
         const int n_tiles = (D.V + TILE_N - 1) / TILE_N;
-        EpiArgs a = base_epi(h, D.V, s0, nb);
-        a.cand = b.cand; a.cand_ms = b.cand_ms; a.n_tiles = n_tiles;
-        a.logits_dump = h->dbg_logits ? h->dbg_logits + (size_t)s0 * RT * D.V : nullptr;
-        const void* w[3] = {h->lm_head, nullptr, nullptr};
-        const int32_t rows[3] = {D.V, 0, 0};
-        int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl);
-        if (rc) return rc;
-        mark(h, KIND_LMHEAD);
-        launch_topk_merge(st0, b.cand, b.cand_ms, n_tiles, D.KP, nb, b.topk + (size_t)s0 * RT * KP_MAX, b.lse + (size_t)s0 * RT, s, pdl);
-        h->launches++;
-        mark(h, KIND_SELECT);
+        // tensor-core path: the LM head and its selection run once per sequence (the candidate lists are shared)
+        const int n_lm = tc ? nb : 1, per = tc ? 1 : nb;
+        for (int q = 0; q < n_lm; ++q) {
+            const int sq = s0 + q;
+            EpiArgs a = base_epi(h, D.V, sq, per);
+            a.cand = b.cand; a.cand_ms = b.cand_ms; a.n_tiles = n_tiles;
+            a.logits_dump = h->dbg_logits ? h->dbg_logits + (size_t)sq * RT * D.V : nullptr;
+            const void* w[3] = {h->lm_head, nullptr, nullptr};
+            const int32_t rows[3] = {D.V, 0, 0};
+            int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl, 1, q * RT);
+            if (rc) return rc;
+            mark(h, KIND_LMHEAD);
+            launch_topk_merge(b.states + sq, b.cand, b.cand_ms, n_tiles, D.KP, per, b.topk + (size_t)sq * RT * KP_MAX, b.lse + (size_t)sq * RT, s, pdl);
+            h->launches++;
+            mark(h, KIND_SELECT);
+        }
     }
     return cuda_ok(cudaGetLastError());
 }
@@ -384,9 +390,15 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
 int forward(esp_handle* h, bool with_lm, int dcap, int only_seq) {
     const bool tc = h->dtype == 1 && h->gemm_impl == 0 && h->p_lm != nullptr;
     if (!tc) return forward_pass(h, with_lm, dcap, 0, h->D.batch, false);
-    for (int i = 0; i < h->D.batch; ++i) {
-        if (only_seq >= 0 ? i != only_seq : !h->ready[i]) continue;
-        const int rc = forward_pass(h, with_lm, dcap, i, 1, true);
+    if (only_seq >= 0) return forward_pass(h, with_lm, dcap, only_seq, 1, true);
+    // consecutive sequences share a pass (and a weight stream); sequences that are not ready are inactive in it
+    const int per_pass = tc_gemm_max_nq();
+    for (int s0 = 0; s0 < h->D.batch; s0 += per_pass) {
+        const int nb = h->D.batch - s0 < per_pass ? h->D.batch - s0 : per_pass;
+        bool any = false;
+        for (int i = s0; i < s0 + nb; ++i) any = any || h->ready[i];
+        if (!any) continue;
+        const int rc = forward_pass(h, with_lm, dcap, s0, nb, true);
         if (rc) return rc;
     }
     return ESP_OK;
@@ -486,44 +498,45 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
     if (model->dtype == 1 && attn_tc_supported(D.h, D.Hq, D.Hkv)) {
         const size_t seq_bytes = (size_t)D.Hkv * D.cap * D.h * 2;
         for (int l = 0; l < D.n_layers; ++l) {
-            for (int i = 0; i < D.batch; ++i) {      // one sequence per pass: its slice of the layer's cache, the shared q buffer
+            for (int i = 0; i < D.batch; ++i) {      // a pass starting at sequence i: the layer's cache from there on, the shared q buffer
                 AttnTc* t = nullptr;
                 char* kc = reinterpret_cast<char*>(layer_ptr(h->b.kcache, h->layer_kv_stride, l)) + seq_bytes * i;
                 char* vc = reinterpret_cast<char*>(layer_ptr(h->b.vcache, h->layer_kv_stride, l)) + seq_bytes * i;
-                if (attn_tc_create(&t, h->b.qbuf, kc, vc, 1, D.Hq, D.Hkv, D.cap)) { esp_free(h); return ESP_E_CUDA; }
+                if (attn_tc_create(&t, h->b.qbuf, kc, vc, D.batch - i, D.Hq, D.Hkv, D.cap)) { esp_free(h); return ESP_E_CUDA; }
                 h->p_attn.push_back(t);
             }
         }
     }
     if (model->dtype == 1) {
         const int dq = D.Hq * D.h, dkv = D.Hkv * D.h;
+        const int nq_max = D.batch < tc_gemm_max_nq() ? D.batch : tc_gemm_max_nq();   // sequences sharing a weight stream
         bool ok = true;
         for (int l = 0; l < D.n_layers && ok; ++l) {
             TcGemm* p = nullptr;
             char* pk = h->b.packed + h->b.pk_layer * l;
             const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t r1[3] = {dq, dkv, dkv};
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, D.batch * RT, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream);
             h->p_qkv.push_back(p);
             const void* w2[3] = {h->wo[l], nullptr, nullptr};
             const int32_t r2[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, D.batch * RT, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream);
             h->p_o.push_back(p);
             const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t r3[3] = {D.F, D.F, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, D.batch * RT, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream);
             h->p_gu.push_back(p);
             const void* w4[3] = {h->wd[l], nullptr, nullptr};
             const int32_t r4[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, D.batch * RT, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream);
             h->p_down.push_back(p);
         }
         const void* w5[3] = {h->lm_head, nullptr, nullptr};
         const int32_t r5[3] = {D.V, 0, 0};
-        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
+        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, D.batch * RT, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
         if (!ok) { esp_free(h); return ESP_E_CUDA; }
     }
     if (cudaStreamSynchronize(h->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) { esp_free(h); return ESP_E_CUDA; }
@@ -927,7 +940,7 @@ int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const
     if (cudaMemsetAsync(counters, 0, sizeof(int) * tc_gemm_counter_ints() , s) != cudaSuccess) return ESP_E_CUDA;
     if (cudaMemsetAsync(err, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
     TcGemm* plan = nullptr;
-    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err, nullptr, 0, nullptr, s)) return ESP_E_CUDA;
+    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, RT, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err, nullptr, 0, nullptr, s)) return ESP_E_CUDA;
     int rc = tc_gemm_launch(plan, a, s, false);
     int e = 0;
     if (!rc && cudaMemcpyAsync(&e, err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) rc = ESP_E_CUDA;

@@ -81,7 +81,8 @@ enum Epi : int { EPI_STORE_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, 
 // Stream-K partition of a GEMM: the n_tiles*KB (tile, k-block) units are dealt out in equal contiguous
 // ranges to G persistent CTAs; CTA c owns units [c*U/G, (c+1)*U/G).  The piece of tile t a CTA computed is
 // kept in slot min(t - first tile of the CTA, slots - 1) of that CTA:
-// partials[((cta*slots + slot)*RT + row)*TILE_N + feature].
+// partials[((cta*slots + slot)*rows + row)*TILE_N + feature], rows = RT x the sequences one launch covers (row =
+// sequence-in-launch * RT + block row).
 // `table` (device memory, one entry per tile, written once when the GEMM plan is made) lists, in CTA order,
 // the cta*slots+slot index of every piece of the tile, so consumer kernels need no partition arithmetic.
 struct TileSrc {
@@ -92,6 +93,7 @@ struct StreamK {
     const float* partials;  // NULL: nothing to sum
     const TileSrc* table;
     int32_t n_tiles, KB, G, slots;
+    int32_t rows;           // rows per slot
 };
 __host__ __device__ __forceinline__ long long sk_begin(long long c, long long U, long long G) { return c * U / G; }
 __host__ __device__ __forceinline__ int sk_cta_of_unit(long long u, long long U, long long G) {
@@ -110,7 +112,7 @@ __host__ __device__ __forceinline__ int sk_slot(const StreamK& s, int c, int til
 }
 // address of contributor c's partial row of a tile
 __device__ __forceinline__ const float* sk_partial(const StreamK& s, int c, int tile, int row) {
-    return s.partials + ((size_t)(c * s.slots + sk_slot(s, c, tile)) * RT + row) * TILE_N;
+    return s.partials + ((size_t)(c * s.slots + sk_slot(s, c, tile)) * s.rows + row) * TILE_N;
 }
 // Sum over the contributors of `tile`, in CTA order, of the four floats at column f of row r.  The loads of up
 // to eight contributors are issued before the first addition (adding the zeros of absent ones changes nothing).
@@ -131,7 +133,7 @@ __device__ __forceinline__ float4 sk_sum4(const StreamK& s, int tile, int r, int
                 t[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (hw < 16 && cb + u < n) {
                     const uint32_t idx = (w[hw >> 1] >> ((hw & 1) * 16)) & 0xffffu;
-                    t[u] = __ldcg(reinterpret_cast<const float4*>(base + (size_t)idx * (RT * TILE_N)));
+                    t[u] = __ldcg(reinterpret_cast<const float4*>(base + (size_t)idx * ((size_t)s.rows * TILE_N)));
                 }
             }
 #pragma unroll

@@ -41,19 +41,25 @@ namespace {
 using namespace tc;
 
 constexpr int BK = 64;                       // k elements per stage (128 bytes of bf16)
+// NQ = sequences one launch covers: their activation blocks ([RT][K] each, consecutive) form one B operand of
+// NQ*RT rows, so the weights are streamed once for all of them (partial-only output only).
+//
 // Ring depth.  The bytes in flight per SM (depth x 16 KB of weights) over the load round trip bound the stream rate,
 // and the ring is also what is requested before the preceding kernel has finished: deeper is better.  The
 // partial-only kernel keeps no accumulator copy in shared memory and spends that room on the ring.
-__host__ __device__ constexpr int stages_of(int epi) { return epi == EPI_PARTIAL ? 8 : 6; }
+__host__ __device__ constexpr int stages_of(int epi, int nq) { return nq == 3 ? 4 : (nq == 2 ? 6 : (epi == EPI_PARTIAL ? 8 : 6)); }
 constexpr int A_BYTES = TILE_N * BK * 2;     // 16384
-constexpr int B_BYTES = RT * BK * 2;         // 10240
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int TMEM_COLS = 256;               // two accumulator buffers of 128 columns
+__host__ __device__ constexpr int b_bytes_of(int nq) { return nq * RT * BK * 2; }   // 10240 per sequence
+__host__ __device__ constexpr int stage_bytes_of(int nq) { return A_BYTES + b_bytes_of(nq); }
+// two accumulator buffers in tensor memory: 128 columns each for one sequence, 256 each for two or three
+__host__ __device__ constexpr int acc_cols_of(int nq) { return nq == 1 ? 128 : 256; }
 constexpr int NUM_THREADS = 192;
+constexpr int MAX_NQ = 3;
 
 struct TcParams {
     CUtensorMap map_a[3];
-    CUtensorMap map_b;
+    CUtensorMap map_b;      // activations [rows][K], box = NQ*RT rows (one map per NQ, picked at launch)
+    int32_t b_row0;         // first activation row of this launch
     int32_t rows_w[3];
     int32_t n_tiles, KB, grid, epi;
     int32_t map_swiglu;  // tile = 64 rows of w[0] (gate) + the matching 64 rows of w[1] (up)
@@ -65,8 +71,10 @@ struct TcParams {
     EpiArgs a;
 };
 
-// kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = 80
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RT >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
+// kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = 80 per sequence
+__host__ __device__ constexpr uint32_t idesc_of(int nq) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((nq * RT) >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
+}
 
 // One (tile, k-range) piece of a CTA's stream-K range.
 struct Seg {
@@ -118,11 +126,14 @@ __device__ __forceinline__ void tile_source(const TcParams& p, int tile, int hal
     row = feat + half * 64;
 }
 
-template <int EPI>
+template <int EPI, int NQ>
 __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constant__ TcParams p) {
+    static_assert(NQ == 1 || EPI == EPI_PARTIAL, "several sequences per launch: partial-only output");
+    constexpr int STAGE_BYTES = stage_bytes_of(NQ), ACC_COLS = acc_cols_of(NQ), TMEM_COLS = 2 * ACC_COLS;
+    constexpr uint32_t IDESC = idesc_of(NQ);
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int STAGES = stages_of(EPI);
+    constexpr int STAGES = stages_of(EPI, NQ);
     unsigned char* stages = smem;
     float* s_acc = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES);
     float* s_aux = s_acc + (EPI == EPI_PARTIAL ? 0 : RT * ACC_LD);
@@ -183,7 +194,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                                 tma_load_2d_hint(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it], pol_w);
                             }
                         } else {
-                            tma_load_2d_hint(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[it], pol_x);
+                            tma_load_2d_hint(sa + A_BYTES, &p.map_b, kb * BK, p.b_row0, &full[it], pol_x);
                         }
                     }
                 }
@@ -208,7 +219,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                             tma_load_2d_hint(sa, &p.map_a[m0], kb * BK, r0, &full[stage], pol_w);
                             tma_load_2d_hint(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage], pol_w);
                         }
-                        tma_load_2d_hint(sa + A_BYTES, &p.map_b, kb * BK, 0, &full[stage], pol_x);
+                        tma_load_2d_hint(sa + A_BYTES, &p.map_b, kb * BK, p.b_row0, &full[stage], pol_x);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -226,7 +237,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                 const int buf = i & 1;
                 if (!mbar_wait(&tempty[buf], ((i >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t tmem_d = tmem_base + buf * 128;
+                const uint32_t tmem_d = tmem_base + buf * ACC_COLS;
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
                     if (!mbar_wait(&full[stage], phase, s_abort)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -252,6 +263,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
         const int n_rows = p.a.st ? (p.a.st->active ? p.a.st->n_rows : 0) : p.a.rows_fixed;
         StreamK sk;
         sk.partials = p.partials; sk.table = nullptr; sk.n_tiles = p.n_tiles; sk.KB = p.KB; sk.G = p.grid; sk.slots = p.slots;
+        sk.rows = NQ * RT;
         bool ok = true;
         for (int i = 0; i < rng.n_seg && ok; ++i) {
             const Seg sg = get_seg(rng, i);
@@ -262,8 +274,27 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
             epi_bar(2);
             if (s_flag[0]) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t taddr = tmem_base + buf * 128 + ((uint32_t)(q * 32) << 16);
+            const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(q * 32) << 16);
             uint32_t v[RT];
+            if constexpr (NQ > 1) {
+                // sequence by sequence: 80 accumulator columns -> that sequence's rows of the partial
+                float* part = p.partials + ((size_t)(blockIdx.x * p.slots + sg.slot) * (NQ * RT)) * TILE_N + f;
+#pragma unroll 1
+                for (int sq = 0; sq < NQ; ++sq) {
+#pragma unroll
+                    for (int c = 0; c < RT / 16; ++c)
+                        tmem_ld16_issue(taddr + sq * RT + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    const SeqState* sst = p.a.st + sq;
+                    const int nr = sst->active ? sst->n_rows : 0;
+#pragma unroll
+                    for (int r = 0; r < RT; ++r)
+                        if (r < nr) __stcg(part + (size_t)(sq * RT + r) * TILE_N, __uint_as_float(v[r]));
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mbar_arrive(&tempty[buf]);
+                continue;
+            }
 #pragma unroll
             for (int c = 0; c < RT / 16; ++c) tmem_ld16_issue(taddr + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -386,8 +417,8 @@ __global__ void __launch_bounds__(128) k_pack_weights(PackArgs g, unsigned char*
     }
 }
 
-constexpr size_t smem_bytes_of(int epi) {
-    return 1024 + (size_t)stages_of(epi) * STAGE_BYTES + (epi == EPI_PARTIAL ? 0 : sizeof(float) * (RT * ACC_LD + RT * 4)) + 256;
+constexpr size_t smem_bytes_of(int epi, int nq) {
+    return 1024 + (size_t)stages_of(epi, nq) * stage_bytes_of(nq) + (epi == EPI_PARTIAL ? 0 : sizeof(float) * (RT * ACC_LD + RT * 4)) + 256;
 }
 
 // [rows][K] bf16 row-major, box = 64 k-elements x box_rows rows, 128-byte swizzle, out-of-range reads give zero
@@ -409,10 +440,13 @@ int make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
 struct TcGemm {
     TcParams p;
     const TileSrc* table = nullptr;
+    CUtensorMap map_b_nq[MAX_NQ];   // activation maps with a box of (i+1)*RT rows
+    int nq_max = 1;
 };
 
 constexpr int MAX_SLOTS = 4;
-size_t tc_gemm_partial_bytes(int n_sm) { return (size_t)n_sm * MAX_SLOTS * RT * TILE_N * sizeof(float); }
+size_t tc_gemm_partial_bytes(int n_sm, int nq) { return (size_t)n_sm * MAX_SLOTS * nq * RT * TILE_N * sizeof(float); }
+int tc_gemm_max_nq() { return MAX_NQ; }
 int tc_gemm_counter_ints() { return 4096; }
 size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K) {
     const long long total = (long long)rows_w[0] + rows_w[1] + rows_w[2];
@@ -422,9 +456,10 @@ size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K) {
 int tc_gemm_tiles(const TcGemm* g) { return g ? g->p.n_tiles : 0; }
 
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
-                   int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
+                   int x_rows, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
                    int table_entries, void* packed, cudaStream_t stream) {
-    if (!out || batch != 1 || K % 8 || n_sm < 1) return -1;
+    if (!out || nq_max < 1 || nq_max > MAX_NQ || x_rows < nq_max * RT || K % 8 || n_sm < 1) return -1;
+    if (nq_max > 1 && !defer) return -1;
     if (reinterpret_cast<uintptr_t>(x) % 16) return -1;
     TcGemm* g = new (std::nothrow) TcGemm();
     if (!g) return -1;
@@ -440,14 +475,17 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
             p.map_a[i] = p.map_a[0];
         }
     }
-    if (make_map(&p.map_b, x, RT, K, RT)) { delete g; return -1; }
+    for (int i = 0; i < nq_max; ++i)
+        if (make_map(&g->map_b_nq[i], x, x_rows, K, (i + 1) * RT)) { delete g; return -1; }
+    g->nq_max = nq_max;
+    p.map_b = g->map_b_nq[0];
     p.map_swiglu = epi == EPI_SWIGLU;
     p.epi = defer ? (int)EPI_PARTIAL : epi;
     p.n_tiles = epi == EPI_SWIGLU ? (rows_w[0] + 63) / 64 : (total_rows + TILE_N - 1) / TILE_N;
     p.KB = (K + BK - 1) / BK;
     const long long U = (long long)p.n_tiles * p.KB;
     p.grid = (int)(U < n_sm ? U : n_sm);
-    if (p.n_tiles > tc_gemm_counter_ints() || tc_gemm_partial_bytes(p.grid) > partial_bytes) { delete g; return -1; }
+    if (p.n_tiles > tc_gemm_counter_ints() || tc_gemm_partial_bytes(p.grid, nq_max) > partial_bytes) { delete g; return -1; }
     // fused epilogues store only the head and tail pieces of a range (2 slots); partial-only output stores every
     // piece, one slot per tile the range touches
     p.slots = 2;
@@ -463,7 +501,7 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
         // contributor table for the consumer kernels
         if (!table_dev || p.n_tiles > table_entries) { delete g; return -1; }
         StreamK k;
-        k.partials = nullptr; k.table = nullptr; k.n_tiles = p.n_tiles; k.KB = p.KB; k.G = p.grid; k.slots = p.slots;
+        k.partials = nullptr; k.table = nullptr; k.n_tiles = p.n_tiles; k.KB = p.KB; k.G = p.grid; k.slots = p.slots; k.rows = RT;
         TileSrc* tab = new (std::nothrow) TileSrc[p.n_tiles];
         if (!tab) { delete g; return -1; }
         bool fits = true;
@@ -515,8 +553,9 @@ int tc_wait_selftest(int* err_dev, cudaStream_t s) {
     return cudaGetLastError() == cudaSuccess ? 0 : -1;
 }
 
-StreamK tc_gemm_streamk(const TcGemm* g) {
+StreamK tc_gemm_streamk(const TcGemm* g, int nq) {
     StreamK k;
+    k.rows = nq * RT;
     k.partials = g ? g->p.partials : nullptr;
     k.table = g ? g->table : nullptr;
     k.n_tiles = g ? g->p.n_tiles : 0;
@@ -526,26 +565,30 @@ StreamK tc_gemm_streamk(const TcGemm* g) {
     return k;
 }
 
-int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl) {
-    if (!g) return ESP_E_ARG;
+// nq sequences (their activation rows start at row b_row0 of the plan's activation buffer, RT apart)
+int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl, int nq, int b_row0) {
+    if (!g || nq < 1 || nq > g->nq_max || b_row0 < 0) return ESP_E_ARG;
+    if (nq > 1 && g->p.epi != EPI_PARTIAL) return ESP_E_ARG;
     TcParams p = g->p;
     p.a = a;
+    p.map_b = g->map_b_nq[nq - 1];
+    p.b_row0 = b_row0;
     cudaError_t e = cudaSuccess;
-#define ESP_TC_CASE(E)                                                                                        \
-    case E: {                                                                                                 \
+#define ESP_TC_CASE(E, Q)                                                                                     \
+    {                                                                                                         \
         static bool attr_set = false;                                                                         \
         if (!attr_set) {                                                                                      \
-            if (cudaFuncSetAttribute(k_gemm_tc<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(E)) != cudaSuccess) return ESP_E_CUDA; \
+            if (cudaFuncSetAttribute(k_gemm_tc<E, Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(E, Q)) != cudaSuccess) return ESP_E_CUDA; \
             attr_set = true;                                                                                  \
         }                                                                                                     \
-        e = launch_k(k_gemm_tc<E>, dim3(p.grid), dim3(NUM_THREADS), smem_bytes_of(E), s, pdl, p);                    \
-    } break;
-    switch (p.epi) {
-        ESP_TC_CASE(EPI_STORE_F32)
-        ESP_TC_CASE(EPI_LOGITS)
-        ESP_TC_CASE(EPI_PARTIAL)
-        default: return ESP_E_ARG;
+        e = launch_k(k_gemm_tc<E, Q>, dim3(p.grid), dim3(NUM_THREADS), smem_bytes_of(E, Q), s, pdl, p);       \
     }
+    if (p.epi == EPI_STORE_F32) ESP_TC_CASE(EPI_STORE_F32, 1)
+    else if (p.epi == EPI_LOGITS) ESP_TC_CASE(EPI_LOGITS, 1)
+    else if (p.epi == EPI_PARTIAL && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1)
+    else if (p.epi == EPI_PARTIAL && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2)
+    else if (p.epi == EPI_PARTIAL && nq == 3) ESP_TC_CASE(EPI_PARTIAL, 3)
+    else return ESP_E_ARG;
 #undef ESP_TC_CASE
     return e == cudaSuccess ? ESP_OK : ESP_E_CUDA;
 }

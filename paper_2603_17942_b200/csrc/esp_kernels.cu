@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, flo
     for (int j = threadIdx.x * 4; j < d; j += STRIDE, ++it) {
         float4 x = *reinterpret_cast<const float4*>(xr + j);
         if (sk.partials) {
-            const float4 acc = sk_sum4(sk, j / TILE_N, r, j % TILE_N);
+            const float4 acc = sk_sum4(sk, j / TILE_N, seq * RT + r, j % TILE_N);
             x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
             *reinterpret_cast<float4*>(xr + j) = x;
         }
@@ -158,19 +158,20 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
     typedef __nv_bfloat16 T;
     constexpr int NE = HD / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int hs = blockIdx.x * 4 + warp, r = blockIdx.y;
-    const SeqState* st = a.st;
+    const int hs = blockIdx.x * 4 + warp, r = blockIdx.y, seq = blockIdx.z;   // seq: sequence within this launch
+    const SeqState* st = a.st ? a.st + seq : nullptr;
     const int n_rows = st ? (st->active ? st->n_rows : 0) : a.rows_fixed;
     if (r >= n_rows || hs >= a.Hq + 2 * a.Hkv) return;
+    const int pr = seq * RT + r;                 // row in the partials and in the query buffer
     const int j0 = hs * HD + lane * NE;          // feature in the concatenated [q | k | v] space
     const int tile = j0 / TILE_N, f = j0 % TILE_N;
     float v[NE];
     if constexpr (NE == 4) {
-        const float4 t = sk_sum4(sk, tile, r, f);
+        const float4 t = sk_sum4(sk, tile, pr, f);
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
     } else {
         // narrower heads: the same sum through the four-float helper on the enclosing aligned group
-        const float4 t = sk_sum4(sk, tile, r, f & ~3);
+        const float4 t = sk_sum4(sk, tile, pr, f & ~3);
         const float tv[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
         for (int i = 0; i < NE; ++i) v[i] = tv[(f & 3) + i];
@@ -201,8 +202,8 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
         }
     }
     T* dst;
-    if (which == 0) dst = reinterpret_cast<T*>(a.q_out) + (size_t)r * a.Hq * HD + head * HD + lane * NE;
-    else dst = reinterpret_cast<T*>(which == 1 ? a.kcache : a.vcache) + ((size_t)head * a.cap + (L + r)) * HD + lane * NE;
+    if (which == 0) dst = reinterpret_cast<T*>(a.q_out) + (size_t)pr * a.Hq * HD + head * HD + lane * NE;
+    else dst = reinterpret_cast<T*>(which == 1 ? a.kcache : a.vcache) + (((size_t)seq * a.Hkv + head) * a.cap + (L + r)) * HD + lane * NE;
     T o[NE];
 #pragma unroll
     for (int i = 0; i < NE; ++i) o[i] = from_f32<T>(v[i]);
@@ -216,17 +217,17 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
 __global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, int rows_fixed, StreamK sk, __nv_bfloat16* act, int F) {
     pdl_wait();
     if (threadIdx.x == 0) pdl_launch_dependents();
-    const int r = blockIdx.y;
-    const int n_rows = states ? (states->active ? states->n_rows : 0) : rows_fixed;
+    const int r = blockIdx.y, seq = blockIdx.z;
+    const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;
     const int j = (blockIdx.x * 256 + threadIdx.x) * 4;
     if (r >= n_rows || j >= F) return;
-    const int tile = j / 64, f = j % 64;
-    const float4 g = sk_sum4(sk, tile, r, f), u = sk_sum4(sk, tile, r, 64 + f);
+    const int tile = j / 64, f = j % 64, pr = seq * RT + r;
+    const float4 g = sk_sum4(sk, tile, pr, f), u = sk_sum4(sk, tile, pr, 64 + f);
     const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
     __nv_bfloat16 o[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) o[i] = __float2bfloat16_rn((gv[i] / (1.0f + expf(-gv[i]))) * uv[i]);
-    *reinterpret_cast<uint2*>(act + (size_t)r * F + j) = *reinterpret_cast<const uint2*>(o);
+    *reinterpret_cast<uint2*>(act + (size_t)pr * F + j) = *reinterpret_cast<const uint2*>(o);
 }
 
 // ------------------------------------------------------------------ CUDA-core GEMM
@@ -1014,16 +1015,16 @@ void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g
     else launch_k(k_rmsnorm<__nv_bfloat16>, grid, dim3(256), 0, s, pdl, st, x, (const __nv_bfloat16*)g, (__nv_bfloat16*)y, d, eps, copy_out);
 }
 void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
-                       float* copy_out, cudaStream_t s, bool pdl) {
-    launch_k(k_resid_norm<__nv_bfloat16>, dim3(RT, 1), dim3(1024), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
+                       float* copy_out, int nq, cudaStream_t s, bool pdl) {
+    launch_k(k_resid_norm<__nv_bfloat16>, dim3(RT, nq), dim3(1024), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
              (__nv_bfloat16*)y, d, eps, copy_out);
 }
-void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, cudaStream_t s, bool pdl) {
-    launch_k(k_swiglu_finish, dim3((F / 4 + 255) / 256, RT), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act, F);
+void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl) {
+    launch_k(k_swiglu_finish, dim3((F / 4 + 255) / 256, RT, nq), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act, F);
 }
-int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, cudaStream_t s, bool pdl) {
+int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl) {
     const int n_heads = a.Hq + 2 * a.Hkv;
-    dim3 grid((n_heads + 3) / 4, RT);
+    dim3 grid((n_heads + 3) / 4, RT, nq);
     if (a.h == 128) launch_k(k_qkv_finish<128>, grid, dim3(128), 0, s, pdl, a, sk);
     else if (a.h == 64) launch_k(k_qkv_finish<64>, grid, dim3(128), 0, s, pdl, a, sk);
     else if (a.h == 32) launch_k(k_qkv_finish<32>, grid, dim3(128), 0, s, pdl, a, sk);

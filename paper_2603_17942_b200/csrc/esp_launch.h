@@ -42,11 +42,11 @@ void launch_assemble(int dtype, const SeqState* st, const void* embed, const flo
                      int batch, cudaStream_t s, bool pdl);
 void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
                     float* copy_out, cudaStream_t s, bool pdl);
-// consumers of the split (EPI_PARTIAL) tensor-core GEMMs, bf16 models, one sequence
+// consumers of the split (EPI_PARTIAL) tensor-core GEMMs, bf16 models; nq = sequences the GEMM launch covered
 void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
-                       float* copy_out, cudaStream_t s, bool pdl);
-int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, cudaStream_t s, bool pdl);
-void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, cudaStream_t s, bool pdl);
+                       float* copy_out, int nq, cudaStream_t s, bool pdl);
+int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl);
+void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl);
 void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int off, int n, int last, int k, cudaStream_t s);
 void launch_set_tree(SeqState* st, int seq, const int32_t* tokens, const int32_t* parents, int n, int k, int n_anchor,
                      int* err, cudaStream_t s);
@@ -72,18 +72,21 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
 // tcgen05 GEMM: a plan holds the TMA descriptors and the stream-K partition of one weight shape
 struct TcGemm;
 // epi selects the tile -> weight-row mapping and the fused epilogue; with defer the kernel only stores partials
-// (EPI_PARTIAL) and the caller runs the matching consumer kernel
+// (EPI_PARTIAL) and the caller runs the matching consumer kernel.  x: activations [x_rows][K]; a deferred plan may
+// cover up to nq_max sequences per launch (their RT-row blocks are consecutive in x), so that the weights are
+// streamed once for all of them
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
-                   int batch, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
+                   int x_rows, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
                    int table_entries, void* packed, cudaStream_t stream);
 // bytes of the repacked copy of a weight set (tc_gemm_create's `packed`; NULL there = stream the caller's matrices)
 size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K);
 void tc_gemm_destroy(TcGemm* g);
-int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl);
-StreamK tc_gemm_streamk(const TcGemm* g);
+int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl, int nq = 1, int b_row0 = 0);
+StreamK tc_gemm_streamk(const TcGemm* g, int nq = 1);
 int tc_wait_selftest(int* err_dev, cudaStream_t s);
 int tc_gemm_tiles(const TcGemm* g);
-size_t tc_gemm_partial_bytes(int n_sm);
+size_t tc_gemm_partial_bytes(int n_sm, int nq = 1);
+int tc_gemm_max_nq();
 int tc_gemm_counter_ints();
 
 }  // namespace esp

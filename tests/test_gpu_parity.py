@@ -192,34 +192,38 @@ def test_bf16_forced_acceptance_bitwise_equals_greedy(pu):
     h.close()
 
 
-def test_bf16_batch_of_sequences_equals_each_sequence_alone(pu):
-    """Sequences are independent (each has its own cache, masks and tree): a handle holding three of them,
-    prefilled with different prompts (one of them later than the others), must emit for each exactly the stream
-    a single-sequence handle emits -- on the tensor-core path, which takes the sequences one at a time."""
+@pytest.mark.parametrize("n_seq", [2, 3, 5])
+def test_bf16_batch_of_sequences_equals_each_sequence_alone(pu, n_seq):
+    """Sequences are independent (each has its own cache, masks and tree): a handle holding several of them,
+    prefilled with different prompts (the last one later than the others), must emit for each exactly the stream
+    a single-sequence handle emits.  On the tensor-core path up to three consecutive sequences share one pass
+    through the layers (one weight stream, MMA N = 80 per sequence): 2 -> one pass of 2, 3 -> one pass of 3,
+    5 -> passes of 3 and 2."""
     import paper_2603_17942_b200 as P
     shape = BF16_SMALL
     w = synth.make_weights(shape, seed=5, gain_jitter=True, std=0.05)
     wd = pu.to_device(w)
     spec = O.SpecCfg(n_probes=3, topk=5, max_nodes=16, expand_width=0, n_anchor=1)
-    prompts = [synth.make_prompt(shape.vocab, n, 10 + i) for i, n in enumerate((90, 300, 17))]
+    lens = (90, 300, 17, 130, 64)[:n_seq]
+    prompts = [synth.make_prompt(shape.vocab, n, 10 + i) for i, n in enumerate(lens)]
     n_new, max_seq = 24, 400
     alone = []
     for pr in prompts:
         h1 = P.Handle(shape, pu.c_spec(spec), wd, max_seq_len=max_seq)
         alone.append(h1.generate(pr, n_new))
         h1.close()
-    h = P.Handle(shape, pu.c_spec(spec), wd, max_seq_len=max_seq, max_batch=3)
-    outs = [[h.prefill(prompts[0], 0)], [h.prefill(prompts[1], 1)], []]
+    h = P.Handle(shape, pu.c_spec(spec), wd, max_seq_len=max_seq, max_batch=n_seq)
+    outs = [[h.prefill(prompts[i], i)] for i in range(n_seq - 1)] + [[]]
     for step in range(200):
         if step == 3:
-            outs[2].append(h.prefill(prompts[2], 2))          # a sequence joins while the others are decoding
+            outs[-1].append(h.prefill(prompts[-1], n_seq - 1))   # a sequence joins while the others are decoding
         if all(len(o) >= n_new for o in outs):
             break
         P.esp_step(h.h, h.tokens_out, h.n_out)
-        for i in range(3):
+        for i in range(n_seq):
             outs[i].extend(int(t) for t in h.tokens_out[i, :h.n_out[i]])
     assert h.stats().device_error == 0
-    for i in range(3):
+    for i in range(n_seq):
         assert outs[i][:n_new] == alone[i], f"sequence {i}"
     h.close()
 
