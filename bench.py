@@ -307,13 +307,18 @@ def run_ours(args, shape, plen, k, K, B):
     w = synth.make_weights(shape, seed=rank, device="cuda")
     prompt = synth.make_prompt(shape.vocab, plen, rank)
     spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1, temperature=args.temperature, seed=1)
-    max_seq = plen + (k + 1) * (2 * steps + 2 * warm + 16) + 64
+    # room for one leg (at most k+1 tokens per step): the end-to-end leg starts again from the prompt
+    max_seq = plen + (k + 1) * (steps + warm + 20 + 16) + 64
     stream = torch.cuda.Stream()
     nbatch = max(1, args.batch)
     h = P.Handle(shape, spec, w, max_seq_len=max_seq, max_batch=nbatch, stream=stream)
-    h.prefill(prompt)
-    for i in range(1, nbatch):
-        h.prefill(synth.make_prompt(shape.vocab, plen, 1000 * rank + i), i)
+
+    def prefill_all():
+        h.prefill(prompt)
+        for i in range(1, nbatch):
+            h.prefill(synth.make_prompt(shape.vocab, plen, 1000 * rank + i), i)
+
+    prefill_all()
 
     def emitted_steps():
         st = h.stats()
@@ -349,7 +354,8 @@ def run_ours(args, shape, plen, k, K, B):
     launches = int(st.kernels_per_step) * steps
     rows = h.state()["n_rows"]
 
-    # ---- end to end: the synchronous call, tokens land in host memory every step
+    # ---- end to end: the synchronous call, tokens land in host memory every step (again from the prompt)
+    prefill_all()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()

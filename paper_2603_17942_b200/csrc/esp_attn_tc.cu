@@ -43,10 +43,12 @@ constexpr int MP = 128;                   // (row, head) pairs per CTA
 constexpr int HALF_BYTES = 128 * 128;     // one 128-row x 64-element (128-byte) swizzled tile
 constexpr int Q_BYTES = 2 * HALF_BYTES, K_BYTES = 2 * HALF_BYTES, V_BYTES = 2 * HALF_BYTES, P_BYTES = 2 * HALF_BYTES;
 constexpr int KV_STAGE = K_BYTES + V_BYTES;
-constexpr int OFF_Q = 0, OFF_KV = Q_BYTES, OFF_P = OFF_KV + 2 * KV_STAGE, OFF_BAR = OFF_P + P_BYTES;
+constexpr int STG_BYTES = 4 * 32 * 128;     // output staging: 32 rows x 128 bytes for each of the 4 output warps
+constexpr int OFF_Q = 0, OFF_KV = Q_BYTES, OFF_P = OFF_KV + 2 * KV_STAGE, OFF_STG = OFF_P + P_BYTES, OFF_BAR = OFF_STG + STG_BYTES;
 constexpr size_t SMEM_BYTES = 1024 + OFF_BAR + 256;
-constexpr int TMEM_COLS = 512;            // S0 at 0, S1 at 128, O at 256
-constexpr int NUM_THREADS = 320;           // producer warp, MMA warp, 8 softmax warps
+constexpr int TMEM_COLS = 512;            // S0 at 0, S1 at 128, O0 at 256, O1 at 384
+constexpr int MAX_T0_ENTRIES = 256;       // sequences x row tiles one launch may cover
+constexpr int NUM_THREADS = 448;           // producer warp, MMA warp, 8 softmax warps, 4 output warps
 
 struct BulkParams {
     CUtensorMap map_q;   // [batch*RT][Hq][128], box 64 x group x rows_per_tile
@@ -54,6 +56,7 @@ struct BulkParams {
     CUtensorMap map_v;
     AttnArgs a;
     int32_t group, rows_per_tile, n_row_tiles;
+    int32_t n_splits, n_seq, seq0;   // work items of this launch: n_splits x KV heads x row tiles x sequences [seq0, seq0 + n_seq)
 };
 
 __device__ __forceinline__ int tail_start_tc(int P, int dcap) {
@@ -72,12 +75,18 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_constant__ BulkParams p) {
+// ---- one item per CTA (grid = splits x (KV heads x row tiles) x sequences): used when the launch has at most
+// about one and a half items per SM, where start-up latency is all that counts.
+constexpr int ONCE_THREADS = 320;          // producer warp, MMA warp, 8 softmax warps (they also write the output)
+constexpr int ONCE_OFF_BAR = OFF_P + P_BYTES;
+constexpr size_t ONCE_SMEM_BYTES = 1024 + ONCE_OFF_BAR + 256;
+
+__global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __grid_constant__ BulkParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ int s_T0max;
     __shared__ float s_xchg[2][2 * MP];   // [exchange parity][half][pair]
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);   // [2]
+    uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + ONCE_OFF_BAR);   // [2]
     uint64_t* kv_empty = kv_full + 2;                                  // [2]
     uint64_t* s_full = kv_empty + 2;                                   // [2]
     uint64_t* q_full = s_full + 2;
@@ -343,6 +352,374 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
     }
 }
 
+// ---- persistent CTAs: used when the launch has clearly more items than SMs.
+// One work item = (split of the cache, KV head, row tile, sequence); what a role needs to know about it.
+struct Item {
+    int split, kvh, rtile, seq, row0, n_rows, L, beg, n_chunks;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_constant__ BulkParams p) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ int s_T0[MAX_T0_ENTRIES];  // [sequence][row tile]: largest T0 among the tile's rows
+    __shared__ int2 s_seq[MAX_T0_ENTRIES];  // [sequence]: (rows in its block, cached positions L)
+    __shared__ float s_xchg[2][2 * MP];   // [exchange parity][half][pair]
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);   // [2]
+    uint64_t* kv_empty = kv_full + 2;                                  // [2]
+    uint64_t* s_full = kv_empty + 2;                                   // [2]
+    uint64_t* o_free = s_full + 2;                                     // [2] an O accumulator has been read out
+    uint64_t* o_full = o_free + 2;                                     // [2] an item's last P V has completed
+    uint64_t* q_full = o_full + 2;
+    uint64_t* q_free = q_full + 1;                                     // the item's last Q K^T has completed
+    uint64_t* p_ready = q_free + 1;
+    uint64_t* pv_done = p_ready + 1;
+    uint64_t* xchg = pv_done + 1;                                      // the two threads of a pair exchanged a value
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(xchg + 1);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+    const AttnArgs& a = p.a;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // Read before pdl_wait(): the sequence state and the cache below T0, both written by earlier steps.
+    if (threadIdx.x == 0) pdl_launch_dependents();
+    for (int e = warp; e < p.n_seq * p.n_row_tiles; e += NUM_THREADS / 32) {   // one warp per entry, a lane per row
+        const int seq = p.seq0 + e / p.n_row_tiles, row0 = (e % p.n_row_tiles) * p.rows_per_tile;
+        int n_rows, L;
+        if (a.st) { n_rows = a.st[seq].active ? a.st[seq].n_rows : 0; L = a.st[seq].L; }
+        else { n_rows = a.n_rows_fixed; L = a.L_fixed; }
+        int t0 = 0;
+        for (int r = row0 + lane; r < row0 + p.rows_per_tile && r < n_rows; r += 32)
+            t0 = max(t0, tail_start_tc(L + (a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r]), a.dcap));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t0 = max(t0, __shfl_xor_sync(0xffffffffu, t0, o));
+        if (lane == 0) {
+            s_T0[e] = t0;
+            if (e % p.n_row_tiles == 0) s_seq[e / p.n_row_tiles] = make_int2(n_rows, L);
+        }
+    }
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); mbar_init(&s_full[i], 1); mbar_init(&o_free[i], 128);
+            mbar_init(&o_full[i], 1);
+        }
+        mbar_init(q_full, 1);
+        mbar_init(q_free, 1);
+        mbar_init(p_ready, 256);
+        mbar_init(pv_done, 1);
+        mbar_init(xchg, 256);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *s_tmem;
+    unsigned char* sQ = smem + OFF_Q;
+    unsigned char* sP = smem + OFF_P;
+
+    // Items are dealt round-robin; every role walks the same list and skips the same empty items, so the
+    // per-chunk and per-item counters below advance identically in all of them.
+    const int n_items = p.n_splits * a.Hkv * p.n_row_tiles * p.n_seq;
+    auto get_item = [&](int idx, Item& it) -> bool {
+        it.split = idx % p.n_splits;
+        int y = idx / p.n_splits;
+        it.rtile = y % p.n_row_tiles;
+        y /= p.n_row_tiles;
+        it.kvh = y % a.Hkv;
+        const int lseq = y / a.Hkv;
+        it.seq = p.seq0 + lseq;
+        it.n_rows = s_seq[lseq].x;
+        it.L = s_seq[lseq].y;
+        it.row0 = it.rtile * p.rows_per_tile;
+        if (it.row0 >= it.n_rows) return false;
+        const int T0max = s_T0[lseq * p.n_row_tiles + it.rtile];
+        it.beg = it.split * a.split_len;
+        if (it.beg >= T0max) return false;
+        const int end = min(it.beg + a.split_len, T0max);
+        it.n_chunks = (end - it.beg + CK - 1) / CK;
+        return true;
+    };
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            bool ok = true, first = true;
+            uint32_t gc = 0, n_it = 0;       // chunks and items issued so far
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                Item it;
+                if (!get_item(idx, it)) continue;
+                const int kvrow0 = (it.seq * a.Hkv + it.kvh) * a.cap + it.beg;
+                auto load_chunk = [&](int c) -> bool {
+                    const uint32_t g = gc + c;
+                    // a fresh barrier passes a wait on parity 1: the first use of a stage does not block
+                    if (!mbar_wait(&kv_empty[g & 1], ((g >> 1) & 1) ^ 1, s_abort)) return false;
+                    unsigned char* st = smem + OFF_KV + (g & 1) * KV_STAGE;
+                    mbar_expect_tx(&kv_full[g & 1], KV_STAGE);
+                    tma_load_2d(st, &p.map_k, 0, kvrow0 + c * CK, &kv_full[g & 1]);
+                    tma_load_2d(st + HALF_BYTES, &p.map_k, 64, kvrow0 + c * CK, &kv_full[g & 1]);
+                    tma_load_2d(st + K_BYTES, &p.map_v, 0, kvrow0 + c * CK, &kv_full[g & 1]);
+                    tma_load_2d(st + K_BYTES + HALF_BYTES, &p.map_v, 64, kvrow0 + c * CK, &kv_full[g & 1]);
+                    return true;
+                };
+                int c0 = 0;
+                if (first) {
+                    // the cache does not depend on the kernel before this one, the queries do
+                    for (; c0 < it.n_chunks && c0 < 2 && ok; ++c0) ok = load_chunk(c0);
+                    pdl_wait();
+                    first = false;
+                } else {
+                    // Q is single buffered: the previous item's last Q K^T must have completed
+                    ok = mbar_wait(q_free, (n_it - 1) & 1, s_abort);
+                }
+                if (!ok) break;
+                mbar_expect_tx(q_full, Q_BYTES);
+                tma_load_3d(sQ, &p.map_q, 0, it.kvh * p.group, it.seq * RT + it.row0, q_full);
+                tma_load_3d(sQ + HALF_BYTES, &p.map_q, 64, it.kvh * p.group, it.seq * RT + it.row0, q_full);
+                for (int c = c0; c < it.n_chunks && ok; ++c) ok = load_chunk(c);
+                gc += it.n_chunks;
+                ++n_it;
+            }
+            if (first) pdl_wait();
+            if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            uint32_t gc = 0, n_it = 0;
+            const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                Item it;
+                if (!get_item(idx, it)) continue;
+                const uint32_t tmem_o = tmem_base + 256 + (n_it & 1) * 128;
+                auto issue_qk = [&](int c) {
+                    const uint32_t g = gc + c;
+                    const uint32_t k_addr = smem_u32(smem + OFF_KV + (g & 1) * KV_STAGE);
+                    const uint32_t tmem_s = tmem_base + (g & 1) * 128;
+#pragma unroll
+                    for (int kk = 0; kk < HD / 16; ++kk) {
+                        const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+                        umma(tmem_s, smem_desc(q_addr + off, 16), smem_desc(k_addr + off, 16), IDESC_QK, kk > 0 ? 1u : 0u);
+                    }
+                    umma_commit(&s_full[g & 1]);
+                    if (c == it.n_chunks - 1) umma_commit(q_free);
+                };
+                ok = mbar_wait(q_full, n_it & 1, s_abort) && mbar_wait(&kv_full[gc & 1], (gc >> 1) & 1, s_abort) &&
+                     mbar_wait(&o_free[n_it & 1], ((n_it >> 1) & 1) ^ 1, s_abort);   // this O buffer's previous item was read out
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                issue_qk(0);
+                for (int c = 0; c < it.n_chunks && ok; ++c) {
+                    const uint32_t g = gc + c;
+                    if (c + 1 < it.n_chunks) {     // S of the next chunk while the softmax of this one runs
+                        if (!mbar_wait(&kv_full[(g + 1) & 1], ((g + 1) >> 1) & 1, s_abort)) { ok = false; break; }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        issue_qk(c + 1);
+                    }
+                    if (!mbar_wait(p_ready, g & 1, s_abort)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t v_addr = smem_u32(smem + OFF_KV + (g & 1) * KV_STAGE + K_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < CK / 16; ++kk) {
+                        const uint32_t p_off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;     // P: K-major over keys
+                        const uint32_t v_off = kk * 16 * 128;                              // V: 16 key rows of 128 bytes further
+                        umma(tmem_o, smem_desc(p_addr + p_off, 16), smem_desc(v_addr + v_off, HALF_BYTES), IDESC_PV,
+                             (c > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    umma_commit(pv_done);
+                    umma_commit(&kv_empty[g & 1]);
+                    if (c == it.n_chunks - 1) umma_commit(&o_full[n_it & 1]);
+                }
+                gc += it.n_chunks;
+                ++n_it;
+            }
+            if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
+        }
+    } else if (warp < 10) {
+        // ---------------- softmax warps 2..9: a thread owns one pair (= tensor-memory lane) and one half of the
+        // chunk's 128 keys (warps 2-5 keys 0..63, warps 6-9 keys 64..127); the two threads of a pair exchange
+        // their maxima (per chunk) and their sums (at the end of an item) through shared memory
+        const int q4 = warp & 3;
+        const int hf = (warp - 2) >> 2;
+        const int pair = q4 * 32 + lane;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16) + hf * 64;   // this thread's 64 columns of S / O
+        uint32_t gc = 0, n_it = 0, xc = 0;   // chunks, items, exchanges so far
+        bool ok = true;
+        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            Item it;
+            if (!get_item(idx, it)) continue;
+            const int r = it.row0 + pair / p.group, head = it.kvh * p.group + pair % p.group;
+            const bool pv = pair / p.group < p.rows_per_tile && r < it.n_rows && r < RT;
+            int T0row = 0;
+            if (pv) T0row = tail_start_tc(it.L + (a.st ? a.st[it.seq].row_depth[r] : a.depth[it.seq * RT + r]), a.dcap);
+            const uint32_t o_addr = lane_addr + 256 + (n_it & 1) * 128;
+            float m_run = -INFINITY, l_run = 0.f;
+            for (int c = 0; c < it.n_chunks && ok; ++c) {
+                const uint32_t g = gc + c;
+                // (a wait that fails must take the whole warp out: the tensor-memory accesses below are warp-wide)
+                if (!__all_sync(0xffffffffu, mbar_wait(&s_full[g & 1], (g >> 1) & 1, s_abort))) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t s_addr = lane_addr + (g & 1) * 128;
+                const int cbase = it.beg + c * CK + hf * 64;
+                // the row's scores for this half, masked to its visible keys and scaled to the log2 domain
+                uint32_t sv[64];
+                tmem_ld64(s_addr, sv);
+                float cmax = -INFINITY;
+                if (__all_sync(0xffffffffu, cbase + 64 <= T0row)) {     // every key of the half is visible to every row of the warp
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) {
+                        const float sc = __uint_as_float(sv[i]) * a.scale_log2;
+                        sv[i] = __float_as_uint(sc);
+                        cmax = fmaxf(cmax, sc);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) {
+                        const float sc = cbase + i < T0row ? __uint_as_float(sv[i]) * a.scale_log2 : -INFINITY;
+                        sv[i] = __float_as_uint(sc);
+                        cmax = fmaxf(cmax, sc);
+                    }
+                }
+                // the chunk maximum over both halves
+                // (double buffered by exchange parity: a thread can be one exchange ahead of its partner, not two)
+                s_xchg[xc & 1][hf * MP + pair] = cmax;
+                mbar_arrive(xchg);
+                if (!__all_sync(0xffffffffu, mbar_wait(xchg, xc & 1, s_abort))) { ok = false; break; }
+                cmax = fmaxf(s_xchg[xc & 1][pair], s_xchg[xc & 1][MP + pair]);
+                ++xc;
+                const float m_new = fmaxf(m_run, cmax);
+                const float m_use = m_new == -INFINITY ? 0.f : m_new;
+                const float alpha = exp2f(m_run - m_use);
+                // P of the previous chunk must have been consumed before it is overwritten, and O must be final
+                // before it is rescaled
+                if (g > 0 && !__all_sync(0xffffffffu, mbar_wait(pv_done, (g - 1) & 1, s_abort))) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                // probabilities, their sum (key order), P as bf16 in the A-operand layout (this half = one swizzled tile)
+                float csum = 0.f;
+                unsigned char* prow = sP + hf * HALF_BYTES + pair * 128;
+#pragma unroll
+                for (int blk = 0; blk < 2; ++blk) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float p0 = exp2f(__uint_as_float(sv[blk * 32 + i]) - m_use), p1 = exp2f(__uint_as_float(sv[blk * 32 + i + 1]) - m_use);
+                        csum += p0;
+                        csum += p1;
+                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+                        pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int chunk16 = blk * 4 + j;
+                        *reinterpret_cast<uint4*>(prow + ((chunk16 ^ (pair & 7)) << 4)) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                    }
+                }
+                if (c > 0) {
+                    // O <- alpha * O (in tensor memory), this thread's 64 of the 128 columns
+                    if (__any_sync(0xffffffffu, alpha != 1.0f)) {   // warp-uniform: skip when no lane's maximum moved
+                        tmem_ld64(o_addr, sv);
+#pragma unroll
+                        for (int blk = 0; blk < 2; ++blk) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) sv[blk * 32 + i] = __float_as_uint(__uint_as_float(sv[blk * 32 + i]) * alpha);
+                            tmem_st32(o_addr + blk * 32, *reinterpret_cast<const uint32_t(*)[32]>(&sv[blk * 32]));
+                        }
+                        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    }
+                }
+                l_run = l_run * alpha + csum;     // this half's share of the row sum
+                m_run = m_new;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes -> tensor-core reads
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mbar_arrive(p_ready);
+            }
+            if (!ok) break;
+            gc += it.n_chunks;
+            // the row sum = first half's share + second half's share; the output warps take care of O
+            s_xchg[xc & 1][hf * MP + pair] = l_run;
+            mbar_arrive(xchg);
+            if (!__all_sync(0xffffffffu, mbar_wait(xchg, xc & 1, s_abort))) { ok = false; break; }
+            const float l_tot = s_xchg[xc & 1][pair] + s_xchg[xc & 1][MP + pair];
+            ++xc;
+            if (pv && hf == 0) a.part_ml[((size_t)(it.seq * RT + r) * a.Hq + head) * a.n_split_max + it.split] = make_float2(m_run, l_tot);
+            ++n_it;
+        }
+        if (!ok && lane == 0) {
+            set_error(a.err, DEV_E_WAIT_TIMEOUT);
+            *s_abort = 1;
+        }
+    } else {
+        // ---------------- output warps 10..13: when an item's last P V has completed, its O accumulator goes tensor
+        // memory -> registers -> (transposed through 4 KB of shared memory per warp) -> global, so that every store
+        // instruction writes whole 128-byte lines, while the softmax warps are already on the next item.  The
+        // tensor-memory loads are warp-wide: every lane takes part.
+        const int q4 = warp & 3;
+        const uint32_t lane_o = tmem_base + ((uint32_t)(q4 * 32) << 16) + 256;
+        unsigned char* stg = smem + OFF_STG + (warp - 10) * (32 * 128);
+        uint32_t n_it = 0;
+        bool ok = true;
+        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            Item it;
+            if (!get_item(idx, it)) continue;
+            const int b = n_it & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(&o_full[b], (n_it >> 1) & 1, s_abort))) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // where the 8 rows this lane stores per pass go (-1: no such pair)
+            const int j = lane & 7;
+            long long obase[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int pr = q4 * 32 + i * 4 + (lane >> 3);
+                const int r2 = it.row0 + pr / p.group, head2 = it.kvh * p.group + pr % p.group;
+                const bool valid = pr / p.group < p.rows_per_tile && r2 < it.n_rows && r2 < RT;
+                obase[i] = valid ? (long long)((((size_t)(it.seq * RT + r2) * a.Hq + head2) * a.n_split_max + it.split) * HD + j * 4) : -1;
+            }
+#pragma unroll 1
+            for (int t = 0; t < 4; ++t) {
+                uint32_t ov[32];
+                tmem_ld32(lane_o + b * 128 + t * 32, ov);
+                if (t == 3) {   // the accumulator is in registers: hand it back to the MMA warp
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    mbar_arrive(&o_free[b]);
+                }
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj)
+                    *reinterpret_cast<uint4*>(stg + lane * 128 + ((jj ^ (lane & 7)) << 4)) =
+                        make_uint4(ov[4 * jj], ov[4 * jj + 1], ov[4 * jj + 2], ov[4 * jj + 3]);
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = i * 4 + (lane >> 3);                      // pair within the warp
+                    if (obase[i] >= 0) {
+                        const uint4 val = *reinterpret_cast<const uint4*>(stg + rr * 128 + ((j ^ (rr & 7)) << 4));
+                        __stcg(reinterpret_cast<uint4*>(a.part_o + obase[i] + t * 32), val);
+                    }
+                }
+                __syncwarp();
+            }
+            ++n_it;
+        }
+        if (!ok && lane == 0) {
+            set_error(a.err, DEV_E_WAIT_TIMEOUT);
+            *s_abort = 1;
+        }
+    }
+    // ---------------- teardown (every thread arrives here)
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (*s_abort) {
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);   // let copies in flight land before shared memory goes away
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
 // ---- tail + merge: one warp per (row, head) pair
 __device__ __forceinline__ int nth_set_bit128(unsigned long long lo, unsigned long long hi, int n) {
     int c = __popcll(lo);
@@ -568,8 +945,38 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
     BulkParams p = t->p;
     p.a = a;
     if (n_split_launch > 0) {
-        dim3 grid(n_split_launch, a.Hkv * p.n_row_tiles, batch);
-        if (launch_k(k_attn_bulk_tc, grid, dim3(NUM_THREADS), SMEM_BYTES, s, pdl, p) != cudaSuccess) return -1;
+        static int n_sm = 0;
+        if (n_sm == 0) {
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1) {
+                n_sm = 0;
+                return -1;
+            }
+        }
+        const long long all_items = (long long)n_split_launch * a.Hkv * p.n_row_tiles * batch;
+        if (all_items <= n_sm + n_sm / 2) {
+            // (nearly) every CTA runs once: one item per CTA.  Measured crossover: the persistent kernel wins from
+            // about 1.2 waves when timed alone, a little later inside a step, where its larger register and
+            // shared-memory footprint delays its start behind the kernel before it
+            static bool once_attr = false;
+            if (!once_attr) {
+                if (cudaFuncSetAttribute(k_attn_bulk_tc_once, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ONCE_SMEM_BYTES) != cudaSuccess) return -1;
+                once_attr = true;
+            }
+            dim3 grid(n_split_launch, a.Hkv * p.n_row_tiles, batch);
+            if (launch_k(k_attn_bulk_tc_once, grid, dim3(ONCE_THREADS), ONCE_SMEM_BYTES, s, pdl, p) != cudaSuccess) return -1;
+        } else {
+            // persistent CTAs, one per SM, walk the (split, KV head, row tile, sequence) items round-robin
+            const int per_launch = MAX_T0_ENTRIES / p.n_row_tiles;
+            for (int s0 = 0; s0 < batch; s0 += per_launch) {
+                p.seq0 = s0;
+                p.n_seq = batch - s0 < per_launch ? batch - s0 : per_launch;
+                p.n_splits = n_split_launch;
+                const long long items = (long long)p.n_splits * a.Hkv * p.n_row_tiles * p.n_seq;
+                const int grid = (int)(items < n_sm ? items : n_sm);
+                if (launch_k(k_attn_bulk_tc, dim3(grid), dim3(NUM_THREADS), SMEM_BYTES, s, pdl, p) != cudaSuccess) return -1;
+            }
+        }
     }
     if (launch_k(k_attn_tail_merge_tc, dim3((RT + 3) / 4, a.Hq, batch), dim3(128), 0, s, pdl, a) != cudaSuccess) return -1;
     return 0;
