@@ -306,7 +306,12 @@ def run_ours(args, shape, plen, k, K, B):
     steps, warm = args.steps, max(args.warmup, 3)
     w = synth.make_weights(shape, seed=rank, device="cuda")
     prompt = synth.make_prompt(shape.vocab, plen, rank)
-    spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1, temperature=args.temperature, seed=1)
+    if args.per_node_probes:
+        # the paper's block layout: k = 3 masks behind every one of 30 tree nodes, BC = (k+1) * 30 = 120 rows
+        k, K, B = 3, 10, 30
+        spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=1, n_anchor=0, temperature=args.temperature, seed=1)
+    else:
+        spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1, temperature=args.temperature, seed=1)
     # room for one leg (at most k+1 tokens per step): the end-to-end leg starts again from the prompt
     max_seq = plen + (k + 1) * (steps + warm + 20 + 16) + 64
     stream = torch.cuda.Stream()
@@ -397,7 +402,7 @@ def run_ours(args, shape, plen, k, K, B):
         hg.close()
 
     replay = None
-    if rank == 0 and not args.no_greedy and nbatch == 1:
+    if rank == 0 and not args.no_greedy and nbatch == 1 and not args.per_node_probes:
         replay = replay_leg(P, shape, w, prompt, stream, k, B, min(256, steps))
 
     # ---- aggregate over ranks: slowest rank's time, all ranks' tokens
@@ -524,6 +529,8 @@ def main():
     ap.add_argument("--batch", type=int, default=1, help="independent sequences in one handle (long-context / batch sweep)")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="0 = greedy matching (default); > 0 = sample matching at that temperature")
+    ap.add_argument("--per-node-probes", action="store_true",
+                    help="k = 3 probes behind each of 30 tree nodes (block complexity 120) instead of the default block")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer count (smaller captures under a profiler)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-greedy", action="store_true", help="skip the greedy-decoding leg")

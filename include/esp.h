@@ -39,7 +39,7 @@ enum {
     ESP_E_ARG = -8        /* NULL or out-of-range argument */
 };
 
-#define ESP_MAX_ROWS 80   /* rows of one block per sequence: tree nodes + mask probes */
+#define ESP_MAX_ROWS 128  /* rows of one block per sequence: tree nodes + mask probes */
 #define ESP_MAX_PROBES 8  /* k */
 #define ESP_MAX_KPRIME 32 /* Top-K entries kept per probe, K + pruner refills */
 
@@ -159,7 +159,9 @@ int esp_set_mask(esp_handle* h, int32_t seq, const float* mask);
  * tokens/parents [host] n nodes in breadth-first order (parents[0] = -1,
  * parents[i] < i); node 0 must carry the current root token.  Has no
  * counterpart in the paper; it exists to drive acceptance lengths that
- * random-init models never produce. */
+ * random-init models never produce.  The tree with its probe rows must fit the
+ * block the handle was configured for (the larger of the spec's rows and
+ * 64 + n_probes), else ESP_E_ARG. */
 int esp_set_tree(esp_handle* h, int32_t seq, const int32_t* tokens, const int32_t* parents, int32_t n);
 
 /* Debug/parity access to device state of sequence `seq`, copied to [host] buffers (any may be NULL):
@@ -231,17 +233,17 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
  * point of the call: a serving loop whose device memory was budgeted up front and handed to other owners, a
  * plug-in running inside somebody else's process that must not touch the allocator, code between the
  * begin and end of work where an allocation would stall the whole device.  The split partials live in a
- * fixed array inside the library instead (ESP_STATIC_SCRATCH_BYTES, 16 MiB, held on every GPU that loads
+ * fixed array inside the library instead (ESP_STATIC_SCRATCH_BYTES, 32 MiB, held on every GPU that loads
  * the library until the process exits).  Same arguments, layouts and results as esp_tree_attention, minus
  * the scratch pair.  Returns ESP_E_WORKSPACE when the shape needs more than the array holds
  * (esp_tree_attention_scratch_bytes(batch, n_q_heads, head_dim, cap) > ESP_STATIC_SCRATCH_BYTES; e.g. 32
- * query heads of 128 with cap <= 2128 at batch 1 fit).  It allocates and frees nothing, on the host or the
+ * query heads of 128 with cap <= 3584 at batch 1 fit).  It allocates and frees nothing, on the host or the
  * device.  The first call on each device looks up the array's device address (a one-time query, no
  * allocation); make that first call outside any stream capture.  All calls share the one array and it keeps
  * the previous call's contents: the entry point re-zeroes the error word it reads, everything else is
  * overwritten before it is read.  Two calls whose kernels can overlap on the GPU (different streams, no
  * dependency between them) would write the same partials and race: keep them ordered. */
-#define ESP_STATIC_SCRATCH_BYTES (16u << 20)
+#define ESP_STATIC_SCRATCH_BYTES (32u << 20)
 int esp_tree_attention_static(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, int32_t cap, int32_t n_q_heads,
                               int32_t n_kv_heads, int32_t head_dim, int32_t dcap, const void* q, const void* kcache,
                               const void* vcache, const uint64_t* anc, const int32_t* depth, void* out,

@@ -16,7 +16,7 @@ import numpy as np
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libesp_b200.so")
 
-ESP_MAX_ROWS = 80
+ESP_MAX_ROWS = 128
 ESP_MAX_PROBES = 8
 ESP_MAX_KPRIME = 32
 
@@ -232,7 +232,7 @@ def esp_tree_attention(dtype: int, batch: int, n_rows: int, L: int, cap: int, n_
         "esp_tree_attention")
 
 
-ESP_STATIC_SCRATCH_BYTES = 16 << 20
+ESP_STATIC_SCRATCH_BYTES = 32 << 20
 
 
 def esp_tree_attention_static(dtype: int, batch: int, n_rows: int, L: int, cap: int, n_q_heads: int, n_kv_heads: int,

@@ -124,6 +124,8 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
         for (int i = 0; i < PROBES_MAX; ++i) D->static_w[i] = is_static && i < s->n_probes ? s->static_widths[i] : 0;
         D->n_anchor = s->n_anchor; D->prune_parent = s->prune_parent; D->prune_root = s->prune_root;
         D->ema_per_token = s->ema_per_token; D->lambda = s->lambda;
+        // rows of a block the tensor-core GEMMs carry: 80 covers every tree of at most 80 rows and the prefill blocks
+        D->gemm_rows = spec_rows(*s) <= 80 ? 80 : RT;
         D->inv_temp = s->temperature > 0.f ? 1.0f / s->temperature : 0.f;
         D->seed_lo = s->seed_lo; D->seed_hi = s->seed_hi;
     }
@@ -160,7 +162,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.tree_dev = c.take<int32_t>(2 * RT);
     o.rope_cos = c.take<float>((size_t)D.cap * (D.h / 2));
     o.rope_sin = c.take<float>((size_t)D.cap * (D.h / 2));
-    o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm, D.batch < tc_gemm_max_nq() ? D.batch : tc_gemm_max_nq()));
+    o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm, D.batch < tc_gemm_max_nq(D.gemm_rows) ? D.batch : tc_gemm_max_nq(D.gemm_rows), D.gemm_rows));
     o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
     o.sk_tables = c.take<TileSrc>(4 * SK_TABLE_TILES);
     o.packed = nullptr;
@@ -188,6 +190,7 @@ struct esp_handle {
     Buffers b;
     cudaStream_t stream;
     int dtype, gemm_impl, n_sm;
+    int rows_cap = RT;   // no block (step or prefill) has more rows than this
     const void *embed, *lm_head, *final_norm;
     std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, na, nf, qn, kn;
     std::vector<TcGemm*> p_qkv, p_o, p_gu, p_down;
@@ -272,12 +275,13 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
     const size_t kv_seq_off = (size_t)s0 * D.Hkv * D.cap * D.h * es;   // this pass's first sequence inside a layer's cache
     float* mvec0 = b.mvec + (size_t)s0 * D.mask_slots * D.d;
     StreamK pending;   // partials of the last down projection, summed by the next norm
-    pending.partials = nullptr; pending.table = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2; pending.rows = RT;
+    pending.partials = nullptr; pending.table = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2; pending.rows = RT; pending.seq_rows = RT;
     mark(h, -1);
-    launch_assemble(h->dtype, st0, h->embed, mvec0, b.hres, D.d, D.mask_slots, nb, s, false);
+    const int rc_rows = h->rows_cap;     // no block has more rows: sizes the row dimension of the grids
+    launch_assemble(h->dtype, st0, h->embed, mvec0, b.hres, D.d, D.mask_slots, nb, s, false, rc_rows);
     h->launches++;
     for (int l = 0; l < D.n_layers; ++l) {
-        if (tc) launch_resid_norm(st0, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl);
+        if (tc) launch_resid_norm(st0, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->na[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -294,7 +298,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             if (rc) return rc;
             mark(h, KIND_QKV);
             if (tc) {
-                if (launch_qkv_finish(a, tc_gemm_streamk(h->p_qkv[l], nb), nb, s, pdl)) return ESP_E_BADCFG;
+                if (launch_qkv_finish(a, tc_gemm_streamk(h->p_qkv[l], nb), nb, s, pdl, rc_rows)) return ESP_E_BADCFG;
                 h->launches++;
                 mark(h, KIND_MISC);
             }
@@ -310,6 +314,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.st = st0;
             a.Hq = D.Hq; a.Hkv = D.Hkv; a.h = D.h; a.cap = D.cap; a.split_len = D.split_len; a.n_split_max = D.n_split_max;
             a.dcap = dcap;
+            a.rows_cap = rc_rows;
             a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
             a.err = b.err;
             if (tc) {
@@ -330,7 +335,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             if (rc) return rc;
             mark(h, KIND_O);
         }
-        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(h->p_o[l], nb), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl);
+        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(h->p_o[l], nb), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -343,7 +348,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             if (rc) return rc;
             mark(h, KIND_GATEUP);
             if (tc) {
-                launch_swiglu_finish(st0, tc_gemm_streamk(h->p_gu[l], nb), b.act, D.F, nb, s, pdl);
+                launch_swiglu_finish(st0, tc_gemm_streamk(h->p_gu[l], nb), b.act, D.F, nb, s, pdl, rc_rows);
                 h->launches++;
                 mark(h, KIND_MISC);
             }
@@ -361,7 +366,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
     }
     if (with_lm) {
         float* dbg_hidden = h->dbg_hidden ? h->dbg_hidden + (size_t)s0 * RT * D.d : nullptr;
-        if (tc) launch_resid_norm(st0, b.hres, pending, h->final_norm, b.xn, D.d, D.rms_eps, dbg_hidden, nb, s, pdl);
+        if (tc) launch_resid_norm(st0, b.hres, pending, h->final_norm, b.xn, D.d, D.rms_eps, dbg_hidden, nb, s, pdl, rc_rows);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, nb, dbg_hidden, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -375,10 +380,10 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.logits_dump = h->dbg_logits ? h->dbg_logits + (size_t)sq * RT * D.V : nullptr;
             const void* w[3] = {h->lm_head, nullptr, nullptr};
             const int32_t rows[3] = {D.V, 0, 0};
-            int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl, 1, q * RT);
+            int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl, 1, q);
             if (rc) return rc;
             mark(h, KIND_LMHEAD);
-            launch_topk_merge(b.states + sq, b.cand, b.cand_ms, n_tiles, D.KP, per, b.topk + (size_t)sq * RT * KP_MAX, b.lse + (size_t)sq * RT, s, pdl);
+            launch_topk_merge(b.states + sq, b.cand, b.cand_ms, n_tiles, D.KP, per, b.topk + (size_t)sq * RT * KP_MAX, b.lse + (size_t)sq * RT, s, pdl, rc_rows);
             h->launches++;
             mark(h, KIND_SELECT);
         }
@@ -392,7 +397,7 @@ int forward(esp_handle* h, bool with_lm, int dcap, int only_seq) {
     if (!tc) return forward_pass(h, with_lm, dcap, 0, h->D.batch, false);
     if (only_seq >= 0) return forward_pass(h, with_lm, dcap, only_seq, 1, true);
     // consecutive sequences share a pass (and a weight stream); sequences that are not ready are inactive in it
-    const int per_pass = tc_gemm_max_nq();
+    const int per_pass = tc_gemm_max_nq(h->D.gemm_rows);
     for (int s0 = 0; s0 < h->D.batch; s0 += per_pass) {
         const int nb = h->D.batch - s0 < per_pass ? h->D.batch - s0 : per_pass;
         bool any = false;
@@ -478,6 +483,11 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
     h->dtype = model->dtype;
     h->gemm_impl = model->dtype == 0 ? 1 : 0;
     h->n_sm = n_sm;
+    {
+        const int step_rows = spec_rows(*spec), pre_rows = PREFILL_CHUNK + spec->n_probes;
+        h->rows_cap = step_rows > pre_rows ? step_rows : pre_rows;
+        if (h->rows_cap > RT) h->rows_cap = RT;
+    }
     carve_all(D, model->dtype, 148, reinterpret_cast<char*>(workspace), &h->b);
     h->embed = w->embed; h->lm_head = w->lm_head; h->final_norm = w->final_norm;
     for (int l = 0; l < D.n_layers; ++l) {
@@ -509,34 +519,35 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
     }
     if (model->dtype == 1) {
         const int dq = D.Hq * D.h, dkv = D.Hkv * D.h;
-        const int nq_max = D.batch < tc_gemm_max_nq() ? D.batch : tc_gemm_max_nq();   // sequences sharing a weight stream
+        const int nrs = D.gemm_rows;
+        const int nq_max = D.batch < tc_gemm_max_nq(nrs) ? D.batch : tc_gemm_max_nq(nrs);   // sequences sharing a weight stream
         bool ok = true;
         for (int l = 0; l < D.n_layers && ok; ++l) {
             TcGemm* p = nullptr;
             char* pk = h->b.packed + h->b.pk_layer * l;
             const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t r1[3] = {dq, dkv, dkv};
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, D.batch * RT, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream);
             h->p_qkv.push_back(p);
             const void* w2[3] = {h->wo[l], nullptr, nullptr};
             const int32_t r2[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, D.batch * RT, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream);
             h->p_o.push_back(p);
             const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t r3[3] = {D.F, D.F, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, D.batch * RT, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream);
             h->p_gu.push_back(p);
             const void* w4[3] = {h->wd[l], nullptr, nullptr};
             const int32_t r4[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, D.batch * RT, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream);
             h->p_down.push_back(p);
         }
         const void* w5[3] = {h->lm_head, nullptr, nullptr};
         const int32_t r5[3] = {D.V, 0, 0};
-        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, D.batch * RT, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
+        ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, D.batch, nrs, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
         if (!ok) { esp_free(h); return ESP_E_CUDA; }
     }
     if (cudaStreamSynchronize(h->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) { esp_free(h); return ESP_E_CUDA; }
@@ -677,7 +688,7 @@ int esp_set_tree(esp_handle* h, int32_t seq, const int32_t* tokens, const int32_
     if (seq < 0 || seq >= h->D.batch || !h->ready[seq]) return ESP_E_STATE;
     const int k = h->D.k;
     const int nA = k > 0 ? (h->D.n_anchor == 0 ? n : (h->D.n_anchor < n ? h->D.n_anchor : n)) : 0;
-    if (n < 1 || n + nA * k > RT) return ESP_E_ARG;
+    if (n < 1 || n + nA * k > h->rows_cap) return ESP_E_ARG;   // the kernels are sized for the configured block
     std::vector<int> depth(n, 0);
     for (int i = 0; i < n; ++i) {
         if (tokens[i] < 0 || tokens[i] >= h->D.V) return ESP_E_ARG;
@@ -908,7 +919,7 @@ int esp_tree_attention_static(int32_t dtype, int32_t batch, int32_t n_rows, int3
 
 int esp_gemm_scratch_bytes(size_t* bytes_out) {
     if (!bytes_out) return ESP_E_ARG;
-    *bytes_out = align_up(tc_gemm_partial_bytes(148), 256) + align_up(sizeof(int) * tc_gemm_counter_ints(), 256) + 256;
+    *bytes_out = align_up(tc_gemm_partial_bytes(148, 1, RT), 256) + align_up(sizeof(int) * tc_gemm_counter_ints(), 256) + 256;
     return ESP_OK;
 }
 
@@ -935,12 +946,12 @@ int esp_gemm_bf16(int32_t impl, int32_t rows, int32_t n_out, int32_t k_in, const
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return ESP_E_CUDA;
     if (n_sm > 148) n_sm = 148;
     char* sc = reinterpret_cast<char*>(scratch);
-    int* counters = reinterpret_cast<int*>(sc + align_up(tc_gemm_partial_bytes(148), 256));
+    int* counters = reinterpret_cast<int*>(sc + align_up(tc_gemm_partial_bytes(148, 1, RT), 256));
     int* err = reinterpret_cast<int*>(sc + need - 256);
     if (cudaMemsetAsync(counters, 0, sizeof(int) * tc_gemm_counter_ints() , s) != cudaSuccess) return ESP_E_CUDA;
     if (cudaMemsetAsync(err, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
     TcGemm* plan = nullptr;
-    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, RT, 1, sc, tc_gemm_partial_bytes(148), counters, n_sm, err, nullptr, 0, nullptr, s)) return ESP_E_CUDA;
+    if (tc_gemm_create(&plan, EPI_STORE_F32, false, wv, rw, k_in, x, 1, rows <= 80 ? 80 : RT, 1, sc, tc_gemm_partial_bytes(148, 1, RT), counters, n_sm, err, nullptr, 0, nullptr, s)) return ESP_E_CUDA;
     int rc = tc_gemm_launch(plan, a, s, false);
     int e = 0;
     if (!rc && cudaMemcpyAsync(&e, err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) rc = ESP_E_CUDA;

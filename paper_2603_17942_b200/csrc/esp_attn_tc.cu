@@ -944,6 +944,8 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
     }
     BulkParams p = t->p;
     p.a = a;
+    const int rows_cap = a.rows_cap > 0 && a.rows_cap < RT ? a.rows_cap : RT;
+    p.n_row_tiles = (rows_cap + p.rows_per_tile - 1) / p.rows_per_tile;   // row tiles that can hold rows
     if (n_split_launch > 0) {
         static int n_sm = 0;
         if (n_sm == 0) {
@@ -978,7 +980,7 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
             }
         }
     }
-    if (launch_k(k_attn_tail_merge_tc, dim3((RT + 3) / 4, a.Hq, batch), dim3(128), 0, s, pdl, a) != cudaSuccess) return -1;
+    if (launch_k(k_attn_tail_merge_tc, dim3((rows_cap + 3) / 4, a.Hq, batch), dim3(128), 0, s, pdl, a) != cudaSuccess) return -1;
     return 0;
 }
 

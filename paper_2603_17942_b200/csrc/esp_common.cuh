@@ -70,6 +70,7 @@ struct Dims {
     int32_t static_w[PROBES_MAX];   // fixed branch widths per depth; static_w[0] == 0: Algorithm 1
     int32_t mask_slots;             // mask vectors per sequence: max(k, 1)
     float lambda;
+    int32_t gemm_rows;              // rows of a block the tensor-core GEMMs carry: 80, or RT for larger blocks
     float inv_temp;                 // 1 / temperature, 0 = greedy matching
     uint32_t seed_lo, seed_hi;      // key of the sampling noise
 };
@@ -81,8 +82,8 @@ enum Epi : int { EPI_STORE_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, 
 // Stream-K partition of a GEMM: the n_tiles*KB (tile, k-block) units are dealt out in equal contiguous
 // ranges to G persistent CTAs; CTA c owns units [c*U/G, (c+1)*U/G).  The piece of tile t a CTA computed is
 // kept in slot min(t - first tile of the CTA, slots - 1) of that CTA:
-// partials[((cta*slots + slot)*rows + row)*TILE_N + feature], rows = RT x the sequences one launch covers (row =
-// sequence-in-launch * RT + block row).
+// partials[((cta*slots + slot)*rows + row)*TILE_N + feature], rows = seq_rows x the sequences one launch covers
+// (row = sequence-in-launch * seq_rows + block row; seq_rows = 80, or RT for blocks of more than 80 rows).
 // `table` (device memory, one entry per tile, written once when the GEMM plan is made) lists, in CTA order,
 // the cta*slots+slot index of every piece of the tile, so consumer kernels need no partition arithmetic.
 struct TileSrc {
@@ -94,6 +95,7 @@ struct StreamK {
     const TileSrc* table;
     int32_t n_tiles, KB, G, slots;
     int32_t rows;           // rows per slot
+    int32_t seq_rows;       // rows per sequence within a slot
 };
 __host__ __device__ __forceinline__ long long sk_begin(long long c, long long U, long long G) { return c * U / G; }
 __host__ __device__ __forceinline__ int sk_cta_of_unit(long long u, long long U, long long G) {

@@ -41,39 +41,45 @@ namespace {
 using namespace tc;
 
 constexpr int BK = 64;                       // k elements per stage (128 bytes of bf16)
-// NQ = sequences one launch covers: their activation blocks ([RT][K] each, consecutive) form one B operand of
-// NQ*RT rows, so the weights are streamed once for all of them (partial-only output only).
+// NRS = rows of a sequence's block that take part (80, or 128 for blocks of more than 80 rows); NQ = sequences
+// one launch covers: the first NRS rows of their activation blocks ([RT][K] each, consecutive) are gathered by
+// one 3-D TMA box into one B operand of NQ*NRS <= 256 rows, so the weights are streamed once for all of them
+// (partial-only output only).
 //
 // Ring depth.  The bytes in flight per SM (depth x 16 KB of weights) over the load round trip bound the stream rate,
 // and the ring is also what is requested before the preceding kernel has finished: deeper is better.  The
 // partial-only kernel keeps no accumulator copy in shared memory and spends that room on the ring.
-__host__ __device__ constexpr int stages_of(int epi, int nq) { return nq == 3 ? 4 : (nq == 2 ? 6 : (epi == EPI_PARTIAL ? 8 : 6)); }
+__host__ __device__ constexpr int stages_of(int epi, int nq, int nrs) {
+    return nrs == 80 ? (nq == 3 ? 4 : (nq == 2 ? 6 : (epi == EPI_PARTIAL ? 8 : 6)))
+                     : (nq == 2 ? 4 : (epi == EPI_PARTIAL ? 7 : 4));
+}
 constexpr int A_BYTES = TILE_N * BK * 2;     // 16384
-__host__ __device__ constexpr int b_bytes_of(int nq) { return nq * RT * BK * 2; }   // 10240 per sequence
-__host__ __device__ constexpr int stage_bytes_of(int nq) { return A_BYTES + b_bytes_of(nq); }
-// two accumulator buffers in tensor memory: 128 columns each for one sequence, 256 each for two or three
-__host__ __device__ constexpr int acc_cols_of(int nq) { return nq == 1 ? 128 : 256; }
+__host__ __device__ constexpr int b_bytes_of(int nq, int nrs) { return nq * nrs * BK * 2; }   // 10240 per 80-row sequence
+__host__ __device__ constexpr int stage_bytes_of(int nq, int nrs) { return A_BYTES + b_bytes_of(nq, nrs); }
+// two accumulator buffers in tensor memory: 128 columns each for up to 128 rows, 256 each beyond
+__host__ __device__ constexpr int acc_cols_of(int nr) { return nr <= 128 ? 128 : 256; }
 constexpr int NUM_THREADS = 192;
 constexpr int MAX_NQ = 3;
+__host__ __device__ constexpr int max_nq_of(int nrs) { return nrs == 80 ? 3 : 2; }
 
 struct TcParams {
     CUtensorMap map_a[3];
-    CUtensorMap map_b;      // activations [rows][K], box = NQ*RT rows (one map per NQ, picked at launch)
-    int32_t b_row0;         // first activation row of this launch
+    CUtensorMap map_b;      // activations [sequence][RT][K], box = NQ sequences x NRS rows x 64 (one map per NQ)
+    int32_t b_seq0;         // first sequence (block of RT activation rows) of this launch
     int32_t rows_w[3];
     int32_t n_tiles, KB, grid, epi;
     int32_t map_swiglu;  // tile = 64 rows of w[0] (gate) + the matching 64 rows of w[1] (up)
     int32_t slots;       // partial slots per CTA
     const unsigned char* a_packed;  // weights repacked per (tile, k-block) unit, or NULL: read w[] through map_a
-    float* partials;   // [grid][slots][RT][TILE_N]
+    float* partials;   // [grid][slots][NQ*NRS][TILE_N]
     int* counters;     // [n_tiles], zero between launches
     int* err;
     EpiArgs a;
 };
 
 // kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = 80 per sequence
-__host__ __device__ constexpr uint32_t idesc_of(int nq) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((nq * RT) >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
+__host__ __device__ constexpr uint32_t idesc_of(int nr) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nr >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
 }
 
 // One (tile, k-range) piece of a CTA's stream-K range.
@@ -126,18 +132,19 @@ __device__ __forceinline__ void tile_source(const TcParams& p, int tile, int hal
     row = feat + half * 64;
 }
 
-template <int EPI, int NQ>
+template <int EPI, int NQ, int NRS>
 __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constant__ TcParams p) {
     static_assert(NQ == 1 || EPI == EPI_PARTIAL, "several sequences per launch: partial-only output");
-    constexpr int STAGE_BYTES = stage_bytes_of(NQ), ACC_COLS = acc_cols_of(NQ), TMEM_COLS = 2 * ACC_COLS;
-    constexpr uint32_t IDESC = idesc_of(NQ);
+    static_assert(NQ * NRS <= 256 && NRS % 16 == 0 && NRS <= RT, "MMA N");
+    constexpr int STAGE_BYTES = stage_bytes_of(NQ, NRS), ACC_COLS = acc_cols_of(NQ * NRS), TMEM_COLS = 2 * ACC_COLS;
+    constexpr uint32_t IDESC = idesc_of(NQ * NRS);
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int STAGES = stages_of(EPI, NQ);
+    constexpr int STAGES = stages_of(EPI, NQ, NRS);
     unsigned char* stages = smem;
     float* s_acc = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES);
-    float* s_aux = s_acc + (EPI == EPI_PARTIAL ? 0 : RT * ACC_LD);
-    uint64_t* full = reinterpret_cast<uint64_t*>(s_aux + (EPI == EPI_PARTIAL ? 0 : RT * 4));
+    float* s_aux = s_acc + (EPI == EPI_PARTIAL ? 0 : NRS * ACC_LD);
+    uint64_t* full = reinterpret_cast<uint64_t*>(s_aux + (EPI == EPI_PARTIAL ? 0 : NRS * 4));
     uint64_t* empty = full + STAGES;
     uint64_t* tfull = empty + STAGES;
     uint64_t* tempty = tfull + 2;
@@ -194,7 +201,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                                 tma_load_2d_hint(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it], pol_w);
                             }
                         } else {
-                            tma_load_2d_hint(sa + A_BYTES, &p.map_b, kb * BK, p.b_row0, &full[it], pol_x);
+                            tma_load_3d_hint(sa + A_BYTES, &p.map_b, kb * BK, 0, p.b_seq0, &full[it], pol_x);
                         }
                     }
                 }
@@ -219,7 +226,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                             tma_load_2d_hint(sa, &p.map_a[m0], kb * BK, r0, &full[stage], pol_w);
                             tma_load_2d_hint(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage], pol_w);
                         }
-                        tma_load_2d_hint(sa + A_BYTES, &p.map_b, kb * BK, p.b_row0, &full[stage], pol_x);
+                        tma_load_3d_hint(sa + A_BYTES, &p.map_b, kb * BK, 0, p.b_seq0, &full[stage], pol_x);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -263,7 +270,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
         const int n_rows = p.a.st ? (p.a.st->active ? p.a.st->n_rows : 0) : p.a.rows_fixed;
         StreamK sk;
         sk.partials = p.partials; sk.table = nullptr; sk.n_tiles = p.n_tiles; sk.KB = p.KB; sk.G = p.grid; sk.slots = p.slots;
-        sk.rows = NQ * RT;
+        sk.rows = NQ * NRS; sk.seq_rows = NRS;
         bool ok = true;
         for (int i = 0; i < rng.n_seg && ok; ++i) {
             const Seg sg = get_seg(rng, i);
@@ -275,28 +282,28 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
             if (s_flag[0]) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(q * 32) << 16);
-            uint32_t v[RT];
+            uint32_t v[NRS];
             if constexpr (NQ > 1) {
                 // sequence by sequence: 80 accumulator columns -> that sequence's rows of the partial
-                float* part = p.partials + ((size_t)(blockIdx.x * p.slots + sg.slot) * (NQ * RT)) * TILE_N + f;
+                float* part = p.partials + ((size_t)(blockIdx.x * p.slots + sg.slot) * (NQ * NRS)) * TILE_N + f;
 #pragma unroll 1
                 for (int sq = 0; sq < NQ; ++sq) {
 #pragma unroll
-                    for (int c = 0; c < RT / 16; ++c)
-                        tmem_ld16_issue(taddr + sq * RT + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
+                    for (int c = 0; c < NRS / 16; ++c)
+                        tmem_ld16_issue(taddr + sq * NRS + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     const SeqState* sst = p.a.st + sq;
                     const int nr = sst->active ? sst->n_rows : 0;
 #pragma unroll
-                    for (int r = 0; r < RT; ++r)
-                        if (r < nr) __stcg(part + (size_t)(sq * RT + r) * TILE_N, __uint_as_float(v[r]));
+                    for (int r = 0; r < NRS; ++r)
+                        if (r < nr) __stcg(part + (size_t)(sq * NRS + r) * TILE_N, __uint_as_float(v[r]));
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 mbar_arrive(&tempty[buf]);
                 continue;
             }
 #pragma unroll
-            for (int c = 0; c < RT / 16; ++c) tmem_ld16_issue(taddr + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
+            for (int c = 0; c < NRS / 16; ++c) tmem_ld16_issue(taddr + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             // the accumulator is in registers: hand the tensor-memory buffer back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -304,11 +311,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
             const bool direct = EPI != EPI_PARTIAL && sg.whole;
             if (direct) {
 #pragma unroll
-                for (int r = 0; r < RT; ++r) s_acc[r * ACC_LD + f] = __uint_as_float(v[r]);
+                for (int r = 0; r < NRS; ++r) s_acc[r * ACC_LD + f] = __uint_as_float(v[r]);
             } else {
-                float* part = p.partials + ((size_t)(blockIdx.x * p.slots + sg.slot) * RT) * TILE_N + f;
+                float* part = p.partials + ((size_t)(blockIdx.x * p.slots + sg.slot) * NRS) * TILE_N + f;
 #pragma unroll
-                for (int r = 0; r < RT; ++r)
+                for (int r = 0; r < NRS; ++r)
                     if (r < n_rows) __stcg(part + r * TILE_N, __uint_as_float(v[r]));
             }
             if (EPI == EPI_PARTIAL) continue;   // the consumer kernel sums the partials
@@ -329,7 +336,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                     __threadfence();
                     // thread et: features 4*(et%32)..+3, rows et/32 + 4*i; every load of a batch is issued before the sums
                     const int f4 = (et & 31) * 4, rg = et >> 5;
-                    for (int i0 = 0; i0 < RT / 4; i0 += 4) {
+                    for (int i0 = 0; i0 < NRS / 4; i0 += 4) {
                         if (rg + 4 * i0 >= n_rows) break;
                         float4 acc[4];
 #pragma unroll
@@ -359,7 +366,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
 #pragma unroll
                         for (int ii = 0; ii < 4; ++ii) {
                             const int r = rg + 4 * (i0 + ii);
-                            if (r < RT) {
+                            if (r < NRS) {
                                 float* d = s_acc + r * ACC_LD + f4;
                                 d[0] = acc[ii].x; d[1] = acc[ii].y; d[2] = acc[ii].z; d[3] = acc[ii].w;
                             }
@@ -417,8 +424,9 @@ __global__ void __launch_bounds__(128) k_pack_weights(PackArgs g, unsigned char*
     }
 }
 
-constexpr size_t smem_bytes_of(int epi, int nq) {
-    return 1024 + (size_t)stages_of(epi, nq) * stage_bytes_of(nq) + (epi == EPI_PARTIAL ? 0 : sizeof(float) * (RT * ACC_LD + RT * 4)) + 256;
+constexpr size_t smem_bytes_of(int epi, int nq, int nrs) {
+    return 1024 + (size_t)stages_of(epi, nq, nrs) * stage_bytes_of(nq, nrs) +
+           (epi == EPI_PARTIAL ? 0 : sizeof(float) * (nrs * ACC_LD + nrs * 4)) + 256;
 }
 
 // [rows][K] bf16 row-major, box = 64 k-elements x box_rows rows, 128-byte swizzle, out-of-range reads give zero
@@ -435,18 +443,33 @@ int make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
     return r == CUDA_SUCCESS ? 0 : -1;
 }
 
+// activations [n_seq][RT][K] bf16: box = 64 k-elements x box_rows rows x box_seqs sequences, 128-byte swizzle
+int make_map_b(CUtensorMap* m, const void* base, int n_seq, int K, int box_rows, int box_seqs) {
+    EncodeFn enc = get_encode();
+    if (!enc) return -1;
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)RT, (cuuint64_t)n_seq};
+    cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)RT * K * 2};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)box_rows, (cuuint32_t)box_seqs};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : -1;
+}
+
 }  // namespace
 
 struct TcGemm {
     TcParams p;
     const TileSrc* table = nullptr;
-    CUtensorMap map_b_nq[MAX_NQ];   // activation maps with a box of (i+1)*RT rows
+    CUtensorMap map_b_nq[MAX_NQ];   // activation maps with a box of nrs rows x (i+1) sequences
     int nq_max = 1;
+    int nrs = 80;                   // rows of a sequence's block that take part: 80 or RT
 };
 
 constexpr int MAX_SLOTS = 4;
-size_t tc_gemm_partial_bytes(int n_sm, int nq) { return (size_t)n_sm * MAX_SLOTS * nq * RT * TILE_N * sizeof(float); }
-int tc_gemm_max_nq() { return MAX_NQ; }
+size_t tc_gemm_partial_bytes(int n_sm, int nq, int nrs) { return (size_t)n_sm * MAX_SLOTS * nq * nrs * TILE_N * sizeof(float); }
+int tc_gemm_max_nq(int nrs) { return max_nq_of(nrs); }
 int tc_gemm_counter_ints() { return 4096; }
 size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K) {
     const long long total = (long long)rows_w[0] + rows_w[1] + rows_w[2];
@@ -456,9 +479,9 @@ size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K) {
 int tc_gemm_tiles(const TcGemm* g) { return g ? g->p.n_tiles : 0; }
 
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
-                   int x_rows, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
+                   int x_seqs, int nrs, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
                    int table_entries, void* packed, cudaStream_t stream) {
-    if (!out || nq_max < 1 || nq_max > MAX_NQ || x_rows < nq_max * RT || K % 8 || n_sm < 1) return -1;
+    if (!out || (nrs != 80 && nrs != RT) || nq_max < 1 || nq_max > max_nq_of(nrs) || x_seqs < nq_max || K % 8 || n_sm < 1) return -1;
     if (nq_max > 1 && !defer) return -1;
     if (reinterpret_cast<uintptr_t>(x) % 16) return -1;
     TcGemm* g = new (std::nothrow) TcGemm();
@@ -476,8 +499,9 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
         }
     }
     for (int i = 0; i < nq_max; ++i)
-        if (make_map(&g->map_b_nq[i], x, x_rows, K, (i + 1) * RT)) { delete g; return -1; }
+        if (make_map_b(&g->map_b_nq[i], x, x_seqs, K, nrs, i + 1)) { delete g; return -1; }
     g->nq_max = nq_max;
+    g->nrs = nrs;
     p.map_b = g->map_b_nq[0];
     p.map_swiglu = epi == EPI_SWIGLU;
     p.epi = defer ? (int)EPI_PARTIAL : epi;
@@ -485,7 +509,7 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
     p.KB = (K + BK - 1) / BK;
     const long long U = (long long)p.n_tiles * p.KB;
     p.grid = (int)(U < n_sm ? U : n_sm);
-    if (p.n_tiles > tc_gemm_counter_ints() || tc_gemm_partial_bytes(p.grid, nq_max) > partial_bytes) { delete g; return -1; }
+    if (p.n_tiles > tc_gemm_counter_ints() || tc_gemm_partial_bytes(p.grid, nq_max, nrs) > partial_bytes) { delete g; return -1; }
     // fused epilogues store only the head and tail pieces of a range (2 slots); partial-only output stores every
     // piece, one slot per tile the range touches
     p.slots = 2;
@@ -501,7 +525,7 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
         // contributor table for the consumer kernels
         if (!table_dev || p.n_tiles > table_entries) { delete g; return -1; }
         StreamK k;
-        k.partials = nullptr; k.table = nullptr; k.n_tiles = p.n_tiles; k.KB = p.KB; k.G = p.grid; k.slots = p.slots; k.rows = RT;
+        k.partials = nullptr; k.table = nullptr; k.n_tiles = p.n_tiles; k.KB = p.KB; k.G = p.grid; k.slots = p.slots; k.rows = nrs; k.seq_rows = nrs;
         TileSrc* tab = new (std::nothrow) TileSrc[p.n_tiles];
         if (!tab) { delete g; return -1; }
         bool fits = true;
@@ -555,7 +579,8 @@ int tc_wait_selftest(int* err_dev, cudaStream_t s) {
 
 StreamK tc_gemm_streamk(const TcGemm* g, int nq) {
     StreamK k;
-    k.rows = nq * RT;
+    k.seq_rows = g ? g->nrs : 80;
+    k.rows = nq * k.seq_rows;
     k.partials = g ? g->p.partials : nullptr;
     k.table = g ? g->table : nullptr;
     k.n_tiles = g ? g->p.n_tiles : 0;
@@ -565,29 +590,34 @@ StreamK tc_gemm_streamk(const TcGemm* g, int nq) {
     return k;
 }
 
-// nq sequences (their activation rows start at row b_row0 of the plan's activation buffer, RT apart)
-int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl, int nq, int b_row0) {
-    if (!g || nq < 1 || nq > g->nq_max || b_row0 < 0) return ESP_E_ARG;
+// nq sequences starting at sequence b_seq0 of the plan's activation buffer
+int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl, int nq, int b_seq0) {
+    if (!g || nq < 1 || nq > g->nq_max || b_seq0 < 0) return ESP_E_ARG;
     if (nq > 1 && g->p.epi != EPI_PARTIAL) return ESP_E_ARG;
     TcParams p = g->p;
     p.a = a;
     p.map_b = g->map_b_nq[nq - 1];
-    p.b_row0 = b_row0;
+    p.b_seq0 = b_seq0;
     cudaError_t e = cudaSuccess;
-#define ESP_TC_CASE(E, Q)                                                                                     \
+#define ESP_TC_CASE(E, Q, N)                                                                                  \
     {                                                                                                         \
         static bool attr_set = false;                                                                         \
         if (!attr_set) {                                                                                      \
-            if (cudaFuncSetAttribute(k_gemm_tc<E, Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(E, Q)) != cudaSuccess) return ESP_E_CUDA; \
+            if (cudaFuncSetAttribute(k_gemm_tc<E, Q, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(E, Q, N)) != cudaSuccess) return ESP_E_CUDA; \
             attr_set = true;                                                                                  \
         }                                                                                                     \
-        e = launch_k(k_gemm_tc<E, Q>, dim3(p.grid), dim3(NUM_THREADS), smem_bytes_of(E, Q), s, pdl, p);       \
+        e = launch_k(k_gemm_tc<E, Q, N>, dim3(p.grid), dim3(NUM_THREADS), smem_bytes_of(E, Q, N), s, pdl, p); \
     }
-    if (p.epi == EPI_STORE_F32) ESP_TC_CASE(EPI_STORE_F32, 1)
-    else if (p.epi == EPI_LOGITS) ESP_TC_CASE(EPI_LOGITS, 1)
-    else if (p.epi == EPI_PARTIAL && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1)
-    else if (p.epi == EPI_PARTIAL && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2)
-    else if (p.epi == EPI_PARTIAL && nq == 3) ESP_TC_CASE(EPI_PARTIAL, 3)
+    const bool wide = g->nrs != 80;
+    if (p.epi == EPI_STORE_F32 && !wide) ESP_TC_CASE(EPI_STORE_F32, 1, 80)
+    else if (p.epi == EPI_STORE_F32) ESP_TC_CASE(EPI_STORE_F32, 1, RT)
+    else if (p.epi == EPI_LOGITS && !wide) ESP_TC_CASE(EPI_LOGITS, 1, 80)
+    else if (p.epi == EPI_LOGITS) ESP_TC_CASE(EPI_LOGITS, 1, RT)
+    else if (p.epi == EPI_PARTIAL && !wide && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1, 80)
+    else if (p.epi == EPI_PARTIAL && !wide && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2, 80)
+    else if (p.epi == EPI_PARTIAL && !wide && nq == 3) ESP_TC_CASE(EPI_PARTIAL, 3, 80)
+    else if (p.epi == EPI_PARTIAL && wide && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1, RT)
+    else if (p.epi == EPI_PARTIAL && wide && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2, RT)
     else return ESP_E_ARG;
 #undef ESP_TC_CASE
     return e == cudaSuccess ? ESP_OK : ESP_E_CUDA;

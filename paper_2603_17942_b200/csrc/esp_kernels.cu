@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, flo
     for (int j = threadIdx.x * 4; j < d; j += STRIDE, ++it) {
         float4 x = *reinterpret_cast<const float4*>(xr + j);
         if (sk.partials) {
-            const float4 acc = sk_sum4(sk, j / TILE_N, seq * RT + r, j % TILE_N);
+            const float4 acc = sk_sum4(sk, j / TILE_N, seq * sk.seq_rows + r, j % TILE_N);
             x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
             *reinterpret_cast<float4*>(xr + j) = x;
         }
@@ -162,16 +162,17 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
     const SeqState* st = a.st ? a.st + seq : nullptr;
     const int n_rows = st ? (st->active ? st->n_rows : 0) : a.rows_fixed;
     if (r >= n_rows || hs >= a.Hq + 2 * a.Hkv) return;
-    const int pr = seq * RT + r;                 // row in the partials and in the query buffer
+    const int pr = seq * RT + r;                 // row in the query buffer
+    const int sr = seq * sk.seq_rows + r;        // row in the partials
     const int j0 = hs * HD + lane * NE;          // feature in the concatenated [q | k | v] space
     const int tile = j0 / TILE_N, f = j0 % TILE_N;
     float v[NE];
     if constexpr (NE == 4) {
-        const float4 t = sk_sum4(sk, tile, pr, f);
+        const float4 t = sk_sum4(sk, tile, sr, f);
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
     } else {
         // narrower heads: the same sum through the four-float helper on the enclosing aligned group
-        const float4 t = sk_sum4(sk, tile, pr, f & ~3);
+        const float4 t = sk_sum4(sk, tile, sr, f & ~3);
         const float tv[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
         for (int i = 0; i < NE; ++i) v[i] = tv[(f & 3) + i];
@@ -221,8 +222,8 @@ __global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, i
     const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;
     const int j = (blockIdx.x * 256 + threadIdx.x) * 4;
     if (r >= n_rows || j >= F) return;
-    const int tile = j / 64, f = j % 64, pr = seq * RT + r;
-    const float4 g = sk_sum4(sk, tile, pr, f), u = sk_sum4(sk, tile, pr, 64 + f);
+    const int tile = j / 64, f = j % 64, pr = seq * RT + r, sr = seq * sk.seq_rows + r;
+    const float4 g = sk_sum4(sk, tile, sr, f), u = sk_sum4(sk, tile, sr, 64 + f);
     const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
     __nv_bfloat16 o[4];
 #pragma unroll
@@ -618,8 +619,8 @@ __global__ void __launch_bounds__(TOPK_THREADS) k_topk_merge(const SeqState* sta
 }
 
 void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
-                       Cand* topk, float* lse, cudaStream_t s, bool pdl) {
-    dim3 grid(RT, batch);
+                       Cand* topk, float* lse, cudaStream_t s, bool pdl, int rows_cap) {
+    dim3 grid(rows_cap, batch);
     size_t smem = (size_t)n_tiles * KP * sizeof(Cand);
     int stage = smem <= 160 * 1024 ? 1 : 0;
     if (!stage) smem = 0;
@@ -1003,8 +1004,8 @@ void launch_mask_init(int dtype, const void* embed, const int32_t* prompt, int t
     else k_mask_init<__nv_bfloat16><<<(d + 127) / 128, 128, 0, s>>>((const __nv_bfloat16*)embed, prompt, t, d, m, slots, mode);
 }
 void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int mask_slots,
-                     int batch, cudaStream_t s, bool pdl) {
-    dim3 grid(RT, batch);
+                     int batch, cudaStream_t s, bool pdl, int rows_cap) {
+    dim3 grid(rows_cap, batch);
     if (dtype == 0) launch_k(k_assemble<float>, grid, dim3(128), 0, s, pdl, st, (const float*)embed, mvec, hres, d, mask_slots);
     else launch_k(k_assemble<__nv_bfloat16>, grid, dim3(128), 0, s, pdl, st, (const __nv_bfloat16*)embed, mvec, hres, d, mask_slots);
 }
@@ -1015,16 +1016,16 @@ void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g
     else launch_k(k_rmsnorm<__nv_bfloat16>, grid, dim3(256), 0, s, pdl, st, x, (const __nv_bfloat16*)g, (__nv_bfloat16*)y, d, eps, copy_out);
 }
 void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
-                       float* copy_out, int nq, cudaStream_t s, bool pdl) {
-    launch_k(k_resid_norm<__nv_bfloat16>, dim3(RT, nq), dim3(1024), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
+                       float* copy_out, int nq, cudaStream_t s, bool pdl, int rows_cap) {
+    launch_k(k_resid_norm<__nv_bfloat16>, dim3(rows_cap, nq), dim3(1024), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
              (__nv_bfloat16*)y, d, eps, copy_out);
 }
-void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl) {
-    launch_k(k_swiglu_finish, dim3((F / 4 + 255) / 256, RT, nq), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act, F);
+void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl, int rows_cap) {
+    launch_k(k_swiglu_finish, dim3((F / 4 + 255) / 256, rows_cap, nq), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act, F);
 }
-int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl) {
+int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl, int rows_cap) {
     const int n_heads = a.Hq + 2 * a.Hkv;
-    dim3 grid((n_heads + 3) / 4, RT, nq);
+    dim3 grid((n_heads + 3) / 4, rows_cap, nq);
     if (a.h == 128) launch_k(k_qkv_finish<128>, grid, dim3(128), 0, s, pdl, a, sk);
     else if (a.h == 64) launch_k(k_qkv_finish<64>, grid, dim3(128), 0, s, pdl, a, sk);
     else if (a.h == 32) launch_k(k_qkv_finish<32>, grid, dim3(128), 0, s, pdl, a, sk);

@@ -15,6 +15,7 @@ struct AttnArgs {
     const SeqState* st;   // NULL -> use the explicit fields below
     const unsigned long long* anc;  // [batch][RT][2]
     const int32_t* depth;           // [batch][RT]
+    int32_t rows_cap;               // no block of this launch has more rows than this (0: RT); sizes the grids
     int32_t n_rows_fixed, L_fixed;
     int32_t Hq, Hkv, h, cap, split_len, n_split_max, dcap;
     float scale_log2;     // log2(e)/sqrt(h)
@@ -39,19 +40,19 @@ void launch_rope_table(float* cs, float* sn, int n_pos, int h, float base, cudaS
 void launch_gumbel_noise(uint32_t key0, uint32_t key1, uint32_t position, int n, float* out, cudaStream_t s);
 void launch_mask_init(int dtype, const void* embed, const int32_t* prompt, int t, int d, float* m, int slots, int mode, cudaStream_t s);
 void launch_assemble(int dtype, const SeqState* st, const void* embed, const float* mvec, float* hres, int d, int mask_slots,
-                     int batch, cudaStream_t s, bool pdl);
+                     int batch, cudaStream_t s, bool pdl, int rows_cap = RT);
 void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
                     float* copy_out, cudaStream_t s, bool pdl);
 // consumers of the split (EPI_PARTIAL) tensor-core GEMMs, bf16 models; nq = sequences the GEMM launch covered
 void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
-                       float* copy_out, int nq, cudaStream_t s, bool pdl);
-int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl);
-void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl);
+                       float* copy_out, int nq, cudaStream_t s, bool pdl, int rows_cap = RT);
+int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl, int rows_cap = RT);
+void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl, int rows_cap = RT);
 void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int off, int n, int last, int k, cudaStream_t s);
 void launch_set_tree(SeqState* st, int seq, const int32_t* tokens, const int32_t* parents, int n, int k, int n_anchor,
                      int* err, cudaStream_t s);
 void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
-                       Cand* topk, float* lse, cudaStream_t s, bool pdl);
+                       Cand* topk, float* lse, cudaStream_t s, bool pdl, int rows_cap = RT);
 void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s, bool pdl);
 
 // CUDA-core GEMM (fp32 models; on-GPU cross-check for bf16)
@@ -72,21 +73,21 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
 // tcgen05 GEMM: a plan holds the TMA descriptors and the stream-K partition of one weight shape
 struct TcGemm;
 // epi selects the tile -> weight-row mapping and the fused epilogue; with defer the kernel only stores partials
-// (EPI_PARTIAL) and the caller runs the matching consumer kernel.  x: activations [x_rows][K]; a deferred plan may
-// cover up to nq_max sequences per launch (their RT-row blocks are consecutive in x), so that the weights are
-// streamed once for all of them
+// (EPI_PARTIAL) and the caller runs the matching consumer kernel.  x: activations [x_seqs][RT][K]; nrs = rows of a
+// block that take part (80, or RT for blocks of more than 80 rows); a deferred plan may cover up to nq_max
+// sequences per launch, so that the weights are streamed once for all of them
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
-                   int x_rows, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
+                   int x_seqs, int nrs, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
                    int table_entries, void* packed, cudaStream_t stream);
 // bytes of the repacked copy of a weight set (tc_gemm_create's `packed`; NULL there = stream the caller's matrices)
 size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K);
 void tc_gemm_destroy(TcGemm* g);
-int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl, int nq = 1, int b_row0 = 0);
+int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl, int nq = 1, int b_seq0 = 0);
 StreamK tc_gemm_streamk(const TcGemm* g, int nq = 1);
 int tc_wait_selftest(int* err_dev, cudaStream_t s);
 int tc_gemm_tiles(const TcGemm* g);
-size_t tc_gemm_partial_bytes(int n_sm, int nq = 1);
-int tc_gemm_max_nq();
+size_t tc_gemm_partial_bytes(int n_sm, int nq = 1, int nrs = 80);
+int tc_gemm_max_nq(int nrs = 80);
 int tc_gemm_counter_ints();
 
 }  // namespace esp

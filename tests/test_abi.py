@@ -45,8 +45,8 @@ def test_workspace_bytes_and_config_checks(lib):
     # static trees: [7,2] and [15,4] with a mask pair per node are 30 and 60 rows
     for widths in ((7, 2), (15, 4), (14,)):
         P.esp_workspace_bytes(m, P.spec_cfg(n_probes=len(widths), n_anchor=0, static_widths=widths))
-    bad = [P.spec_cfg(n_probes=4, topk=10, max_nodes=64, n_anchor=0),      # (k+1)*64 rows > 80
-           P.spec_cfg(n_probes=3, n_anchor=0, static_widths=(7, 5, 9)),    # (k+1)*(1+21) rows > 80
+    bad = [P.spec_cfg(n_probes=4, topk=10, max_nodes=64, n_anchor=0),      # (k+1)*64 rows > 128
+           P.spec_cfg(n_probes=3, n_anchor=0, static_widths=(7, 5, 20)),   # (k+1)*(1+32) rows > 128
            P.spec_cfg(n_probes=2, n_anchor=1, static_widths=(40, 2)),      # K' beyond the kept list length
            P.spec_cfg(n_probes=9, topk=4, max_nodes=8),                    # too many probes
            P.spec_cfg(n_probes=2, topk=40, max_nodes=8),                   # K' beyond the kept list length

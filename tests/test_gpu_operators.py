@@ -165,6 +165,32 @@ def test_tree_attention_rows_equal_decoding_each_path_alone():
         assert torch.equal(alone[0, 0], tree_out[0, r]), f"row {r} (depth {d})"
 
 
+def test_tree_attention_one_item_and_persistent_kernels_agree_bitwise():
+    """The cache below T0 is summed by one of two tensor-core kernels, picked by the number of (split, KV head,
+    row tile, sequence) items in the launch.  One sequence at KV 2048 stays below the switch (8 x 24 = 192 items),
+    three copies of it in one call are above it (576 items): every copy must come out bit for bit like the single
+    one, and a different sequence in the same call must not disturb them."""
+    Hq, Hkv, h, n_nodes, n_probes, L = 32, 8, 128, 64, 4, 2048
+    M = n_nodes + n_probes
+    cap = L + R
+    q, kc, vc, kb, vb = synth.random_qkv((1, R, Hq, h), (1, Hkv, cap, h), (1, Hkv, M, h), seed=77, device="cuda")
+    kc[:, :, L:L + M] = kb
+    vc[:, :, L:L + M] = vb
+    _, d, vis = _tree_block(n_nodes, n_probes, 5, seed=5)
+    anc = _anc_words(vis)[None]
+    depth = np.zeros((1, R), np.int32)
+    depth[0, :M] = d
+    single = _run_attention(1, q, kc, vc, anc, depth, M, L, Hq, Hkv, h)
+    q2, kc2, vc2, _, _ = synth.random_qkv((1, R, Hq, h), (1, Hkv, cap, h), (1, Hkv, M, h), seed=78, device="cuda")
+    qq = torch.cat([q, q2, q, q]).contiguous()
+    kk = torch.cat([kc, kc2, kc, kc]).contiguous()
+    vv = torch.cat([vc, vc2, vc, vc]).contiguous()
+    many = _run_attention(1, qq, kk, vv, np.repeat(anc, 4, 0), np.repeat(depth, 4, 0), M, L, Hq, Hkv, h)
+    for s in (0, 2, 3):
+        assert torch.equal(many[s, :M], single[0, :M]), f"copy {s}"
+    assert not torch.equal(many[1, :M], single[0, :M])
+
+
 def test_tree_attention_long_context_against_oracle():
     """KV length 32768 (the longest context of the batch sweep): the cache is cut in 32 splits of 1024; every
     row and head against the oracle."""

@@ -247,6 +247,71 @@ def test_full_width_shapes_parity(pu, base, topk, B):
     run.close()
 
 
+# ------------------------------------------------------------------ blocks of more than 80 rows (BC = 120)
+@pytest.mark.parametrize("widths", [(), (15, 10, 4)])
+def test_tiny_fp32_block_complexity_120_parity(pu, widths):
+    """The paper's largest block: k = 3 masks behind every one of 30 tree nodes, BC = (k+1) * 30 = 120 rows
+    (Section 3.3; Appendix on increasing block complexity), dynamic and static tree."""
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=2, gain_jitter=True, std=0.3)
+    prompt = synth.make_prompt(shape.vocab, 70, 4)
+    spec = O.SpecCfg(n_probes=3, topk=10, max_nodes=30, expand_width=1, n_anchor=0, prune_parent=False, static_widths=widths)
+    run = pu.ParityRun(shape, w, spec, prompt, 40, TOL_FP32)
+    out = run.run()
+    assert out == O.greedy_generate(O.OracleModel(shape, w), prompt, 40, 256)
+    assert run.h.state()["n_rows"] == 120
+    g, _ = pu.gpu_generate(shape, run.wd, pu.GREEDY, prompt, 40)
+    assert g == out
+    run.close()
+
+
+def test_bf16_block_complexity_120_parity_and_batch(pu):
+    """The same block on the tensor-core path (MMA N = 128 per sequence, two sequences per weight stream): parity
+    per step, bitwise equal to greedy decoding, and two sequences in one handle equal to each alone."""
+    import paper_2603_17942_b200 as P
+    shape = BF16_SMALL
+    w = synth.make_weights(shape, seed=6, gain_jitter=True, std=0.05)
+    spec = O.SpecCfg(n_probes=3, topk=10, max_nodes=30, expand_width=1, n_anchor=0)
+    prompts = [synth.make_prompt(shape.vocab, n, 20 + i) for i, n in enumerate((210, 75, 140))]
+    run = pu.ParityRun(shape, w, spec, prompts[0], 24, TOL_BF16)
+    out = run.run()
+    assert run.h.state()["n_rows"] == 120
+    g, _ = pu.gpu_generate(shape, run.wd, pu.GREEDY, prompts[0], 24)
+    assert g == out
+    n_new, max_seq = 20, 400
+    alone = []
+    for pr in prompts:
+        h1 = P.Handle(shape, pu.c_spec(spec), run.wd, max_seq_len=max_seq)
+        alone.append(h1.generate(pr, n_new))
+        h1.close()
+    h = P.Handle(shape, pu.c_spec(spec), run.wd, max_seq_len=max_seq, max_batch=3)     # passes of 2 and 1
+    outs = [[h.prefill(prompts[i], i)] for i in range(3)]
+    while not all(len(o) >= n_new for o in outs):
+        P.esp_step(h.h, h.tokens_out, h.n_out)
+        for i in range(3):
+            outs[i].extend(int(t) for t in h.tokens_out[i, :h.n_out[i]])
+    assert h.stats().device_error == 0
+    for i in range(3):
+        assert outs[i][:n_new] == alone[i], f"sequence {i}"
+    h.close()
+    run.close()
+
+
+def test_full_width_block_complexity_120_parity(pu):
+    """Llama-3-8B-shape GEMMs, attention and LM head with 120-row blocks (two layers)."""
+    shape = synth.LLAMA3_8B.replace(n_layers=2)
+    w = synth.make_weights(shape, seed=0, device="cuda")
+    wh = synth.weights_to_host(w)
+    prompt = synth.make_prompt(shape.vocab, 200, 0)
+    spec = O.SpecCfg(n_probes=3, topk=10, max_nodes=30, expand_width=1, n_anchor=0)
+    run = pu.ParityRun(shape, wh, spec, prompt, 3, TOL_BF16, w_dev=w)
+    out = run.run()
+    g, _ = pu.gpu_generate(shape, w, pu.GREEDY, prompt, 3)
+    assert g == out
+    assert run.h.state()["n_rows"] == 120 and run.h.stats().device_error == 0
+    run.close()
+
+
 # ------------------------------------------------------------------ sample matching (temperature > 0)
 def test_sampling_noise_bitwise_equals_oracle():
     """The Gumbel noise of the CUDA path and of the oracle are the same fp32 numbers, bit for bit."""

@@ -86,7 +86,7 @@ def test_static_scratch_attention_matches_caller_scratch_twice_in_a_row():
 
 def test_static_scratch_attention_rejects_shapes_beyond_its_array():
     x = _inputs(L=64, seed=23)
-    big_cap = 1 << 16                                                     # partials for 64k positions do not fit in 16 MiB
+    big_cap = 1 << 16                                                     # partials for 64k positions do not fit in the array
     assert P.esp_tree_attention_scratch_bytes(1, 32, 128, big_cap) > P.ESP_STATIC_SCRATCH_BYTES
     out = torch.zeros_like(x["q"])
     with pytest.raises(P.EspError) as e:
