@@ -36,6 +36,10 @@ if ROOT not in sys.path:
 METRIC = "esp_accepted_tokens_per_s"
 UNIT = "tok/s"
 
+# DRAM bytes (read + written) of one gate/up GEMM launch from the ncu capture summarised under profiles/
+# (Llama-3-8B shape, 68 rows, one sequence); None for workloads without a capture of the current kernel.
+GATEUP_DRAM_TRAFFIC = {"llama3-8b": 242.8e6}
+
 WORKLOADS = {
     # name: (shape attr in synth, prompt length, probes, topk, max_nodes)
     "llama3-8b": ("LLAMA3_8B", 1024, 4, 10, 64),
@@ -435,7 +439,8 @@ def run_ours(args, shape, plen, k, K, B):
             "gpu_launches": launches,
             "roofline": {"bound": "hbm", "kernel": "k_gemm_tc<EPI_PARTIAL>, gate/up projection (235 MB of weights per launch)",
                          "achieved": gu_ach, "peak": peak, "unit": "GB/s", "frac": gu_ach / peak if gu_ach else None,
-                         "traffic": None, "peak_source": peak_src, "bytes_per_launch": gu_bytes,
+                         "traffic": GATEUP_DRAM_TRAFFIC.get(args.config) if nbatch == 1 and not args.per_node_probes else None,
+                         "peak_source": peak_src, "bytes_per_launch": gu_bytes,
                          "us_per_launch": gu_ms * 1e3,
                          "measured_in": f"{n_prof} profiled steps after the timed region (an event after every kernel)"},
             "step_roofline": {"bound": "hbm", "bytes_per_step": wbytes + kvbytes, "weight_bytes": wbytes,
