@@ -312,6 +312,43 @@ def test_full_width_block_complexity_120_parity(pu):
     run.close()
 
 
+# ------------------------------------------------------------------ limits of the configuration space
+@pytest.mark.parametrize("spec_kw,plen", [
+    (dict(n_probes=3, topk=12, max_nodes=32, expand_width=1, n_anchor=0, prune_parent=False), 64),   # 128 rows: the largest block
+    (dict(n_probes=8, topk=2, max_nodes=12, expand_width=1, n_anchor=1), 33),                        # the most probes
+    (dict(n_probes=1, topk=31, max_nodes=32, expand_width=0, n_anchor=1), 5),                        # the longest Top-K' list (32 with the pruner's spare)
+    (dict(n_probes=2, topk=3, max_nodes=8, expand_width=0, n_anchor=0), 1),                          # a one-token prompt
+    (dict(n_probes=2, topk=3, max_nodes=8, expand_width=1, n_anchor=2), 2),
+    (dict(n_probes=1, topk=1, max_nodes=2, expand_width=1, n_anchor=1), 129),                        # the smallest tree, a ragged third prefill block
+])
+def test_tiny_fp32_limits_parity(pu, spec_kw, plen):
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=8, gain_jitter=True, std=0.3)
+    prompt = synth.make_prompt(shape.vocab, plen, 9)
+    spec = O.SpecCfg(**spec_kw)
+    run = pu.ParityRun(shape, w, spec, prompt, 24, TOL_FP32)
+    out = run.run()
+    assert out == O.greedy_generate(O.OracleModel(shape, w), prompt, 24, 256)
+    if spec.n_probes == 3:
+        assert run.h.state()["n_rows"] == 128
+    assert run.h.stats().device_error == 0
+    run.close()
+
+
+def test_bf16_largest_block_parity(pu):
+    """128 rows (32 nodes x (3 probes + 1)) on the tensor-core path."""
+    shape = BF16_SMALL
+    w = synth.make_weights(shape, seed=9, gain_jitter=True, std=0.05)
+    prompt = synth.make_prompt(shape.vocab, 100, 3)
+    spec = O.SpecCfg(n_probes=3, topk=12, max_nodes=32, expand_width=1, n_anchor=0, prune_parent=False)
+    run = pu.ParityRun(shape, w, spec, prompt, 16, TOL_BF16)
+    out = run.run()
+    assert run.h.state()["n_rows"] == 128
+    g, _ = pu.gpu_generate(shape, run.wd, pu.GREEDY, prompt, 16)
+    assert g == out
+    run.close()
+
+
 # ------------------------------------------------------------------ sample matching (temperature > 0)
 def test_sampling_noise_bitwise_equals_oracle():
     """The Gumbel noise of the CUDA path and of the oracle are the same fp32 numbers, bit for bit."""
