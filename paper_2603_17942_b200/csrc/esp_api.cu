@@ -33,6 +33,7 @@ struct Buffers {
     float2* part_ml;
     Cand* cand;
     float2* cand_ms;
+    uint32_t* cand_floor;
     Cand* topk;
     float* lse;
     float* mvec;
@@ -152,6 +153,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.part_ml = c.take<float2>(Mtot * D.Hq * D.n_split_max);
     o.cand = c.take<Cand>((size_t)n_tiles_v * Mtot * D.KP);
     o.cand_ms = c.take<float2>((size_t)n_tiles_v * Mtot);
+    o.cand_floor = c.take<uint32_t>(Mtot);
     o.topk = c.take<Cand>(Mtot * KP_MAX);
     o.lse = c.take<float>(Mtot);
     o.mvec = c.take<float>((size_t)D.batch * D.mask_slots * D.d);
@@ -376,14 +378,14 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
         for (int q = 0; q < n_lm; ++q) {
             const int sq = s0 + q;
             EpiArgs a = base_epi(h, D.V, sq, per);
-            a.cand = b.cand; a.cand_ms = b.cand_ms; a.n_tiles = n_tiles;
+            a.cand = b.cand; a.cand_ms = b.cand_ms; a.cand_floor = b.cand_floor; a.n_tiles = n_tiles;
             a.logits_dump = h->dbg_logits ? h->dbg_logits + (size_t)sq * RT * D.V : nullptr;
             const void* w[3] = {h->lm_head, nullptr, nullptr};
             const int32_t rows[3] = {D.V, 0, 0};
             int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl, 1, q);
             if (rc) return rc;
             mark(h, KIND_LMHEAD);
-            launch_topk_merge(b.states + sq, b.cand, b.cand_ms, n_tiles, D.KP, per, b.topk + (size_t)sq * RT * KP_MAX, b.lse + (size_t)sq * RT, s, pdl, rc_rows);
+            launch_topk_merge(b.states + sq, b.cand, b.cand_ms, n_tiles, D.KP, per, b.topk + (size_t)sq * RT * KP_MAX, b.lse + (size_t)sq * RT, s, pdl, rc_rows, b.cand_floor);
             h->launches++;
             mark(h, KIND_SELECT);
         }

@@ -174,6 +174,9 @@ struct EpiArgs {
     int32_t KP;
     int32_t n_tiles;
     float* logits_dump;       // optional [batch*RT][V]
+    // optional [batch*RT]: per probe row, a running lower bound of its K'-th largest logit, as an order-preserving
+    // unsigned key (0 = nothing known yet).  Tiles add to it; entries below it cannot be in the row's Top-K'.
+    uint32_t* cand_floor;
     // sample matching: tree rows pick argmax(logit * samp_inv_temp + Gumbel noise); 0 = greedy matching
     float samp_inv_temp;
     uint32_t samp_key0, samp_key1;

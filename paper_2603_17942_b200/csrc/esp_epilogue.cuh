@@ -15,6 +15,17 @@ namespace esp {
 
 constexpr int ACC_LD = TILE_N + 1;  // padded row stride of s_acc (floats)
 
+// order-preserving map of a float onto an unsigned integer (larger float <=> larger key; every key > 0)
+// (-0 and +0 share a key, as they compare equal)
+__device__ __forceinline__ uint32_t float_order_key(float v) {
+    uint32_t b = __float_as_uint(v);
+    if ((b << 1) == 0u) b = 0u;
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float float_from_order_key(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
 __device__ __forceinline__ void epi_bar(int bar_id) {
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
 }
@@ -136,6 +147,10 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
                 s = warp_sum(s);
                 if (lane == 0) a.cand_ms[(size_t)tile * Mtot + grow0 + r] = make_float2(tmax, s);
             }
+            // what other tiles have already established about this row's K'-th largest logit: a tile's own K'-th
+            // best is a lower bound of it, so an entry strictly below the bound cannot make the final list
+            uint32_t floor_key = 0;
+            if (probe && a.cand_floor) floor_key = __ldcg(a.cand_floor + grow0 + r);
             unsigned used = 0;
             for (int j = 0; j < kp; ++j) {
                 // lane-local best among unused, then warp-wide best by (value desc, id asc)
@@ -144,16 +159,21 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     if (!(used >> i & 1) && id[i] < a.n_out && cand_before(v[i], id[i], bv, bi)) { bv = v[i]; bi = id[i]; bslot = i; }
-                float wv = bv;
-                int wi = bi;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    float ov = __shfl_xor_sync(0xffffffffu, wv, o);
-                    int oi = __shfl_xor_sync(0xffffffffu, wi, o);
-                    if (cand_before(ov, oi, wv, wi)) { wv = ov; wi = oi; }
-                }
+                // two warp-wide integer reductions: the largest value (as an order-preserving key), then the smallest
+                // token id among the lanes that hold it
+                const uint32_t key = bslot >= 0 ? float_order_key(bv) : 0u;
+                const uint32_t wkey = __reduce_max_sync(0xffffffffu, key);
+                const uint32_t wid = __reduce_min_sync(0xffffffffu, (bslot >= 0 && key == wkey) ? (uint32_t)bi : 0xffffffffu);
+                const int wi = wkey == 0u ? 0x7fffffff : (int)wid;
+                const float wv = wkey == 0u ? -INFINITY : float_from_order_key(wkey);
                 if (wi == bi && bslot >= 0) used |= 1u << bslot;
+                if (probe && wi != 0x7fffffff && float_order_key(wv) < floor_key) {   // warp-uniform: this and all later entries are out
+                    if (lane == 0) for (int jj = j; jj < kp; ++jj) { out[jj].val = -INFINITY; out[jj].id = -1; }
+                    break;
+                }
                 if (lane == 0) { out[j].val = wv; out[j].id = wi == 0x7fffffff ? -1 : wi; }
+                if (probe && a.cand_floor && j == kp - 1 && wi != 0x7fffffff && lane == 0)
+                    atomicMax(a.cand_floor + grow0 + r, float_order_key(wv));          // this tile holds kp entries >= wv
             }
         }
     }

@@ -533,7 +533,8 @@ int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch
 constexpr int TOPK_THREADS = 256;
 constexpr int TOPK_MAXT = 8;   // tiles per thread (n_tiles <= 2048)
 __global__ void __launch_bounds__(TOPK_THREADS) k_topk_merge(const SeqState* states, const Cand* cand, const float2* cand_ms,
-                                                             int n_tiles, int KP, int batch, Cand* topk, float* lse, int stage) {
+                                                             int n_tiles, int KP, int batch, Cand* topk, float* lse, int stage,
+                                                             uint32_t* cand_floor) {
     extern __shared__ __align__(16) unsigned char tk_smem[];
     Cand* s_c = reinterpret_cast<Cand*>(tk_smem);
     __shared__ float s_v[TOPK_THREADS];
@@ -615,11 +616,12 @@ __global__ void __launch_bounds__(TOPK_THREADS) k_topk_merge(const SeqState* sta
             __syncthreads();
         }
         if (tid == 0) lse[grow] = s_v[0] + logf(s_s[0]);
+        if (tid == 0 && cand_floor) cand_floor[grow] = 0;     // nothing is known about the next forward's logits
     }
 }
 
 void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
-                       Cand* topk, float* lse, cudaStream_t s, bool pdl, int rows_cap) {
+                       Cand* topk, float* lse, cudaStream_t s, bool pdl, int rows_cap, uint32_t* cand_floor) {
     dim3 grid(rows_cap, batch);
     size_t smem = (size_t)n_tiles * KP * sizeof(Cand);
     int stage = smem <= 160 * 1024 ? 1 : 0;
@@ -629,7 +631,7 @@ void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_
         cudaFuncSetAttribute(k_topk_merge, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         attr_bytes = smem;
     }
-    launch_k(k_topk_merge, grid, dim3(TOPK_THREADS), smem, s, pdl, st, cand, cand_ms, n_tiles, KP, batch, topk, lse, stage);
+    launch_k(k_topk_merge, grid, dim3(TOPK_THREADS), smem, s, pdl, st, cand, cand_ms, n_tiles, KP, batch, topk, lse, stage, cand_floor);
 }
 
 // ------------------------------------------------------------------ sampling noise, stand-alone (for checking)

@@ -52,7 +52,7 @@ void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int of
 void launch_set_tree(SeqState* st, int seq, const int32_t* tokens, const int32_t* parents, int n, int k, int n_anchor,
                      int* err, cudaStream_t s);
 void launch_topk_merge(const SeqState* st, const Cand* cand, const float2* cand_ms, int n_tiles, int KP, int batch,
-                       Cand* topk, float* lse, cudaStream_t s, bool pdl, int rows_cap = RT);
+                       Cand* topk, float* lse, cudaStream_t s, bool pdl, int rows_cap = RT, uint32_t* cand_floor = nullptr);
 void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s, bool pdl);
 
 // CUDA-core GEMM (fp32 models; on-GPU cross-check for bf16)
