@@ -204,8 +204,10 @@ def run_reference(args, shape, plen, k, K, B):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
             "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.config + "-shape bf16 weights, b=1", "prompt_len": plen, "n_probes": k, "topk": K,
-                       "max_nodes": B},
+            "config": {"workload": f"{args.config}-shape bf16 decoder, random-init seeded weights, b=1",
+                       "prompt_len": plen, "batch": 1, "temperature": 0.0, "n_probes": k, "topk": K, "max_nodes": B,
+                       "rows_per_step": B + k, "replicas": 1,
+                       "note": "bf16 weights widened exactly, fp32 arithmetic (the oracle's precision)"},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": smp.describe()},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
