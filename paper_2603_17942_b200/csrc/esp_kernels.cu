@@ -43,8 +43,10 @@ __global__ void k_mask_init(const T* embed, const int32_t* prompt, int t, int d,
 // tree nodes hold the chains back to back, k rows each).
 template <typename T>
 __global__ void k_assemble(const SeqState* states, const T* embed, const float* mvec, float* hres, int d, int mask_slots) {
-    pdl_wait();
+    // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
+    // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
+    pdl_wait();
     int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
     if (!st->active || r >= st->n_rows) return;
@@ -76,8 +78,10 @@ __global__ void k_assemble(const SeqState* states, const T* embed, const float* 
 template <typename T>
 __global__ void __launch_bounds__(256) k_rmsnorm(const SeqState* states, const float* x, const T* g, T* y, int d, float eps,
                                                 float* copy_out) {
-    pdl_wait();
+    // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
+    // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
+    pdl_wait();
     int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
     if (!st->active || r >= st->n_rows) return;
@@ -105,8 +109,10 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const SeqState* states, const f
 template <typename T>
 __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, float* hres, StreamK sk, const T* g, T* y, int d,
                                                     float eps, float* copy_out) {
-    pdl_wait();
+    // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
+    // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
+    pdl_wait();
     const int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
     if (!st->active || r >= st->n_rows) return;
@@ -153,8 +159,10 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, flo
 // a lane owns HD/32 consecutive features; the rotate-half partner (i, i + HD/2) sits 16 lanes away.
 template <int HD>
 __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
-    pdl_wait();
+    // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
+    // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
+    pdl_wait();
     typedef __nv_bfloat16 T;
     constexpr int NE = HD / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -216,19 +224,34 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
 // Consumer of the split gate/up GEMM: a tile holds 64 gate features (columns 0..63) and the matching 64 up
 // features (columns 64..127); sums both over the tile's contributors in CTA order and stores silu(gate) * up.
 __global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, int rows_fixed, StreamK sk, __nv_bfloat16* act, int F) {
-    pdl_wait();
+    // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
+    // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.y, seq = blockIdx.z;
     const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;
-    const int j = (blockIdx.x * 256 + threadIdx.x) * 4;
-    if (r >= n_rows || j >= F) return;
-    const int tile = j / 64, f = j % 64, pr = seq * RT + r, sr = seq * sk.seq_rows + r;
-    const float4 g = sk_sum4(sk, tile, sr, f), u = sk_sum4(sk, tile, sr, 64 + f);
-    const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
-    __nv_bfloat16 o[4];
+    // eight features per thread: half the threads, so that the next GEMM's CTA finds registers free beside this
+    // kernel's CTAs and can start its weight stream while they run
+    const int j0 = (blockIdx.x * 256 + threadIdx.x) * 8;
+    if (r >= n_rows || j0 >= F) return;
+    const int pr = seq * RT + r, sr = seq * sk.seq_rows + r;
+    float4 g[2], u[2];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) o[i] = __float2bfloat16_rn((gv[i] / (1.0f + expf(-gv[i]))) * uv[i]);
-    *reinterpret_cast<uint2*>(act + (size_t)pr * F + j) = *reinterpret_cast<const uint2*>(o);
+    for (int q = 0; q < 2; ++q) {
+        const int j = j0 + 4 * q, tile = j / 64, f = j % 64;
+        if (j >= F) { g[q] = u[q] = make_float4(0.f, 0.f, 0.f, 0.f); continue; }
+        g[q] = sk_sum4(sk, tile, sr, f);
+        u[q] = sk_sum4(sk, tile, sr, 64 + f);
+    }
+    __nv_bfloat16 o[8];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        const float gv[4] = {g[q].x, g[q].y, g[q].z, g[q].w}, uv[4] = {u[q].x, u[q].y, u[q].z, u[q].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[4 * q + i] = __float2bfloat16_rn((gv[i] / (1.0f + expf(-gv[i]))) * uv[i]);
+    }
+    if (j0 + 8 <= F) *reinterpret_cast<uint4*>(act + (size_t)pr * F + j0) = *reinterpret_cast<const uint4*>(o);
+    else *reinterpret_cast<uint2*>(act + (size_t)pr * F + j0) = *reinterpret_cast<const uint2*>(o);
 }
 
 // ------------------------------------------------------------------ CUDA-core GEMM
@@ -448,8 +471,10 @@ __global__ void __launch_bounds__(128) k_attn_bulk_simt(AttnArgs a, int n_split_
 template <typename T, int HD>
 __global__ void __launch_bounds__(128) k_attn_tail_merge(AttnArgs a) {
     __shared__ float s_qall[4][HD];
-    pdl_wait();
+    // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
+    // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * 4 + warp, head = blockIdx.y, seq = blockIdx.z;
     int n_rows, L, depth;
@@ -539,6 +564,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) k_topk_merge(const SeqState* sta
     Cand* s_c = reinterpret_cast<Cand*>(tk_smem);
     __shared__ float s_v[TOPK_THREADS];
     __shared__ int s_i[TOPK_THREADS];
+    if (threadIdx.x == 0) pdl_launch_dependents();
     pdl_wait();
     const int seq = blockIdx.y, r = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const SeqState* st = states + seq;
@@ -1023,7 +1049,7 @@ void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const
              (__nv_bfloat16*)y, d, eps, copy_out);
 }
 void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl, int rows_cap) {
-    launch_k(k_swiglu_finish, dim3((F / 4 + 255) / 256, rows_cap, nq), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act, F);
+    launch_k(k_swiglu_finish, dim3((F / 8 + 255) / 256, rows_cap, nq), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act, F);
 }
 int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl, int rows_cap) {
     const int n_heads = a.Hq + 2 * a.Hkv;
