@@ -580,11 +580,15 @@ __global__ void __launch_bounds__(TOPK_THREADS) k_topk_merge(const SeqState* sta
         __syncthreads();
     }
     auto entry = [&](int t, int q) -> Cand { return stage ? s_c[t * kp + q] : cand[((size_t)t * Mtot + grow) * KP + q]; };
+    // Two levels, both by (value desc, id asc).  Level 1: each warp merges the sorted lists of its tiles (tile t
+    // belongs to thread t mod 256) into its own top kp -- a round is the lane-local best head, then two warp-wide
+    // integer reductions (largest order-preserving key, smallest id among its holders); no block barrier.
+    // Level 2: warp 0 merges the 8 warp lists the same way, one list per lane.
+    __shared__ Cand s_w[TOPK_THREADS / 32][KP_MAX];
     unsigned char cur[TOPK_MAXT];
 #pragma unroll
     for (int i = 0; i < TOPK_MAXT; ++i) cur[i] = 0;
     for (int j = 0; j < kp; ++j) {
-        // this thread's best remaining entry: lists are sorted, so it is the best head among its tiles
         float bv = -INFINITY;
         int bi = 0x7fffffff, bt = -1;
 #pragma unroll
@@ -595,28 +599,40 @@ __global__ void __launch_bounds__(TOPK_THREADS) k_topk_merge(const SeqState* sta
                 if (c.id >= 0 && cand_before(c.val, c.id, bv, bi)) { bv = c.val; bi = c.id; bt = i; }
             }
         }
-        float wv = bv;
-        int wi = bi;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, wv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, wi, o);
-            if (cand_before(ov, oi, wv, wi)) { wv = ov; wi = oi; }
-        }
-        if (lane == 0) { s_v[warp] = wv; s_i[warp] = wi; }
-        __syncthreads();
-        wv = s_v[0];
-        wi = s_i[0];
-#pragma unroll
-        for (int w = 1; w < TOPK_THREADS / 32; ++w)
-            if (cand_before(s_v[w], s_i[w], wv, wi)) { wv = s_v[w]; wi = s_i[w]; }
-        if (bt >= 0 && wi == bi) {     // token ids are unique across tiles: exactly one thread owns the winner
+        const uint32_t key = bt >= 0 ? float_order_key(bv) : 0u;
+        const uint32_t wkey = __reduce_max_sync(0xffffffffu, key);
+        const uint32_t wid = __reduce_min_sync(0xffffffffu, (bt >= 0 && key == wkey) ? (uint32_t)bi : 0xffffffffu);
+        if (bt >= 0 && key == wkey && (uint32_t)bi == wid) {   // token ids are unique across tiles: one owner
 #pragma unroll
             for (int i = 0; i < TOPK_MAXT; ++i) if (i == bt) cur[i]++;
+            s_w[warp][j].val = bv;
+            s_w[warp][j].id = bi;
         }
-        if (tid == 0) { topk[(size_t)grow * KP_MAX + j].val = wv; topk[(size_t)grow * KP_MAX + j].id = wi == 0x7fffffff ? -1 : wi; }
-        __syncthreads();
+        if (wkey == 0u && lane == 0) { s_w[warp][j].val = -INFINITY; s_w[warp][j].id = -1; }
     }
+    __syncthreads();
+    if (warp == 0) {
+        int c2 = 0;     // this lane's cursor into warp list `lane`
+        for (int j = 0; j < kp; ++j) {
+            float bv = -INFINITY;
+            int bi = 0x7fffffff;
+            bool have = false;
+            if (lane < TOPK_THREADS / 32 && c2 < kp) {
+                const Cand c = s_w[lane][c2];
+                if (c.id >= 0) { bv = c.val; bi = c.id; have = true; }
+            }
+            const uint32_t key = have ? float_order_key(bv) : 0u;
+            const uint32_t wkey = __reduce_max_sync(0xffffffffu, key);
+            const uint32_t wid = __reduce_min_sync(0xffffffffu, (have && key == wkey) ? (uint32_t)bi : 0xffffffffu);
+            if (have && key == wkey && (uint32_t)bi == wid) {
+                ++c2;
+                topk[(size_t)grow * KP_MAX + j].val = bv;
+                topk[(size_t)grow * KP_MAX + j].id = bi;
+            }
+            if (wkey == 0u && lane == 0) { topk[(size_t)grow * KP_MAX + j].val = -INFINITY; topk[(size_t)grow * KP_MAX + j].id = -1; }
+        }
+    }
+    __syncthreads();
     if (probe) {
         // thread-strided partial merges in tile order, then a fixed tree over threads
         float m = -INFINITY, sm = 0.f;
