@@ -779,10 +779,12 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     __shared__ int s_na, s_ustar, s_delta, s_nexp, s_ncreated, s_abort;
     __shared__ int s_exp[RT], s_sel[RT], s_new[RT];
     __shared__ int s_rtok[RT], s_rpar[RT], s_rdep[RT], s_arg[RT];   // this step's row table and per-row argmax
+    __shared__ int s_cnt[3], s_nsurv;
     __shared__ int s_keep[PROBES_MAX * RT], s_nkeep;                  // per depth, the B-1 best nodes: the only ones the final pick can take
     __shared__ Cand s_list[PROBES_MAX][KP_MAX];                       // Top-K' lists of the probes the next tree uses
     __shared__ float s_lse[PROBES_MAX];
     unsigned long long* c_key = reinterpret_cast<unsigned long long*>(c_rank + MAX_CAND);   // total-order keys
+    unsigned long long* c_sort = c_key + MAX_CAND;                                           // scratch of the sorts
 
     pdl_wait();
     const Dims& D = A.D;
@@ -881,14 +883,34 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     {
         const T* E = reinterpret_cast<const T*>(A.embed);
         float* m = A.mvec + (size_t)seq * D.mask_slots * D.d;
-        for (int j = tid; j < D.d; j += nt) {
-            float ev[PROBES_MAX + 2];
-            const int e0 = D.ema_per_token ? 0 : n_emit - 1;
-            for (int e = e0; e < n_emit; ++e) ev[e] = to_f32(E[(size_t)s_out[e] * D.d + j]);
-            for (int slot = 0; slot < D.mask_slots; ++slot) {      // every mask vector follows the same update
-                float mv = m[(size_t)slot * D.d + j];
-                for (int e = e0; e < n_emit; ++e) mv = __fadd_rn(mv, __fmul_rn(D.lambda, __fsub_rn(ev[e], mv)));
-                m[(size_t)slot * D.d + j] = mv;
+        // four consecutive elements per thread; every load of a pass is issued before the first store
+        const int e0 = D.ema_per_token ? 0 : n_emit - 1;
+        for (int j = tid * 4; j < D.d; j += nt * 4) {
+            float ev[PROBES_MAX + 2][4];
+            float4 mv[PROBES_MAX];
+            for (int e = e0; e < n_emit; ++e)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) ev[e][i] = j + i < D.d ? to_f32(E[(size_t)s_out[e] * D.d + j + i]) : 0.f;
+            const bool vec = j + 4 <= D.d;
+#pragma unroll
+            for (int slot = 0; slot < PROBES_MAX; ++slot) {
+                if (slot < D.mask_slots) {
+                    float* ms = m + (size_t)slot * D.d + j;
+                    mv[slot] = vec ? *reinterpret_cast<const float4*>(ms)
+                                   : make_float4(ms[0], j + 1 < D.d ? ms[1] : 0.f, j + 2 < D.d ? ms[2] : 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int slot = 0; slot < PROBES_MAX; ++slot) {      // every mask vector follows the same update
+                if (slot < D.mask_slots) {
+                    float x[4] = {mv[slot].x, mv[slot].y, mv[slot].z, mv[slot].w};
+                    for (int e = e0; e < n_emit; ++e)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) x[i] = __fadd_rn(x[i], __fmul_rn(D.lambda, __fsub_rn(ev[e][i], x[i])));
+                    float* ms = m + (size_t)slot * D.d + j;
+                    if (vec) *reinterpret_cast<float4*>(ms) = make_float4(x[0], x[1], x[2], x[3]);
+                    else for (int i = 0; i < 4 && j + i < D.d; ++i) ms[i] = x[i];
+                }
             }
         }
     }
@@ -946,16 +968,56 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
         }
         __syncthreads();
         const int width = D.W == 0 ? D.B - i : min(D.W, D.B - i);
-        for (int w = tid; w < n_new; w += nt) {
-            const int c = base + w;
-            const unsigned long long key = c_key[c];   // same depth: (logP desc, creation asc)
+        // Ranks of the new nodes among themselves (same depth: logP desc, creation asc) matter only below
+        // R = max(width, B-1).  With many new nodes, first find by bisection on the keys' high words (the logP
+        // part) the smallest bound that at least R keys do not exceed; only the nodes within it are ranked.
+        const int R = min(max(width, D.B - 1), RT);
+        const int n_kept = min(min(D.B - 1, RT), n_new), keep0 = s_nkeep;
+        int* surv = reinterpret_cast<int*>(c_sort);     // creation indices of the nodes that may rank below R
+        int n_surv = n_new;
+        if (n_new > 4 * R) {
+            unsigned hk[MAX_CAND / 1024];               // high words of this thread's keys (n_new <= MAX_CAND)
+            bool hv[MAX_CAND / 1024];
+#pragma unroll
+            for (int q = 0; q < MAX_CAND / 1024; ++q) {
+                const int w = tid + q * nt;
+                hv[q] = w < n_new;
+                hk[q] = hv[q] ? (unsigned)(c_key[base + w] >> 32) : 0u;
+            }
+            if (tid == 0) { s_cnt[0] = 0; s_cnt[1] = 0; s_cnt[2] = 0; s_nsurv = 0; }
+            __syncthreads();
+            unsigned lo = 0u, hi = 0xffffffffu;         // count(high word <= hi) >= R throughout
+            for (int it = 0; lo < hi; ++it) {
+                const unsigned mid = lo + ((hi - lo) >> 1);
+                if (tid == 0) s_cnt[(it + 1) % 3] = 0;  // last read two barriers ago
+                int mine = 0;
+#pragma unroll
+                for (int q = 0; q < MAX_CAND / 1024; ++q) mine += (hv[q] && hk[q] <= mid) ? 1 : 0;
+                mine = __reduce_add_sync(0xffffffffu, mine);
+                if ((tid & 31) == 0 && mine) atomicAdd(&s_cnt[it % 3], mine);
+                __syncthreads();
+                if (s_cnt[it % 3] >= R) hi = mid; else lo = mid + 1;
+            }
+#pragma unroll
+            for (int q = 0; q < MAX_CAND / 1024; ++q)
+                if (hv[q] && hk[q] <= lo) surv[atomicAdd(&s_nsurv, 1)] = base + tid + q * nt;
+            __syncthreads();
+            n_surv = s_nsurv;
+        } else {
+            for (int w = tid; w < n_new; w += nt) surv[w] = base + w;
+            __syncthreads();
+        }
+        for (int w = tid; w < n_surv; w += nt) {
+            const int c = surv[w];
+            const unsigned long long key = c_key[c];
             int rank = 0;
-            for (int o = 0; o < n_new; ++o) rank += c_key[base + o] < key ? 1 : 0;
+            for (int o = 0; o < n_surv; ++o) rank += c_key[surv[o]] < key ? 1 : 0;
             if (rank < width && c_tok[c] >= 0) s_exp[rank] = c;
             // a node with B-1 or more nodes of its own depth before it cannot be among the B-1 best overall
-            if (rank < D.B - 1 && rank < RT) s_keep[atomicAdd(&s_nkeep, 1)] = c;
+            if (rank < n_kept) s_keep[keep0 + rank] = c;
         }
-        if (tid == 0) { s_ncreated = base + n_new; s_nexp = min(width, n_new); }
+        __syncthreads();
+        if (tid == 0) { s_ncreated = base + n_new; s_nexp = min(width, n_new); s_nkeep = keep0 + n_kept; }
         __syncthreads();
     }
     // final selection: root + the B-1 best created nodes by (logP desc, depth asc, creation asc)
@@ -1028,7 +1090,7 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
 }
 
 void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s, bool pdl) {
-    size_t smem = (size_t)MAX_CAND * 28;
+    size_t smem = (size_t)MAX_CAND * 36;
     if (dtype == 0) {
         cudaFuncSetAttribute(k_tree_step<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         launch_k(k_tree_step<float>, dim3(A.D.batch), dim3(1024), smem, s, pdl, A);
