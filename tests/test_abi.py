@@ -32,6 +32,33 @@ def test_every_declared_symbol_is_exported(lib):
     assert sorted(P.EXPORTS) == names
 
 
+def test_binding_mirrors_the_header():
+    """The constants and the struct members of the ctypes mirror are the header's, in the header's order."""
+    import ctypes
+    text = open(os.path.join(ROOT, "include", "esp.h")).read()
+    for name, value in (("ESP_MAX_ROWS", P.ESP_MAX_ROWS), ("ESP_MAX_PROBES", P.ESP_MAX_PROBES),
+                        ("ESP_MAX_KPRIME", P.ESP_MAX_KPRIME)):
+        m = re.search(r"#define\s+%s\s+(\d+)" % name, text)
+        assert m and int(m.group(1)) == value, name
+    m = re.search(r"#define\s+ESP_STATIC_SCRATCH_BYTES\s+\((\d+)u\s*<<\s*(\d+)\)", text)
+    assert m and (int(m.group(1)) << int(m.group(2))) == P.ESP_STATIC_SCRATCH_BYTES
+    code = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    for cname, ctype in (("esp_model_cfg", P.esp_model_cfg), ("esp_spec_cfg", P.esp_spec_cfg)):
+        end = code.index("} %s;" % cname)
+        body = code[code.rindex("typedef struct {", 0, end) + len("typedef struct {"):end]
+        members = []
+        for decl in body.split(";"):
+            decl = decl.strip()
+            if not decl:
+                continue
+            names = decl.split(None, 1)[1]
+            members += [n.strip().split("[")[0] for n in names.split(",")]
+        mirror = [f[0] for f in ctype._fields_]
+        assert [("lam" if n == "lambda" else n) for n in members] == mirror, cname
+    # two floats, two 32-bit seed words and the 32-bit members: no padding anywhere
+    assert ctypes.sizeof(P.esp_spec_cfg) == 4 * (len(P.esp_spec_cfg._fields_) - 1 + P.ESP_MAX_PROBES)
+
+
 def test_workspace_bytes_and_config_checks(lib):
     m = P.model_cfg(synth.LLAMA3_8B, 1024 + 256 + 16)
     s = P.spec_cfg(n_probes=4, topk=10, max_nodes=64, expand_width=0, n_anchor=1)
