@@ -118,7 +118,7 @@ typedef struct esp_handle esp_handle;
 
 /* Bytes of [device] workspace esp_init needs (KV cache for max_batch sequences of
  * max_seq_len + ESP_MAX_ROWS positions, activations, split-K and attention
- * partials, per-sequence state and -- for bf16 models with max_batch 1 -- a copy of
+ * partials, per-sequence state and -- for bf16 models -- a copy of
  * every layer matrix and of the LM head repacked into the 16 KB blocks the GEMM
  * main loop streams, i.e. about the size of the model again).
  * ESP_E_BADCFG if the configuration is unsupported. */
@@ -143,7 +143,8 @@ int esp_prefill(esp_handle* h, int32_t seq, const int32_t* prompt, int32_t n_pro
 
 /* One decode-and-verify step for every prefilled sequence (Figure 1 right):
  * forward over [last accepted token, draft-tree nodes, mask probes] under the
- * tree mask, argmax / Top-K' + log-sum-exp, lossless verification (Section 2),
+ * tree mask, argmax (or the sampled token, see esp_spec_cfg.temperature) / Top-K' +
+ * log-sum-exp, lossless verification (Section 2),
  * KV compaction of the accepted path, mask update (Eq. mask_update_mean) and
  * the next tree (Algorithm 1 + pruner).  esp_step = esp_step_async + esp_read.
  * tokens_out [host] [max_batch][ESP_MAX_PROBES+1], n_out [host] [max_batch]. */
