@@ -366,8 +366,11 @@ def run_ours(args, shape, plen, k, K, B):
     rows = h.state()["n_rows"]
 
     # ---- end to end: the synchronous call, tokens land in host memory every step (again from the prompt)
-    prefill_all()
     torch.cuda.synchronize()
+    tp0 = time.perf_counter()
+    prefill_all()                      # host prompt in, first token out: the time to the first token of a warm library
+    torch.cuda.synchronize()
+    prefill_ms = (time.perf_counter() - tp0) * 1e3
     if dist is not None:
         dist.barrier()
     te0 = time.perf_counter()
@@ -439,6 +442,8 @@ def run_ours(args, shape, plen, k, K, B):
                     "d2h_bytes_per_step": d2h,
                     "note": "synchronous esp_step; a step's inputs are the device state left by the previous step"},
             "gpu_launches": launches,
+            "prefill": {"ms": prefill_ms, "prompt_tokens": plen * nbatch, "tokens_per_s": plen * nbatch / (prefill_ms * 1e-3),
+                        "note": "esp_prefill of every sequence from host memory, blocks of %d prompt rows" % P.ESP_PREFILL_CHUNK},
             "roofline": {"bound": "hbm", "kernel": "k_gemm_tc<EPI_PARTIAL>, gate/up projection (235 MB of weights per launch)",
                          "achieved": gu_ach, "peak": peak, "unit": "GB/s", "frac": gu_ach / peak if gu_ach else None,
                          "traffic": GATEUP_DRAM_TRAFFIC.get(args.config) if nbatch == 1 and not args.per_node_probes else None,

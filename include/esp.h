@@ -42,6 +42,7 @@ enum {
 #define ESP_MAX_ROWS 128  /* rows of one block per sequence: tree nodes + mask probes */
 #define ESP_MAX_PROBES 8  /* k */
 #define ESP_MAX_KPRIME 32 /* Top-K entries kept per probe, K + pruner refills */
+#define ESP_PREFILL_CHUNK 120 /* prompt rows esp_prefill runs per block (the last block adds the k mask rows) */
 
 /* The frozen decoder f_theta (Section 2; LLaMA3 / Qwen3 shapes, Section 4 "Models"). */
 typedef struct {
@@ -161,8 +162,7 @@ int esp_set_mask(esp_handle* h, int32_t seq, const float* mask);
  * parents[i] < i); node 0 must carry the current root token.  Has no
  * counterpart in the paper; it exists to drive acceptance lengths that
  * random-init models never produce.  The tree with its probe rows must fit the
- * block the handle was configured for (the larger of the spec's rows and
- * 64 + n_probes), else ESP_E_ARG. */
+ * block the handle was configured for (the spec's rows), else ESP_E_ARG. */
 int esp_set_tree(esp_handle* h, int32_t seq, const int32_t* tokens, const int32_t* parents, int32_t n);
 
 /* Debug/parity access to device state of sequence `seq`, copied to [host] buffers (any may be NULL):

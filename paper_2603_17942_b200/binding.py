@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(HERE, "libesp_b200.so")
 ESP_MAX_ROWS = 128
 ESP_MAX_PROBES = 8
 ESP_MAX_KPRIME = 32
+ESP_PREFILL_CHUNK = 120
 
 ERRORS = {0: "ESP_OK", -1: "ESP_E_BADCFG", -2: "ESP_E_WORKSPACE", -3: "ESP_E_PROMPT", -4: "ESP_E_FULL",
           -5: "ESP_E_DEVICE", -6: "ESP_E_CUDA", -7: "ESP_E_STATE", -8: "ESP_E_ARG"}
@@ -30,7 +31,7 @@ EXPORTS = ["esp_workspace_bytes", "esp_init", "esp_prefill", "esp_step", "esp_st
            "esp_gemm_bf16"]
 
 __all__ = ["EspError", "esp_model_cfg", "esp_spec_cfg", "esp_weights", "esp_stats", "load_library", "model_cfg",
-           "spec_cfg", "Handle", "ESP_MAX_ROWS", "ESP_MAX_PROBES", "ESP_MAX_KPRIME", "ESP_STATIC_SCRATCH_BYTES", "EXPORTS", "LIB_PATH", "KINDS"] + EXPORTS
+           "spec_cfg", "Handle", "ESP_MAX_ROWS", "ESP_MAX_PROBES", "ESP_MAX_KPRIME", "ESP_PREFILL_CHUNK", "ESP_STATIC_SCRATCH_BYTES", "EXPORTS", "LIB_PATH", "KINDS"] + EXPORTS
 
 
 class EspError(RuntimeError):

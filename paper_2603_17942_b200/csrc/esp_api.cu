@@ -118,7 +118,7 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
         int S = 256;
         while ((m->max_seq_len + S - 1) / S > 16) S *= 2;   // at most 16 splits: the partials stay small next to the cache
         D->split_len = S;
-        D->n_split_max = (m->max_seq_len + S - 1) / S + 1;
+        D->n_split_max = (m->max_seq_len + RT + S - 1) / S + 1;   // a prefill block's own rows count as cache positions
         D->rms_eps = m->rms_eps;
         D->k = s->n_probes; D->K = topk; D->KP = s->n_probes > 0 ? KP : 1; D->B = n_nodes; D->W = is_static ? 1 : s->expand_width;
         D->mask_slots = s->n_probes > 0 ? s->n_probes : 1;
@@ -164,7 +164,12 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.tree_dev = c.take<int32_t>(2 * RT);
     o.rope_cos = c.take<float>((size_t)D.cap * (D.h / 2));
     o.rope_sin = c.take<float>((size_t)D.cap * (D.h / 2));
-    o.gemm_partials = c.take<char>(tc_gemm_partial_bytes(n_sm, D.batch < tc_gemm_max_nq(D.gemm_rows) ? D.batch : tc_gemm_max_nq(D.gemm_rows), D.gemm_rows));
+    {
+        // the decode steps' passes (several sequences of gemm_rows rows) or one 128-row prefill block, whichever is larger
+        const size_t step_b = tc_gemm_partial_bytes(n_sm, D.batch < tc_gemm_max_nq(D.gemm_rows) ? D.batch : tc_gemm_max_nq(D.gemm_rows), D.gemm_rows);
+        const size_t pre_b = tc_gemm_partial_bytes(n_sm, 1, RT);
+        o.gemm_partials = c.take<char>(step_b > pre_b ? step_b : pre_b);
+    }
     o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
     o.sk_tables = c.take<TileSrc>(4 * SK_TABLE_TILES);
     o.packed = nullptr;
@@ -196,6 +201,10 @@ struct esp_handle {
     const void *embed, *lm_head, *final_norm;
     std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, na, nf, qn, kn;
     std::vector<TcGemm*> p_qkv, p_o, p_gu, p_down;
+    // the same GEMMs with 128 rows per block for the prefill, when the decode steps use the 80-row kernels
+    std::vector<TcGemm*> p_qkv_w, p_o_w, p_gu_w, p_down_w;
+    TcGemm* p_lm_w = nullptr;
+    int rows_cap_prefill = RT;
     std::vector<AttnTc*> p_attn;   // per layer, bf16 models with head_dim 128
     TcGemm* p_lm = nullptr;
     std::vector<int> L_host, ready;
@@ -263,7 +272,7 @@ int run_gemm(esp_handle* h, TcGemm* plan, int epi, int n_tiles, const void* cons
 // their weights once for all nb sequences and store stream-K partials that the next kernel sums (k_qkv_finish;
 // k_resid_norm = residual add + RMSNorm; k_swiglu_finish); the LM head runs once per sequence and finishes
 // in-kernel.  CUDA-core path (fp32 models): the same layer with every epilogue fused in the GEMM.
-int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc) {
+int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc, bool prefill) {
     const Dims& D = h->D;
     Buffers& b = h->b;
     cudaStream_t s = h->stream;
@@ -271,7 +280,8 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
     const size_t es = h->dtype ? 2 : 4;
     int Lmax = 0;
     for (int i = s0; i < s0 + nb; ++i) Lmax = h->L_host[i] > Lmax ? h->L_host[i] : Lmax;
-    const int n_split_launch = (Lmax + D.split_len - 1) / D.split_len;
+    // a prefill block's rows attend to the block's earlier rows through the cache as well
+    const int n_split_launch = (Lmax + (prefill ? RT : 0) + D.split_len - 1) / D.split_len;
     const bool pdl = h->use_pdl && !h->prof;
     SeqState* st0 = b.states + s0;
     const size_t kv_seq_off = (size_t)s0 * D.Hkv * D.cap * D.h * es;   // this pass's first sequence inside a layer's cache
@@ -279,7 +289,9 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
     StreamK pending;   // partials of the last down projection, summed by the next norm
     pending.partials = nullptr; pending.table = nullptr; pending.n_tiles = 0; pending.KB = 1; pending.G = 1; pending.slots = 2; pending.rows = RT; pending.seq_rows = RT;
     mark(h, -1);
-    const int rc_rows = h->rows_cap;     // no block has more rows: sizes the row dimension of the grids
+    const int rc_rows = prefill ? h->rows_cap_prefill : h->rows_cap;   // no block has more rows: sizes the row dimension of the grids
+    const bool wide = prefill && !h->p_qkv_w.empty();                  // 128-row GEMM plans for the prefill blocks
+    auto plan = [&](std::vector<TcGemm*>& narrow, std::vector<TcGemm*>& w128, int l) -> TcGemm* { return wide ? w128[l] : narrow[l]; };
     launch_assemble(h->dtype, st0, h->embed, mvec0, b.hres, D.d, D.mask_slots, nb, s, false, rc_rows);
     h->launches++;
     for (int l = 0; l < D.n_layers; ++l) {
@@ -296,11 +308,11 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.k_norm = D.qk_norm ? h->kn[l] : nullptr;
             const void* w[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t rows[3] = {dq, dkv, dkv};
-            int rc = run_gemm(h, tc ? h->p_qkv[l] : nullptr, EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a, tc, pdl, tc ? nb : 1);
+            int rc = run_gemm(h, tc ? plan(h->p_qkv, h->p_qkv_w, l) : nullptr, EPI_QKV, (dq + 2 * dkv) / TILE_N, w, rows, b.xn, D.d, a, tc, pdl, tc ? nb : 1);
             if (rc) return rc;
             mark(h, KIND_QKV);
             if (tc) {
-                if (launch_qkv_finish(a, tc_gemm_streamk(h->p_qkv[l], nb), nb, s, pdl, rc_rows)) return ESP_E_BADCFG;
+                if (launch_qkv_finish(a, tc_gemm_streamk(plan(h->p_qkv, h->p_qkv_w, l), nb), nb, s, pdl, rc_rows)) return ESP_E_BADCFG;
                 h->launches++;
                 mark(h, KIND_MISC);
             }
@@ -317,6 +329,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.Hq = D.Hq; a.Hkv = D.Hkv; a.h = D.h; a.cap = D.cap; a.split_len = D.split_len; a.n_split_max = D.n_split_max;
             a.dcap = dcap;
             a.rows_cap = rc_rows;
+            a.cache_in_flight = prefill ? 1 : 0;
             a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
             a.err = b.err;
             if (tc) {
@@ -333,11 +346,11 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.hres = b.hres;
             const void* w[3] = {h->wo[l], nullptr, nullptr};
             const int32_t rows[3] = {D.d, 0, 0};
-            int rc = run_gemm(h, tc ? h->p_o[l] : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.attn_out, dq, a, tc, pdl, tc ? nb : 1);
+            int rc = run_gemm(h, tc ? plan(h->p_o, h->p_o_w, l) : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.attn_out, dq, a, tc, pdl, tc ? nb : 1);
             if (rc) return rc;
             mark(h, KIND_O);
         }
-        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(h->p_o[l], nb), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
+        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(plan(h->p_o, h->p_o_w, l), nb), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -346,11 +359,11 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.act_out = b.act;
             const void* w[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t rows[3] = {D.F, D.F, 0};
-            int rc = run_gemm(h, tc ? h->p_gu[l] : nullptr, EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a, tc, pdl, tc ? nb : 1);
+            int rc = run_gemm(h, tc ? plan(h->p_gu, h->p_gu_w, l) : nullptr, EPI_SWIGLU, (D.F + 63) / 64, w, rows, b.xn, D.d, a, tc, pdl, tc ? nb : 1);
             if (rc) return rc;
             mark(h, KIND_GATEUP);
             if (tc) {
-                launch_swiglu_finish(st0, tc_gemm_streamk(h->p_gu[l], nb), b.act, D.F, nb, s, pdl, rc_rows);
+                launch_swiglu_finish(st0, tc_gemm_streamk(plan(h->p_gu, h->p_gu_w, l), nb), b.act, D.F, nb, s, pdl, rc_rows);
                 h->launches++;
                 mark(h, KIND_MISC);
             }
@@ -360,9 +373,9 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.hres = b.hres;
             const void* w[3] = {h->wd[l], nullptr, nullptr};
             const int32_t rows[3] = {D.d, 0, 0};
-            int rc = run_gemm(h, tc ? h->p_down[l] : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.act, D.F, a, tc, pdl, tc ? nb : 1);
+            int rc = run_gemm(h, tc ? plan(h->p_down, h->p_down_w, l) : nullptr, EPI_RESID, (D.d + TILE_N - 1) / TILE_N, w, rows, b.act, D.F, a, tc, pdl, tc ? nb : 1);
             if (rc) return rc;
-            if (tc) pending = tc_gemm_streamk(h->p_down[l], nb);
+            if (tc) pending = tc_gemm_streamk(plan(h->p_down, h->p_down_w, l), nb);
             mark(h, KIND_DOWN);
         }
     }
@@ -382,7 +395,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
             a.logits_dump = h->dbg_logits ? h->dbg_logits + (size_t)sq * RT * D.V : nullptr;
             const void* w[3] = {h->lm_head, nullptr, nullptr};
             const int32_t rows[3] = {D.V, 0, 0};
-            int rc = run_gemm(h, h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl, 1, q);
+            int rc = run_gemm(h, wide ? h->p_lm_w : h->p_lm, EPI_LOGITS, n_tiles, w, rows, b.xn, D.d, a, tc, pdl, 1, q);
             if (rc) return rc;
             mark(h, KIND_LMHEAD);
             launch_topk_merge(b.states + sq, b.cand, b.cand_ms, n_tiles, D.KP, per, b.topk + (size_t)sq * RT * KP_MAX, b.lse + (size_t)sq * RT, s, pdl, rc_rows, b.cand_floor);
@@ -396,8 +409,9 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc)
 // Forward over the sequences that take part: `only_seq` (prefill) or every prefilled sequence (a step).
 int forward(esp_handle* h, bool with_lm, int dcap, int only_seq) {
     const bool tc = h->dtype == 1 && h->gemm_impl == 0 && h->p_lm != nullptr;
-    if (!tc) return forward_pass(h, with_lm, dcap, 0, h->D.batch, false);
-    if (only_seq >= 0) return forward_pass(h, with_lm, dcap, only_seq, 1, true);
+    const bool prefill = only_seq >= 0;
+    if (!tc) return forward_pass(h, with_lm, dcap, 0, h->D.batch, false, prefill);
+    if (only_seq >= 0) return forward_pass(h, with_lm, dcap, only_seq, 1, true, true);
     // consecutive sequences share a pass (and a weight stream); sequences that are not ready are inactive in it
     const int per_pass = tc_gemm_max_nq(h->D.gemm_rows);
     for (int s0 = 0; s0 < h->D.batch; s0 += per_pass) {
@@ -405,7 +419,7 @@ int forward(esp_handle* h, bool with_lm, int dcap, int only_seq) {
         bool any = false;
         for (int i = s0; i < s0 + nb; ++i) any = any || h->ready[i];
         if (!any) continue;
-        const int rc = forward_pass(h, with_lm, dcap, s0, nb, true);
+        const int rc = forward_pass(h, with_lm, dcap, s0, nb, true, false);
         if (rc) return rc;
     }
     return ESP_OK;
@@ -487,8 +501,8 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
     h->n_sm = n_sm;
     {
         const int step_rows = spec_rows(*spec), pre_rows = PREFILL_CHUNK + spec->n_probes;
-        h->rows_cap = step_rows > pre_rows ? step_rows : pre_rows;
-        if (h->rows_cap > RT) h->rows_cap = RT;
+        h->rows_cap = step_rows > RT ? RT : step_rows;
+        h->rows_cap_prefill = pre_rows > RT ? RT : pre_rows;
     }
     carve_all(D, model->dtype, 148, reinterpret_cast<char*>(workspace), &h->b);
     h->embed = w->embed; h->lm_head = w->lm_head; h->final_norm = w->final_norm;
@@ -550,6 +564,34 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
         const void* w5[3] = {h->lm_head, nullptr, nullptr};
         const int32_t r5[3] = {D.V, 0, 0};
         ok = ok && !tc_gemm_create(&h->p_lm, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, D.batch, nrs, 1, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
+        if (ok && nrs != RT) {
+            // the prefill runs 120-row blocks: the same weights (already repacked) behind 128-row GEMM plans
+            const size_t pbytes = tc_gemm_partial_bytes(148, 1, RT);
+            for (int l = 0; l < D.n_layers && ok; ++l) {
+                TcGemm* p = nullptr;
+                char* pk = h->b.packed + h->b.pk_layer * l;
+                const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
+                const int32_t r1[3] = {dq, dkv, dkv};
+                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream);
+                h->p_qkv_w.push_back(p);
+                const void* w2[3] = {h->wo[l], nullptr, nullptr};
+                const int32_t r2[3] = {D.d, 0, 0};
+                p = nullptr;
+                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream);
+                h->p_o_w.push_back(p);
+                const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
+                const int32_t r3[3] = {D.F, D.F, 0};
+                p = nullptr;
+                ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream);
+                h->p_gu_w.push_back(p);
+                const void* w4[3] = {h->wd[l], nullptr, nullptr};
+                const int32_t r4[3] = {D.d, 0, 0};
+                p = nullptr;
+                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream);
+                h->p_down_w.push_back(p);
+            }
+            ok = ok && !tc_gemm_create(&h->p_lm_w, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
+        }
         if (!ok) { esp_free(h); return ESP_E_CUDA; }
     }
     if (cudaStreamSynchronize(h->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) { esp_free(h); return ESP_E_CUDA; }
@@ -813,6 +855,11 @@ void esp_free(esp_handle* h) {
     for (auto* p : h->p_gu) tc_gemm_destroy(p);
     for (auto* p : h->p_down) tc_gemm_destroy(p);
     tc_gemm_destroy(h->p_lm);
+    for (auto* p : h->p_qkv_w) tc_gemm_destroy(p);
+    for (auto* p : h->p_o_w) tc_gemm_destroy(p);
+    for (auto* p : h->p_gu_w) tc_gemm_destroy(p);
+    for (auto* p : h->p_down_w) tc_gemm_destroy(p);
+    tc_gemm_destroy(h->p_lm_w);
     for (auto* t : h->p_attn) attn_tc_destroy(t);
     if (h->pinned) cudaFreeHost(h->pinned);
     drop_graphs(h);

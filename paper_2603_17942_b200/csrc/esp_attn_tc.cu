@@ -166,8 +166,10 @@ __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __g
                 tma_load_2d(st + K_BYTES, &p.map_v, 0, kvrow0 + c * CK, &kv_full[c & 1]);
                 tma_load_2d(st + K_BYTES + HALF_BYTES, &p.map_v, 64, kvrow0 + c * CK, &kv_full[c & 1]);
             };
+            // the cache below T0 is settled in a decode step: request it before waiting for the kernel that wrote the queries
+            if (a.cache_in_flight) pdl_wait();
             for (int c = 0; c < n_chunks && c < 2; ++c) load_chunk(c);
-            pdl_wait();     // the queries come from the kernel before this one
+            if (!a.cache_in_flight) pdl_wait();
             mbar_expect_tx(q_full, Q_BYTES);
             tma_load_3d(sQ, &p.map_q, 0, kvh * p.group, seq * RT + row0, q_full);
             tma_load_3d(sQ + HALF_BYTES, &p.map_q, 64, kvh * p.group, seq * RT + row0, q_full);
@@ -468,8 +470,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                 int c0 = 0;
                 if (first) {
                     // the cache does not depend on the kernel before this one, the queries do
+                    if (a.cache_in_flight) pdl_wait();
                     for (; c0 < it.n_chunks && c0 < 2 && ok; ++c0) ok = load_chunk(c0);
-                    pdl_wait();
+                    if (!a.cache_in_flight) pdl_wait();
                     first = false;
                 } else {
                     // Q is single buffered: the previous item's last Q K^T must have completed

@@ -16,9 +16,9 @@ constexpr int KP_MAX = ESP_MAX_KPRIME;  // Top-K' entries kept per row
 constexpr int PROBES_MAX = ESP_MAX_PROBES;
 constexpr int TILE_N = 128;             // output features per GEMM tile
 constexpr int MAX_CAND = 4096;          // nodes Algorithm 1 may create in one step
-constexpr int PREFILL_CHUNK = 64;       // prompt rows per prefill block
+constexpr int PREFILL_CHUNK = ESP_PREFILL_CHUNK;   // prompt rows per prefill block
 constexpr int DCAP_STEP = 16;           // tail cap of decode steps (>= 2k)
-constexpr int DCAP_PREFILL = 80;        // tail cap of prefill chain blocks
+constexpr int DCAP_PREFILL = 16;        // tail cap of prefill blocks: their earlier rows are cache positions already
 constexpr int RING = ESP_MAX_PROBES + 4; // per-sequence result record: n_out, L, tokens
 
 // device error codes (first one recorded wins)

@@ -133,8 +133,8 @@ class ParityRun:
         ref, kb, vb, _ = self.model.block_forward(self.kc, self.vc, 0, x, np.arange(M), np.tril(np.ones((M, M), np.uint8)), want)
         self.kc[:, :t], self.vc[:, :t] = kb[:, :t], vb[:, :t]
         self.L = t
-        # the last prefill chunk holds the final (t-1) % 64 + 1 prompt rows followed by the k mask rows
-        r0 = (t - 1) % 64
+        # the last prefill chunk holds the final (t-1) % chunk + 1 prompt rows followed by the k mask rows
+        r0 = (t - 1) % P.ESP_PREFILL_CHUNK
         rng = self._cmp_logits(gl[r0:r0 + 1 + k], ref[t - 1:], "prefill")
         self._check_selection(gl, st, [r0], range(r0 + 1, r0 + 1 + k), {r0: t - 1})
         assert first == st["topk_ids"][r0, 0]
