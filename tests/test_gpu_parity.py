@@ -247,6 +247,34 @@ def test_full_width_shapes_parity(pu, base, topk, B):
     run.close()
 
 
+def test_full_width_stream_is_invariant_across_cache_split_growth(pu):
+    """While a sequence grows, the number of cache splits grows, the captured step graph changes with it and the
+    attention launch moves from one CTA per (split, head group, row tile) to the persistent kernel.  None of this
+    may change a bit: the ESP stream with forced multi-token acceptances stays equal to plain decoding while the
+    length crosses several split boundaries, that hand-over among them."""
+    import paper_2603_17942_b200 as P
+    shape = synth.LLAMA3_8B.replace(n_layers=2)
+    w = synth.make_weights(shape, seed=2, device="cuda")
+    prompt = synth.make_prompt(shape.vocab, 1990, 8)
+    n_new, max_seq = 640, 3000
+    truth, _ = pu.gpu_generate(shape, w, pu.GREEDY, prompt, n_new, max_seq_len=max_seq)
+    spec = O.SpecCfg(n_probes=4, topk=10, max_nodes=64, expand_width=0, n_anchor=1)
+    h = P.Handle(shape, pu.c_spec(spec), w, max_seq_len=max_seq)
+    out = [h.prefill(prompt)]
+    rng = np.random.default_rng(3)
+    while len(out) < n_new - 8:
+        n = len(out)
+        if rng.integers(0, 2):
+            depth = int(rng.integers(1, 6))
+            toks = [out[-1]] + [truth[n + i] for i in range(depth)]
+            h.set_tree(np.array(toks, np.int32), np.arange(-1, depth, dtype=np.int32))
+        out.extend(h.step())
+    assert out == truth[:len(out)]
+    assert len(prompt) + len(out) > 2304 + 256          # past the hand-over (10 splits of 256 keys) and one more split
+    assert h.stats().device_error == 0
+    h.close()
+
+
 # ------------------------------------------------------------------ blocks of more than 80 rows (BC = 120)
 @pytest.mark.parametrize("widths", [(), (15, 10, 4)])
 def test_tiny_fp32_block_complexity_120_parity(pu, widths):
