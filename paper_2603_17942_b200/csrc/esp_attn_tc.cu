@@ -81,6 +81,12 @@ constexpr int ONCE_THREADS = 320;          // producer warp, MMA warp, 8 softmax
 constexpr int ONCE_OFF_BAR = OFF_P + P_BYTES;
 constexpr size_t ONCE_SMEM_BYTES = 1024 + ONCE_OFF_BAR + 256;
 
+// The producer thread waits for the kernel before this one and only then releases the kernel after it.
+__device__ __forceinline__ void trigger_after_wait() {
+    pdl_wait();
+    pdl_launch_dependents();
+}
+
 __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __grid_constant__ BulkParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ int s_T0max;
@@ -103,7 +109,8 @@ __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __g
     const int seq = blockIdx.z;
 
     // Read before pdl_wait(): the sequence state and the cache below T0, both written by earlier steps.
-    if (threadIdx.x == 0) pdl_launch_dependents();
+    // The tail kernel is released only after this kernel's wait has returned (trigger_after_wait), so that it may
+    // work on this step's queries and keys while the CTAs here are still running.
     int n_rows, L;
     if (a.st) {
         const SeqState* st = a.st + seq;
@@ -167,9 +174,9 @@ __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __g
                 tma_load_2d(st + K_BYTES + HALF_BYTES, &p.map_v, 64, kvrow0 + c * CK, &kv_full[c & 1]);
             };
             // the cache below T0 is settled in a decode step: request it before waiting for the kernel that wrote the queries
-            if (a.cache_in_flight) pdl_wait();
+            if (a.cache_in_flight) trigger_after_wait();
             for (int c = 0; c < n_chunks && c < 2; ++c) load_chunk(c);
-            if (!a.cache_in_flight) pdl_wait();
+            if (!a.cache_in_flight) trigger_after_wait();
             mbar_expect_tx(q_full, Q_BYTES);
             tma_load_3d(sQ, &p.map_q, 0, kvh * p.group, seq * RT + row0, q_full);
             tma_load_3d(sQ + HALF_BYTES, &p.map_q, 64, kvh * p.group, seq * RT + row0, q_full);
@@ -383,7 +390,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     // Read before pdl_wait(): the sequence state and the cache below T0, both written by earlier steps.
-    if (threadIdx.x == 0) pdl_launch_dependents();
+    // The dependent kernel is released by the producer thread once its wait has returned (trigger_after_wait).
     for (int e = warp; e < p.n_seq * p.n_row_tiles; e += NUM_THREADS / 32) {   // one warp per entry, a lane per row
         const int seq = p.seq0 + e / p.n_row_tiles, row0 = (e % p.n_row_tiles) * p.rows_per_tile;
         int n_rows, L;
@@ -470,9 +477,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                 int c0 = 0;
                 if (first) {
                     // the cache does not depend on the kernel before this one, the queries do
-                    if (a.cache_in_flight) pdl_wait();
+                    if (a.cache_in_flight) trigger_after_wait();
                     for (; c0 < it.n_chunks && c0 < 2 && ok; ++c0) ok = load_chunk(c0);
-                    if (!a.cache_in_flight) pdl_wait();
+                    if (!a.cache_in_flight) trigger_after_wait();
                     first = false;
                 } else {
                     // Q is single buffered: the previous item's last Q K^T must have completed
@@ -486,7 +493,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                 gc += it.n_chunks;
                 ++n_it;
             }
-            if (first) pdl_wait();
+            if (first) trigger_after_wait();
             if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
         }
     } else if (warp == 1) {
@@ -761,8 +768,10 @@ __global__ void __launch_bounds__(128, 4) k_attn_tail_merge_tc(AttnArgs a) {
         L = a.L_fixed;
         if (r < n_rows) { depth = a.depth[seq * RT + r]; lo = a.anc[(size_t)(seq * RT + r) * 2]; hi = a.anc[(size_t)(seq * RT + r) * 2 + 1]; }
     }
-    pdl_wait();
-    if (r >= n_rows) return;
+    // After a bulk launch this kernel starts once every bulk CTA's wait has returned: the kernel that wrote this
+    // step's queries, keys and values has completed by then, and the tail may be computed while the bulk CTAs run.
+    if (!a.tail_first) pdl_wait();
+    if (r >= n_rows) { pdl_wait(); return; }
     const int kvh = head / (a.Hq / a.Hkv);
     const int P = L + depth, T0 = tail_start_tc(P, a.dcap);
     const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.kc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
@@ -776,18 +785,20 @@ __global__ void __launch_bounds__(128, 4) k_attn_tail_merge_tc(AttnArgs a) {
         s_q[lane * 4 + 2] = __low2float(q23); s_q[lane * 4 + 3] = __high2float(q23);
     }
     __syncwarp();
-    // bulk partials: request the first eight now, they are summed after the tail is done
     const int n_sp = (T0 + a.split_len - 1) / a.split_len;
     const size_t base = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max;
     float2 ml0[8];
     float4 c40[8];
+    auto request_partials = [&]() {     // the first eight bulk partials
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-        if (u < n_sp) {
-            ml0[u] = __ldcg(a.part_ml + base + u);
-            c40[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (base + u) * HD + lane * 4));
+        for (int u = 0; u < 8; ++u) {
+            if (u < n_sp) {
+                ml0[u] = __ldcg(a.part_ml + base + u);
+                c40[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (base + u) * HD + lane * 4));
+            }
         }
-    }
+    };
+    if (!a.tail_first) request_partials();      // in flight while the tail is computed
     // ---- tail
     float tm = -INFINITY, tl = 0.f, to[4] = {0.f, 0.f, 0.f, 0.f};
     const int n_tail = P - T0 + 1;
@@ -854,6 +865,7 @@ __global__ void __launch_bounds__(128, 4) k_attn_tail_merge_tc(AttnArgs a) {
         merge_ml(tm, tl, to, cm, cl, co);
     }
     // ---- merge: splits in order, then the tail
+    if (a.tail_first) { pdl_wait(); request_partials(); }
     float m = -INFINITY, l = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
@@ -947,6 +959,7 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
     }
     BulkParams p = t->p;
     p.a = a;
+    p.a.tail_first = 0;
     const int rows_cap = a.rows_cap > 0 && a.rows_cap < RT ? a.rows_cap : RT;
     p.n_row_tiles = (rows_cap + p.rows_per_tile - 1) / p.rows_per_tile;   // row tiles that can hold rows
     if (n_split_launch > 0) {
@@ -983,7 +996,9 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
             }
         }
     }
-    if (launch_k(k_attn_tail_merge_tc, dim3((rows_cap + 3) / 4, a.Hq, batch), dim3(128), 0, s, pdl, a) != cudaSuccess) return -1;
+    AttnArgs ta = a;
+    ta.tail_first = n_split_launch > 0;     // the bulk kernels release their dependent after their own wait
+    if (launch_k(k_attn_tail_merge_tc, dim3((rows_cap + 3) / 4, a.Hq, batch), dim3(128), 0, s, pdl, ta) != cudaSuccess) return -1;
     return 0;
 }
 

@@ -211,7 +211,9 @@ __device__ __forceinline__ void set_error(int* err, int code) {
 // Programmatic dependent launch.  A kernel launched with the attribute may start while its predecessor in
 // the stream still runs; pdl_wait() returns once the predecessor has completed and its writes are visible.
 // Rule used throughout: before pdl_wait() a kernel touches only immutable inputs (weights) and its own
-// shared/tensor memory.  Both calls are no-ops for a plain launch.
+// shared/tensor memory, and data that kernels before the predecessor wrote only where the predecessor releases
+// its dependents after its own wait (the attention kernels; a kernel can only start once all CTAs of the one
+// before it have released it or exited).  Both calls are no-ops for a plain launch.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
