@@ -750,7 +750,8 @@ __device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], floa
 
 // The tail: positions T0..P in position order, lane j owns key j of a 32-key chunk (chunk grid anchored at T0).
 // Then the merge: bulk partials in split order, the tail last; a lane owns 4 of the 128 output dims.
-__global__ void __launch_bounds__(128, 4) k_attn_tail_merge_tc(AttnArgs a) {
+template <bool TAIL_FIRST>
+__global__ void __launch_bounds__(128, TAIL_FIRST ? 5 : 4) k_attn_tail_merge_tc(AttnArgs a) {
     __shared__ float s_qall[4][HD];
     if (threadIdx.x == 0) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -770,7 +771,7 @@ __global__ void __launch_bounds__(128, 4) k_attn_tail_merge_tc(AttnArgs a) {
     }
     // After a bulk launch this kernel starts once every bulk CTA's wait has returned: the kernel that wrote this
     // step's queries, keys and values has completed by then, and the tail may be computed while the bulk CTAs run.
-    if (!a.tail_first) pdl_wait();
+    if (!TAIL_FIRST) pdl_wait();
     if (r >= n_rows) { pdl_wait(); return; }
     const int kvh = head / (a.Hq / a.Hkv);
     const int P = L + depth, T0 = tail_start_tc(P, a.dcap);
@@ -798,7 +799,7 @@ __global__ void __launch_bounds__(128, 4) k_attn_tail_merge_tc(AttnArgs a) {
             }
         }
     };
-    if (!a.tail_first) request_partials();      // in flight while the tail is computed
+    if (!TAIL_FIRST) request_partials();      // in flight while the tail is computed
     // ---- tail
     float tm = -INFINITY, tl = 0.f, to[4] = {0.f, 0.f, 0.f, 0.f};
     const int n_tail = P - T0 + 1;
@@ -865,7 +866,7 @@ __global__ void __launch_bounds__(128, 4) k_attn_tail_merge_tc(AttnArgs a) {
         merge_ml(tm, tl, to, cm, cl, co);
     }
     // ---- merge: splits in order, then the tail
-    if (a.tail_first) { pdl_wait(); request_partials(); }
+    if (TAIL_FIRST) { pdl_wait(); request_partials(); }
     float m = -INFINITY, l = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
@@ -959,7 +960,6 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
     }
     BulkParams p = t->p;
     p.a = a;
-    p.a.tail_first = 0;
     const int rows_cap = a.rows_cap > 0 && a.rows_cap < RT ? a.rows_cap : RT;
     p.n_row_tiles = (rows_cap + p.rows_per_tile - 1) / p.rows_per_tile;   // row tiles that can hold rows
     if (n_split_launch > 0) {
@@ -996,9 +996,11 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
             }
         }
     }
-    AttnArgs ta = a;
-    ta.tail_first = n_split_launch > 0;     // the bulk kernels release their dependent after their own wait
-    if (launch_k(k_attn_tail_merge_tc, dim3((rows_cap + 3) / 4, a.Hq, batch), dim3(128), 0, s, pdl, ta) != cudaSuccess) return -1;
+    // the bulk kernels release their dependent after their own wait: behind them the tail is computed first
+    const dim3 tgrid((rows_cap + 3) / 4, a.Hq, batch);
+    const cudaError_t e = n_split_launch > 0 ? launch_k(k_attn_tail_merge_tc<true>, tgrid, dim3(128), 0, s, pdl, a)
+                                             : launch_k(k_attn_tail_merge_tc<false>, tgrid, dim3(128), 0, s, pdl, a);
+    if (e != cudaSuccess) return -1;
     return 0;
 }
 

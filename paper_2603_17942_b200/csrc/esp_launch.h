@@ -18,7 +18,6 @@ struct AttnArgs {
     int32_t rows_cap;               // no block of this launch has more rows than this (0: RT); sizes the grids
     int32_t cache_in_flight;        // 1: positions below T0 may have been written by the kernel before this one
                                     // (prefill blocks: a row's earlier rows sit in the cache already)
-    int32_t tail_first;             // set by attn_tc_launch: the tail kernel computes the tail before it waits
     int32_t n_rows_fixed, L_fixed;
     int32_t Hq, Hkv, h, cap, split_len, n_split_max, dcap;
     float scale_log2;     // log2(e)/sqrt(h)
