@@ -997,8 +997,9 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
         }
     }
     // the bulk kernels release their dependent after their own wait: behind them the tail is computed first
+    // (plain launches run one after the other: there the partials are requested before the tail instead)
     const dim3 tgrid((rows_cap + 3) / 4, a.Hq, batch);
-    const cudaError_t e = n_split_launch > 0 ? launch_k(k_attn_tail_merge_tc<true>, tgrid, dim3(128), 0, s, pdl, a)
+    const cudaError_t e = n_split_launch > 0 && pdl ? launch_k(k_attn_tail_merge_tc<true>, tgrid, dim3(128), 0, s, pdl, a)
                                              : launch_k(k_attn_tail_merge_tc<false>, tgrid, dim3(128), 0, s, pdl, a);
     if (e != cudaSuccess) return -1;
     return 0;
