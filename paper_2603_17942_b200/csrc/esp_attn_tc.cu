@@ -771,6 +771,8 @@ __global__ void __launch_bounds__(128, TAIL_FIRST ? 5 : 4) k_attn_tail_merge_tc(
     }
     // After a bulk launch this kernel starts once every bulk CTA's wait has returned: the kernel that wrote this
     // step's queries, keys and values has completed by then, and the tail may be computed while the bulk CTAs run.
+    // (Nothing reads those buffers through L1 between that kernel's writes and this point: the bulk kernels fetch
+    // them by TMA, so no SM can hold a line of them from before the writes.)
     if (!TAIL_FIRST) pdl_wait();
     if (r >= n_rows) { pdl_wait(); return; }
     const int kvh = head / (a.Hq / a.Hkv);
