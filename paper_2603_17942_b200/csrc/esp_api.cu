@@ -903,6 +903,7 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     a.anc = reinterpret_cast<const unsigned long long*>(anc);
     a.depth = depth;
     a.n_rows_fixed = n_rows; a.L_fixed = L;
+    a.rows_cap = n_rows;      // sizes the grids: no block has more rows
     a.Hq = n_q_heads; a.Hkv = n_kv_heads; a.h = head_dim; a.cap = cap; a.split_len = S; a.n_split_max = (int)ns; a.dcap = dcap;
     a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)head_dim));
     a.err = reinterpret_cast<int*>(reinterpret_cast<char*>(scratch) + need - 256);
