@@ -750,8 +750,14 @@ __device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], floa
 
 // The tail: positions T0..P in position order, lane j owns key j of a 32-key chunk (chunk grid anchored at T0).
 // Then the merge: bulk partials in split order, the tail last; a lane owns 4 of the 128 output dims.
-template <bool TAIL_FIRST>
-__global__ void __launch_bounds__(128, TAIL_FIRST ? 5 : 4) k_attn_tail_merge_tc(AttnArgs a) {
+// TAIL_FIRST: launched behind a bulk kernel with programmatic dependent launch (see below).  LEAN: smaller load
+// batches and 64 registers, eight CTAs per SM, for grids of many waves where occupancy counts for more than one
+// warp's latency.  All instances add in the same order and give the same bits.
+template <bool TAIL_FIRST, bool LEAN>
+__global__ void __launch_bounds__(128, LEAN ? 8 : (TAIL_FIRST ? 5 : 4)) k_attn_tail_merge_tc(AttnArgs a) {
+    constexpr int KB8 = LEAN ? 8 : HD / 8;      // 16-byte pieces of a key row loaded before they are used
+    constexpr int VB = LEAN ? 8 : 16;           // value rows loaded before they are used
+    constexpr int PB = LEAN ? 4 : 8;            // split partials loaded before they are merged
     __shared__ float s_qall[4][HD];
     if (threadIdx.x == 0) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -790,11 +796,11 @@ __global__ void __launch_bounds__(128, TAIL_FIRST ? 5 : 4) k_attn_tail_merge_tc(
     __syncwarp();
     const int n_sp = (T0 + a.split_len - 1) / a.split_len;
     const size_t base = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max;
-    float2 ml0[8];
-    float4 c40[8];
-    auto request_partials = [&]() {     // the first eight bulk partials
+    float2 ml0[PB];
+    float4 c40[PB];
+    auto request_partials = [&]() {     // the first bulk partials
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < PB; ++u) {
             if (u < n_sp) {
                 ml0[u] = __ldcg(a.part_ml + base + u);
                 c40[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (base + u) * HD + lane * 4));
@@ -821,19 +827,22 @@ __global__ void __launch_bounds__(128, TAIL_FIRST ? 5 : 4) k_attn_tail_merge_tc(
         float sc = -INFINITY;
         if (valid) {
             const uint4* kr = reinterpret_cast<const uint4*>(kbase + (size_t)slot * HD);
-            uint4 kreg[HD / 8];
-#pragma unroll
-            for (int d8 = 0; d8 < HD / 8; ++d8) kreg[d8] = kr[d8];
             float acc = 0.f;
 #pragma unroll
-            for (int d8 = 0; d8 < HD / 8; ++d8) {
-                const uint4 kk = kreg[d8];
+            for (int dh = 0; dh < HD / 8; dh += KB8) {
+            uint4 kreg[KB8];
+#pragma unroll
+            for (int d8 = 0; d8 < KB8; ++d8) kreg[d8] = kr[dh + d8];
+#pragma unroll
+            for (int d8 = dh; d8 < dh + KB8; ++d8) {
+                const uint4 kk = kreg[d8 - dh];
                 const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kk);
                 const float4 qa = *reinterpret_cast<const float4*>(s_q + d8 * 8), qb = *reinterpret_cast<const float4*>(s_q + d8 * 8 + 4);
                 acc = fmaf(qa.x, __low2float(k2[0]), acc); acc = fmaf(qa.y, __high2float(k2[0]), acc);
                 acc = fmaf(qa.z, __low2float(k2[1]), acc); acc = fmaf(qa.w, __high2float(k2[1]), acc);
                 acc = fmaf(qb.x, __low2float(k2[2]), acc); acc = fmaf(qb.y, __high2float(k2[2]), acc);
                 acc = fmaf(qb.z, __low2float(k2[3]), acc); acc = fmaf(qb.w, __high2float(k2[3]), acc);
+            }
             }
             sc = acc * a.scale_log2;
         }
@@ -845,19 +854,19 @@ __global__ void __launch_bounds__(128, TAIL_FIRST ? 5 : 4) k_attn_tail_merge_tc(
 #pragma unroll
         for (int of = 16; of > 0; of >>= 1) cl += __shfl_xor_sync(0xffffffffu, cl, of);
         float co[4] = {0.f, 0.f, 0.f, 0.f};
-        // weighted values, keys in position order; the loads of 16 keys are issued before their sums
+        // weighted values, keys in position order; the loads of VB keys are issued before their sums
         // (a key that is not in the chunk reads slot 0 with weight 0 and is skipped)
-        for (int j0 = 0; j0 < 32; j0 += 16) {
-            float pj[16];
-            uint2 vv[16];
+        for (int j0 = 0; j0 < 32; j0 += VB) {
+            float pj[VB];
+            uint2 vv[VB];
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
+            for (int u = 0; u < VB; ++u) {
                 pj[u] = __shfl_sync(0xffffffffu, pe, j0 + u);
                 const int sj = __shfl_sync(0xffffffffu, slot, j0 + u);
                 vv[u] = *reinterpret_cast<const uint2*>(vbase + (size_t)sj * HD + lane * 4);
             }
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
+            for (int u = 0; u < VB; ++u) {
                 if (pj[u] != 0.f) {
                     const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vv[u].x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vv[u].y);
                     co[0] = fmaf(pj[u], __low2float(v01), co[0]); co[1] = fmaf(pj[u], __high2float(v01), co[1]);
@@ -871,24 +880,24 @@ __global__ void __launch_bounds__(128, TAIL_FIRST ? 5 : 4) k_attn_tail_merge_tc(
     if (TAIL_FIRST) { pdl_wait(); request_partials(); }
     float m = -INFINITY, l = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < PB; ++u) {
         if (u < n_sp) {
             const float co[4] = {c40[u].x, c40[u].y, c40[u].z, c40[u].w};
             merge_ml(m, l, o, ml0[u].x, ml0[u].y, co);
         }
     }
-    for (int s0 = 8; s0 < n_sp; s0 += 8) {
-        float2 ml[8];
-        float4 c4[8];
+    for (int s0 = PB; s0 < n_sp; s0 += PB) {
+        float2 ml[PB];
+        float4 c4[PB];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < PB; ++u) {
             if (s0 + u < n_sp) {
                 ml[u] = __ldcg(a.part_ml + base + s0 + u);
                 c4[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (base + s0 + u) * HD + lane * 4));
             }
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < PB; ++u) {
             if (s0 + u < n_sp) {
                 const float co[4] = {c4[u].x, c4[u].y, c4[u].z, c4[u].w};
                 merge_ml(m, l, o, ml[u].x, ml[u].y, co);
@@ -1001,8 +1010,12 @@ int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_la
     // the bulk kernels release their dependent after their own wait: behind them the tail is computed first
     // (plain launches run one after the other: there the partials are requested before the tail instead)
     const dim3 tgrid((rows_cap + 3) / 4, a.Hq, batch);
-    const cudaError_t e = n_split_launch > 0 && pdl ? launch_k(k_attn_tail_merge_tc<true>, tgrid, dim3(128), 0, s, pdl, a)
-                                             : launch_k(k_attn_tail_merge_tc<false>, tgrid, dim3(128), 0, s, pdl, a);
+    // several waves of CTAs launched on their own: the lean instance (measured: 333 against 368 us for 16
+    // sequences of 4k positions; inside a step, where the tail overlaps the bulk kernel, it is the slower one)
+    const bool many = !pdl && (long long)tgrid.x * tgrid.y * tgrid.z > 8 * 148;
+    const cudaError_t e = n_split_launch > 0 && many ? launch_k(k_attn_tail_merge_tc<true, true>, tgrid, dim3(128), 0, s, pdl, a)
+                          : n_split_launch > 0 && pdl ? launch_k(k_attn_tail_merge_tc<true, false>, tgrid, dim3(128), 0, s, pdl, a)
+                                                      : launch_k(k_attn_tail_merge_tc<false, false>, tgrid, dim3(128), 0, s, pdl, a);
     if (e != cudaSuccess) return -1;
     return 0;
 }
