@@ -118,10 +118,19 @@ __device__ __forceinline__ const float* sk_partial(const StreamK& s, int c, int 
 }
 // Sum over the contributors of `tile`, in CTA order, of the four floats at column f of row r.  The loads of up
 // to eight contributors are issued before the first addition (adding the zeros of absent ones changes nothing).
-__device__ __forceinline__ float4 sk_sum4(const StreamK& s, int tile, int r, int f) {
+// A tile's table entry does not change after the plan was built: a consumer may fetch it before it waits for the GEMM.
+struct SkEntry {
+    uint4 e0, e1;
+};
+__device__ __forceinline__ SkEntry sk_entry(const StreamK& s, int tile) {
     const uint4* e = reinterpret_cast<const uint4*>(s.table + tile);
-    const uint4 e0 = __ldg(e), e1 = __ldg(e + 1);
-    const uint32_t w[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
+    SkEntry en;
+    en.e0 = __ldg(e);
+    en.e1 = __ldg(e + 1);
+    return en;
+}
+__device__ __forceinline__ float4 sk_sum4(const StreamK& s, const SkEntry& en, int r, int f) {
+    const uint32_t w[8] = {en.e0.x, en.e0.y, en.e0.z, en.e0.w, en.e1.x, en.e1.y, en.e1.z, en.e1.w};
     const int n = (int)(w[0] & 0xffffu);
     const float* base = s.partials + (size_t)r * TILE_N + f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -144,6 +153,8 @@ __device__ __forceinline__ float4 sk_sum4(const StreamK& s, int tile, int r, int
     }
     return acc;
 }
+
+__device__ __forceinline__ float4 sk_sum4(const StreamK& s, int tile, int r, int f) { return sk_sum4(s, sk_entry(s, tile), r, f); }
 
 // Everything an epilogue may need.  One struct for all variants keeps the
 // GEMM kernels identical across call sites.

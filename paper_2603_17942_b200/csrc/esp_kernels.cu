@@ -112,6 +112,16 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, flo
     // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
     // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
+    // fetched before the wait: the tile's contributor entry and the norm weights of this thread's first four
+    // features (neither changes after initialisation), so that only the partials are loaded behind the wait
+    const int jf = threadIdx.x * 4;
+    SkEntry en0;
+    if (sk.partials && jf < d) en0 = sk_entry(sk, jf / TILE_N);
+    T g0[4];
+    if (jf < d) {
+        if constexpr (sizeof(T) == 2) *reinterpret_cast<uint2*>(g0) = __ldg(reinterpret_cast<const uint2*>(g + jf));
+        else *reinterpret_cast<float4*>(g0) = __ldg(reinterpret_cast<const float4*>(g + jf));
+    }
     pdl_wait();
     const int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
@@ -125,7 +135,8 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, flo
     for (int j = threadIdx.x * 4; j < d; j += STRIDE, ++it) {
         float4 x = *reinterpret_cast<const float4*>(xr + j);
         if (sk.partials) {
-            const float4 acc = sk_sum4(sk, j / TILE_N, seq * sk.seq_rows + r, j % TILE_N);
+            const float4 acc = it == 0 ? sk_sum4(sk, en0, seq * sk.seq_rows + r, j % TILE_N)
+                                       : sk_sum4(sk, j / TILE_N, seq * sk.seq_rows + r, j % TILE_N);
             x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
             *reinterpret_cast<float4*>(xr + j) = x;
         }
@@ -146,7 +157,7 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, flo
         const float xv[4] = {x.x, x.y, x.z, x.w};
         T o[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) o[i] = from_f32<T>(xv[i] * rinv * to_f32(g[j + i]));
+        for (int i = 0; i < 4; ++i) o[i] = from_f32<T>(xv[i] * rinv * to_f32(it == 0 ? g0[i] : g[j + i]));
         if constexpr (sizeof(T) == 2) *reinterpret_cast<uint2*>(yr + j) = *reinterpret_cast<const uint2*>(o);
         else *reinterpret_cast<float4*>(yr + j) = *reinterpret_cast<const float4*>(o);
         if (copy_out) *reinterpret_cast<float4*>(copy_out + (size_t)(seq * RT + r) * d + j) = x;
@@ -162,32 +173,55 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
     // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
     // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
-    pdl_wait();
     typedef __nv_bfloat16 T;
     constexpr int NE = HD / 32;
+    constexpr int half = HD / 2;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hs = blockIdx.x * 4 + warp, r = blockIdx.y, seq = blockIdx.z;   // seq: sequence within this launch
+    // Fetched before the wait, so that only the partials are loaded behind it: the row table (written by an earlier
+    // step), the tile's contributor entry, the rotary factors of the row's position and the norm weights
     const SeqState* st = a.st ? a.st + seq : nullptr;
     const int n_rows = st ? (st->active ? st->n_rows : 0) : a.rows_fixed;
-    if (r >= n_rows || hs >= a.Hq + 2 * a.Hkv) return;
+    const bool work = r < n_rows && hs < a.Hq + 2 * a.Hkv;
     const int pr = seq * RT + r;                 // row in the query buffer
     const int sr = seq * sk.seq_rows + r;        // row in the partials
     const int j0 = hs * HD + lane * NE;          // feature in the concatenated [q | k | v] space
     const int tile = j0 / TILE_N, f = j0 % TILE_N;
+    const int which = hs < a.Hq ? 0 : (hs < a.Hq + a.Hkv ? 1 : 2);
+    const int head = which == 0 ? hs : (which == 1 ? hs - a.Hq : hs - a.Hq - a.Hkv);
+    const int L = st ? st->L : 0;
+    SkEntry en;
+    float cs[NE], sn[NE], gw[NE];
+    if (work) {
+        en = sk_entry(sk, tile);
+        if (which != 2) {
+            const int pos = L + (st ? st->row_depth[r] : r);
+#pragma unroll
+            for (int i = 0; i < NE; ++i) {
+                const int idx = (lane * NE + i) % half;
+                cs[i] = __ldg(a.rope_cos + (size_t)pos * half + idx);
+                sn[i] = __ldg(a.rope_sin + (size_t)pos * half + idx);
+            }
+            if (a.qk_norm) {
+                const T* g = reinterpret_cast<const T*>(which == 0 ? a.q_norm : a.k_norm);
+#pragma unroll
+                for (int i = 0; i < NE; ++i) gw[i] = to_f32(g[lane * NE + i]);
+            }
+        }
+    }
+    pdl_wait();
+    if (!work) return;
     float v[NE];
     if constexpr (NE == 4) {
-        const float4 t = sk_sum4(sk, tile, sr, f);
+        const float4 t = sk_sum4(sk, en, sr, f);
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
     } else {
         // narrower heads: the same sum through the four-float helper on the enclosing aligned group
-        const float4 t = sk_sum4(sk, tile, sr, f & ~3);
+        const float4 t = sk_sum4(sk, en, sr, f & ~3);
         const float tv[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
         for (int i = 0; i < NE; ++i) v[i] = tv[(f & 3) + i];
     }
-    const int which = hs < a.Hq ? 0 : (hs < a.Hq + a.Hkv ? 1 : 2);
-    const int head = which == 0 ? hs : (which == 1 ? hs - a.Hq : hs - a.Hq - a.Hkv);
-    const int L = st ? st->L : 0;
     if (which != 2) {
         if (a.qk_norm) {
             float ss = 0.f;
@@ -195,19 +229,14 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
             for (int i = 0; i < NE; ++i) ss += v[i] * v[i];
             ss = warp_sum(ss);
             const float rinv = 1.0f / sqrtf(ss / (float)HD + a.rms_eps);
-            const T* g = reinterpret_cast<const T*>(which == 0 ? a.q_norm : a.k_norm);
 #pragma unroll
-            for (int i = 0; i < NE; ++i) v[i] = v[i] * rinv * to_f32(g[lane * NE + i]);
+            for (int i = 0; i < NE; ++i) v[i] = v[i] * rinv * gw[i];
         }
-        constexpr int half = HD / 2;
-        const int pos = L + (st ? st->row_depth[r] : r);
         const bool low = lane < 16;
 #pragma unroll
         for (int i = 0; i < NE; ++i) {
             const float other = __shfl_xor_sync(0xffffffffu, v[i], 16);
-            const int idx = (lane * NE + i) % half;
-            const float cs = a.rope_cos[(size_t)pos * half + idx], sn = a.rope_sin[(size_t)pos * half + idx];
-            v[i] = low ? v[i] * cs - other * sn : v[i] * cs + other * sn;
+            v[i] = low ? v[i] * cs[i] - other * sn[i] : v[i] * cs[i] + other * sn[i];
         }
     }
     T* dst;
@@ -227,21 +256,23 @@ __global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, i
     // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
     // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
-    pdl_wait();
-    const int r = blockIdx.y, seq = blockIdx.z;
-    const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;
     // eight features per thread: half the threads, so that the next GEMM's CTA finds registers free beside this
     // kernel's CTAs and can start its weight stream while they run
     const int j0 = (blockIdx.x * 256 + threadIdx.x) * 8;
+    SkEntry en;      // fixed since the plan was built: fetched before the wait (the eight features share a tile)
+    if (j0 < F) en = sk_entry(sk, j0 / 64);
+    pdl_wait();
+    const int r = blockIdx.y, seq = blockIdx.z;
+    const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;
     if (r >= n_rows || j0 >= F) return;
     const int pr = seq * RT + r, sr = seq * sk.seq_rows + r;
     float4 g[2], u[2];
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
-        const int j = j0 + 4 * q, tile = j / 64, f = j % 64;
+        const int j = j0 + 4 * q, f = j % 64;
         if (j >= F) { g[q] = u[q] = make_float4(0.f, 0.f, 0.f, 0.f); continue; }
-        g[q] = sk_sum4(sk, tile, sr, f);
-        u[q] = sk_sum4(sk, tile, sr, 64 + f);
+        g[q] = sk_sum4(sk, en, sr, f);
+        u[q] = sk_sum4(sk, en, sr, 64 + f);
     }
     __nv_bfloat16 o[8];
 #pragma unroll
