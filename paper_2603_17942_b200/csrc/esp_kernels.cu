@@ -122,10 +122,11 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, flo
         if constexpr (sizeof(T) == 2) *reinterpret_cast<uint2*>(g0) = __ldg(reinterpret_cast<const uint2*>(g + jf));
         else *reinterpret_cast<float4*>(g0) = __ldg(reinterpret_cast<const float4*>(g + jf));
     }
-    pdl_wait();
     const int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
-    if (!st->active || r >= st->n_rows) return;
+    const bool idle = !st->active || r >= st->n_rows;     // the row table was written by an earlier step
+    pdl_wait();
+    if (idle) return;
     float* xr = hres + (size_t)(seq * RT + r) * d;
     __shared__ float red[32];
     constexpr int STRIDE = 1024 * 4;
@@ -261,9 +262,9 @@ __global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, i
     const int j0 = (blockIdx.x * 256 + threadIdx.x) * 8;
     SkEntry en;      // fixed since the plan was built: fetched before the wait (the eight features share a tile)
     if (j0 < F) en = sk_entry(sk, j0 / 64);
-    pdl_wait();
     const int r = blockIdx.y, seq = blockIdx.z;
-    const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;
+    const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;   // written by an earlier step
+    pdl_wait();
     if (r >= n_rows || j0 >= F) return;
     const int pr = seq * RT + r, sr = seq * sk.seq_rows + r;
     float4 g[2], u[2];
