@@ -740,11 +740,12 @@ __device__ __forceinline__ int nth_set_bit128(unsigned long long lo, unsigned lo
     return m ? base + __ffsll((long long)m) - 1 : -1;
 }
 __device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], float cm, float cl, const float (&co)[4]) {
+    // products and sums are rounded one by one, so that every instance of the kernel rounds alike
     const float mn = fmaxf(m, cm);
-    const float a = exp2f(m - mn), b = exp2f(cm - mn);
-    l = l * a + cl * b;
+    const float a = exp2f(__fsub_rn(m, mn)), b = exp2f(__fsub_rn(cm, mn));
+    l = __fmaf_rn(l, a, __fmul_rn(cl, b));
 #pragma unroll
-    for (int i = 0; i < 4; ++i) o[i] = o[i] * a + co[i] * b;
+    for (int i = 0; i < 4; ++i) o[i] = __fmaf_rn(o[i], a, __fmul_rn(co[i], b));
     m = mn;
 }
 
