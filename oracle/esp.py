@@ -477,6 +477,22 @@ def call_reduction_percent(tau: float) -> float:
     return 100.0 * (1.0 - 1.0 / tau)
 
 
+def draft_source(tree: Tree, blk: Block, path: Sequence[int], spec: SpecCfg) -> Tuple[int, int, List[int]]:
+    """Which mask rows of the block just verified feed which depth of the next tree (Section 2: mask i
+    elicits the token i+1 positions ahead; Appendix E position ids).
+
+    u* is the deepest anchored node on the accepted path p_0..p_a.  Its probe j sits at pos(u*) + j and
+    predicts the token at pos(u*) + j + 1.  The next root sits at L + a + 1, so depth i of the next tree
+    is the token at L + a + 1 + i: it needs probe j = delta + i with delta = a - depth(u*).  Returns
+    (u*, delta, rows) with rows[i-1] the block row that proposes depth i, i = 1..k-delta.
+    """
+    a = len(path) - 1
+    ustar = max(p for p in path if p in blk.anchors)
+    delta = a - int(tree.depths[ustar])
+    rows = [blk.probe_row[(ustar, j)] for j in range(delta + 1, spec.n_probes + 1)]
+    return ustar, delta, rows
+
+
 def next_tree(root_token: int, cand_ids, cand_logits, lses, spec: SpecCfg) -> Tree:
     """The tree the next step verifies: Algorithm 1, or the fixed-width tree when spec.static_widths is set."""
     if spec.static_widths:
@@ -561,8 +577,10 @@ class EspOracle:
             self.m = mask_update(self.m, self.model.embed(y), sp.lam)
         ids, vals, lses = self._probe_lists(logits, range(t, t + k))
         self.tree = next_tree(y, ids, vals, lses, sp) if k else root_only(y)
+        rec = {"kind": "prefill", "first": y, "L_after": t, "probe_pos": list(range(t, t + k))}
         if self.keep_logits:
-            self.log.append({"kind": "prefill", "logits": logits[t - 1:].copy(), "first": y})
+            rec["logits"] = logits[t - 1:].copy()
+        self.log.append(rec)
         return y
 
     # -- one decode-and-verify step (Figure 1 right)
@@ -587,16 +605,15 @@ class EspOracle:
             self._emit(y)
         if not sp.ema_per_token:
             self.m = mask_update(self.m, self.model.embed(out[-1]), sp.lam)
-        # next proposals come from the mask chain of the deepest anchored node on the accepted path;
-        # probe j of node u predicts position pos(u)+j+1, so depth i of the next tree needs j = delta+i
+        # next proposals come from the mask chain of the deepest anchored node on the accepted path
         ids = vals = lses = ()
+        rows: List[int] = []
         if k:
-            ustar = max(p for p in path if p in blk.anchors)
-            delta = a - int(tree.depths[ustar])
-            rows = [blk.probe_row[(ustar, j)] for j in range(delta + 1, k + 1)]
+            _, _, rows = draft_source(tree, blk, path, sp)
             ids, vals, lses = self._probe_lists(logits, rows)
         rec = {"kind": "step", "tree": tree, "block": blk, "next_of_node": nxt, "path": path, "emitted": out,
-               "cand_ids": ids, "cand_vals": vals, "lses": lses}
+               "cand_ids": ids, "cand_vals": vals, "lses": lses, "L_after": self.L,
+               "probe_pos": [int(pos[r]) for r in rows]}
         if self.keep_logits:
             rec["logits"] = logits
         self.log.append(rec)

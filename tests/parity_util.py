@@ -186,9 +186,7 @@ class ParityRun:
         np.testing.assert_allclose(st["mask_vec"], self.m, rtol=0, atol=2e-6 * max(1.0, float(np.abs(self.m).max())))
         ids = vals = lses = ()
         if k:
-            ustar = max(p for p in path if p in blk.anchors)
-            delta = a - int(tree.depths[ustar])
-            rows = [blk.probe_row[(ustar, j)] for j in range(delta + 1, k + 1)]
+            _, _, rows = O.draft_source(tree, blk, path, sp)   # pinned by the position-predictor test of the oracle
             kp = sp.k_prime
             ids = [st["topk_ids"][r, :kp] for r in rows]
             vals = [st["topk_vals"][r, :kp] for r in rows]

@@ -439,3 +439,89 @@ def test_sample_matching_is_lossless_token_by_token(W, n_anchor, temperature):
 def dataclasses_replace(spec, **kw):
     import dataclasses
     return dataclasses.replace(spec, **kw)
+
+
+# ---------------------------------------------------------------- which mask row proposes which depth (Section 2; Appendix E)
+class _PositionPredictor:
+    """Stand-in for the frozen model with a known answer at every position: whatever a row holds, a row at
+    position p puts token g(p + 1) first (and g(p + 1) + 1, ... after it).  Section 2 says mask i elicits the
+    token i + 1 positions ahead, i.e. a mask row at position p proposes the token of position p + 1: under
+    this model every drafted node is right exactly when each depth of the tree was drawn from the mask row one
+    position before it, and the walk then accepts the whole tree."""
+
+    def __init__(self, vocab=61, d=4):
+        self.V, self.d, self.n_layers = vocab, d, 1
+        self.calls = []
+
+    def g(self, p):          # token at position p; consecutive tokens differ, so the pruner never removes a right draft
+        return (7 * p + 3) % self.V
+
+    def embed(self, token):
+        return np.full(self.d, float(token), np.float32)
+
+    def new_cache(self, cap):
+        z = np.zeros((1, cap, 1, 1), np.float32)
+        return z, z.copy()
+
+    def block_forward(self, kc, vc, L, x, pos, vis, want=None, need_hidden=False):
+        M = len(pos)
+        self.calls.append([int(p) for p in pos])
+        logits = np.zeros((M, self.V), np.float32)
+        for r in range(M):
+            first = self.g(int(pos[r]) + 1)
+            for j in range(self.V):
+                logits[r, (first + j) % self.V] = -0.5 * j
+        kb = np.zeros((1, M, 1, 1), np.float32)
+        return logits, kb, kb.copy(), None
+
+
+@pytest.mark.parametrize("n_anchor,k", [(0, 3), (1, 3), (2, 4), (0, 1)])
+def test_mask_rows_feed_the_depth_one_position_ahead(n_anchor, k):
+    model = _PositionPredictor()
+    t = 9
+    prompt = [model.g(p) for p in range(t)]
+    spec = esp.SpecCfg(n_probes=k, topk=3, max_nodes=3 * k + 1, expand_width=1, n_anchor=n_anchor)
+    dec = esp.EspOracle(model, spec, 256)
+    out = dec.generate(prompt, 40)
+    assert out == [model.g(p) for p in range(t, t + 40)]
+    # position identity, every record: the row proposing depth i of the next tree sits at (new L) + i - 1
+    for rec in dec.log:
+        assert rec["probe_pos"] == [rec["L_after"] + i - 1 for i in range(1, len(rec["probe_pos"]) + 1)], rec["kind"]
+    assert dec.log[0]["probe_pos"] == [t + j - 1 for j in range(1, k + 1)]          # prefill: mask j at t + j - 1
+    # behaviour: each step accepts every depth it drafted.  Paper mode (all nodes anchored): k per step.
+    # Fewer anchors: the chain behind the deepest anchored accepted node has k - delta rows left.
+    steps = [r for r in dec.log if r["kind"] == "step"]
+    drafted = [int(r["tree"].depths.max()) for r in steps]
+    assert dec.accept_hist == drafted
+    if n_anchor == 0:
+        assert all(a == k for a in dec.accept_hist)
+    else:
+        assert max(dec.accept_hist) == k and any(len(r["probe_pos"]) < k for r in steps)   # delta > 0 occurs
+
+
+def test_a_shifted_mask_row_choice_is_caught():
+    """Negative control for the pin above: feeding depth i from the row one further along the chain (delta
+    off by one) or from the chain in reverse order drafts wrong tokens under the position predictor."""
+    model = _PositionPredictor()
+    t, k = 9, 3
+    prompt = [model.g(p) for p in range(t)]
+    spec = esp.SpecCfg(n_probes=k, topk=3, max_nodes=3 * k + 1, expand_width=1, n_anchor=0)
+    for wrong in ("shift", "reverse"):
+        dec = esp.EspOracle(model, spec, 256)
+        dec.prefill(prompt)
+        tree, blk = dec.tree, esp.layout_block(dec.tree, spec)
+        pos = dec.L + blk.row_pos_off
+        logits, _, _, _ = model.block_forward(None, None, dec.L, None, pos, blk.vis)
+        nxt = [int(np.argmax(logits[r])) for r in range(blk.n_nodes)]
+        path, emitted = esp.verify_walk(tree, nxt)
+        _, _, rows = esp.draft_source(tree, blk, path, spec)
+        bad = rows[1:] if wrong == "shift" else rows[::-1]
+        lists = [esp.topk_desc(logits[r], spec.k_prime) for r in bad]
+        nt = esp.build_tree(emitted[-1], [l[0] for l in lists], [l[1] for l in lists],
+                            [esp.log_sum_exp(logits[r]) for r in bad], spec)
+        L_new = dec.L + len(path)
+        right = esp.build_tree(emitted[-1], *zip(*[(esp.topk_desc(logits[r], spec.k_prime)[0], esp.topk_desc(logits[r], spec.k_prime)[1],
+                                                    esp.log_sum_exp(logits[r])) for r in rows]), spec)
+        top = lambda tr: [int(tr.tokens[i]) for i in range(1, tr.n) if tr.logp[i] == max(tr.logp[j] for j in range(tr.n) if tr.depths[j] == tr.depths[i])]
+        assert top(right)[:2] == [model.g(L_new + 1), model.g(L_new + 2)]
+        assert top(nt)[:1] != [model.g(L_new + 1)]
