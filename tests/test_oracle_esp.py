@@ -250,7 +250,7 @@ def test_esp_output_equals_greedy_decoding(W, n_anchor, prune):
     assert len(set(ref)) > 5                      # not a degenerate constant stream
     assert 1.0 <= dec.tau <= spec.n_probes + 1    # at most k drafts + the bonus token per call
     assert sum(a + 1 for a in dec.accept_hist) == len(dec.emitted) - 1
-    for rec in dec.log:
+    for rec in (r for r in dec.log if r["kind"] == "step"):
         _check_tree_invariants(rec["tree"], spec)
         expect_rows = (spec.n_probes + 1) * rec["tree"].n if n_anchor == 0 else rec["tree"].n + spec.n_probes
         assert rec["block"].m == expect_rows
