@@ -27,26 +27,21 @@
 // DEV_E_WAIT_TIMEOUT, frees its tensor memory and returns.
 #include <new>
 #include <string.h>
+#include <new>
+#include <string.h>
 
-#include "esp_launch.h"
-#include "esp_tc.cuh"
+#include "esp_attn_tc.cuh"
 
 namespace esp {
 
 namespace {
 
 using namespace tc;
+using namespace attn;
 
-constexpr int HD = 128;
-constexpr int CK = 128;                   // keys per chunk
-constexpr int MP = 128;                   // (row, head) pairs per CTA
-constexpr int HALF_BYTES = 128 * 128;     // one 128-row x 64-element (128-byte) swizzled tile
-constexpr int Q_BYTES = 2 * HALF_BYTES, K_BYTES = 2 * HALF_BYTES, V_BYTES = 2 * HALF_BYTES, P_BYTES = 2 * HALF_BYTES;
-constexpr int KV_STAGE = K_BYTES + V_BYTES;
 constexpr int STG_BYTES = 4 * 32 * 128;     // output staging: 32 rows x 128 bytes for each of the 4 output warps
-constexpr int OFF_Q = 0, OFF_KV = Q_BYTES, OFF_P = OFF_KV + 2 * KV_STAGE, OFF_STG = OFF_P + P_BYTES, OFF_BAR = OFF_STG + STG_BYTES;
+constexpr int OFF_STG = OFF_P + P_BYTES, OFF_BAR = OFF_STG + STG_BYTES;
 constexpr size_t SMEM_BYTES = 1024 + OFF_BAR + 256;
-constexpr int TMEM_COLS = 512;            // S0 at 0, S1 at 128, O0 at 256, O1 at 384
 constexpr int MAX_T0_ENTRIES = 256;       // sequences x row tiles one launch may cover
 constexpr int NUM_THREADS = 448;           // producer warp, MMA warp, 8 softmax warps, 4 output warps
 
@@ -59,95 +54,73 @@ struct BulkParams {
     int32_t n_splits, n_seq, seq0;   // work items of this launch: n_splits x KV heads x row tiles x sequences [seq0, seq0 + n_seq)
 };
 
-__device__ __forceinline__ int tail_start_tc(int P, int dcap) {
-    int t = P - dcap;
-    return t <= 0 ? 0 : (t / 16) * 16;
-}
-
-// kind::f16 instruction descriptors: D = f32, A = B = bf16, M = 128, N = 128; PV takes B (V) MN-major
-constexpr uint32_t IDESC_QK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-constexpr uint32_t IDESC_PV = IDESC_QK | (1u << 16);
-
-// 64 consecutive columns of this lane: two loads in flight, one wait
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
-    tmem_ld32_issue(taddr, &r[0]);
-    tmem_ld32_issue(taddr + 32, &r[32]);
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
 // ---- one item per CTA (grid = splits x (KV heads x row tiles) x sequences): used when the launch has at most
 // about one and a half items per SM, where start-up latency is all that counts.
 constexpr int ONCE_THREADS = 320;          // producer warp, MMA warp, 8 softmax warps (they also write the output)
-constexpr int ONCE_OFF_BAR = OFF_P + P_BYTES;
+constexpr int ONCE_OFF_BAR = ITEM_BYTES;
 constexpr size_t ONCE_SMEM_BYTES = 1024 + ONCE_OFF_BAR + 256;
-
-// The producer thread waits for the kernel before this one and only then releases the kernel after it.
-__device__ __forceinline__ void trigger_after_wait() {
-    pdl_wait();
-    pdl_launch_dependents();
-}
 
 __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __grid_constant__ BulkParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ int s_T0max;
     __shared__ float s_xchg[2][2 * MP];   // [exchange parity][half][pair]
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + ONCE_OFF_BAR);   // [2]
-    uint64_t* kv_empty = kv_full + 2;                                  // [2]
-    uint64_t* s_full = kv_empty + 2;                                   // [2]
-    uint64_t* q_full = s_full + 2;
-    uint64_t* p_ready = q_full + 1;
-    uint64_t* pv_done = p_ready + 1;
-    uint64_t* xchg = pv_done + 1;                                      // the two threads of a pair exchanged a value
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(xchg + 1);
-    volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+    BulkShared sm;
+    sm.buf = smem;
+    sm.kv_full = reinterpret_cast<uint64_t*>(smem + ONCE_OFF_BAR);   // [2]
+    sm.kv_empty = sm.kv_full + 2;                                    // [2]
+    sm.s_full = sm.kv_empty + 2;                                     // [2]
+    sm.q_full = sm.s_full + 2;
+    sm.p_ready = sm.q_full + 1;
+    sm.pv_done = sm.p_ready + 1;
+    sm.xchg = sm.pv_done + 1;                                        // the two threads of a pair exchanged a value
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm.xchg + 1);
+    sm.s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+    sm.s_xchg = &s_xchg[0][0];
 
     const AttnArgs& a = p.a;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int split = blockIdx.x;
-    const int kvh = blockIdx.y / p.n_row_tiles, rtile = blockIdx.y % p.n_row_tiles;
-    const int seq = blockIdx.z;
+    BulkItem it;
+    it.split = blockIdx.x;
+    it.kvh = blockIdx.y / p.n_row_tiles;
+    const int rtile = blockIdx.y % p.n_row_tiles;
+    it.seq = blockIdx.z;
 
     // Read before pdl_wait(): the sequence state and the cache below T0, both written by earlier steps.
     // The tail kernel is released only after this kernel's wait has returned (trigger_after_wait), so that it may
     // work on this step's queries and keys while the CTAs here are still running.
-    int n_rows, L;
     if (a.st) {
-        const SeqState* st = a.st + seq;
-        n_rows = st->active ? st->n_rows : 0;
-        L = st->L;
+        const SeqState* st = a.st + it.seq;
+        it.n_rows = st->active ? st->n_rows : 0;
+        it.L = st->L;
     } else {
-        n_rows = a.n_rows_fixed;
-        L = a.L_fixed;
+        it.n_rows = a.n_rows_fixed;
+        it.L = a.L_fixed;
     }
-    const int row0 = rtile * p.rows_per_tile;
-    if (row0 >= n_rows) { pdl_wait(); return; }
+    it.row0 = rtile * p.rows_per_tile;
+    if (it.row0 >= it.n_rows) { pdl_wait(); return; }
     if (warp == 2) {
         int t0 = 0;
-        for (int r = row0 + lane; r < row0 + p.rows_per_tile && r < n_rows; r += 32) {
-            const int depth = a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r];
-            t0 = max(t0, tail_start_tc(L + depth, a.dcap));
+        for (int r = it.row0 + lane; r < it.row0 + p.rows_per_tile && r < it.n_rows; r += 32) {
+            const int depth = a.st ? a.st[it.seq].row_depth[r] : a.depth[it.seq * RT + r];
+            t0 = max(t0, tail_start_tc(it.L + depth, a.dcap));
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) t0 = max(t0, __shfl_xor_sync(0xffffffffu, t0, o));
         if (lane == 0) s_T0max = t0;
     }
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 2; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); mbar_init(&s_full[i], 1); }
-        mbar_init(q_full, 1);
-        mbar_init(p_ready, 256);
-        mbar_init(pv_done, 1);
-        mbar_init(xchg, 256);
-        *s_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        bulk_init_barriers(sm);
+        *sm.s_abort = 0;
     }
     __syncthreads();
     const int T0max = s_T0max;
     const int n_bulk = (T0max + a.split_len - 1) / a.split_len;
-    if (split >= n_bulk) { pdl_wait(); return; }     // block-uniform: nobody holds tensor memory yet
-    const int beg = split * a.split_len;
-    const int end = min(beg + a.split_len, T0max);
-    const int n_chunks = (end - beg + CK - 1) / CK;
+    if (it.split >= n_bulk) { pdl_wait(); return; }     // block-uniform: nobody holds tensor memory yet
+    it.beg = it.split * a.split_len;
+    const int end = min(it.beg + a.split_len, T0max);
+    it.n_chunks = (end - it.beg + CK - 1) / CK;
+    it.kv_row0 = (it.seq * a.Hkv + it.kvh) * a.cap;
 
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
@@ -157,202 +130,13 @@ __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __g
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *s_tmem;
-    unsigned char* sQ = smem + OFF_Q;
-    unsigned char* sP = smem + OFF_P;
-
-    if (warp == 0) {
-        // ---------------- TMA producer
-        if (lane == 0) {
-            const int kvrow0 = (seq * a.Hkv + kvh) * a.cap + beg;
-            bool ok = true;
-            auto load_chunk = [&](int c) {
-                unsigned char* st = smem + OFF_KV + (c & 1) * KV_STAGE;
-                mbar_expect_tx(&kv_full[c & 1], KV_STAGE);
-                tma_load_2d(st, &p.map_k, 0, kvrow0 + c * CK, &kv_full[c & 1]);
-                tma_load_2d(st + HALF_BYTES, &p.map_k, 64, kvrow0 + c * CK, &kv_full[c & 1]);
-                tma_load_2d(st + K_BYTES, &p.map_v, 0, kvrow0 + c * CK, &kv_full[c & 1]);
-                tma_load_2d(st + K_BYTES + HALF_BYTES, &p.map_v, 64, kvrow0 + c * CK, &kv_full[c & 1]);
-            };
-            // the cache below T0 is settled in a decode step: request it before waiting for the kernel that wrote the queries
-            if (a.cache_in_flight) trigger_after_wait();
-            for (int c = 0; c < n_chunks && c < 2; ++c) load_chunk(c);
-            if (!a.cache_in_flight) trigger_after_wait();
-            mbar_expect_tx(q_full, Q_BYTES);
-            tma_load_3d(sQ, &p.map_q, 0, kvh * p.group, seq * RT + row0, q_full);
-            tma_load_3d(sQ + HALF_BYTES, &p.map_q, 64, kvh * p.group, seq * RT + row0, q_full);
-            for (int c = 2; c < n_chunks && ok; ++c) {
-                if (!mbar_wait(&kv_empty[c & 1], ((c >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
-                load_chunk(c);
-            }
-            if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
-        }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer
-        if (lane == 0) {
-            bool ok = true;
-            const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
-            auto issue_qk = [&](int c) {
-                const uint32_t k_addr = smem_u32(smem + OFF_KV + (c & 1) * KV_STAGE);
-                const uint32_t tmem_s = tmem_base + (c & 1) * 128;
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                    umma(tmem_s, smem_desc(q_addr + off, 16), smem_desc(k_addr + off, 16), IDESC_QK, kk > 0 ? 1u : 0u);
-                }
-                umma_commit(&s_full[c & 1]);
-            };
-            ok = mbar_wait(q_full, 0, s_abort) && mbar_wait(&kv_full[0], 0, s_abort);
-            if (ok) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                issue_qk(0);
-            }
-            for (int c = 0; c < n_chunks && ok; ++c) {
-                if (c + 1 < n_chunks) {     // S of the next chunk while the softmax of this one runs
-                    if (!mbar_wait(&kv_full[(c + 1) & 1], ((c + 1) >> 1) & 1, s_abort)) { ok = false; break; }
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    issue_qk(c + 1);
-                }
-                if (!mbar_wait(p_ready, c & 1, s_abort)) { ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t v_addr = smem_u32(smem + OFF_KV + (c & 1) * KV_STAGE + K_BYTES);
-#pragma unroll
-                for (int kk = 0; kk < CK / 16; ++kk) {
-                    const uint32_t p_off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;     // P: K-major over keys
-                    const uint32_t v_off = kk * 16 * 128;                              // V: 16 key rows of 128 bytes further
-                    umma(tmem_base + 256, smem_desc(p_addr + p_off, 16), smem_desc(v_addr + v_off, HALF_BYTES), IDESC_PV,
-                         (c > 0 || kk > 0) ? 1u : 0u);
-                }
-                umma_commit(pv_done);
-                umma_commit(&kv_empty[c & 1]);
-            }
-            if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
-        }
-    } else {
-        // ---------------- softmax warps 2..9: a thread owns one pair (= tensor-memory lane) and one half of the
-        // chunk's 128 keys (warps 2-5 keys 0..63, warps 6-9 keys 64..127); the two threads of a pair exchange
-        // their maxima (per chunk) and their sums (at the end) through shared memory
-        const int q4 = warp & 3;
-        const int hf = (warp - 2) >> 2;
-        const int pair = q4 * 32 + lane;
-        const int r = row0 + pair / p.group, head = kvh * p.group + pair % p.group;
-        const bool pv = pair / p.group < p.rows_per_tile && r < n_rows && r < RT;
-        int T0row = 0;
-        if (pv) T0row = tail_start_tc(L + (a.st ? a.st[seq].row_depth[r] : a.depth[seq * RT + r]), a.dcap);
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16) + hf * 64;   // this thread's 64 columns of S / O
-        float m_run = -INFINITY, l_run = 0.f;
-        bool ok = true;
-        for (int c = 0; c < n_chunks && ok; ++c) {
-            // (a wait that fails must take the whole warp out: the tensor-memory accesses below are warp-wide)
-            if (!__all_sync(0xffffffffu, mbar_wait(&s_full[c & 1], (c >> 1) & 1, s_abort))) { ok = false; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t s_addr = lane_addr + (c & 1) * 128;
-            const int cbase = beg + c * CK + hf * 64;
-            // the row's scores for this half, masked to its visible keys and scaled to the log2 domain
-            uint32_t sv[64];
-            tmem_ld64(s_addr, sv);
-            float cmax = -INFINITY;
-            if (__all_sync(0xffffffffu, cbase + 64 <= T0row)) {     // every key of the half is visible to every row of the warp
-#pragma unroll
-                for (int i = 0; i < 64; ++i) {
-                    const float sc = __uint_as_float(sv[i]) * a.scale_log2;
-                    sv[i] = __float_as_uint(sc);
-                    cmax = fmaxf(cmax, sc);
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 64; ++i) {
-                    const float sc = cbase + i < T0row ? __uint_as_float(sv[i]) * a.scale_log2 : -INFINITY;
-                    sv[i] = __float_as_uint(sc);
-                    cmax = fmaxf(cmax, sc);
-                }
-            }
-            // the chunk maximum over both halves
-            // (double buffered by exchange parity: a thread can be one exchange ahead of its partner, not two)
-            s_xchg[c & 1][hf * MP + pair] = cmax;
-            mbar_arrive(xchg);
-            if (!__all_sync(0xffffffffu, mbar_wait(xchg, c & 1, s_abort))) { ok = false; break; }
-            cmax = fmaxf(s_xchg[c & 1][pair], s_xchg[c & 1][MP + pair]);
-            const float m_new = fmaxf(m_run, cmax);
-            const float m_use = m_new == -INFINITY ? 0.f : m_new;
-            const float alpha = exp2f(m_run - m_use);
-            // P of the previous chunk must have been consumed before it is overwritten, and O must be final
-            // before it is rescaled
-            if (c > 0 && !__all_sync(0xffffffffu, mbar_wait(pv_done, (c - 1) & 1, s_abort))) { ok = false; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // probabilities, their sum (key order), P as bf16 in the A-operand layout (this half = one swizzled tile)
-            float csum = 0.f;
-            unsigned char* prow = sP + hf * HALF_BYTES + pair * 128;
-#pragma unroll
-            for (int blk = 0; blk < 2; ++blk) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float p0 = exp2f(__uint_as_float(sv[blk * 32 + i]) - m_use), p1 = exp2f(__uint_as_float(sv[blk * 32 + i + 1]) - m_use);
-                    csum += p0;
-                    csum += p1;
-                    const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int chunk16 = blk * 4 + j;
-                    *reinterpret_cast<uint4*>(prow + ((chunk16 ^ (pair & 7)) << 4)) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                }
-            }
-            if (c > 0) {
-                // O <- alpha * O (in tensor memory), this thread's 64 of the 128 columns
-                if (__any_sync(0xffffffffu, alpha != 1.0f)) {   // warp-uniform: skip when no lane's maximum moved
-                    tmem_ld64(lane_addr + 256, sv);
-#pragma unroll
-                    for (int blk = 0; blk < 2; ++blk) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) sv[blk * 32 + i] = __float_as_uint(__uint_as_float(sv[blk * 32 + i]) * alpha);
-                        tmem_st32(lane_addr + 256 + blk * 32, *reinterpret_cast<const uint32_t(*)[32]>(&sv[blk * 32]));
-                    }
-                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                }
-            }
-            l_run = l_run * alpha + csum;     // this half's share of the row sum
-            m_run = m_new;
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes -> tensor-core reads
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            mbar_arrive(p_ready);
-        }
-        if (ok && !__all_sync(0xffffffffu, mbar_wait(pv_done, (n_chunks - 1) & 1, s_abort))) ok = false;
-        if (ok) {
-            // the row sum = first half's share + second half's share
-            s_xchg[n_chunks & 1][hf * MP + pair] = l_run;
-            mbar_arrive(xchg);
-            if (!__all_sync(0xffffffffu, mbar_wait(xchg, n_chunks & 1, s_abort))) ok = false;
-        }
-        if (ok) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // O half-row -> shared memory (the K/V stages are free now) -> one 256-byte bulk copy per thread.  The
-            // tensor-memory load is warp-wide: every lane takes part, lanes without a pair copy nothing.
-            uint32_t ov[64];
-            tmem_ld64(lane_addr + 256, ov);
-            float* orow = reinterpret_cast<float*>(smem + OFF_KV) + pair * (HD + 4) + hf * 64;   // rows padded by 16 bytes: no bank conflicts
-#pragma unroll
-            for (int i = 0; i < 64; i += 4)
-                *reinterpret_cast<uint4*>(orow + i) = make_uint4(ov[i], ov[i + 1], ov[i + 2], ov[i + 3]);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            if (pv) {
-                const size_t idx = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max + split;
-                if (hf == 0) a.part_ml[idx] = make_float2(m_run, s_xchg[n_chunks & 1][pair] + s_xchg[n_chunks & 1][MP + pair]);
-                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                             ::"l"(a.part_o + idx * HD + hf * 64), "r"(smem_u32(orow)), "r"(64 * 4) : "memory");
-            }
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");        // copies complete: shared memory may be released
-        } else if (lane == 0) {
-            set_error(a.err, DEV_E_WAIT_TIMEOUT);
-            *s_abort = 1;
-        }
-    }
+    BulkMaps mp;
+    mp.q = &p.map_q; mp.k = &p.map_k; mp.v = &p.map_v; mp.group = p.group; mp.rows_per_tile = p.rows_per_tile;
+    bulk_item_roles<true>(mp, a, it, sm, tmem_base, warp, lane);
     // ---------------- teardown (every thread arrives here)
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (*s_abort) {
+    if (*sm.s_abort) {
         for (int i = 0; i < 64; ++i) __nanosleep(10000);   // let copies in flight land before shared memory goes away
     }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -573,79 +357,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                 // (a wait that fails must take the whole warp out: the tensor-memory accesses below are warp-wide)
                 if (!__all_sync(0xffffffffu, mbar_wait(&s_full[g & 1], (g >> 1) & 1, s_abort))) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t s_addr = lane_addr + (g & 1) * 128;
-                const int cbase = it.beg + c * CK + hf * 64;
-                // the row's scores for this half, masked to its visible keys and scaled to the log2 domain
-                uint32_t sv[64];
-                tmem_ld64(s_addr, sv);
-                float cmax = -INFINITY;
-                if (__all_sync(0xffffffffu, cbase + 64 <= T0row)) {     // every key of the half is visible to every row of the warp
-#pragma unroll
-                    for (int i = 0; i < 64; ++i) {
-                        const float sc = __uint_as_float(sv[i]) * a.scale_log2;
-                        sv[i] = __float_as_uint(sc);
-                        cmax = fmaxf(cmax, sc);
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 64; ++i) {
-                        const float sc = cbase + i < T0row ? __uint_as_float(sv[i]) * a.scale_log2 : -INFINITY;
-                        sv[i] = __float_as_uint(sc);
-                        cmax = fmaxf(cmax, sc);
-                    }
-                }
-                // the chunk maximum over both halves
-                // (double buffered by exchange parity: a thread can be one exchange ahead of its partner, not two)
-                s_xchg[xc & 1][hf * MP + pair] = cmax;
-                mbar_arrive(xchg);
-                if (!__all_sync(0xffffffffu, mbar_wait(xchg, xc & 1, s_abort))) { ok = false; break; }
-                cmax = fmaxf(s_xchg[xc & 1][pair], s_xchg[xc & 1][MP + pair]);
+                ok = softmax_chunk(lane_addr + (g & 1) * 128, o_addr, it.beg + c * CK + hf * 64, T0row, a.scale_log2, m_run, l_run,
+                                   &s_xchg[xc & 1][0], xchg, xc & 1, g > 0, pv_done, (g - 1) & 1, c > 0,
+                                   sP + hf * HALF_BYTES + pair * 128, pair, hf, p_ready, s_abort);
                 ++xc;
-                const float m_new = fmaxf(m_run, cmax);
-                const float m_use = m_new == -INFINITY ? 0.f : m_new;
-                const float alpha = exp2f(m_run - m_use);
-                // P of the previous chunk must have been consumed before it is overwritten, and O must be final
-                // before it is rescaled
-                if (g > 0 && !__all_sync(0xffffffffu, mbar_wait(pv_done, (g - 1) & 1, s_abort))) { ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                // probabilities, their sum (key order), P as bf16 in the A-operand layout (this half = one swizzled tile)
-                float csum = 0.f;
-                unsigned char* prow = sP + hf * HALF_BYTES + pair * 128;
-#pragma unroll
-                for (int blk = 0; blk < 2; ++blk) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float p0 = exp2f(__uint_as_float(sv[blk * 32 + i]) - m_use), p1 = exp2f(__uint_as_float(sv[blk * 32 + i + 1]) - m_use);
-                        csum += p0;
-                        csum += p1;
-                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-                        pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int chunk16 = blk * 4 + j;
-                        *reinterpret_cast<uint4*>(prow + ((chunk16 ^ (pair & 7)) << 4)) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                    }
-                }
-                if (c > 0) {
-                    // O <- alpha * O (in tensor memory), this thread's 64 of the 128 columns
-                    if (__any_sync(0xffffffffu, alpha != 1.0f)) {   // warp-uniform: skip when no lane's maximum moved
-                        tmem_ld64(o_addr, sv);
-#pragma unroll
-                        for (int blk = 0; blk < 2; ++blk) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) sv[blk * 32 + i] = __float_as_uint(__uint_as_float(sv[blk * 32 + i]) * alpha);
-                            tmem_st32(o_addr + blk * 32, *reinterpret_cast<const uint32_t(*)[32]>(&sv[blk * 32]));
-                        }
-                        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                    }
-                }
-                l_run = l_run * alpha + csum;     // this half's share of the row sum
-                m_run = m_new;
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes -> tensor-core reads
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                mbar_arrive(p_ready);
             }
             if (!ok) break;
             gc += it.n_chunks;
@@ -653,9 +368,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
             s_xchg[xc & 1][hf * MP + pair] = l_run;
             mbar_arrive(xchg);
             if (!__all_sync(0xffffffffu, mbar_wait(xchg, xc & 1, s_abort))) { ok = false; break; }
-            const float l_tot = s_xchg[xc & 1][pair] + s_xchg[xc & 1][MP + pair];
+            const float l_tot = __fadd_rn(s_xchg[xc & 1][pair], s_xchg[xc & 1][MP + pair]);
             ++xc;
-            if (pv && hf == 0) a.part_ml[((size_t)(it.seq * RT + r) * a.Hq + head) * a.n_split_max + it.split] = make_float2(m_run, l_tot);
+            if (pv && hf == 0) __stcg(a.part_ml + ((size_t)(it.seq * RT + r) * a.Hq + head) * a.n_split_max + it.split, make_float2(m_run, l_tot));
             ++n_it;
         }
         if (!ok && lane == 0) {
@@ -729,28 +444,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
-
-// ---- tail + merge: one warp per (row, head) pair
-__device__ __forceinline__ int nth_set_bit128(unsigned long long lo, unsigned long long hi, int n) {
-    int c = __popcll(lo);
-    unsigned long long m = lo;
-    int base = 0;
-    if (n >= c) { n -= c; m = hi; base = 64; }
-    for (int i = 0; i < n; ++i) m &= m - 1;
-    return m ? base + __ffsll((long long)m) - 1 : -1;
-}
-__device__ __forceinline__ void merge_ml(float& m, float& l, float (&o)[4], float cm, float cl, const float (&co)[4]) {
-    // products and sums are rounded one by one, so that every instance of the kernel rounds alike
-    const float mn = fmaxf(m, cm);
-    const float a = exp2f(__fsub_rn(m, mn)), b = exp2f(__fsub_rn(cm, mn));
-    l = __fmaf_rn(l, a, __fmul_rn(cl, b));
-#pragma unroll
-    for (int i = 0; i < 4; ++i) o[i] = __fmaf_rn(o[i], a, __fmul_rn(co[i], b));
-    m = mn;
-}
-
-// The tail: positions T0..P in position order, lane j owns key j of a 32-key chunk (chunk grid anchored at T0).
-// Then the merge: bulk partials in split order, the tail last; a lane owns 4 of the 128 output dims.
+// ---- tail + merge: one warp per (row, head) pair (tail_pair, merge_pair).
 // TAIL_FIRST: launched behind a bulk kernel with programmatic dependent launch (see below).  LEAN: smaller load
 // batches and 64 registers, eight CTAs per SM, for grids of many waves where occupancy counts for more than one
 // warp's latency.  All instances add in the same order and give the same bits.
@@ -762,157 +456,32 @@ __global__ void __launch_bounds__(128, LEAN ? 8 : (TAIL_FIRST ? 5 : 4)) k_attn_t
     __shared__ float s_qall[4][HD];
     if (threadIdx.x == 0) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int r = blockIdx.x * 4 + warp, head = blockIdx.y, seq = blockIdx.z;
+    PairCtx c;
+    c.r = blockIdx.x * 4 + warp; c.head = blockIdx.y; c.seq = blockIdx.z;
+    c.depth = 0; c.lo = 0; c.hi = 0;
     // the sequence state was written by an earlier step; everything else is read after the wait
-    int n_rows, L, depth = 0;
-    unsigned long long lo = 0, hi = 0;
+    int n_rows;
     if (a.st) {
-        const SeqState* st = a.st + seq;
+        const SeqState* st = a.st + c.seq;
         n_rows = st->active ? st->n_rows : 0;
-        L = st->L;
-        if (r < n_rows) { depth = st->row_depth[r]; lo = st->row_anc[r][0]; hi = st->row_anc[r][1]; }
+        c.L = st->L;
+        if (c.r < n_rows) { c.depth = st->row_depth[c.r]; c.lo = st->row_anc[c.r][0]; c.hi = st->row_anc[c.r][1]; }
     } else {
         n_rows = a.n_rows_fixed;
-        L = a.L_fixed;
-        if (r < n_rows) { depth = a.depth[seq * RT + r]; lo = a.anc[(size_t)(seq * RT + r) * 2]; hi = a.anc[(size_t)(seq * RT + r) * 2 + 1]; }
+        c.L = a.L_fixed;
+        if (c.r < n_rows) { c.depth = a.depth[c.seq * RT + c.r]; c.lo = a.anc[(size_t)(c.seq * RT + c.r) * 2]; c.hi = a.anc[(size_t)(c.seq * RT + c.r) * 2 + 1]; }
     }
     // After a bulk launch this kernel starts once every bulk CTA's wait has returned: the kernel that wrote this
     // step's queries, keys and values has completed by then, and the tail may be computed while the bulk CTAs run.
-    // (Nothing reads those buffers through L1 between that kernel's writes and this point: the bulk kernels fetch
-    // them by TMA, so no SM can hold a line of them from before the writes.)
+    // The tail reads those buffers with L2 loads only, so no stale line of an SM's L1 can be seen.
     if (!TAIL_FIRST) pdl_wait();
-    if (r >= n_rows) { pdl_wait(); return; }
-    const int kvh = head / (a.Hq / a.Hkv);
-    const int P = L + depth, T0 = tail_start_tc(P, a.dcap);
-    const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(a.kc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
-    const __nv_bfloat16* vbase = reinterpret_cast<const __nv_bfloat16*>(a.vc) + ((size_t)seq * a.Hkv + kvh) * a.cap * HD;
-    const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((size_t)(seq * RT + r) * a.Hq + head) * HD;
-    float* s_q = s_qall[warp];
-    {
-        const uint2 qq = *reinterpret_cast<const uint2*>(q + lane * 4);
-        const __nv_bfloat162 q01 = *reinterpret_cast<const __nv_bfloat162*>(&qq.x), q23 = *reinterpret_cast<const __nv_bfloat162*>(&qq.y);
-        s_q[lane * 4 + 0] = __low2float(q01); s_q[lane * 4 + 1] = __high2float(q01);
-        s_q[lane * 4 + 2] = __low2float(q23); s_q[lane * 4 + 3] = __high2float(q23);
-    }
-    __syncwarp();
-    const int n_sp = (T0 + a.split_len - 1) / a.split_len;
-    const size_t base = ((size_t)(seq * RT + r) * a.Hq + head) * a.n_split_max;
-    float2 ml0[PB];
-    float4 c40[PB];
-    auto request_partials = [&]() {     // the first bulk partials
-#pragma unroll
-        for (int u = 0; u < PB; ++u) {
-            if (u < n_sp) {
-                ml0[u] = __ldcg(a.part_ml + base + u);
-                c40[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (base + u) * HD + lane * 4));
-            }
-        }
-    };
-    if (!TAIL_FIRST) request_partials();      // in flight while the tail is computed
-    // ---- tail
-    float tm = -INFINITY, tl = 0.f, to[4] = {0.f, 0.f, 0.f, 0.f};
-    const int n_tail = P - T0 + 1;
-    for (int t0 = 0; t0 < n_tail; t0 += 32) {
-        const int t = t0 + lane;
-        bool valid = t < n_tail;
-        int slot = 0;
-        if (valid) {
-            const int pos = T0 + t;
-            if (pos < L) slot = pos;
-            else {
-                const int b = nth_set_bit128(lo, hi, pos - L);
-                if (b < 0) { set_error(a.err, DEV_E_INDEX); valid = false; }
-                else slot = L + b;
-            }
-        }
-        float sc = -INFINITY;
-        if (valid) {
-            const uint4* kr = reinterpret_cast<const uint4*>(kbase + (size_t)slot * HD);
-            float acc = 0.f;
-#pragma unroll
-            for (int dh = 0; dh < HD / 8; dh += KB8) {
-            uint4 kreg[KB8];
-#pragma unroll
-            for (int d8 = 0; d8 < KB8; ++d8) kreg[d8] = kr[dh + d8];
-#pragma unroll
-            for (int d8 = dh; d8 < dh + KB8; ++d8) {
-                const uint4 kk = kreg[d8 - dh];
-                const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kk);
-                const float4 qa = *reinterpret_cast<const float4*>(s_q + d8 * 8), qb = *reinterpret_cast<const float4*>(s_q + d8 * 8 + 4);
-                acc = fmaf(qa.x, __low2float(k2[0]), acc); acc = fmaf(qa.y, __high2float(k2[0]), acc);
-                acc = fmaf(qa.z, __low2float(k2[1]), acc); acc = fmaf(qa.w, __high2float(k2[1]), acc);
-                acc = fmaf(qb.x, __low2float(k2[2]), acc); acc = fmaf(qb.y, __high2float(k2[2]), acc);
-                acc = fmaf(qb.z, __low2float(k2[3]), acc); acc = fmaf(qb.w, __high2float(k2[3]), acc);
-            }
-            }
-            sc = acc * a.scale_log2;
-        }
-        float cm = sc;
-#pragma unroll
-        for (int of = 16; of > 0; of >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, of));
-        const float pe = valid ? exp2f(sc - cm) : 0.f;
-        float cl = pe;
-#pragma unroll
-        for (int of = 16; of > 0; of >>= 1) cl += __shfl_xor_sync(0xffffffffu, cl, of);
-        float co[4] = {0.f, 0.f, 0.f, 0.f};
-        // weighted values, keys in position order; the loads of VB keys are issued before their sums
-        // (a key that is not in the chunk reads slot 0 with weight 0 and is skipped)
-        for (int j0 = 0; j0 < 32; j0 += VB) {
-            float pj[VB];
-            uint2 vv[VB];
-#pragma unroll
-            for (int u = 0; u < VB; ++u) {
-                pj[u] = __shfl_sync(0xffffffffu, pe, j0 + u);
-                const int sj = __shfl_sync(0xffffffffu, slot, j0 + u);
-                vv[u] = *reinterpret_cast<const uint2*>(vbase + (size_t)sj * HD + lane * 4);
-            }
-#pragma unroll
-            for (int u = 0; u < VB; ++u) {
-                if (pj[u] != 0.f) {
-                    const __nv_bfloat162 v01 = *reinterpret_cast<const __nv_bfloat162*>(&vv[u].x), v23 = *reinterpret_cast<const __nv_bfloat162*>(&vv[u].y);
-                    co[0] = fmaf(pj[u], __low2float(v01), co[0]); co[1] = fmaf(pj[u], __high2float(v01), co[1]);
-                    co[2] = fmaf(pj[u], __low2float(v23), co[2]); co[3] = fmaf(pj[u], __high2float(v23), co[3]);
-                }
-            }
-        }
-        merge_ml(tm, tl, to, cm, cl, co);
-    }
-    // ---- merge: splits in order, then the tail
-    if (TAIL_FIRST) { pdl_wait(); request_partials(); }
-    float m = -INFINITY, l = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int u = 0; u < PB; ++u) {
-        if (u < n_sp) {
-            const float co[4] = {c40[u].x, c40[u].y, c40[u].z, c40[u].w};
-            merge_ml(m, l, o, ml0[u].x, ml0[u].y, co);
-        }
-    }
-    for (int s0 = PB; s0 < n_sp; s0 += PB) {
-        float2 ml[PB];
-        float4 c4[PB];
-#pragma unroll
-        for (int u = 0; u < PB; ++u) {
-            if (s0 + u < n_sp) {
-                ml[u] = __ldcg(a.part_ml + base + s0 + u);
-                c4[u] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (base + s0 + u) * HD + lane * 4));
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < PB; ++u) {
-            if (s0 + u < n_sp) {
-                const float co[4] = {c4[u].x, c4[u].y, c4[u].z, c4[u].w};
-                merge_ml(m, l, o, ml[u].x, ml[u].y, co);
-            }
-        }
-    }
-    merge_ml(m, l, o, tm, tl, to);
-    const float inv = 1.0f / l;
-    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out) + ((size_t)(seq * RT + r) * a.Hq + head) * HD + lane * 4;
-    const __nv_bfloat162 o01 = __floats2bfloat162_rn(o[0] * inv, o[1] * inv), o23 = __floats2bfloat162_rn(o[2] * inv, o[3] * inv);
-    uint2 pk;
-    pk.x = *reinterpret_cast<const uint32_t*>(&o01);
-    pk.y = *reinterpret_cast<const uint32_t*>(&o23);
-    *reinterpret_cast<uint2*>(out) = pk;
+    if (c.r >= n_rows) { pdl_wait(); return; }
+    FirstPartials<PB> fp;
+    if (!TAIL_FIRST) request_partials<PB>(fp, a, c, lane);      // in flight while the tail is computed
+    TailAcc t;
+    tail_pair<KB8, VB>(t, a, c, s_qall[warp], lane);
+    if (TAIL_FIRST) { pdl_wait(); request_partials<PB>(fp, a, c, lane); }
+    merge_pair<PB>(fp, t, a, c, lane);
 }
 
 }  // namespace

@@ -32,7 +32,7 @@
 
 #include "esp_epilogue.cuh"
 #include "esp_launch.h"
-#include "esp_tc.cuh"
+#include "esp_gemm_tc.cuh"
 
 namespace esp {
 
@@ -40,7 +40,6 @@ namespace {
 
 using namespace tc;
 
-constexpr int BK = 64;                       // k elements per stage (128 bytes of bf16)
 // NRS = rows of a sequence's block that take part (80, or 128 for blocks of more than 80 rows); NQ = sequences
 // one launch covers: the first NRS rows of their activation blocks ([RT][K] each, consecutive) are gathered by
 // one 3-D TMA box into one B operand of NQ*NRS <= 256 rows, so the weights are streamed once for all of them
@@ -53,7 +52,6 @@ __host__ __device__ constexpr int stages_of(int epi, int nq, int nrs) {
     return nrs == 80 ? (nq == 3 ? 4 : (nq == 2 ? 6 : (epi == EPI_PARTIAL ? 8 : 6)))
                      : (nq == 2 ? 4 : (epi == EPI_PARTIAL ? 7 : 4));
 }
-constexpr int A_BYTES = TILE_N * BK * 2;     // 16384
 __host__ __device__ constexpr int b_bytes_of(int nq, int nrs) { return nq * nrs * BK * 2; }   // 10240 per 80-row sequence
 __host__ __device__ constexpr int stage_bytes_of(int nq, int nrs) { return A_BYTES + b_bytes_of(nq, nrs); }
 // two accumulator buffers in tensor memory: 128 columns each for up to 128 rows, 256 each beyond
@@ -76,52 +74,6 @@ struct TcParams {
     int* err;
     EpiArgs a;
 };
-
-// kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = 80 per sequence
-__host__ __device__ constexpr uint32_t idesc_of(int nr) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nr >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
-}
-
-// One (tile, k-range) piece of a CTA's stream-K range.
-struct Seg {
-    int tile, kb0, kb1, slot;
-    bool whole;
-};
-
-// A CTA's unit range [u0, u1) cut at tile boundaries.  Segments are handed out with the partial ones first
-// (tail piece, then head piece), whole tiles after them: partial tiles are then complete early in every
-// CTA's timeline and the CTA that finishes one does so while the weight stream of its whole tiles is running.
-struct Range {
-    int first_tile, last_tile, head_kb0, tail_kb1, KB, n_seg, slots;
-    bool tail_partial;
-};
-__device__ __forceinline__ Range make_range(long long u0, long long u1, int KB, int slots) {
-    Range r;
-    r.KB = KB;
-    r.slots = slots;
-    r.first_tile = (int)(u0 / KB);
-    r.head_kb0 = (int)(u0 % KB);
-    r.last_tile = (int)((u1 - 1) / KB);
-    r.tail_kb1 = (int)((u1 - 1) % KB) + 1;
-    r.n_seg = r.last_tile - r.first_tile + 1;
-    r.tail_partial = r.n_seg > 1 && r.tail_kb1 < KB;
-    return r;
-}
-__device__ __forceinline__ Seg get_seg(const Range& r, int i) {
-    Seg s;
-    if (r.n_seg == 1) {
-        s.tile = r.first_tile; s.kb0 = r.head_kb0; s.kb1 = r.tail_kb1; s.slot = 0;
-    } else {
-        // order: [tail if partial] head, middle tiles, [tail if whole]
-        int idx = r.tail_partial ? i - 1 : i;
-        if (idx < 0 || idx == r.n_seg - 1) { s.tile = r.last_tile; s.kb0 = 0; s.kb1 = r.tail_kb1; s.slot = 1; }
-        else if (idx == 0) { s.tile = r.first_tile; s.kb0 = r.head_kb0; s.kb1 = r.KB; s.slot = 0; }
-        else { s.tile = r.first_tile + idx; s.kb0 = 0; s.kb1 = r.KB; s.slot = 1; }
-    }
-    s.slot = s.tile - r.first_tile < r.slots - 1 ? s.tile - r.first_tile : r.slots - 1;
-    s.whole = s.kb0 == 0 && s.kb1 == r.KB;
-    return s;
-}
 
 // which weight matrix / row the two 64-row halves of a tile come from
 __device__ __forceinline__ void tile_source(const TcParams& p, int tile, int half, int& m, int& row) {
@@ -477,6 +429,11 @@ size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K) {
     return (size_t)(n_tiles * ((K + BK - 1) / BK)) * A_BYTES;
 }
 int tc_gemm_tiles(const TcGemm* g) { return g ? g->p.n_tiles : 0; }
+void tc_gemm_geometry(const TcGemm* g, TcGemmGeom* out) {
+    out->n_tiles = g->p.n_tiles; out->KB = g->p.KB; out->grid = g->p.grid; out->slots = g->p.slots;
+    out->table = g->table; out->packed = g->p.a_packed; out->partials = g->p.partials; out->nrs = g->nrs;
+    out->map_b = g->map_b_nq[0];
+}
 
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
                    int x_seqs, int nrs, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,

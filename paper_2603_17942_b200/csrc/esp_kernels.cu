@@ -3,6 +3,7 @@
 // tail + merge), Top-K' merge, and the single-block tree kernel (verify walk,
 // KV compaction, mask update, Algorithm 1 + pruner, next row table).
 #include "esp_epilogue.cuh"
+#include "esp_consumers.cuh"
 #include "esp_launch.h"
 
 namespace esp {
@@ -104,65 +105,28 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const SeqState* states, const f
 
 // Consumer of a split GEMM (O or down projection) fused with the residual add and the next RMSNorm:
 //   hres[r] += sum over the tile's contributors, in CTA order, of their fp32 partials;  y = rmsnorm(hres[r]) * g.
-// One block per row; with sk.partials == NULL it is a plain RMSNorm of hres.  The sum order depends only on
-// the GEMM's shape, never on the number of rows in the block.
+// One block per row (resid_norm_row); with sk.partials == NULL it is a plain RMSNorm of hres.  The sum order
+// depends only on the GEMM's shape, never on the number of rows in the block.
 template <typename T>
 __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, float* hres, StreamK sk, const T* g, T* y, int d,
                                                     float eps, float* copy_out) {
     // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
     // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
-    // fetched before the wait: the tile's contributor entry and the norm weights of this thread's first four
-    // features (neither changes after initialisation), so that only the partials are loaded behind the wait
-    const int jf = threadIdx.x * 4;
-    SkEntry en0;
-    if (sk.partials && jf < d) en0 = sk_entry(sk, jf / TILE_N);
-    T g0[4];
-    if (jf < d) {
-        if constexpr (sizeof(T) == 2) *reinterpret_cast<uint2*>(g0) = __ldg(reinterpret_cast<const uint2*>(g + jf));
-        else *reinterpret_cast<float4*>(g0) = __ldg(reinterpret_cast<const float4*>(g + jf));
-    }
+    // fetched before the wait: the tile's contributor entry and the norm weights of this warp's first group
+    // (neither changes after initialisation), so that only the partials are loaded behind the wait
+    __shared__ float red[128];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    NormFirst<T> pf;
+    norm_prefetch(pf, sk, g, d, warp, lane);
     const int seq = blockIdx.y, r = blockIdx.x;
     const SeqState* st = states + seq;
     const bool idle = !st->active || r >= st->n_rows;     // the row table was written by an earlier step
     pdl_wait();
     if (idle) return;
-    float* xr = hres + (size_t)(seq * RT + r) * d;
-    __shared__ float red[32];
-    constexpr int STRIDE = 1024 * 4;
-    float4 keep[2];
-    float ss = 0.f;
-    int it = 0;
-    for (int j = threadIdx.x * 4; j < d; j += STRIDE, ++it) {
-        float4 x = *reinterpret_cast<const float4*>(xr + j);
-        if (sk.partials) {
-            const float4 acc = it == 0 ? sk_sum4(sk, en0, seq * sk.seq_rows + r, j % TILE_N)
-                                       : sk_sum4(sk, j / TILE_N, seq * sk.seq_rows + r, j % TILE_N);
-            x.x += acc.x; x.y += acc.y; x.z += acc.z; x.w += acc.w;
-            *reinterpret_cast<float4*>(xr + j) = x;
-        }
-        if (it < 2) keep[it] = x;
-        ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-    }
-    ss = warp_sum(ss);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 32; ++w) tot += red[w];
-    const float rinv = 1.0f / sqrtf(tot / (float)d + eps);
-    T* yr = y + (size_t)(seq * RT + r) * d;
-    it = 0;
-    for (int j = threadIdx.x * 4; j < d; j += STRIDE, ++it) {
-        const float4 x = it < 2 ? keep[it] : *reinterpret_cast<const float4*>(xr + j);   // beyond: this thread's own writes
-        const float xv[4] = {x.x, x.y, x.z, x.w};
-        T o[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) o[i] = from_f32<T>(xv[i] * rinv * to_f32(it == 0 ? g0[i] : g[j + i]));
-        if constexpr (sizeof(T) == 2) *reinterpret_cast<uint2*>(yr + j) = *reinterpret_cast<const uint2*>(o);
-        else *reinterpret_cast<float4*>(yr + j) = *reinterpret_cast<const float4*>(o);
-        if (copy_out) *reinterpret_cast<float4*>(copy_out + (size_t)(seq * RT + r) * d + j) = x;
-    }
+    const size_t row = (size_t)(seq * RT + r) * d;
+    resid_norm_row<T, 32>(hres + row, sk, seq * sk.seq_rows + r, g, y + row, d, eps, copy_out ? copy_out + row : nullptr, red, pf,
+                          warp, lane, [] { __syncthreads(); });
 }
 
 // Consumer of the split QKV GEMM: sums the partials of one (row, head) in CTA order, then what follows
@@ -174,9 +138,6 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
     // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
     // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
-    typedef __nv_bfloat16 T;
-    constexpr int NE = HD / 32;
-    constexpr int half = HD / 2;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hs = blockIdx.x * 4 + warp, r = blockIdx.y, seq = blockIdx.z;   // seq: sequence within this launch
     // Fetched before the wait, so that only the partials are loaded behind it: the row table (written by an earlier
@@ -184,71 +145,16 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
     const SeqState* st = a.st ? a.st + seq : nullptr;
     const int n_rows = st ? (st->active ? st->n_rows : 0) : a.rows_fixed;
     const bool work = r < n_rows && hs < a.Hq + 2 * a.Hkv;
-    const int pr = seq * RT + r;                 // row in the query buffer
-    const int sr = seq * sk.seq_rows + r;        // row in the partials
-    const int j0 = hs * HD + lane * NE;          // feature in the concatenated [q | k | v] space
-    const int tile = j0 / TILE_N, f = j0 % TILE_N;
-    const int which = hs < a.Hq ? 0 : (hs < a.Hq + a.Hkv ? 1 : 2);
-    const int head = which == 0 ? hs : (which == 1 ? hs - a.Hq : hs - a.Hq - a.Hkv);
     const int L = st ? st->L : 0;
-    SkEntry en;
-    float cs[NE], sn[NE], gw[NE];
-    if (work) {
-        en = sk_entry(sk, tile);
-        if (which != 2) {
-            const int pos = L + (st ? st->row_depth[r] : r);
-#pragma unroll
-            for (int i = 0; i < NE; ++i) {
-                const int idx = (lane * NE + i) % half;
-                cs[i] = __ldg(a.rope_cos + (size_t)pos * half + idx);
-                sn[i] = __ldg(a.rope_sin + (size_t)pos * half + idx);
-            }
-            if (a.qk_norm) {
-                const T* g = reinterpret_cast<const T*>(which == 0 ? a.q_norm : a.k_norm);
-#pragma unroll
-                for (int i = 0; i < NE; ++i) gw[i] = to_f32(g[lane * NE + i]);
-            }
-        }
-    }
+    QkvArgs qa;
+    qa.q_out = a.q_out; qa.kcache = a.kcache; qa.vcache = a.vcache; qa.q_norm = a.q_norm; qa.k_norm = a.k_norm;
+    qa.rope_cos = a.rope_cos; qa.rope_sin = a.rope_sin; qa.Hq = a.Hq; qa.Hkv = a.Hkv; qa.cap = a.cap; qa.qk_norm = a.qk_norm;
+    qa.rms_eps = a.rms_eps;
+    QkvPre<HD> pf;
+    if (work) qkv_prefetch<HD>(pf, qa, sk, hs, L + (st ? st->row_depth[r] : r), lane);
     pdl_wait();
     if (!work) return;
-    float v[NE];
-    if constexpr (NE == 4) {
-        const float4 t = sk_sum4(sk, en, sr, f);
-        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-    } else {
-        // narrower heads: the same sum through the four-float helper on the enclosing aligned group
-        const float4 t = sk_sum4(sk, en, sr, f & ~3);
-        const float tv[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-        for (int i = 0; i < NE; ++i) v[i] = tv[(f & 3) + i];
-    }
-    if (which != 2) {
-        if (a.qk_norm) {
-            float ss = 0.f;
-#pragma unroll
-            for (int i = 0; i < NE; ++i) ss += v[i] * v[i];
-            ss = warp_sum(ss);
-            const float rinv = 1.0f / sqrtf(ss / (float)HD + a.rms_eps);
-#pragma unroll
-            for (int i = 0; i < NE; ++i) v[i] = v[i] * rinv * gw[i];
-        }
-        const bool low = lane < 16;
-#pragma unroll
-        for (int i = 0; i < NE; ++i) {
-            const float other = __shfl_xor_sync(0xffffffffu, v[i], 16);
-            v[i] = low ? v[i] * cs[i] - other * sn[i] : v[i] * cs[i] + other * sn[i];
-        }
-    }
-    T* dst;
-    if (which == 0) dst = reinterpret_cast<T*>(a.q_out) + (size_t)pr * a.Hq * HD + head * HD + lane * NE;
-    else dst = reinterpret_cast<T*>(which == 1 ? a.kcache : a.vcache) + (((size_t)seq * a.Hkv + head) * a.cap + (L + r)) * HD + lane * NE;
-    T o[NE];
-#pragma unroll
-    for (int i = 0; i < NE; ++i) o[i] = from_f32<T>(v[i]);
-    if constexpr (NE == 4) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(o);
-    else if constexpr (NE == 2) *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(o);
-    else dst[0] = o[0];
+    qkv_finish_task<HD>(pf, qa, sk, seq, seq * sk.seq_rows + r, seq * RT + r, L + r, hs, lane);
 }
 
 // Consumer of the split gate/up GEMM: a tile holds 64 gate features (columns 0..63) and the matching 64 up
@@ -266,24 +172,7 @@ __global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, i
     const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;   // written by an earlier step
     pdl_wait();
     if (r >= n_rows || j0 >= F) return;
-    const int pr = seq * RT + r, sr = seq * sk.seq_rows + r;
-    float4 g[2], u[2];
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-        const int j = j0 + 4 * q, f = j % 64;
-        if (j >= F) { g[q] = u[q] = make_float4(0.f, 0.f, 0.f, 0.f); continue; }
-        g[q] = sk_sum4(sk, en, sr, f);
-        u[q] = sk_sum4(sk, en, sr, 64 + f);
-    }
-    __nv_bfloat16 o[8];
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-        const float gv[4] = {g[q].x, g[q].y, g[q].z, g[q].w}, uv[4] = {u[q].x, u[q].y, u[q].z, u[q].w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) o[4 * q + i] = __float2bfloat16_rn((gv[i] / (1.0f + expf(-gv[i]))) * uv[i]);
-    }
-    if (j0 + 8 <= F) *reinterpret_cast<uint4*>(act + (size_t)pr * F + j0) = *reinterpret_cast<const uint4*>(o);
-    else *reinterpret_cast<uint2*>(act + (size_t)pr * F + j0) = *reinterpret_cast<const uint2*>(o);
+    swiglu_task(sk, en, seq * sk.seq_rows + r, act + (size_t)(seq * RT + r) * F, j0, F);
 }
 
 // ------------------------------------------------------------------ CUDA-core GEMM

@@ -92,4 +92,42 @@ size_t tc_gemm_partial_bytes(int n_sm, int nq = 1, int nrs = 80);
 int tc_gemm_max_nq(int nrs = 80);
 int tc_gemm_counter_ints();
 
+
+// All layers of a step in one persistent cooperative launch (esp_layers_tc.cu): bf16, head_dim 128, blocks of at
+// most 80 rows, one sequence per pass.  Same phases, same partition and same bits as the kernels above.
+struct LayersTc;
+struct LayersTcDesc {
+    const TcGemm* gemm[4];         // layer 0's QKV, O, gate/up and down plans (every layer has the same geometry)
+    const void* packed;            // layer 0's repacked weights; pk_layer bytes per layer
+    size_t pk_layer;
+    float* hres;
+    void *xn, *qbuf, *attn_out, *act;
+    void *kcache, *vcache;         // [n_layers][batch][Hkv][cap][h]
+    size_t layer_kv_stride;        // bytes
+    const void* const* norm_attn;  // device arrays of n_layers device pointers
+    const void* const* norm_ffn;
+    const void* const* q_norm;
+    const void* const* k_norm;
+    const float *rope_cos, *rope_sin;
+    int32_t n_layers, d, Hq, Hkv, h, F, cap, qk_norm, batch;
+    float rms_eps;
+    float* part_o;
+    float2* part_ml;
+    int32_t split_len, n_split_max, dcap;
+    float scale_log2;
+    unsigned int* sync_counter;    // zero when the plan is made; the kernel counts it up
+    int* err;
+    int32_t n_sm;
+};
+bool layers_tc_supported(const LayersTcDesc& d);
+int layers_tc_create(LayersTc** out, const LayersTcDesc& d);
+void layers_tc_destroy(LayersTc* t);
+int layers_tc_grid(const LayersTc* t);
+int layers_tc_syncs_per_layer();
+unsigned int layers_tc_arrivals(const LayersTc* t);   // what one launch adds to the barrier counter
+// seq: the sequence's index in the cache; sync_base: the counter's value when the kernel starts;
+// timeline: optional [n_layers * layers_tc_syncs_per_layer()] device words, CTA 0's global timer after every barrier
+int layers_tc_launch(LayersTc* t, const SeqState* st, int seq, void* kcache_seq, void* vcache_seq, unsigned int sync_base,
+                     unsigned long long* timeline, cudaStream_t s);
+
 }  // namespace esp
