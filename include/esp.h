@@ -182,13 +182,37 @@ int esp_debug_capture(esp_handle* h, float* logits, float* hidden);
  * 1 = CUDA-core reference kernels (same epilogues; for A/B checks on the GPU).  fp32 models always use 1. */
 int esp_debug_set_gemm(esp_handle* h, int32_t impl);
 
+/* Selects how the decoder layers of a step are launched for bf16 models with head_dim 128, max_batch 1 and blocks
+ * of at most 80 rows: 1 = one kernel per operation, chained by programmatic dependent launch (default; what
+ * batches, prefill blocks and larger blocks always use), 0 = all layers in one persistent cooperative kernel (the
+ * weight ring keeps running across the operations of a layer, grid-wide barriers with bounded waits between
+ * them).  Both run the same arithmetic in the same order and give the same bits.  Mode 0 is kept for A/B
+ * checks and tracing (esp_debug_layer_timeline): on a B200 its step is slower, because every phase between two
+ * GEMMs pays two grid barriers plus its own chain of L2 round trips with 14 warps per SM, where the chained
+ * kernels overlap neighbouring launches.  No counterpart in the paper.
+ * ESP_E_BADCFG if mode 0 is not available for the handle's configuration. */
+int esp_debug_set_layer_kernel(esp_handle* h, int32_t mode);
+
 /* Measurement hook (no counterpart in the paper): one esp_step with a CUDA event recorded on the handle's
  * stream after every kernel group; ms_by_kind [host] [8] receives the device time per group in this order:
  * 0 row assembly, RMSNorm and the kernels that sum GEMM partials (residual add + norm, RoPE + cache write,
  * SiLU*up), 1 QKV GEMM, 2 tree attention, 3 O GEMM, 4 gate/up GEMM, 5 down GEMM, 6 LM-head GEMM with fused
  * selection, 7 Top-K' merge + tree kernel.  The kernels run back to back without overlap in this mode, so the
- * groups add up to more than an unprofiled step.  tokens_out / n_out as esp_step. */
+ * groups add up to more than an unprofiled step.  When all layers run in one kernel (esp_debug_set_layer_kernel
+ * mode 0) that kernel's share is split by the global-timer stamps its first CTA takes after every grid barrier.
+ * tokens_out / n_out as esp_step. */
 int esp_step_profiled(esp_handle* h, float* ms_by_kind, int32_t* tokens_out, int32_t* n_out);
+
+/* Tracing (no counterpart in the paper): the time stamps of the last esp_step_profiled whose layers ran in one
+ * kernel.  stamps_ns [host] [capacity] receives the GPU's global timer (ns) as read by that kernel's first CTA:
+ * eight words per grid barrier -- [0] its arrival at the barrier, [1] its exit, and inside the phase that
+ * follows, when that is a GEMM, [2] the activation tiles of the ring's first items requested, [3] the first
+ * item consumed by the tensor cores, [4] the last one issued, [5] the last accumulator stored ([6], [7] and the
+ * words of other phases are unused and hold stale values) -- ten barriers per layer, one behind each phase in
+ * the order: attention norm, QKV GEMM, q/k/v finish, attention over the cache, attention tail + merge, O GEMM,
+ * FFN norm, gate/up GEMM, SiLU*up, down GEMM.  *n_out [host] = words per step (n_layers * 80).  Synchronises.
+ * ESP_E_BADCFG if the handle has no such kernel. */
+int esp_debug_layer_timeline(esp_handle* h, uint64_t* stamps_ns, int32_t capacity, int32_t* n_out);
 
 int esp_get_stats(esp_handle* h, esp_stats* out);
 

@@ -25,7 +25,7 @@ ERRORS = {0: "ESP_OK", -1: "ESP_E_BADCFG", -2: "ESP_E_WORKSPACE", -3: "ESP_E_PRO
           -5: "ESP_E_DEVICE", -6: "ESP_E_CUDA", -7: "ESP_E_STATE", -8: "ESP_E_ARG"}
 
 EXPORTS = ["esp_workspace_bytes", "esp_init", "esp_prefill", "esp_step", "esp_step_async", "esp_read", "esp_set_mask", "esp_set_tree",
-           "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_step_profiled", "esp_get_stats",
+           "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_debug_set_layer_kernel", "esp_debug_layer_timeline", "esp_step_profiled", "esp_get_stats",
            "esp_debug_wait_selftest", "esp_debug_gumbel", "esp_free",
            "esp_tree_attention_scratch_bytes", "esp_tree_attention", "esp_tree_attention_static", "esp_gemm_scratch_bytes",
            "esp_gemm_bf16"]
@@ -182,6 +182,19 @@ def esp_debug_capture(h, logits=None, hidden=None):
 
 def esp_debug_set_gemm(h, impl: int):
     _check(load_library().esp_debug_set_gemm(h, ctypes.c_int32(impl)), "esp_debug_set_gemm")
+
+
+def esp_debug_set_layer_kernel(h, mode: int):
+    """1: one kernel per operation (default), 0: all decoder layers in one persistent cooperative kernel."""
+    _check(load_library().esp_debug_set_layer_kernel(h, ctypes.c_int32(mode)), "esp_debug_set_layer_kernel")
+
+
+def esp_debug_layer_timeline(h, n_layers: int) -> np.ndarray:
+    """Global-timer stamps (ns) of the last profiled step: [n_layers][10 barriers][8 words] (see esp.h)."""
+    out = np.zeros(n_layers * 80, np.uint64)
+    n = ctypes.c_int32(0)
+    _check(load_library().esp_debug_layer_timeline(h, _vp(out), ctypes.c_int32(out.size), ctypes.byref(n)), "esp_debug_layer_timeline")
+    return out[:n.value].reshape(-1, 10, 8)
 
 
 KINDS = ("norm_and_partial_consumers", "qkv_gemm", "tree_attention", "o_gemm", "gateup_gemm", "down_gemm", "lmhead_topk", "select_tree")

@@ -49,6 +49,11 @@ struct Buffers {
     // weights repacked for streaming (bf16 models, one sequence): per layer [qkv | o | gate/up | down], then the LM head
     char* packed;
     size_t pk_qkv, pk_o, pk_gu, pk_down, pk_lm, pk_layer;
+    // the all-layers kernel: per-layer pointer tables [4][n_layers] (attention norm, FFN norm, q norm, k norm),
+    // its barrier counter and the time stamps of a profiled step
+    const void** layer_ptrs;
+    unsigned int* sync_counter;
+    unsigned long long* timeline;
 };
 constexpr int SK_TABLE_TILES = 2048;
 
@@ -84,6 +89,7 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
     if (m->n_kv_heads < 1 || m->n_q_heads % m->n_kv_heads) return ESP_E_BADCFG;
     if ((m->n_q_heads * m->head_dim) % TILE_N || (m->n_kv_heads * m->head_dim) % TILE_N) return ESP_E_BADCFG;
     if (m->d_model % 8 || m->d_ffn % 8) return ESP_E_BADCFG;  // 16-byte rows for TMA and vector loads
+    if (m->dtype == 1 && m->d_model > 128 * TILE_N) return ESP_E_BADCFG;   // the norm kernels keep one partial per 128 features
     if (m->vocab > 2048 * TILE_N) return ESP_E_BADCFG;
     if (m->max_batch < 1 || m->max_seq_len < 1) return ESP_E_BADCFG;
     if (s->n_probes < 0 || s->n_probes > PROBES_MAX) return ESP_E_BADCFG;
@@ -172,6 +178,9 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     }
     o.gemm_counters = c.take<int>(tc_gemm_counter_ints());
     o.sk_tables = c.take<TileSrc>(4 * SK_TABLE_TILES);
+    o.layer_ptrs = c.take<const void*>((size_t)4 * D.n_layers);
+    o.sync_counter = c.take<unsigned int>(64);
+    o.timeline = c.take<unsigned long long>((size_t)layers_tc_trace_slots() * D.n_layers * layers_tc_syncs_per_layer() + 8);
     o.packed = nullptr;
     o.pk_qkv = o.pk_o = o.pk_gu = o.pk_down = o.pk_lm = o.pk_layer = 0;
     if (dtype == 1) {
@@ -207,6 +216,9 @@ struct esp_handle {
     int rows_cap_prefill = RT;
     std::vector<AttnTc*> p_attn;   // per layer, bf16 models with head_dim 128
     TcGemm* p_lm = nullptr;
+    LayersTc* p_layers = nullptr;  // all layers in one launch (one sequence per pass, blocks of at most 80 rows)
+    bool use_layers = false;       // esp_debug_set_layer_kernel (off by default: measured slower than one kernel per operation)
+    unsigned int sync_epoch = 0;   // value of the barrier counter after the launches enqueued so far
     std::vector<int> L_host, ready;
     int32_t* pinned = nullptr;  // [batch][RING] + 4 ints (error words)
     float *dbg_logits = nullptr, *dbg_hidden = nullptr;
@@ -226,7 +238,7 @@ namespace {
 
 int cuda_ok(cudaError_t e) { return e == cudaSuccess ? ESP_OK : ESP_E_CUDA; }
 
-enum { KIND_MISC = 0, KIND_QKV, KIND_ATTN, KIND_O, KIND_GATEUP, KIND_DOWN, KIND_LMHEAD, KIND_SELECT, KIND_N };
+enum { KIND_MISC = 0, KIND_QKV, KIND_ATTN, KIND_O, KIND_GATEUP, KIND_DOWN, KIND_LMHEAD, KIND_SELECT, KIND_N, KIND_FUSED };
 
 void mark(esp_handle* h, int kind) {
     if (!h->prof) return;
@@ -294,7 +306,20 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc,
     auto plan = [&](std::vector<TcGemm*>& narrow, std::vector<TcGemm*>& w128, int l) -> TcGemm* { return wide ? w128[l] : narrow[l]; };
     launch_assemble(h->dtype, st0, h->embed, mvec0, b.hres, D.d, D.mask_slots, nb, s, false, rc_rows);
     h->launches++;
-    for (int l = 0; l < D.n_layers; ++l) {
+    // One sequence, a block of at most 80 rows, bf16: every layer in one persistent launch (same bits as the
+    // kernel-per-operation path below, which serves batches, prefill blocks and larger blocks).
+    const bool fused = tc && nb == 1 && !prefill && h->p_layers && h->use_layers;
+    if (fused) {
+        mark(h, KIND_MISC);
+        const int rc = layers_tc_launch(h->p_layers, st0, s0, reinterpret_cast<char*>(b.kcache) + kv_seq_off,
+                                        reinterpret_cast<char*>(b.vcache) + kv_seq_off, h->sync_epoch, h->prof ? b.timeline : nullptr, s);
+        if (rc) return rc;
+        h->sync_epoch += layers_tc_arrivals(h->p_layers);
+        h->launches++;
+        mark(h, KIND_FUSED);
+        pending = tc_gemm_streamk(h->p_down[D.n_layers - 1], 1);
+    }
+    for (int l = 0; l < D.n_layers && !fused; ++l) {
         if (tc) launch_resid_norm(st0, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->na[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
@@ -593,6 +618,32 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
             ok = ok && !tc_gemm_create(&h->p_lm_w, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
         }
         if (!ok) { esp_free(h); return ESP_E_CUDA; }
+        // the all-layers kernel: per-layer pointer tables and the plan
+        if (nrs == 80 && D.batch == 1) {
+            std::vector<const void*> tab((size_t)4 * D.n_layers, nullptr);
+            for (int l = 0; l < D.n_layers; ++l) {
+                tab[0 * D.n_layers + l] = h->na[l]; tab[1 * D.n_layers + l] = h->nf[l];
+                tab[2 * D.n_layers + l] = h->qn[l]; tab[3 * D.n_layers + l] = h->kn[l];
+            }
+            if (cudaMemcpyAsync(h->b.layer_ptrs, tab.data(), sizeof(void*) * tab.size(), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+                cudaStreamSynchronize(h->stream) != cudaSuccess) { esp_free(h); return ESP_E_CUDA; }
+            LayersTcDesc ld;
+            memset(&ld, 0, sizeof(ld));
+            ld.gemm[0] = h->p_qkv[0]; ld.gemm[1] = h->p_o[0]; ld.gemm[2] = h->p_gu[0]; ld.gemm[3] = h->p_down[0];
+            ld.packed = h->b.packed; ld.pk_layer = h->b.pk_layer;
+            ld.hres = h->b.hres; ld.xn = h->b.xn; ld.qbuf = h->b.qbuf; ld.attn_out = h->b.attn_out; ld.act = h->b.act;
+            ld.kcache = h->b.kcache; ld.vcache = h->b.vcache; ld.layer_kv_stride = h->layer_kv_stride;
+            ld.norm_attn = h->b.layer_ptrs; ld.norm_ffn = h->b.layer_ptrs + D.n_layers;
+            ld.q_norm = h->b.layer_ptrs + 2 * D.n_layers; ld.k_norm = h->b.layer_ptrs + 3 * D.n_layers;
+            ld.rope_cos = h->b.rope_cos; ld.rope_sin = h->b.rope_sin;
+            ld.n_layers = D.n_layers; ld.d = D.d; ld.Hq = D.Hq; ld.Hkv = D.Hkv; ld.h = D.h; ld.F = D.F; ld.cap = D.cap;
+            ld.qk_norm = D.qk_norm; ld.batch = D.batch; ld.rms_eps = D.rms_eps;
+            ld.part_o = h->b.part_o; ld.part_ml = h->b.part_ml;
+            ld.split_len = D.split_len; ld.n_split_max = D.n_split_max; ld.dcap = DCAP_STEP;
+            ld.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
+            ld.sync_counter = h->b.sync_counter; ld.err = h->b.err; ld.n_sm = n_sm;
+            if (layers_tc_supported(ld) && layers_tc_create(&h->p_layers, ld)) { esp_free(h); return ESP_E_CUDA; }
+        }
     }
     if (cudaStreamSynchronize(h->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) { esp_free(h); return ESP_E_CUDA; }
     *handle_out = h;
@@ -647,7 +698,10 @@ int esp_step_async(esp_handle* h) {
     if (!any) return ESP_E_STATE;
     int rc = ESP_OK;
     bool done = false;
-    if (h->use_graph && !h->prof) {
+    // (the all-layers kernel makes a step a handful of launches, and its barrier counter's start value is a launch
+    // parameter: such steps are launched directly)
+    const bool fused_step = h->p_layers && h->use_layers && h->D.batch == 1 && h->gemm_impl == 0;
+    if (h->use_graph && !h->prof && !fused_step) {
         // The launch sequence of a step depends on the host only through the number of attention splits;
         // every other quantity (L, row counts, the tree) is read from device state by the kernels.
         // (key: which sequences take part and how many cache splits each one's attention launches)
@@ -791,6 +845,25 @@ int esp_debug_set_gemm(esp_handle* h, int32_t impl) {
     return ESP_OK;
 }
 
+int esp_debug_set_layer_kernel(esp_handle* h, int32_t mode) {
+    if (!h || (mode != 0 && mode != 1)) return ESP_E_ARG;
+    if (mode == 0 && !h->p_layers) return ESP_E_BADCFG;
+    h->use_layers = mode == 0;
+    drop_graphs(h);
+    return ESP_OK;
+}
+
+int esp_debug_layer_timeline(esp_handle* h, uint64_t* stamps_ns, int32_t capacity, int32_t* n_out) {
+    if (!h || !stamps_ns || !n_out || capacity < 0) return ESP_E_ARG;
+    if (!h->p_layers) return ESP_E_BADCFG;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return ESP_E_CUDA;
+    const int n = layers_tc_trace_slots() * h->D.n_layers * layers_tc_syncs_per_layer();
+    *n_out = n;
+    const int m = n < capacity ? n : capacity;
+    if (m > 0 && cudaMemcpy(stamps_ns, h->b.timeline, sizeof(uint64_t) * m, cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+    return ESP_OK;
+}
+
 int esp_step_profiled(esp_handle* h, float* ms_by_kind, int32_t* tokens_out, int32_t* n_out) {
     if (!h || !ms_by_kind) return ESP_E_ARG;
     h->prof = true;
@@ -805,6 +878,22 @@ int esp_step_profiled(esp_handle* h, float* ms_by_kind, int32_t* tokens_out, int
         if (cudaEventElapsedTime(&ms, h->ev[i - 1], h->ev[i]) != cudaSuccess) return ESP_E_CUDA;
         const int kind = h->ev_kind[i];
         if (kind >= 0 && kind < KIND_N) ms_by_kind[kind] += ms;
+        if (kind == KIND_FUSED) {
+            // inside the all-layers kernel: the global timer after each grid barrier, ten phases per layer
+            // (norm, QKV, q/k/v finish, attention bulk, tail + merge, O, norm, gate/up, SiLU*up, down)
+            static const int kind_of_phase[10] = {KIND_MISC, KIND_QKV, KIND_MISC, KIND_ATTN, KIND_ATTN, KIND_O, KIND_MISC, KIND_GATEUP, KIND_MISC, KIND_DOWN};
+            const int n = h->D.n_layers * layers_tc_syncs_per_layer();
+            const int ts = layers_tc_trace_slots();
+            std::vector<unsigned long long> tl((size_t)ts * n);
+            if (cudaMemcpy(tl.data(), h->b.timeline, sizeof(unsigned long long) * ts * n, cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+            double inside = 0.0;
+            for (int j = 1; j < n; ++j) {
+                const double d_ms = (double)(tl[(size_t)ts * j + 1] - tl[(size_t)ts * (j - 1) + 1]) * 1e-6;   // barrier exit to barrier exit
+                ms_by_kind[kind_of_phase[j % 10]] += (float)d_ms;
+                inside += d_ms;
+            }
+            if (ms > inside) ms_by_kind[KIND_MISC] += (float)(ms - inside);   // launch, set-up and the first norm
+        }
     }
     return rc;
 }
@@ -860,6 +949,7 @@ void esp_free(esp_handle* h) {
     for (auto* p : h->p_gu_w) tc_gemm_destroy(p);
     for (auto* p : h->p_down_w) tc_gemm_destroy(p);
     tc_gemm_destroy(h->p_lm_w);
+    layers_tc_destroy(h->p_layers);
     for (auto* t : h->p_attn) attn_tc_destroy(t);
     if (h->pinned) cudaFreeHost(h->pinned);
     drop_graphs(h);

@@ -338,8 +338,10 @@ __device__ __forceinline__ void request_partials(FirstPartials<PB>& fp, const At
 
 // The tail: positions T0..P in position order, lane j owns key j of a 32-key chunk (chunk grid anchored at T0);
 // in-flight ancestors are found through the ancestor mask.  s_q: 128 floats of shared memory owned by the warp.
-// This step's queries, keys and values were written by another kernel or CTA shortly before: they are read
-// with L2 loads (ld.global.cg), never through L1.  KB8 / VB: 16-byte key pieces / value rows in flight.
+// What this step wrote shortly before, in another kernel or CTA -- the queries and the keys / values of the block's
+// own rows (slots >= L) -- is read with L2 loads (ld.global.cg), never through L1; cache positions below L were
+// written by earlier steps and go through L1, where the pairs that share a KV head find them again.
+// KB8 / VB: 16-byte key pieces / value rows in flight.
 template <int KB8, int VB>
 __device__ __forceinline__ void tail_pair(TailAcc& t, const AttnArgs& a, const PairCtx& c, float* s_q, int lane) {
     const int kvh = c.head / (a.Hq / a.Hkv);
@@ -379,7 +381,7 @@ __device__ __forceinline__ void tail_pair(TailAcc& t, const AttnArgs& a, const P
             for (int dh = 0; dh < HD / 8; dh += KB8) {
                 uint4 kreg[KB8];
 #pragma unroll
-                for (int d8 = 0; d8 < KB8; ++d8) kreg[d8] = __ldcg(kr + dh + d8);
+                for (int d8 = 0; d8 < KB8; ++d8) kreg[d8] = slot < c.L ? kr[dh + d8] : __ldcg(kr + dh + d8);
 #pragma unroll
                 for (int d8 = dh; d8 < dh + KB8; ++d8) {
                     const uint4 kk = kreg[d8 - dh];
@@ -410,7 +412,8 @@ __device__ __forceinline__ void tail_pair(TailAcc& t, const AttnArgs& a, const P
             for (int u = 0; u < VB; ++u) {
                 pj[u] = __shfl_sync(0xffffffffu, pe, j0 + u);
                 const int sj = __shfl_sync(0xffffffffu, slot, j0 + u);
-                vv[u] = __ldcg(reinterpret_cast<const uint2*>(vbase + (size_t)sj * HD + lane * 4));
+                const uint2* vr = reinterpret_cast<const uint2*>(vbase + (size_t)sj * HD + lane * 4);
+                vv[u] = sj < c.L ? *vr : __ldcg(vr);
             }
 #pragma unroll
             for (int u = 0; u < VB; ++u) {

@@ -124,6 +124,7 @@ int layers_tc_create(LayersTc** out, const LayersTcDesc& d);
 void layers_tc_destroy(LayersTc* t);
 int layers_tc_grid(const LayersTc* t);
 int layers_tc_syncs_per_layer();
+int layers_tc_trace_slots();   // time stamps per barrier in the timeline
 unsigned int layers_tc_arrivals(const LayersTc* t);   // what one launch adds to the barrier counter
 // seq: the sequence's index in the cache; sync_base: the counter's value when the kernel starts;
 // timeline: optional [n_layers * layers_tc_syncs_per_layer()] device words, CTA 0's global timer after every barrier

@@ -22,6 +22,7 @@
 // DEV_E_WAIT_TIMEOUT; the other CTAs see the error word in their own waits and leave too; every CTA lets its
 // copies land, frees its tensor memory and returns.
 #include <new>
+#include <stddef.h>
 #include <string.h>
 
 #include "esp_attn_tc.cuh"
@@ -85,7 +86,7 @@ struct LayersParams {
     unsigned int* sync_counter;    // arrivals, counted up launch after launch
     unsigned int sync_base;        // its value before this launch
     int* err;
-    unsigned long long* timeline;  // optional: CTA 0 stamps the global timer after every grid barrier
+    unsigned long long* timeline;  // optional: CTA 0 stamps the global timer when it arrives at and when it leaves every grid barrier
 };
 
 struct Shared {                    // behind the ring
@@ -93,23 +94,38 @@ struct Shared {                    // behind the ring
     uint64_t kv_full[2], kv_empty[2], s_full[2], q_full, p_ready, pv_done, xchg;       // attention item
     uint32_t tmem;
     int abort_flag, T0max, sync_ok;
-    float red[128];
-    float xch[2][2 * attn::MP];
-    float s_q[CONS_WARPS][attn::HD];
+    alignas(16) float red[128];
+    alignas(16) float xch[2][2 * attn::MP];
+    alignas(16) float s_q[CONS_WARPS][attn::HD];      // read as float4
 };
+static_assert(offsetof(Shared, s_q) % 16 == 0 && offsetof(Shared, full) % 8 == 0, "vector and barrier alignment");
 constexpr size_t SMEM_BYTES = 1024 + RING_BYTES + sizeof(Shared);
 
 __device__ __forceinline__ void cons_bar() { asm volatile("bar.sync 1, %0;" ::"n"(CONS_THREADS) : "memory"); }
+__device__ __forceinline__ void main_bar() { __syncthreads(); }
+
+// Tracing: with a timeline buffer, CTA 0 stamps the global timer into TRACE_SLOTS words per barrier: [0] its arrival
+// at the barrier, [1] its exit, [2..] marks inside the phase that follows (GEMM phases: the activation tiles of
+// the ring's first items requested, the first and the last item consumed, the last accumulator stored).
+constexpr int TRACE_SLOTS = 8;
+__device__ __forceinline__ void trace(const LayersParams& p, int stamp, int slot) {
+    if (p.timeline && blockIdx.x == 0) {
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
+        p.timeline[(size_t)stamp * TRACE_SLOTS + slot] = now;
+    }
+}
 
 // Grid-wide barrier.  Every thread's global writes of the phase before it are visible to every thread of the
 // grid after it, to tensor-map (async proxy) loads as well.  false: this CTA or another one gave up.
 __device__ __forceinline__ bool grid_sync(const LayersParams& p, Shared& sh, uint32_t& epoch, int& stamp) {
     asm volatile("fence.proxy.async;" ::: "memory");
-    __syncthreads();
+    main_bar();
     if (threadIdx.x == 0) {
         epoch += gridDim.x;
         const uint32_t target = p.sync_base + epoch;
         bool ok = sh.abort_flag == 0;
+        trace(p, stamp, 0);
         if (ok) {
             asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.sync_counter) : "memory");
             unsigned long long t0 = 0;
@@ -128,15 +144,11 @@ __device__ __forceinline__ bool grid_sync(const LayersParams& p, Shared& sh, uin
         }
         if (!ok) sh.abort_flag = 1;
         sh.sync_ok = ok ? 1 : 0;
-        if (p.timeline && blockIdx.x == 0) {
-            unsigned long long now;
-            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
-            p.timeline[stamp] = now;
-        }
+        trace(p, stamp, 1);
         asm volatile("fence.proxy.async;" ::: "memory");
     }
     ++stamp;
-    __syncthreads();
+    main_bar();
     return sh.sync_ok != 0;
 }
 
@@ -182,7 +194,7 @@ __device__ __forceinline__ bool prefetch_weights(const LayersParams& p, Shared& 
 
 // producer thread: all items of GEMM `g` of layer `l` (the activation tiles, and the weight units not yet requested)
 __device__ __forceinline__ bool produce_gemm(const LayersParams& p, Shared& sh, unsigned char* ring, Ring& rg, int g, int l,
-                                             uint64_t pol_w, uint64_t pol_x) {
+                                             uint64_t pol_w, uint64_t pol_x, int tr) {
     const GemmDesc& gd = p.g[g];
     if ((int)blockIdx.x >= gd.G) return true;
     const Range rng = cta_range(gd, blockIdx.x);
@@ -197,9 +209,10 @@ __device__ __forceinline__ bool produce_gemm(const LayersParams& p, Shared& sh, 
                 if (!mbar_wait(&sh.empty[stage], par ^ 1, &sh.abort_flag)) return false;
                 mbar_expect_tx(&sh.full[stage], STAGE_BYTES);
                 bulk_load(sa, base + ((size_t)sg.tile * gd.KB + kb) * A_BYTES, A_BYTES, &sh.full[stage], pol_w);
-            }
+                }
             tma_load_3d_hint(sa + A_BYTES, &p.map_b[g], kb * BK, 0, 0, &sh.full[stage], pol_x);
             ++rg.it;
+            if (idx + 1 == rg.pre) trace(p, tr, 2);
         }
     }
     rg.pre = 0;
@@ -207,7 +220,7 @@ __device__ __forceinline__ bool produce_gemm(const LayersParams& p, Shared& sh, 
 }
 
 // MMA thread
-__device__ __forceinline__ bool mma_gemm(const LayersParams& p, Shared& sh, unsigned char* ring, Ring& rg, int g, uint32_t tmem_base) {
+__device__ __forceinline__ bool mma_gemm(const LayersParams& p, Shared& sh, unsigned char* ring, Ring& rg, int g, uint32_t tmem_base, int tr) {
     const GemmDesc& gd = p.g[g];
     if ((int)blockIdx.x >= gd.G) return true;
     const Range rng = cta_range(gd, blockIdx.x);
@@ -220,6 +233,7 @@ __device__ __forceinline__ bool mma_gemm(const LayersParams& p, Shared& sh, unsi
         for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++rg.it) {
             const uint32_t stage = rg.it % STAGES, par = (rg.it / STAGES) & 1;
             if (!mbar_wait(&sh.full[stage], par, &sh.abort_flag)) return false;
+            if (i == 0 && kb == sg.kb0) trace(p, tr, 3);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t sa = smem_u32(ring + stage * STAGE_BYTES);
             const uint64_t da = smem_desc(sa, 16), db = smem_desc(sa + A_BYTES, 16);
@@ -230,12 +244,13 @@ __device__ __forceinline__ bool mma_gemm(const LayersParams& p, Shared& sh, unsi
         }
         umma_commit(&sh.tfull[buf]);
     }
+    trace(p, tr, 4);
     return true;
 }
 
 // epilogue warps 2..5: accumulator -> fp32 partial of the (CTA, slot) piece; false (warp-uniform): a wait ran out
 __device__ __forceinline__ bool epilogue_gemm(const LayersParams& p, Shared& sh, Ring& rg, int g, uint32_t tmem_base, int n_rows,
-                                              int warp, int lane) {
+                                              int warp, int lane, int tr) {
     const GemmDesc& gd = p.g[g];
     if ((int)blockIdx.x >= gd.G) return true;
     const Range rng = cta_range(gd, blockIdx.x);
@@ -258,6 +273,7 @@ __device__ __forceinline__ bool epilogue_gemm(const LayersParams& p, Shared& sh,
 #pragma unroll
         for (int r = 0; r < NRS; ++r)
             if (r < n_rows) __stcg(part + r * TILE_N, __uint_as_float(v[r]));
+        if (i == rng.n_seg - 1 && warp == 2 && lane == 0) { trace(p, tr, 5); }
     }
     return true;
 }
@@ -313,13 +329,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
     // one GEMM phase; `next_g` >= 0: afterwards the producer requests the first weight units of that GEMM (of layer next_l)
     auto gemm_phase = [&](int g, int l, int next_g, int next_l) {
         if (producer) {
-            bool ok = produce_gemm(p, sh, ring, rg, g, l, pol_w, pol_x);
+            bool ok = produce_gemm(p, sh, ring, rg, g, l, pol_w, pol_x, stamp - 1);
             if (ok && next_g >= 0) ok = prefetch_weights(p, sh, ring, rg, next_g, next_l, pol_w);
             if (!ok) { set_error(p.err, DEV_E_WAIT_TIMEOUT); sh.abort_flag = 1; }
         } else if (mma) {
-            if (!mma_gemm(p, sh, ring, rg, g, tmem_base)) { set_error(p.err, DEV_E_WAIT_TIMEOUT); sh.abort_flag = 1; }
+            if (!mma_gemm(p, sh, ring, rg, g, tmem_base, stamp - 1)) { set_error(p.err, DEV_E_WAIT_TIMEOUT); sh.abort_flag = 1; }
         } else if (warp >= 2 && warp < 6) {
-            if (!epilogue_gemm(p, sh, rg, g, tmem_base, n_rows, warp, lane) && lane == 0) { set_error(p.err, DEV_E_WAIT_TIMEOUT); sh.abort_flag = 1; }
+            if (!epilogue_gemm(p, sh, rg, g, tmem_base, n_rows, warp, lane, stamp - 1) && lane == 0) { set_error(p.err, DEV_E_WAIT_TIMEOUT); sh.abort_flag = 1; }
         }
     };
     // residual add (partials of GEMM `g_src`, -1: none) + RMSNorm with gain `gain`: row `cta`
@@ -396,7 +412,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
                     if (lane == 0) sh.T0max = t0;
                 }
                 if (threadIdx.x == 0) attn::bulk_init_barriers(bsm);
-                __syncthreads();
+                main_bar();
                 const int T0max = sh.T0max;
                 it.beg = it.split * p.split_len;
                 if (it.beg < T0max) {       // block-uniform
@@ -406,7 +422,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
                     attn::bulk_item_roles<false>(bmp, aa, it, bsm, tmem_base, warp, lane);
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 }
-                __syncthreads();
+                main_bar();
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 ok = sh.abort_flag == 0;
             }
@@ -477,6 +493,7 @@ struct LayersTc {
 };
 
 int layers_tc_syncs_per_layer() { return 10; }
+int layers_tc_trace_slots() { return TRACE_SLOTS; }
 
 bool layers_tc_supported(const LayersTcDesc& d) {
     if (d.h != attn::HD || !attn_tc_supported(d.h, d.Hq, d.Hkv)) return false;
