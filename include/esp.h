@@ -42,6 +42,7 @@ enum {
 #define ESP_MAX_ROWS 128  /* rows of one block per sequence: tree nodes + mask probes */
 #define ESP_MAX_PROBES 8  /* k */
 #define ESP_MAX_KPRIME 32 /* Top-K entries kept per probe, K + pruner refills */
+#define ESP_MAX_UNREAD_STEPS 1024 /* decode steps esp_step_async may enqueue before their results are read */
 #define ESP_PREFILL_CHUNK 120 /* prompt rows esp_prefill runs per block (the last block adds the k mask rows) */
 
 /* The frozen decoder f_theta (Section 2; LLaMA3 / Qwen3 shapes, Section 4 "Models"). */
@@ -113,6 +114,7 @@ typedef struct {
     int64_t accept_hist[ESP_MAX_PROBES + 1]; /* [a] = steps that accepted a draft tokens */
     int32_t device_error;   /* 0, or the first device-side error code recorded */
     int32_t kernels_per_step; /* kernel launches one esp_step enqueues */
+    int64_t rows_hist[4];   /* decode steps by block size (tree nodes + mask rows): <= 16, <= 32, <= 64, more rows */
 } esp_stats;
 
 typedef struct esp_handle esp_handle;
@@ -148,7 +150,14 @@ int esp_prefill(esp_handle* h, int32_t seq, const int32_t* prompt, int32_t n_pro
  * log-sum-exp, lossless verification (Section 2),
  * KV compaction of the accepted path, mask update (Eq. mask_update_mean) and
  * the next tree (Algorithm 1 + pruner).  esp_step = esp_step_async + esp_read.
- * tokens_out [host] [max_batch][ESP_MAX_PROBES+1], n_out [host] [max_batch]. */
+ * tokens_out [host] [max_batch][ESP_MAX_PROBES+1], n_out [host] [max_batch].
+ * esp_step_async only enqueues the step; nothing of it depends on the host, so several may be enqueued back to
+ * back.  Every step leaves its result in a record of its own and esp_read returns the OLDEST unread step (0 tokens
+ * for a sequence that took no part in it; with nothing unread it reports 0 tokens for every sequence and the
+ * device status).  At most ESP_MAX_UNREAD_STEPS steps may be unread: one more esp_step_async returns ESP_E_STATE.
+ * While steps are unread the host knows each cache length only as an upper bound (k + 1 positions per unread
+ * step): ESP_E_FULL may then come that many positions early, and the attention launches are sized for the bound
+ * (splits without work return at once); results do not depend on it. */
 int esp_step(esp_handle* h, int32_t* tokens_out, int32_t* n_out);
 int esp_step_async(esp_handle* h);
 int esp_read(esp_handle* h, int32_t* tokens_out, int32_t* n_out);
@@ -243,6 +252,12 @@ void esp_free(esp_handle* h);
  *   out      [batch][ESP_MAX_ROWS][n_q_heads][head_dim]
  *   scratch  esp_tree_attention_scratch_bytes bytes
  * dtype as in esp_model_cfg; n_rows <= ESP_MAX_ROWS rows are real; L + ESP_MAX_ROWS <= cap.
+ * The tensor-core path reads the cache in chunks of 128 positions that may reach up to position
+ * L + ESP_MAX_ROWS - 1: positions beyond a row's visible keys get weight zero, but their VALUES still enter a
+ * product with that zero, so kcache / vcache must hold finite numbers (zeros will do) up to there.
+ * The call is asynchronous on cuda_stream.  A device-side problem (a bounded wait that ran out, an ancestor
+ * mask that names a row the block does not have) is recorded in the first word of the scratch, which the call
+ * clears when it starts; esp_tree_attention_status reads it back.
  * dcap (a multiple of 16, >= the largest depth) sets where each row's key list switches from the
  * tensor-core chunks to the position-by-position tail: keys at positions below
  * floor((L + depth - dcap) / 16) * 16 go through the chunked path, the rest through the tail. */
@@ -252,6 +267,10 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
                        int32_t n_kv_heads, int32_t head_dim, int32_t dcap, const void* q, const void* kcache,
                        const void* vcache, const uint64_t* anc, const int32_t* depth, void* out, void* scratch,
                        size_t scratch_bytes, void* cuda_stream);
+/* Device status of the last esp_tree_attention that used `scratch` [device] (NULL: of the last
+ * esp_tree_attention_static on the current device): waits for cuda_stream, copies the status word to
+ * *device_status_out [host] (may be NULL) and returns ESP_OK if it is 0, ESP_E_DEVICE otherwise. */
+int esp_tree_attention_status(const void* scratch, void* cuda_stream, int32_t* device_status_out);
 
 /* esp_tree_attention for callers that cannot hand over scratch memory (the paper has no counterpart; this is
  * a packaging variant of the operator above).  Meant for hosts that may not allocate device memory at the
@@ -263,11 +282,12 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
  * the scratch pair.  Returns ESP_E_WORKSPACE when the shape needs more than the array holds
  * (esp_tree_attention_scratch_bytes(batch, n_q_heads, head_dim, cap) > ESP_STATIC_SCRATCH_BYTES; e.g. 32
  * query heads of 128 with cap <= 3584 at batch 1 fit).  It allocates and frees nothing, on the host or the
- * device.  The first call on each device looks up the array's device address (a one-time query, no
- * allocation); make that first call outside any stream capture.  All calls share the one array and it keeps
- * the previous call's contents: the entry point re-zeroes the error word it reads, everything else is
- * overwritten before it is read.  Two calls whose kernels can overlap on the GPU (different streams, no
- * dependency between them) would write the same partials and race: keep them ordered. */
+ * device: the descriptors of the call live in its own stack frame.  The first call on each device looks up the
+ * array's device address (a one-time query, no allocation); make that first call outside any stream capture.
+ * All calls share the one array and it keeps the previous call's contents: the status word at its start is
+ * cleared by every call (esp_tree_attention_status(NULL, ...) reads it), everything else is overwritten before
+ * it is read.  Two calls whose kernels can overlap on the GPU (different streams, no dependency between them)
+ * would write the same partials and race: keep them ordered. */
 #define ESP_STATIC_SCRATCH_BYTES (32u << 20)
 int esp_tree_attention_static(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, int32_t cap, int32_t n_q_heads,
                               int32_t n_kv_heads, int32_t head_dim, int32_t dcap, const void* q, const void* kcache,

@@ -20,6 +20,7 @@ ESP_MAX_ROWS = 128
 ESP_MAX_PROBES = 8
 ESP_MAX_KPRIME = 32
 ESP_PREFILL_CHUNK = 120
+ESP_MAX_UNREAD_STEPS = 1024
 
 ERRORS = {0: "ESP_OK", -1: "ESP_E_BADCFG", -2: "ESP_E_WORKSPACE", -3: "ESP_E_PROMPT", -4: "ESP_E_FULL",
           -5: "ESP_E_DEVICE", -6: "ESP_E_CUDA", -7: "ESP_E_STATE", -8: "ESP_E_ARG"}
@@ -27,11 +28,11 @@ ERRORS = {0: "ESP_OK", -1: "ESP_E_BADCFG", -2: "ESP_E_WORKSPACE", -3: "ESP_E_PRO
 EXPORTS = ["esp_workspace_bytes", "esp_init", "esp_prefill", "esp_step", "esp_step_async", "esp_read", "esp_set_mask", "esp_set_tree",
            "esp_debug_state", "esp_debug_capture", "esp_debug_set_gemm", "esp_debug_set_layer_kernel", "esp_debug_layer_timeline", "esp_step_profiled", "esp_get_stats",
            "esp_debug_wait_selftest", "esp_debug_gumbel", "esp_free",
-           "esp_tree_attention_scratch_bytes", "esp_tree_attention", "esp_tree_attention_static", "esp_gemm_scratch_bytes",
+           "esp_tree_attention_scratch_bytes", "esp_tree_attention", "esp_tree_attention_status", "esp_tree_attention_static", "esp_gemm_scratch_bytes",
            "esp_gemm_bf16"]
 
 __all__ = ["EspError", "esp_model_cfg", "esp_spec_cfg", "esp_weights", "esp_stats", "load_library", "model_cfg",
-           "spec_cfg", "Handle", "ESP_MAX_ROWS", "ESP_MAX_PROBES", "ESP_MAX_KPRIME", "ESP_PREFILL_CHUNK", "ESP_STATIC_SCRATCH_BYTES", "EXPORTS", "LIB_PATH", "KINDS"] + EXPORTS
+           "spec_cfg", "Handle", "ESP_MAX_ROWS", "ESP_MAX_PROBES", "ESP_MAX_KPRIME", "ESP_PREFILL_CHUNK", "ESP_MAX_UNREAD_STEPS", "ESP_STATIC_SCRATCH_BYTES", "EXPORTS", "LIB_PATH", "KINDS"] + EXPORTS
 
 
 class EspError(RuntimeError):
@@ -65,7 +66,7 @@ class esp_weights(ctypes.Structure):
 
 class esp_stats(ctypes.Structure):
     _fields_ = [("steps", ctypes.c_int64), ("emitted", ctypes.c_int64), ("accept_hist", ctypes.c_int64 * (ESP_MAX_PROBES + 1)),
-                ("device_error", ctypes.c_int32), ("kernels_per_step", ctypes.c_int32)]
+                ("device_error", ctypes.c_int32), ("kernels_per_step", ctypes.c_int32), ("rows_hist", ctypes.c_int64 * 4)]
 
 
 _lib = None
@@ -251,11 +252,18 @@ ESP_STATIC_SCRATCH_BYTES = 32 << 20
 
 def esp_tree_attention_static(dtype: int, batch: int, n_rows: int, L: int, cap: int, n_q_heads: int, n_kv_heads: int,
                               head_dim: int, dcap: int, q, kcache, vcache, anc, depth, out, stream=None):
-    """esp_tree_attention with the library's built-in 16 MiB scratch array: no scratch argument, no allocation."""
+    """esp_tree_attention with the library's built-in 32 MiB scratch array: no scratch argument, no allocation."""
     _check(load_library().esp_tree_attention_static(
         ctypes.c_int32(dtype), ctypes.c_int32(batch), ctypes.c_int32(n_rows), ctypes.c_int32(L), ctypes.c_int32(cap),
         ctypes.c_int32(n_q_heads), ctypes.c_int32(n_kv_heads), ctypes.c_int32(head_dim), ctypes.c_int32(dcap), _vp(q),
         _vp(kcache), _vp(vcache), _vp(anc), _vp(depth), _vp(out), _vp(stream)), "esp_tree_attention_static")
+
+
+def esp_tree_attention_status(scratch=None, stream=None) -> int:
+    """Device status word of the last tree attention on `scratch` (None: on the built-in array); raises EspError(ESP_E_DEVICE) if set."""
+    st = ctypes.c_int32(0)
+    _check(load_library().esp_tree_attention_status(_vp(scratch), _vp(stream), ctypes.byref(st)), "esp_tree_attention_status")
+    return st.value
 
 
 def esp_gemm_scratch_bytes() -> int:

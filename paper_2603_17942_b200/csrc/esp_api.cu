@@ -165,7 +165,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.mvec = c.take<float>((size_t)D.batch * D.mask_slots * D.d);
     o.states = c.take<SeqState>(D.batch);
     o.err = c.take<int>(4);
-    o.out_ring = c.take<int32_t>((size_t)D.batch * RING);
+    o.out_ring = c.take<int32_t>((size_t)(NREC + 1) * D.batch * RING);
     o.prompt_dev = c.take<int32_t>(D.cap);
     o.tree_dev = c.take<int32_t>(2 * RT);
     o.rope_cos = c.take<float>((size_t)D.cap * (D.h / 2));
@@ -220,6 +220,8 @@ struct esp_handle {
     bool use_layers = false;       // esp_debug_set_layer_kernel (off by default: measured slower than one kernel per operation)
     unsigned int sync_epoch = 0;   // value of the barrier counter after the launches enqueued so far
     std::vector<int> L_host, ready;
+    unsigned long long issued = 0;      // decode steps enqueued on this handle
+    unsigned long long consumed = 0;    // ... whose records esp_read has returned
     int32_t* pinned = nullptr;  // [batch][RING] + 4 ints (error words)
     float *dbg_logits = nullptr, *dbg_hidden = nullptr;
     int launches = 0, kernels_per_step = 0;
@@ -450,8 +452,9 @@ int forward(esp_handle* h, bool with_lm, int dcap, int only_seq) {
     return ESP_OK;
 }
 
-int tree_step(esp_handle* h) {
+int tree_step(esp_handle* h, bool is_step) {
     TreeArgs A;
+    A.is_step = is_step ? 1 : 0;
     A.D = h->D;
     A.states = h->b.states;
     A.topk = h->b.topk;
@@ -479,9 +482,10 @@ __global__ void k_select(SeqState* st, int batch, int seq_only) {
 }
 __global__ void k_mark_ready(SeqState* st, int seq) { st[seq].ready = 1; }
 
-int read_ring(esp_handle* h) {
+// Copies the records of slot `slot` (all sequences) and the error word to pinned memory; synchronises.
+int read_ring(esp_handle* h, int slot) {
     const int n = h->D.batch * RING;
-    if (cudaMemcpyAsync(h->pinned, h->b.out_ring, sizeof(int32_t) * n, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return ESP_E_CUDA;
+    if (cudaMemcpyAsync(h->pinned, h->b.out_ring + (size_t)slot * n, sizeof(int32_t) * n, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return ESP_E_CUDA;
     if (cudaMemcpyAsync(h->pinned + n, h->b.err, sizeof(int), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return ESP_E_CUDA;
     if (cudaStreamSynchronize(h->stream) != cudaSuccess) return ESP_E_CUDA;
     return h->pinned[n] ? ESP_E_DEVICE : ESP_OK;
@@ -670,13 +674,19 @@ int esp_prefill(esp_handle* h, int32_t seq, const int32_t* prompt, int32_t n_pro
         launch_setup_chain(h->b.states, seq, h->b.prompt_dev, off, cn, last, h->D.k, s);
         h->L_host[seq] = off;
         int rc = forward(h, last, DCAP_PREFILL, seq);
-        if (rc) return rc;
-        rc = tree_step(h);
-        if (rc) return rc;
+        if (!rc) rc = tree_step(h, false);
+        if (rc) {
+            // the other sequences keep their lengths; this one has to be prefilled again before it can step
+            k_select<<<1, 32, 0, s>>>(h->b.states, h->D.batch, -1);
+            h->L_host = saved;
+            h->L_host[seq] = 0;
+            h->ready[seq] = 0;
+            return rc;
+        }
     }
     k_mark_ready<<<1, 1, 0, s>>>(h->b.states, seq);
     k_select<<<1, 32, 0, s>>>(h->b.states, h->D.batch, -1);
-    int rc = read_ring(h);
+    int rc = read_ring(h, NREC);
     h->L_host = saved;
     h->L_host[seq] = n_prompt;
     h->ready[seq] = 1;
@@ -696,6 +706,7 @@ int esp_step_async(esp_handle* h) {
         Lmax = h->L_host[i] > Lmax ? h->L_host[i] : Lmax;
     }
     if (!any) return ESP_E_STATE;
+    if (h->issued - h->consumed >= (unsigned long long)NREC) return ESP_E_STATE;   // every record slot holds an unread step
     int rc = ESP_OK;
     bool done = false;
     // (the all-layers kernel makes a step a handful of launches, and its barrier counter's start value is a launch
@@ -720,7 +731,7 @@ int esp_step_async(esp_handle* h) {
             bool ok = cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
             if (ok) {
                 int r1 = forward(h, true, DCAP_STEP, -1);
-                int r2 = r1 ? r1 : tree_step(h);
+                int r2 = r1 ? r1 : tree_step(h, true);
                 ok = cudaStreamEndCapture(h->stream, &graph) == cudaSuccess && !r2 && graph;
             }
             if (ok) ok = cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess;
@@ -743,9 +754,11 @@ int esp_step_async(esp_handle* h) {
         const int before = h->launches;
         rc = forward(h, true, DCAP_STEP, -1);
         if (rc) return rc;
-        rc = tree_step(h);
+        rc = tree_step(h, true);
         h->kernels_per_step = h->launches - before;
     }
+    if (rc) return rc;
+    ++h->issued;
     // until the result is read the host only knows an upper bound of each cache length
     for (int i = 0; i < h->D.batch; ++i)
         if (h->ready[i]) h->L_host[i] += h->D.k + 1;
@@ -754,11 +767,21 @@ int esp_step_async(esp_handle* h) {
 
 int esp_read(esp_handle* h, int32_t* tokens_out, int32_t* n_out) {
     if (!h) return ESP_E_ARG;
-    int rc = read_ring(h);
+    if (h->consumed == h->issued) {           // nothing unread: only the device status
+        if (n_out)
+            for (int i = 0; i < h->D.batch; ++i) n_out[i] = 0;
+        if (cudaStreamSynchronize(h->stream) != cudaSuccess) return ESP_E_CUDA;
+        int e = 0;
+        if (cudaMemcpy(&e, h->b.err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
+        return e ? ESP_E_DEVICE : ESP_OK;
+    }
+    int rc = read_ring(h, (int)(h->consumed % NREC));
+    ++h->consumed;
+    const int unread = (int)(h->issued - h->consumed);
     for (int i = 0; i < h->D.batch; ++i) {
-        if (!h->ready[i]) { if (n_out) n_out[i] = 0; continue; }
         const int32_t* r = h->pinned + i * RING;
-        h->L_host[i] = r[1];
+        if (!h->ready[i] || r[0] <= 0) { if (n_out) n_out[i] = 0; continue; }   // took no part in that step
+        h->L_host[i] = r[1] + unread * (h->D.k + 1);     // steps still unread can each add at most k + 1 positions
         if (n_out) n_out[i] = r[0];
         if (tokens_out)
             for (int j = 0; j < r[0] && j <= PROBES_MAX; ++j) tokens_out[i * (PROBES_MAX + 1) + j] = r[2 + j];
@@ -908,6 +931,7 @@ int esp_get_stats(esp_handle* h, esp_stats* out) {
         out->steps += (int64_t)st.steps;
         out->emitted += (int64_t)st.emitted;
         for (int a = 0; a <= PROBES_MAX; ++a) out->accept_hist[a] += (int64_t)st.accept_hist[a];
+        for (int a = 0; a < 4; ++a) out->rows_hist[a] += (int64_t)st.rows_hist[a];
     }
     int e = 0;
     if (cudaMemcpy(&e, h->b.err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return ESP_E_CUDA;
@@ -968,6 +992,7 @@ int esp_tree_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t h
     return ESP_OK;
 }
 
+// scratch layout: [error word, 256 bytes][split partials: weighted values][split partials: (max, sum)]
 int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, int32_t cap, int32_t n_q_heads,
                        int32_t n_kv_heads, int32_t head_dim, int32_t dcap, const void* q, const void* kcache,
                        const void* vcache, const uint64_t* anc, const int32_t* depth, void* out, void* scratch,
@@ -984,11 +1009,15 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     while ((cap - RT + S - 1) / S > 16) S *= 2;
     const size_t ns = (cap + S - 1) / S + 1;
     const size_t rows = (size_t)batch * RT * n_q_heads * ns;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    char* sc = reinterpret_cast<char*>(scratch);
+    // the error word starts at zero (the scratch may hold an earlier call's bytes); the partials are written before they are read
+    if (cudaMemsetAsync(sc, 0, 256, s) != cudaSuccess) return ESP_E_CUDA;
     AttnArgs a;
     memset(&a, 0, sizeof(a));
     a.q = q; a.kc = kcache; a.vc = vcache; a.out = out;
-    a.part_o = reinterpret_cast<float*>(scratch);
-    a.part_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(scratch) + align_up(rows * head_dim * sizeof(float), 256));
+    a.part_o = reinterpret_cast<float*>(sc + 256);
+    a.part_ml = reinterpret_cast<float2*>(sc + 256 + align_up(rows * head_dim * sizeof(float), 256));
     a.st = nullptr;
     a.anc = reinterpret_cast<const unsigned long long*>(anc);
     a.depth = depth;
@@ -996,16 +1025,11 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     a.rows_cap = n_rows;      // sizes the grids: no block has more rows
     a.Hq = n_q_heads; a.Hkv = n_kv_heads; a.h = head_dim; a.cap = cap; a.split_len = S; a.n_split_max = (int)ns; a.dcap = dcap;
     a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)head_dim));
-    a.err = reinterpret_cast<int*>(reinterpret_cast<char*>(scratch) + need - 256);
-    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    a.err = reinterpret_cast<int*>(sc);
     const int n_split_launch = (L + S - 1) / S;
     const bool mma = dtype == 1 && attn_tc_supported(head_dim, n_q_heads, n_kv_heads);
     if (mma) {
-        AttnTc* t = nullptr;
-        if (attn_tc_create(&t, q, kcache, vcache, batch, n_q_heads, n_kv_heads, cap)) return ESP_E_CUDA;
-        const int rc = attn_tc_launch(t, a, batch, n_split_launch, s, false);   // the descriptors travel by value
-        attn_tc_destroy(t);
-        if (rc) return ESP_E_BADCFG;
+        if (attn_tc_run(q, kcache, vcache, batch, n_q_heads, n_kv_heads, cap, a, n_split_launch, s)) return ESP_E_BADCFG;
     } else if (launch_attn_simt(dtype, a, batch, n_split_launch, true, s, false)) {
         return ESP_E_BADCFG;
     }
@@ -1049,12 +1073,24 @@ int esp_tree_attention_static(int32_t dtype, int32_t batch, int32_t n_rows, int3
     void* scratch = nullptr;
     rc = static_scratch_ptr(&scratch);
     if (rc) return rc;
-    // the array still holds the previous call's bytes: the error word (last 256 bytes of the used part) must
-    // start at zero; the partials are written by this call before they are read
-    if (cudaMemsetAsync(reinterpret_cast<char*>(scratch) + need - 256, 0, 256, reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
-        return ESP_E_CUDA;
     return esp_tree_attention(dtype, batch, n_rows, L, cap, n_q_heads, n_kv_heads, head_dim, dcap, q, kcache, vcache, anc,
                               depth, out, scratch, need, cuda_stream);
+}
+
+int esp_tree_attention_status(const void* scratch, void* cuda_stream, int32_t* device_status_out) {
+    const void* src = scratch;
+    if (!src) {
+        void* p = nullptr;
+        const int rc = static_scratch_ptr(&p);
+        if (rc) return rc;
+        src = p;
+    }
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    int e = 0;
+    if (cudaMemcpyAsync(&e, src, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return ESP_E_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return ESP_E_CUDA;
+    if (device_status_out) *device_status_out = e;
+    return e ? ESP_E_DEVICE : ESP_OK;
 }
 
 int esp_gemm_scratch_bytes(size_t* bytes_out) {

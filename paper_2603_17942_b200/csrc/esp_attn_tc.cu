@@ -497,12 +497,29 @@ bool attn_tc_supported(int h, int Hq, int Hkv) {
 }
 
 // TMA descriptors of one layer's query buffer [batch*RT][Hq][128] and KV cache [batch*Hkv*cap][128] (bf16).
+static int attn_tc_fill(AttnTc* t, const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap);
+
 int attn_tc_create(AttnTc** out, const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap) {
-    if (!out || !attn_tc_supported(HD, Hq, Hkv)) return -1;
-    EncodeFn enc = get_encode();
-    if (!enc) return -1;
+    if (!out) return -1;
     AttnTc* t = new (std::nothrow) AttnTc();
     if (!t) return -1;
+    if (attn_tc_fill(t, q, kcache, vcache, batch, Hq, Hkv, cap)) { delete t; return -1; }
+    *out = t;
+    return 0;
+}
+
+// One attention with the descriptors built in this call's own frame: nothing is allocated, on the host or the device.
+int attn_tc_run(const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap, const AttnArgs& a,
+                int n_split_launch, cudaStream_t s) {
+    AttnTc t;
+    if (attn_tc_fill(&t, q, kcache, vcache, batch, Hq, Hkv, cap)) return -1;
+    return attn_tc_launch(&t, a, batch, n_split_launch, s, false);     // the descriptors travel by value
+}
+
+static int attn_tc_fill(AttnTc* t, const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap) {
+    if (!attn_tc_supported(HD, Hq, Hkv)) return -1;
+    EncodeFn enc = get_encode();
+    if (!enc) return -1;
     memset(&t->p, 0, sizeof(t->p));
     const int group = Hq / Hkv, rows_per_tile = MP / group;
     t->p.group = group;
@@ -515,7 +532,7 @@ int attn_tc_create(AttnTc** out, const void* q, const void* kcache, const void* 
         cuuint32_t box[3] = {64, (cuuint32_t)group, (cuuint32_t)rows_per_tile};
         if (enc(&t->p.map_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, estr3,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) { delete t; return -1; }
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return -1;
     }
     for (int i = 0; i < 2; ++i) {
         cuuint64_t dims[2] = {(cuuint64_t)HD, (cuuint64_t)batch * Hkv * cap};
@@ -523,9 +540,8 @@ int attn_tc_create(AttnTc** out, const void* q, const void* kcache, const void* 
         cuuint32_t box[2] = {64, (cuuint32_t)CK};
         if (enc(i ? &t->p.map_v : &t->p.map_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(i ? vcache : kcache), dims,
                 strides, box, estr3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) { delete t; return -1; }
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return -1;
     }
-    *out = t;
     return 0;
 }
 
@@ -534,38 +550,24 @@ void attn_tc_destroy(AttnTc* t) { delete t; }
 // Two launches: the bulk kernel (grid = splits x (KV heads x row tiles) x sequences), then tail + merge.
 int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl) {
     if (!t || n_split_launch + 1 > a.n_split_max || a.split_len % CK) return -1;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(k_attn_bulk_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return -1;
-        attr_set = true;
-    }
     BulkParams p = t->p;
     p.a = a;
     const int rows_cap = a.rows_cap > 0 && a.rows_cap < RT ? a.rows_cap : RT;
     p.n_row_tiles = (rows_cap + p.rows_per_tile - 1) / p.rows_per_tile;   // row tiles that can hold rows
     if (n_split_launch > 0) {
-        static int n_sm = 0;
-        if (n_sm == 0) {
-            int dev = 0;
-            if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1) {
-                n_sm = 0;
-                return -1;
-            }
-        }
+        const int n_sm = current_sm_count();
+        if (n_sm < 1) return -1;
         const long long all_items = (long long)n_split_launch * a.Hkv * p.n_row_tiles * batch;
         if (all_items <= n_sm + n_sm / 2) {
             // (nearly) every CTA runs once: one item per CTA.  Measured crossover: the persistent kernel wins from
             // about 1.2 waves when timed alone, a little later inside a step, where its larger register and
             // shared-memory footprint delays its start behind the kernel before it
-            static bool once_attr = false;
-            if (!once_attr) {
-                if (cudaFuncSetAttribute(k_attn_bulk_tc_once, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ONCE_SMEM_BYTES) != cudaSuccess) return -1;
-                once_attr = true;
-            }
+            if (ensure_dynamic_smem(reinterpret_cast<const void*>(k_attn_bulk_tc_once), (int)ONCE_SMEM_BYTES)) return -1;
             dim3 grid(n_split_launch, a.Hkv * p.n_row_tiles, batch);
             if (launch_k(k_attn_bulk_tc_once, grid, dim3(ONCE_THREADS), ONCE_SMEM_BYTES, s, pdl, p) != cudaSuccess) return -1;
         } else {
             // persistent CTAs, one per SM, walk the (split, KV head, row tile, sequence) items round-robin
+            if (ensure_dynamic_smem(reinterpret_cast<const void*>(k_attn_bulk_tc), (int)SMEM_BYTES)) return -1;
             const int per_launch = MAX_T0_ENTRIES / p.n_row_tiles;
             for (int s0 = 0; s0 < batch; s0 += per_launch) {
                 p.seq0 = s0;

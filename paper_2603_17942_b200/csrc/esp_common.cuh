@@ -20,6 +20,9 @@ constexpr int PREFILL_CHUNK = ESP_PREFILL_CHUNK;   // prompt rows per prefill bl
 constexpr int DCAP_STEP = 16;           // tail cap of decode steps (>= 2k)
 constexpr int DCAP_PREFILL = 16;        // tail cap of prefill blocks: their earlier rows are cache positions already
 constexpr int RING = ESP_MAX_PROBES + 4; // per-sequence result record: n_out, L, tokens
+// Result records: a decode step writes every sequence's record into slot (steps so far) % NREC, so that steps
+// enqueued without a read in between keep their results; the prefill uses slot NREC.  [NREC + 1][batch][RING].
+constexpr int NREC = ESP_MAX_UNREAD_STEPS;
 
 // device error codes (first one recorded wins)
 enum : int {
@@ -50,6 +53,8 @@ struct SeqState {
     float row_logp[RT];
     unsigned long long steps, emitted;
     unsigned long long accept_hist[PROBES_MAX + 1];
+    unsigned long long rec;       // decode steps launched on the handle so far (every sequence counts alike): next record slot
+    unsigned long long rows_hist[4];   // decode steps by rows of their block: <= 16, <= 32, <= 64, more
 };
 
 struct Cand {  // one Top-K' entry
@@ -227,6 +232,11 @@ __device__ __forceinline__ void set_error(int* err, int code) {
 // before it have released it or exited).  Both calls are no-ops for a plain launch.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute belongs to the device's copy of the
+// function) and tells how many SMs the current device has; both are cached per device, under a lock.
+int ensure_dynamic_smem(const void* func, int bytes);     // 0 on success
+int current_sm_count();                                   // 0 on failure
 
 // Launch with or without the programmatic-dependent-launch attribute.
 template <typename... KArgs, typename... Args>

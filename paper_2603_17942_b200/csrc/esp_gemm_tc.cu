@@ -558,11 +558,7 @@ int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl, 
     cudaError_t e = cudaSuccess;
 #define ESP_TC_CASE(E, Q, N)                                                                                  \
     {                                                                                                         \
-        static bool attr_set = false;                                                                         \
-        if (!attr_set) {                                                                                      \
-            if (cudaFuncSetAttribute(k_gemm_tc<E, Q, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(E, Q, N)) != cudaSuccess) return ESP_E_CUDA; \
-            attr_set = true;                                                                                  \
-        }                                                                                                     \
+        if (ensure_dynamic_smem(reinterpret_cast<const void*>(k_gemm_tc<E, Q, N>), (int)smem_bytes_of(E, Q, N))) return ESP_E_CUDA;            \
         e = launch_k(k_gemm_tc<E, Q, N>, dim3(p.grid), dim3(NUM_THREADS), smem_bytes_of(E, Q, N), s, pdl, p); \
     }
     const bool wide = g->nrs != 80;

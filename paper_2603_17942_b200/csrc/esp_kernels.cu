@@ -2,11 +2,43 @@
 // (CUDA-core) small-M GEMM, position-canonical tree attention (split partials,
 // tail + merge), Top-K' merge, and the single-block tree kernel (verify walk,
 // KV compaction, mask update, Algorithm 1 + pruner, next row table).
+#include <mutex>
+#include <utility>
+#include <vector>
+
 #include "esp_epilogue.cuh"
 #include "esp_consumers.cuh"
 #include "esp_launch.h"
 
 namespace esp {
+
+// ------------------------------------------------------------------ per-device caches of the launch helpers
+namespace {
+std::mutex g_dev_mutex;
+std::vector<std::pair<const void*, int>> g_smem_done;   // (function, device) pairs whose limit has been raised
+int g_sm_count[64];
+}  // namespace
+int ensure_dynamic_smem(const void* func, int bytes) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    for (const auto& e : g_smem_done)
+        if (e.first == func && e.second == dev) return 0;
+    if (cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return -1;
+    g_smem_done.emplace_back(func, dev);
+    return 0;
+}
+int current_sm_count() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (g_sm_count[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 0;
+        g_sm_count[dev] = n;
+    }
+    return g_sm_count[dev];
+}
 
 // ------------------------------------------------------------------ small helpers
 __global__ void k_rope_table(float* cs, float* sn, int n_pos, int h, float base) {
@@ -711,7 +743,15 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
     const Dims& D = A.D;
     const int seq = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     SeqState* st = A.states + seq;
-    if (!st->active) return;
+    // where this launch's record goes; every sequence, active or not, counts the handle's decode steps
+    const unsigned long long rec_no = st->rec;
+    int32_t* rec = A.out_ring + ((size_t)(A.is_step ? (int)(rec_no % NREC) : NREC) * D.batch + seq) * RING;
+    __syncthreads();      // every thread has read the counter
+    if (A.is_step && tid == 0) st->rec = rec_no + 1;
+    if (!st->active) {
+        if (tid == 0) rec[0] = 0;
+        return;
+    }
     const int mode = st->mode;
     const int N0 = st->n_nodes, L0 = st->L;
     const int grow0 = seq * RT;
@@ -761,10 +801,12 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
         s_na = a;
         st->n_out = n_emit;
         for (int j = 0; j < n_emit; ++j) st->out_tokens[j] = s_out[j];
-        A.out_ring[seq * RING] = n_emit;
-        A.out_ring[seq * RING + 1] = mode == 2 ? L0 + N0 : L0 + a + 1;
-        for (int j = 0; j < n_emit; ++j) A.out_ring[seq * RING + 2 + j] = s_out[j];
+        rec[0] = n_emit;
+        rec[1] = mode == 2 ? L0 + N0 : L0 + a + 1;
+        for (int j = 0; j < n_emit; ++j) rec[2 + j] = s_out[j];
         if (mode == 0) {
+            const int rows = st->n_rows;
+            st->rows_hist[rows <= 16 ? 0 : (rows <= 32 ? 1 : (rows <= 64 ? 2 : 3))] += 1;
             st->steps += 1;
             st->emitted += n_emit;
             st->accept_hist[a < PROBES_MAX ? a : PROBES_MAX] += 1;
@@ -1013,10 +1055,10 @@ __global__ void __launch_bounds__(1024) k_tree_step(TreeArgs A) {
 void launch_tree_step(int dtype, const TreeArgs& A, cudaStream_t s, bool pdl) {
     size_t smem = (size_t)MAX_CAND * 36;
     if (dtype == 0) {
-        cudaFuncSetAttribute(k_tree_step<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        ensure_dynamic_smem(reinterpret_cast<const void*>(k_tree_step<float>), (int)smem);
         launch_k(k_tree_step<float>, dim3(A.D.batch), dim3(1024), smem, s, pdl, A);
     } else {
-        cudaFuncSetAttribute(k_tree_step<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        ensure_dynamic_smem(reinterpret_cast<const void*>(k_tree_step<__nv_bfloat16>), (int)smem);
         launch_k(k_tree_step<__nv_bfloat16>, dim3(A.D.batch), dim3(1024), smem, s, pdl, A);
     }
 }

@@ -34,7 +34,8 @@ struct TreeArgs {
     void* kcache;       // [n_layers][batch][Hkv][cap][h]
     void* vcache;
     int* err;
-    int32_t* out_ring;  // [batch][RING]: n_out, new L, tokens  (copied to the host by esp_read)
+    int32_t* out_ring;  // [NREC + 1][batch][RING]: n_out, new L, tokens  (copied to the host by esp_read)
+    int32_t is_step;    // 1: a decode step (record slot = steps so far % NREC), 0: a prefill block (slot NREC)
 };
 
 
@@ -71,6 +72,9 @@ bool attn_tc_supported(int h, int Hq, int Hkv);
 int attn_tc_create(AttnTc** out, const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap);
 void attn_tc_destroy(AttnTc* t);
 int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl);
+// the same for one call, descriptors built in the call's own frame (no allocation anywhere)
+int attn_tc_run(const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap, const AttnArgs& a,
+                int n_split_launch, cudaStream_t s);
 
 // tcgen05 GEMM: a plan holds the TMA descriptors and the stream-K partition of one weight shape
 struct TcGemm;

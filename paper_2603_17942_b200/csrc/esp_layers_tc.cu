@@ -489,7 +489,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
 struct LayersTc {
     LayersParams p;
     int grid = 0;
-    bool attr_set[64] = {};
 };
 
 int layers_tc_syncs_per_layer() { return 10; }
@@ -571,12 +570,7 @@ unsigned int layers_tc_arrivals(const LayersTc* t) { return t ? (unsigned int)(t
 int layers_tc_launch(LayersTc* t, const SeqState* st, int seq, void* kcache_seq, void* vcache_seq, unsigned int sync_base,
                      unsigned long long* timeline, cudaStream_t s) {
     if (!t || !st) return ESP_E_ARG;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ESP_E_CUDA;
-    if (!t->attr_set[dev]) {
-        if (cudaFuncSetAttribute(k_layers_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess) return ESP_E_CUDA;
-        t->attr_set[dev] = true;
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(k_layers_tc), (int)SMEM_BYTES)) return ESP_E_CUDA;
     LayersParams p = t->p;
     p.st = st;
     p.kcache = reinterpret_cast<char*>(kcache_seq);

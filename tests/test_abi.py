@@ -37,13 +37,14 @@ def test_binding_mirrors_the_header():
     import ctypes
     text = open(os.path.join(ROOT, "include", "esp.h")).read()
     for name, value in (("ESP_MAX_ROWS", P.ESP_MAX_ROWS), ("ESP_MAX_PROBES", P.ESP_MAX_PROBES),
-                        ("ESP_MAX_KPRIME", P.ESP_MAX_KPRIME)):
+                        ("ESP_MAX_KPRIME", P.ESP_MAX_KPRIME), ("ESP_MAX_UNREAD_STEPS", P.ESP_MAX_UNREAD_STEPS),
+                        ("ESP_PREFILL_CHUNK", P.ESP_PREFILL_CHUNK)):
         m = re.search(r"#define\s+%s\s+(\d+)" % name, text)
         assert m and int(m.group(1)) == value, name
     m = re.search(r"#define\s+ESP_STATIC_SCRATCH_BYTES\s+\((\d+)u\s*<<\s*(\d+)\)", text)
     assert m and (int(m.group(1)) << int(m.group(2))) == P.ESP_STATIC_SCRATCH_BYTES
     code = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    for cname, ctype in (("esp_model_cfg", P.esp_model_cfg), ("esp_spec_cfg", P.esp_spec_cfg)):
+    for cname, ctype in (("esp_model_cfg", P.esp_model_cfg), ("esp_spec_cfg", P.esp_spec_cfg), ("esp_stats", P.esp_stats)):
         end = code.index("} %s;" % cname)
         body = code[code.rindex("typedef struct {", 0, end) + len("typedef struct {"):end]
         members = []

@@ -98,7 +98,31 @@ def _run_attention(dtype, q, kc, vc, anc, depth, n_rows, L, Hq, Hkv, h, dcap=16)
     P.esp_tree_attention(dtype, b, n_rows, L, cap, Hq, Hkv, h, dcap, q, kc, vc,
                          torch.from_numpy(anc.view(np.int64)).cuda(), torch.from_numpy(depth).cuda(), out, scratch, nb)
     torch.cuda.synchronize()
+    assert P.esp_tree_attention_status(scratch) == 0       # no bounded wait ran out, no index left its range
     return out
+
+
+def test_tree_attention_status_reports_a_set_error_word():
+    """The operator reports device-side problems through the first word of its scratch.  The read-back is checked
+    from the host side: a word set by hand must come back as ESP_E_DEVICE, and the next call must clear it."""
+    Hq, Hkv, h, L = 32, 8, 128, 300
+    cap = L + R
+    q, kc, vc, _, _ = synth.random_qkv((1, R, Hq, h), (1, Hkv, cap, h), (1, Hkv, 4, h), seed=1, device="cuda")
+    anc = np.zeros((1, R, 2), np.uint64)
+    for i in range(R):
+        anc[0, i, i // 64] = np.uint64(1) << np.uint64(i % 64)
+    nb = P.esp_tree_attention_scratch_bytes(1, Hq, h, cap)
+    scratch = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+    args = (1, 1, 4, L, cap, Hq, Hkv, h, 16, q, kc, vc, torch.from_numpy(anc.view(np.int64)).cuda(),
+            torch.zeros((1, R), dtype=torch.int32, device="cuda"), torch.zeros_like(q), scratch, nb)
+    P.esp_tree_attention(*args)
+    assert P.esp_tree_attention_status(scratch) == 0
+    scratch[:4] = torch.tensor([2, 0, 0, 0], dtype=torch.uint8, device="cuda")     # as a kernel would record DEV_E_INDEX
+    with pytest.raises(P.EspError) as e:
+        P.esp_tree_attention_status(scratch)
+    assert e.value.code == -5                               # ESP_E_DEVICE
+    P.esp_tree_attention(*args)
+    assert P.esp_tree_attention_status(scratch) == 0
 
 
 @pytest.mark.parametrize("batch,L,dt", [(1, 4096, "bf16"), (16, 4096, "bf16"), (2, 777, "bf16"), (1, 0, "bf16"),

@@ -465,3 +465,48 @@ def test_host_side_errors(pu):
     assert e.value.code == -4                                   # sequence full
     assert h.stats().device_error == 0
     h.close()
+
+
+# ------------------------------------------------------------------ asynchronous steps
+def test_async_steps_then_reads_equal_synchronous_steps(pu):
+    """esp_step_async only enqueues; every step keeps its own result record and esp_read hands them back oldest
+    first.  A run of N enqueued steps followed by N reads must give, step by step, the tokens of N synchronous
+    steps, the same final state and the same continuation -- also while the host, which between reads knows
+    the cache length only as an upper bound (k + 1 per unread step), sizes the attention launches for more
+    cache splits than there are (the bound crosses a split boundary here: 256-position splits, L near 250)."""
+    import paper_2603_17942_b200 as P
+    shape = BF16_SMALL
+    w = synth.make_weights(shape, seed=7, gain_jitter=True, std=0.05)
+    wd = pu.to_device(w)
+    prompt = synth.make_prompt(shape.vocab, 236, 9)
+    spec = O.SpecCfg(n_probes=3, topk=5, max_nodes=16, expand_width=0, n_anchor=1)
+    hs = P.Handle(shape, pu.c_spec(spec), wd, max_seq_len=700)
+    ha = P.Handle(shape, pu.c_spec(spec), wd, max_seq_len=700)
+    assert hs.prefill(prompt) == ha.prefill(prompt)
+    n = 40
+    sync_tokens = [hs.step() for _ in range(n)]
+    for _ in range(n):
+        ha.step_async()
+    async_tokens = [ha.read() for _ in range(n)]
+    assert async_tokens == sync_tokens
+    assert ha.read() == []                                   # nothing unread is left
+    sa, ss = ha.state(), hs.state()
+    assert sa["L"] == ss["L"] and sa["n_rows"] == ss["n_rows"]
+    assert list(sa["row_token"][:sa["n_rows"]]) == list(ss["row_token"][:ss["n_rows"]])
+    assert np.array_equal(sa["mask_vec"], ss["mask_vec"])
+    assert ha.stats().emitted == hs.stats().emitted and ha.stats().steps == hs.stats().steps
+    assert [ha.step() for _ in range(6)] == [hs.step() for _ in range(6)]
+    assert sum(hs.stats().rows_hist) == hs.stats().steps        # every step is counted in the block-size histogram
+    assert ha.stats().device_error == 0 and hs.stats().device_error == 0
+    # one step more than there are result records is refused, and nothing is lost
+    hb = P.Handle(shape, pu.c_spec(pu.GREEDY), wd, max_seq_len=236 + P.ESP_MAX_UNREAD_STEPS + 300)
+    hb.prefill(prompt)
+    for _ in range(P.ESP_MAX_UNREAD_STEPS):
+        hb.step_async()
+    with pytest.raises(P.EspError) as e:
+        hb.step_async()
+    assert e.value.code == -7                                # ESP_E_STATE
+    first = hb.read()
+    hb.step_async()                                          # one record is free again
+    assert len(first) == 1
+    ha.close(); hs.close(); hb.close()

@@ -14,6 +14,7 @@ import torch
 
 import synth
 import paper_2603_17942_b200 as P
+from oracle import esp as O
 
 pytestmark = pytest.mark.gpu
 
@@ -82,6 +83,33 @@ def test_static_scratch_attention_matches_caller_scratch_twice_in_a_row():
     assert torch.equal(got1[:, :first["M"]], ref1[:, :first["M"]])
     assert torch.equal(got2[:, :second["M"]], ref2[:, :second["M"]])
     assert torch.equal(_static(first)[:, :first["M"]], ref1[:, :first["M"]])   # and back again
+    assert P.esp_tree_attention_status(None) == 0                              # no device-side problem recorded in the array
+    # the call takes no device memory: free memory is the same before and after a call into a ready output tensor
+    x, out = first, torch.zeros_like(first["q"])
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    P.esp_tree_attention_static(1, x["batch"], x["M"], x["L"], x["cap"], x["Hq"], x["Hkv"], x["h"], 16, x["q"], x["kc"],
+                                x["vc"], x["anc"], x["depth"], out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert torch.equal(out[:, :x["M"]], ref1[:, :x["M"]])
+
+
+def test_static_scratch_attention_against_the_oracle():
+    """Not only equal to the sibling entry point: the rows of one sequence against the CPU oracle's tree attention
+    (two passes over each row's own key list), at the tolerance of the operator tests."""
+    x = _inputs(L=900, seed=24)
+    got = _static(x)[0, :x["M"]].float().cpu().numpy()
+    L, M = x["L"], x["M"]
+    anc = x["anc"].cpu().numpy().view(np.uint64)[0]
+    vis = np.zeros((M, M), np.uint8)
+    for r in range(M):
+        for i in range(M):
+            vis[r, i] = (int(anc[r, i // 64]) >> (i % 64)) & 1
+    kc, vc = x["kc"][0].float().permute(1, 0, 2).cpu().numpy(), x["vc"][0].float().permute(1, 0, 2).cpu().numpy()
+    ref = O.tree_attention(x["q"][0, :M].float().cpu().numpy(), kc[:L], vc[:L], kc[L:L + M], vc[L:L + M], vis)
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= 2e-2
 
 
 def test_static_scratch_attention_rejects_shapes_beyond_its_array():
