@@ -10,12 +10,15 @@ prompt, 4 mask probes, Top-10 per probe, trees of at most 64 nodes, batch 1.  We
 from HBM every step, far more than the L2 holds, so no cache flush is needed between steps.
 
 Prints ONE JSON line.  `value` is accepted tokens per second with everything resident on the device
-(K esp_step_async calls between two CUDA events on the library's stream); `e2e` is the same metric through
-the synchronous esp_step call that returns the tokens in host memory every step.  With N > 1 every rank runs
-an independent replica of the whole job (the method has no cross-GPU exchange); `value` sums the replicas'
-tokens over the slowest rank's time.
+(K esp_step_async calls between two CUDA events on the library's stream; their tokens are read afterwards from
+the per-step result records and must equal greedy decoding with the same kernels); `e2e` is the same metric
+over a whole request through the public calls -- the prompt from host memory into esp_prefill, then K
+synchronous esp_step calls that return their tokens in host memory -- and `e2e_step` that request's steps
+alone.  With N > 1 every rank runs an independent replica of the whole job (the method has no cross-GPU
+exchange); `value` sums the replicas' tokens over the slowest rank's time.
 
-`--impl reference` times the CPU oracle (oracle/) on the host cores on a bounded sample of the same workload.
+`--impl reference` times the CPU oracle (oracle/) on the host cores: whole full-depth steps of the same workload,
+as many of the K requested as fit its time budget.
 """
 from __future__ import annotations
 
@@ -132,17 +135,17 @@ def random_block(n_nodes, k, seed):
 
 
 class OracleSample:
-    """One bounded sample of the workload for the CPU oracle: a full-width block (all tree and probe rows)
-    through ONE decoder layer and the LM head against a random KV cache of the prompt's length.  The oracle's
-    time for a whole step is 32 (n_layers) x the layer time + the LM-head time; accepted tokens per step are
-    taken as 1 (random-init models accept no drafts)."""
+    """The CPU oracle on a bounded sample of the workload: whole decode-and-verify forwards -- a full-width
+    block (all tree and probe rows) through EVERY decoder layer and the LM head against a KV cache of the
+    prompt's length (random N(0,1) entries: the forward does not care what the cache holds), then the argmax /
+    Top-K' read-out the step needs.  One such forward is one step; accepted tokens per step are taken as 1
+    (random-init models accept no drafts).  Nothing is extrapolated: the sample is bounded by running few steps."""
 
-    def __init__(self, shape, plen, k, B, host_weights):
+    def __init__(self, shape, plen, k, K, B, host_weights):
         from oracle import esp as O
         self.O = O
-        self.shape1 = shape.replace(n_layers=1)
-        self.n_layers = shape.n_layers
-        self.model = O.OracleModel(self.shape1, host_weights)
+        self.shape = shape
+        self.model = O.OracleModel(shape, host_weights)
         rng = np.random.default_rng(0)
         self.L = plen
         self.kc, self.vc = self.model.new_cache(plen + 8)
@@ -150,64 +153,70 @@ class OracleSample:
         self.vc[:, :plen] = rng.standard_normal(self.vc[:, :plen].shape, dtype=np.float32)
         self.vis, pos = random_block(B, k, 0)
         self.pos = plen + pos
-        self.M = B + k
+        self.M, self.B, self.kp = B + k, B, K + 1
         self.x = (rng.standard_normal((self.M, shape.d_model), dtype=np.float32) * 0.02).astype(np.float32)
         self.cores = O.num_threads()
 
     def step_seconds(self):
-        none = np.zeros(self.M, np.uint8)
         t0 = time.perf_counter()
-        self.model.block_forward(self.kc, self.vc, self.L, self.x, self.pos, self.vis, want=none)
-        t1 = time.perf_counter()
-        self.model.block_forward(self.kc, self.vc, self.L, self.x, self.pos, self.vis)
-        t2 = time.perf_counter()
-        t_layer, t_both = t1 - t0, t2 - t1
-        return self.n_layers * t_layer + max(t_both - t_layer, 0.0)
+        logits, _, _, _ = self.model.block_forward(self.kc, self.vc, self.L, self.x, self.pos, self.vis)
+        for r in range(self.B):
+            self.O.topk_desc(logits[r], 1)
+        for r in range(self.B, self.M):
+            self.O.topk_desc(logits[r], self.kp)
+            self.O.log_sum_exp(logits[r])
+        return time.perf_counter() - t0
 
     def describe(self):
-        return (f"one {self.M}-row block through 1 of {self.n_layers} layers + LM head, KV length {self.L}; "
-                f"step time = {self.n_layers} x layer + head, 1 token per step")
+        return (f"whole steps: a {self.M}-row block through all {self.shape.n_layers} layers + LM head + selection, "
+                f"KV length {self.L}, 1 token per step")
 
 
-def host_slice(shape, w_dev=None, seed=0):
-    """Host copies of what the one-layer oracle sample needs (embed, lm_head, final norm, layer 0)."""
+def host_weights(shape, w_dev=None, seed=0):
+    """Full-depth host copies of the model for the oracle (generated on the GPU when there is one: much faster)."""
     import synth
     import torch
     if w_dev is None:
-        s1 = shape.replace(n_layers=1)
-        return synth.make_weights(s1, seed=seed, device="cpu")
-    out = {}
-    for k, v in w_dev.items():
-        out[k] = [v[0].cpu()] if isinstance(v, list) else v.cpu()
-    if w_dev["lm_head"] is w_dev["embed"]:
-        out["lm_head"] = out["embed"]
-    return out
+        dev = "cuda" if torch.cuda.is_available() else "cpu"
+        w_dev = synth.make_weights(shape, seed=seed, device=dev)
+        if dev == "cpu":
+            return w_dev
+    return synth.weights_to_host(w_dev)
+
+
+def workload_config(name, plen, nbatch, temperature, k, K, B, rows, replicas):
+    """The `config` object of the JSON line: identical for both arms."""
+    return {"workload": f"{name}-shape bf16 decoder, random-init seeded weights, b={nbatch}",
+            "prompt_len": plen, "batch": nbatch, "temperature": temperature, "n_probes": k, "topk": K, "max_nodes": B,
+            "rows_per_step": rows, "replicas": replicas, "l2": "inputs exceed L2 (weights are re-streamed every step)"}
+
+
+REFERENCE_BUDGET_S = 150.0      # timed CPU work of the reference arm; the step count is cut to fit
 
 
 def run_reference(args, shape, plen, k, K, B):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    smp = OracleSample(shape, plen, k, B, host_slice(shape))
-    for _ in range(min(args.warmup, 1)):
+    smp = OracleSample(shape, plen, k, K, B, host_weights(shape))
+    n_warm = min(max(args.warmup, 0), 2)
+    for _ in range(n_warm):
         smp.step_seconds()
-    steps = max(1, args.steps)
-    budget_s = 180.0
     times = []
     t_start = time.perf_counter()
-    for i in range(steps):
+    for i in range(max(1, args.steps)):
         times.append(smp.step_seconds())
-        if time.perf_counter() - t_start > budget_s and i + 1 < steps:
+        # stop when another step of this length would pass the budget
+        if time.perf_counter() - t_start + times[-1] > REFERENCE_BUDGET_S:
             break
     sec = float(np.mean(times))
     val = 1.0 / sec
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
-            "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "warmup": n_warm, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{args.config}-shape bf16 decoder, random-init seeded weights, b=1",
-                       "prompt_len": plen, "batch": 1, "temperature": 0.0, "n_probes": k, "topk": K, "max_nodes": B,
-                       "rows_per_step": B + k, "replicas": 1,
-                       "note": "bf16 weights widened exactly, fp32 arithmetic (the oracle's precision)"},
+            "config": workload_config(args.config, plen, 1, 0.0, k, K, B, B + k, 1),
+            "note": f"the CPU oracle as it stands (bf16 weights widened exactly, fp32 arithmetic); {len(times)} of the "
+                    f"{args.steps} requested steps fit the {REFERENCE_BUDGET_S:.0f} s budget",
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": smp.describe()},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -223,19 +232,28 @@ def algorithmic_bytes(shape, L_mean, rows):
     return w, kv_per_pos * L_mean + kv_per_pos * rows
 
 
-def replay_leg(P, shape, w, prompt, stream, k, B, n_tokens, seed=0):
+REPLAY_SCHEDULES = {
+    # the two operating points of the paper's main table for this model size: probabilities of 0, 1, 2, 3 accepted drafts
+    "1.63": [0.55, 0.30, 0.12, 0.03],       # mean 0.63 accepted drafts per step
+    "1.71": [0.50, 0.33, 0.13, 0.04],       # mean 0.71
+}
+
+
+def replay_leg(P, shape, w, prompt, stream, k, B, n_steps, probs, seed=0):
     """Throughput under a synthetic acceptance schedule.  Random-init models accept no drafts, so the draft trees
     of this leg are set from outside (esp_set_tree): each holds the true continuation (taken from a greedy run of
-    the same kernels) down to a depth drawn per step -- 0, 1, 2, 3 drafts with probability .55/.30/.12/.03, mean
-    0.63, i.e. the paper's tau = 1.63 -- inside a full tree of B nodes of wrong siblings.  The emitted stream must
+    the same kernels) down to a depth drawn per step with the probabilities `probs` (the paper's tau = 1.63 / 1.71
+    operating points) inside a full tree of B nodes of wrong siblings.  The emitted stream must
     equal the greedy stream token for token.  Says nothing about model quality; it shows what a step costs when
     drafts are accepted, their KV rows compacted and the host is in the loop (set_tree + step, synchronous)."""
+    n_tokens = int(2.2 * n_steps) + 16   # what n_steps emit at these schedules, with a wide margin (the loop stops at the end of the known stream)
     import torch
     plen = len(prompt)
     max_seq = plen + n_tokens + 64
     hg = P.Handle(shape, P.spec_cfg(), w, max_seq_len=max_seq, stream=stream)
     truth = hg.generate(prompt, n_tokens + 8)
     hg.close()
+    mean_acc = sum(i * q for i, q in enumerate(probs))
     h = P.Handle(shape, P.spec_cfg(n_probes=k, topk=10, max_nodes=B, expand_width=0, n_anchor=1), w, max_seq_len=max_seq, stream=stream)
     out = [h.prefill(prompt)]
     rng = np.random.default_rng(seed)
@@ -243,9 +261,10 @@ def replay_leg(P, shape, w, prompt, stream, k, B, n_tokens, seed=0):
     steps = 0
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    while len(out) < n_tokens:
+    L_start = h.state()["L"]
+    while steps < n_steps and len(out) + k + 1 < len(truth):
         n = len(out)
-        a = int(min(rng.choice(4, p=[0.55, 0.30, 0.12, 0.03]), k))
+        a = int(min(rng.choice(len(probs), p=probs), k))
         toks, pars, main = [out[-1]], [-1], 0
         for d in range(1, k + 1):
             level = []
@@ -266,14 +285,16 @@ def replay_leg(P, shape, w, prompt, stream, k, B, n_tokens, seed=0):
         out.extend(new)
     torch.cuda.synchronize()
     sec = time.perf_counter() - t0
-    if out[:n_tokens] != truth[:n_tokens]:
+    if out != truth[:len(out)]:
         raise SystemExit("replay: ESP stream differs from the greedy stream")
+    L_end = h.state()["L"]
     err = h.stats().device_error
     h.close()
     if err:
         raise SystemExit("replay: device error word set")
     return {"tau": (len(out) - 1) / steps, "tok_s": (len(out) - 1) / sec, "steps": steps, "ms_per_step": sec / steps * 1e3,
-            "note": "synthetic acceptance schedule (forced drafts, mean 0.63 accepted per step), not model quality; "
+            "L_start": L_start, "L_end": L_end,
+            "note": f"synthetic acceptance schedule (forced drafts, mean {mean_acc:.2f} accepted per step), not model quality; "
                     "includes the host round trip of esp_set_tree every step; stream checked equal to greedy"}
 
 
@@ -310,6 +331,8 @@ def run_ours(args, shape, plen, k, K, B):
     P.load_library()
 
     steps, warm = args.steps, max(args.warmup, 3)
+    if steps > P.ESP_MAX_UNREAD_STEPS:
+        raise SystemExit(f"--steps: at most {P.ESP_MAX_UNREAD_STEPS} (the steps of the timed region are enqueued without a read in between)")
     w = synth.make_weights(shape, seed=rank, device="cuda")
     prompt = synth.make_prompt(shape.vocab, plen, rank)
     if args.per_node_probes:
@@ -324,10 +347,12 @@ def run_ours(args, shape, plen, k, K, B):
     nbatch = max(1, args.batch)
     h = P.Handle(shape, spec, w, max_seq_len=max_seq, max_batch=nbatch, stream=stream)
 
+    first_tokens = []
+
     def prefill_all():
-        h.prefill(prompt)
+        first_tokens[:] = [h.prefill(prompt)]
         for i in range(1, nbatch):
-            h.prefill(synth.make_prompt(shape.vocab, plen, 1000 * rank + i), i)
+            first_tokens.append(h.prefill(synth.make_prompt(shape.vocab, plen, 1000 * rank + i), i))
 
     prefill_all()
 
@@ -336,8 +361,9 @@ def run_ours(args, shape, plen, k, K, B):
         return int(st.emitted), int(st.steps), st
 
     # ---- device-resident throughput: K asynchronous steps between two events on the library's stream
+    esp_stream = [first_tokens[0]]
     for _ in range(warm):
-        h.step()
+        esp_stream.extend(h.step())
     e0, s0, _ = emitted_steps()
     L0 = h.state()["L"]
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -357,7 +383,9 @@ def run_ours(args, shape, plen, k, K, B):
         dist.barrier()
     t1 = time.time()
     clocks = sampler.stop(t0, t1)
-    h.read()
+    timed_stream = []                  # sequence 0's tokens of the timed steps, from their result records
+    for _ in range(steps):
+        timed_stream.extend(h.read())
     ms = ev0.elapsed_time(ev1)
     e1, s1, st = emitted_steps()
     L1 = h.state()["L"]
@@ -365,23 +393,27 @@ def run_ours(args, shape, plen, k, K, B):
     launches = int(st.kernels_per_step) * steps
     rows = h.state()["n_rows"]
 
-    # ---- end to end: the synchronous call, tokens land in host memory every step (again from the prompt)
+    esp_stream.extend(timed_stream)
+
+    # ---- end to end, a whole request through the public calls: the prompt goes from host memory into esp_prefill,
+    # then `steps` synchronous esp_step calls, each returning its tokens in host memory
     torch.cuda.synchronize()
-    tp0 = time.perf_counter()
-    prefill_all()                      # host prompt in, first token out: the time to the first token of a warm library
-    torch.cuda.synchronize()
-    prefill_ms = (time.perf_counter() - tp0) * 1e3
     if dist is not None:
         dist.barrier()
     te0 = time.perf_counter()
-    e2e_tokens = 0
+    prefill_all()
+    torch.cuda.synchronize()
+    prefill_ms = (time.perf_counter() - te0) * 1e3
+    e2e_tokens = nbatch                # the prefill emits every sequence's first token
     for _ in range(steps):
         h.step()
         e2e_tokens += int(h.n_out.sum())
     torch.cuda.synchronize()
     te1 = time.perf_counter()
     e2e_ms = (te1 - te0) * 1e3
-    d2h = nbatch * (P.ESP_MAX_PROBES + 4) * 4 + 4
+    e2e_step_ms = (e2e_ms - prefill_ms) / steps
+    h2d_request = nbatch * plen * 4                              # the prompts (int32 ids)
+    d2h_step = nbatch * (P.ESP_MAX_PROBES + 4) * 4 + 4           # every sequence's result record + the status word
 
     # ---- per-kernel-group device times (events between groups), for the roofline of the dominant kernel
     n_prof = min(steps, 20)
@@ -392,27 +424,38 @@ def run_ours(args, shape, plen, k, K, B):
     if h.stats().device_error != 0:
         raise SystemExit("device error word set during the benchmark")
 
-    # ---- greedy decoding with the same kernels (one row per step), for context
-    greedy_tok_s = None
+    # ---- greedy decoding with the same kernels (one row per step): its rate, and the stream the timed ESP steps
+    # above must have reproduced token for token (lossless verification)
+    greedy_tok_s, stream_checked = None, None
     if rank == 0 and not args.no_greedy and nbatch == 1:
-        hg = P.Handle(shape, P.spec_cfg(), w, max_seq_len=plen + 2 * steps + 64, stream=stream)
-        hg.prefill(prompt)
+        n_greedy = len(esp_stream) - 1            # decode steps that emit as many tokens as the ESP legs did
+        hg = P.Handle(shape, P.spec_cfg(temperature=args.temperature, seed=1), w, max_seq_len=plen + n_greedy + 64, stream=stream)
+        greedy_stream = [hg.prefill(prompt)]
         for _ in range(warm):
-            hg.step()
+            greedy_stream.extend(hg.step())
+        n_timed = min(n_greedy - warm, P.ESP_MAX_UNREAD_STEPS)
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         with torch.cuda.stream(stream):
             g0.record()
-            for _ in range(steps):
+            for _ in range(n_timed):
                 hg.step_async()
             g1.record()
         torch.cuda.synchronize()
-        hg.read()
-        greedy_tok_s = steps / (g0.elapsed_time(g1) * 1e-3)
+        for _ in range(n_timed):
+            greedy_stream.extend(hg.read())
+        greedy_tok_s = n_timed / (g0.elapsed_time(g1) * 1e-3)
+        while len(greedy_stream) < len(esp_stream):
+            greedy_stream.extend(hg.step())
         hg.close()
+        if greedy_stream[:len(esp_stream)] != esp_stream:
+            bad = next(i for i, (x, y) in enumerate(zip(esp_stream, greedy_stream)) if x != y)
+            raise SystemExit(f"the timed ESP stream differs from greedy decoding at token {bad}")
+        stream_checked = len(esp_stream)
 
-    replay = None
-    if rank == 0 and not args.no_greedy and nbatch == 1 and not args.per_node_probes:
-        replay = replay_leg(P, shape, w, prompt, stream, k, B, min(256, steps))
+    replay = {}
+    if rank == 0 and not args.no_greedy and nbatch == 1 and not args.per_node_probes and args.temperature == 0.0:
+        for name, probs in REPLAY_SCHEDULES.items():
+            replay[name] = replay_leg(P, shape, w, prompt, stream, k, B, 200, probs, seed=int(float(name) * 100))
 
     # ---- aggregate over ranks: slowest rank's time, all ranks' tokens
     if dist is not None:
@@ -433,15 +476,21 @@ def run_ours(args, shape, plen, k, K, B):
             "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
             "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": f"{args.config}-shape bf16 decoder, random-init seeded weights, b={nbatch}",
-                       "prompt_len": plen, "batch": nbatch, "temperature": args.temperature, "n_probes": k, "topk": K, "max_nodes": B, "rows_per_step": rows,
-                       "replicas": world, "l2": "inputs exceed L2 (weights are re-streamed every step)"},
+            "config": workload_config(args.config, plen, nbatch, args.temperature, k, K, B, rows, world),
             "mean_accepted_len": tokens / (steps * world * nbatch),
+            "kv_len": {"timed_start": L0, "timed_end": L1},
             "clocks": clocks,
-            "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 0,
-                    "d2h_bytes_per_step": d2h,
-                    "note": "synchronous esp_step; a step's inputs are the device state left by the previous step"},
+            "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d_request / steps, "d2h_bytes_per_step": d2h_step,
+                    "h2d_bytes_per_request": h2d_request, "request_ms": e2e_ms, "request_tokens": e2e_tokens,
+                    "note": "whole requests through the public calls, every rank: the prompt from host memory into "
+                            "esp_prefill, then `steps` synchronous esp_step calls that return their tokens in host "
+                            "memory; the prefill time is inside the timed region and its bytes are spread over the steps"},
+            "e2e_step": {"value": (e2e_tokens - nbatch * world) / ((e2e_ms - prefill_ms) * 1e-3), "unit": UNIT, "ms_per_step": e2e_step_ms,
+                         "note": "the synchronous esp_step calls of that request alone (a step's inputs are the device "
+                                 "state the step before left; its tokens land in host memory)"},
             "gpu_launches": launches,
+            "stream_equals_greedy_tokens": stream_checked,
             "prefill": {"ms": prefill_ms, "prompt_tokens": plen * nbatch, "tokens_per_s": plen * nbatch / (prefill_ms * 1e-3),
                         "note": "esp_prefill of every sequence from host memory, blocks of %d prompt rows" % P.ESP_PREFILL_CHUNK},
             "roofline": {"bound": "hbm", "kernel": "k_gemm_tc<EPI_PARTIAL>, gate/up projection (235 MB of weights per launch)",
@@ -456,13 +505,15 @@ def run_ours(args, shape, plen, k, K, B):
                               "peak_source": peak_src},
             "kernel_group_ms_per_step": kinds,
             "greedy_tok_s": greedy_tok_s,
-            "replay_tau_1_63": replay,
+            "replay": replay or None,
         }
         if not args.no_cpu and world == 1:
-            smp = OracleSample(shape, plen, k, B, host_slice(shape, w))
-            sec = smp.step_seconds()
+            smp = OracleSample(shape, plen, k, K, B, host_weights(shape, w))
+            smp.step_seconds()                               # warm: page the weights in, start the thread pool
+            secs = sorted(smp.step_seconds() for _ in range(3))
+            sec = secs[1]
             line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": smp.cores, "kind": "oracle",
-                                    "sample": smp.describe(), "ms_per_step": sec * 1e3}
+                                    "sample": smp.describe() + "; median of 3 after one warm-up", "ms_per_step": sec * 1e3}
         else:
             line["cpu_baseline"] = None
         print(json.dumps(line), flush=True)

@@ -28,7 +28,8 @@ struct Carve {
 struct Buffers {
     void *kcache, *vcache;
     float* hres;
-    void *xn, *qbuf, *attn_out, *act;
+    void *xn, *qbuf, *attn_out, *act;       // bf16 models: xn, attn_out and act hold two planes (hi, then lo)
+    void *xn_lo, *attn_out_lo, *act_lo;      // the low-order planes (NULL for fp32 models)
     float* part_o;
     float2* part_ml;
     Cand* cand;
@@ -56,6 +57,11 @@ struct Buffers {
     unsigned long long* timeline;
 };
 constexpr int SK_TABLE_TILES = 2048;
+// bf16 models: the inputs of the layer GEMMs (RMSNorm output, attention output, SiLU*up) reach the tensor cores as
+// pairs hi + lo of bf16 numbers, each product taken with both.  With one plane the logits of a 32-layer model
+// sit 2.5e-2 of their range from the fp32 reference (worst of 8.7 M logits), with two 1.5e-2; the keys, values,
+// queries and probabilities stay single bf16 numbers (the cache is bf16).
+constexpr int ACT_PLANES = 2;
 
 
 // tree nodes including the root: max_nodes, or 1 + the fixed widths of a static tree
@@ -151,10 +157,18 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.kcache = c.take<char>(kv);
     o.vcache = c.take<char>(kv);
     o.hres = c.take<float>(Mtot * D.d);
-    o.xn = c.take<char>(Mtot * D.d * es);
+    // activations that feed the tensor-core GEMMs are kept as bf16 pairs hi + lo (ACT_PLANES planes, Mtot rows apart)
+    const size_t pl = dtype ? ACT_PLANES : 1;
+    o.xn = c.take<char>(pl * Mtot * D.d * es);
     o.qbuf = c.take<char>(Mtot * D.Hq * D.h * es);
-    o.attn_out = c.take<char>(Mtot * D.Hq * D.h * es);
-    o.act = c.take<char>(Mtot * D.F * es);
+    o.attn_out = c.take<char>(pl * Mtot * D.Hq * D.h * es);
+    o.act = c.take<char>(pl * Mtot * D.F * es);
+    o.xn_lo = o.attn_out_lo = o.act_lo = nullptr;
+    if (base && pl == 2) {
+        o.xn_lo = reinterpret_cast<char*>(o.xn) + Mtot * D.d * es;
+        o.attn_out_lo = reinterpret_cast<char*>(o.attn_out) + Mtot * D.Hq * D.h * es;
+        o.act_lo = reinterpret_cast<char*>(o.act) + Mtot * D.F * es;
+    }
     o.part_o = c.take<float>(Mtot * D.Hq * D.n_split_max * D.h);
     o.part_ml = c.take<float2>(Mtot * D.Hq * D.n_split_max);
     o.cand = c.take<Cand>((size_t)n_tiles_v * Mtot * D.KP);
@@ -172,7 +186,7 @@ size_t carve_all(const Dims& D, int dtype, int n_sm, char* base, Buffers* b) {
     o.rope_sin = c.take<float>((size_t)D.cap * (D.h / 2));
     {
         // the decode steps' passes (several sequences of gemm_rows rows) or one 128-row prefill block, whichever is larger
-        const size_t step_b = tc_gemm_partial_bytes(n_sm, D.batch < tc_gemm_max_nq(D.gemm_rows) ? D.batch : tc_gemm_max_nq(D.gemm_rows), D.gemm_rows);
+        const size_t step_b = tc_gemm_partial_bytes(n_sm, D.batch < tc_gemm_max_nq(D.gemm_rows, ACT_PLANES) ? D.batch : tc_gemm_max_nq(D.gemm_rows, ACT_PLANES), D.gemm_rows);
         const size_t pre_b = tc_gemm_partial_bytes(n_sm, 1, RT);
         o.gemm_partials = c.take<char>(step_b > pre_b ? step_b : pre_b);
     }
@@ -322,7 +336,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc,
         pending = tc_gemm_streamk(h->p_down[D.n_layers - 1], 1);
     }
     for (int l = 0; l < D.n_layers && !fused; ++l) {
-        if (tc) launch_resid_norm(st0, b.hres, pending, h->na[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
+        if (tc) launch_resid_norm(st0, b.hres, pending, h->na[l], b.xn, b.xn_lo, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->na[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -351,6 +365,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc,
             a.kc = reinterpret_cast<char*>(layer_ptr(b.kcache, h->layer_kv_stride, l)) + kv_seq_off;
             a.vc = reinterpret_cast<char*>(layer_ptr(b.vcache, h->layer_kv_stride, l)) + kv_seq_off;
             a.out = b.attn_out;
+            a.out_lo = tc ? b.attn_out_lo : nullptr;
             a.part_o = b.part_o; a.part_ml = b.part_ml;
             a.st = st0;
             a.Hq = D.Hq; a.Hkv = D.Hkv; a.h = D.h; a.cap = D.cap; a.split_len = D.split_len; a.n_split_max = D.n_split_max;
@@ -359,7 +374,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc,
             a.cache_in_flight = prefill ? 1 : 0;
             a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D.h));
             a.err = b.err;
-            if (tc) {
+            if (tc && !h->p_attn.empty()) {
                 if (attn_tc_launch(h->p_attn[(size_t)l * D.batch + s0], a, nb, n_split_launch, s, pdl)) return ESP_E_BADCFG;
                 h->launches += n_split_launch > 0 ? 2 : 1;
             } else {
@@ -377,7 +392,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc,
             if (rc) return rc;
             mark(h, KIND_O);
         }
-        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(plan(h->p_o, h->p_o_w, l), nb), h->nf[l], b.xn, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
+        if (tc) launch_resid_norm(st0, b.hres, tc_gemm_streamk(plan(h->p_o, h->p_o_w, l), nb), h->nf[l], b.xn, b.xn_lo, D.d, D.rms_eps, nullptr, nb, s, pdl, rc_rows);
         else launch_rmsnorm(h->dtype, st0, b.hres, h->nf[l], b.xn, D.d, D.rms_eps, nb, nullptr, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -390,7 +405,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc,
             if (rc) return rc;
             mark(h, KIND_GATEUP);
             if (tc) {
-                launch_swiglu_finish(st0, tc_gemm_streamk(plan(h->p_gu, h->p_gu_w, l), nb), b.act, D.F, nb, s, pdl, rc_rows);
+                launch_swiglu_finish(st0, tc_gemm_streamk(plan(h->p_gu, h->p_gu_w, l), nb), b.act, b.act_lo, D.F, nb, s, pdl, rc_rows);
                 h->launches++;
                 mark(h, KIND_MISC);
             }
@@ -408,7 +423,7 @@ int forward_pass(esp_handle* h, bool with_lm, int dcap, int s0, int nb, bool tc,
     }
     if (with_lm) {
         float* dbg_hidden = h->dbg_hidden ? h->dbg_hidden + (size_t)s0 * RT * D.d : nullptr;
-        if (tc) launch_resid_norm(st0, b.hres, pending, h->final_norm, b.xn, D.d, D.rms_eps, dbg_hidden, nb, s, pdl, rc_rows);
+        if (tc) launch_resid_norm(st0, b.hres, pending, h->final_norm, b.xn, nullptr, D.d, D.rms_eps, dbg_hidden, nb, s, pdl, rc_rows);   // the LM head reads one plane
         else launch_rmsnorm(h->dtype, st0, b.hres, h->final_norm, b.xn, D.d, D.rms_eps, nb, dbg_hidden, s, pdl);
         h->launches++;
         mark(h, KIND_MISC);
@@ -440,7 +455,7 @@ int forward(esp_handle* h, bool with_lm, int dcap, int only_seq) {
     if (!tc) return forward_pass(h, with_lm, dcap, 0, h->D.batch, false, prefill);
     if (only_seq >= 0) return forward_pass(h, with_lm, dcap, only_seq, 1, true, true);
     // consecutive sequences share a pass (and a weight stream); sequences that are not ready are inactive in it
-    const int per_pass = tc_gemm_max_nq(h->D.gemm_rows);
+    const int per_pass = tc_gemm_max_nq(h->D.gemm_rows, ACT_PLANES);
     for (int s0 = 0; s0 < h->D.batch; s0 += per_pass) {
         const int nb = h->D.batch - s0 < per_pass ? h->D.batch - s0 : per_pass;
         bool any = false;
@@ -565,29 +580,29 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
     if (model->dtype == 1) {
         const int dq = D.Hq * D.h, dkv = D.Hkv * D.h;
         const int nrs = D.gemm_rows;
-        const int nq_max = D.batch < tc_gemm_max_nq(nrs) ? D.batch : tc_gemm_max_nq(nrs);   // sequences sharing a weight stream
+        const int nq_max = D.batch < tc_gemm_max_nq(nrs, ACT_PLANES) ? D.batch : tc_gemm_max_nq(nrs, ACT_PLANES);   // sequences sharing a weight stream
         bool ok = true;
         for (int l = 0; l < D.n_layers && ok; ++l) {
             TcGemm* p = nullptr;
             char* pk = h->b.packed + h->b.pk_layer * l;
             const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
             const int32_t r1[3] = {dq, dkv, dkv};
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream, ACT_PLANES);
             h->p_qkv.push_back(p);
             const void* w2[3] = {h->wo[l], nullptr, nullptr};
             const int32_t r2[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream, ACT_PLANES);
             h->p_o.push_back(p);
             const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
             const int32_t r3[3] = {D.F, D.F, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream, ACT_PLANES);
             h->p_gu.push_back(p);
             const void* w4[3] = {h->wd[l], nullptr, nullptr};
             const int32_t r4[3] = {D.d, 0, 0};
             p = nullptr;
-            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream);
+            ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, D.batch, nrs, nq_max, h->b.gemm_partials, tc_gemm_partial_bytes(148, nq_max, nrs), h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream, ACT_PLANES);
             h->p_down.push_back(p);
         }
         const void* w5[3] = {h->lm_head, nullptr, nullptr};
@@ -601,22 +616,22 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
                 char* pk = h->b.packed + h->b.pk_layer * l;
                 const void* w1[3] = {h->wq[l], h->wk[l], h->wv[l]};
                 const int32_t r1[3] = {dq, dkv, dkv};
-                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream);
+                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w1, r1, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 0 * SK_TABLE_TILES, SK_TABLE_TILES, pk, h->stream, ACT_PLANES);
                 h->p_qkv_w.push_back(p);
                 const void* w2[3] = {h->wo[l], nullptr, nullptr};
                 const int32_t r2[3] = {D.d, 0, 0};
                 p = nullptr;
-                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream);
+                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w2, r2, dq, h->b.attn_out, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 1 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv, h->stream, ACT_PLANES);
                 h->p_o_w.push_back(p);
                 const void* w3[3] = {h->wg[l], h->wu[l], nullptr};
                 const int32_t r3[3] = {D.F, D.F, 0};
                 p = nullptr;
-                ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream);
+                ok = ok && !tc_gemm_create(&p, EPI_SWIGLU, true, w3, r3, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 2 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o, h->stream, ACT_PLANES);
                 h->p_gu_w.push_back(p);
                 const void* w4[3] = {h->wd[l], nullptr, nullptr};
                 const int32_t r4[3] = {D.d, 0, 0};
                 p = nullptr;
-                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream);
+                ok = ok && !tc_gemm_create(&p, EPI_PARTIAL, true, w4, r4, D.F, h->b.act, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, h->b.sk_tables + 3 * SK_TABLE_TILES, SK_TABLE_TILES, pk + h->b.pk_qkv + h->b.pk_o + h->b.pk_gu, h->stream, ACT_PLANES);
                 h->p_down_w.push_back(p);
             }
             ok = ok && !tc_gemm_create(&h->p_lm_w, EPI_LOGITS, false, w5, r5, D.d, h->b.xn, D.batch, RT, 1, h->b.gemm_partials, pbytes, h->b.gemm_counters, n_sm, h->b.err, nullptr, 0, h->b.packed + h->b.pk_layer * D.n_layers, h->stream);
@@ -636,6 +651,7 @@ int esp_init(const esp_model_cfg* model, const esp_spec_cfg* spec, const esp_wei
             ld.gemm[0] = h->p_qkv[0]; ld.gemm[1] = h->p_o[0]; ld.gemm[2] = h->p_gu[0]; ld.gemm[3] = h->p_down[0];
             ld.packed = h->b.packed; ld.pk_layer = h->b.pk_layer;
             ld.hres = h->b.hres; ld.xn = h->b.xn; ld.qbuf = h->b.qbuf; ld.attn_out = h->b.attn_out; ld.act = h->b.act;
+            ld.xn_lo = h->b.xn_lo; ld.attn_out_lo = h->b.attn_out_lo; ld.act_lo = h->b.act_lo;
             ld.kcache = h->b.kcache; ld.vcache = h->b.vcache; ld.layer_kv_stride = h->layer_kv_stride;
             ld.norm_attn = h->b.layer_ptrs; ld.norm_ffn = h->b.layer_ptrs + D.n_layers;
             ld.q_norm = h->b.layer_ptrs + 2 * D.n_layers; ld.k_norm = h->b.layer_ptrs + 3 * D.n_layers;

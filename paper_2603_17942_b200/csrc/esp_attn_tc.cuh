@@ -463,12 +463,17 @@ __device__ __forceinline__ void merge_pair(const FirstPartials<PB>& fp, const Ta
     merge_ml(m, l, o, t.m, t.l, t.o);
     const float inv = 1.0f / l;
     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out) + ((size_t)(c.seq * RT + c.r) * a.Hq + c.head) * HD + lane * 4;
-    const __nv_bfloat162 o01 = __floats2bfloat162_rn(__fmul_rn(o[0], inv), __fmul_rn(o[1], inv)),
-                         o23 = __floats2bfloat162_rn(__fmul_rn(o[2], inv), __fmul_rn(o[3], inv));
-    uint2 pk;
-    pk.x = *reinterpret_cast<const uint32_t*>(&o01);
-    pk.y = *reinterpret_cast<const uint32_t*>(&o23);
-    *reinterpret_cast<uint2*>(out) = pk;
+    __nv_bfloat16 oh[4], ol[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float v = __fmul_rn(o[i], inv);
+        oh[i] = __float2bfloat16_rn(v);
+        ol[i] = __float2bfloat16_rn(__fsub_rn(v, __bfloat162float(oh[i])));
+    }
+    *reinterpret_cast<uint2*>(out) = *reinterpret_cast<const uint2*>(oh);
+    if (a.out_lo)      // low-order plane for an O projection that reads the output as hi + lo
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.out_lo) + ((size_t)(c.seq * RT + c.r) * a.Hq + c.head) * HD + lane * 4) =
+            *reinterpret_cast<const uint2*>(ol);
 }
 
 }  // namespace attn

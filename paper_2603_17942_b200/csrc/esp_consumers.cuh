@@ -13,6 +13,13 @@
 
 namespace esp {
 
+// An activation that feeds a two-plane GEMM is stored as hi = bf16(x) and lo = bf16(x - hi): hi + lo carries x to
+// about 2^-17, and the tensor cores take the product with both.
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(__fsub_rn(x, __bfloat162float(hi)));
+}
+
 // ------------------------------------------------------------------ residual add + RMSNorm of one row
 // The row is cut into groups of 128 features (= GEMM tiles).  A warp owns a group at a time, lane l the
 // features 128*group + 4*l .. +3.  Sum of squares: per lane x0^2 + x1^2 + x2^2 + x3^2 (fused multiply-adds in
@@ -40,8 +47,9 @@ __device__ __forceinline__ void norm_prefetch(NormFirst<T>& pf, const StreamK& s
 
 // hres[row] += partial sums (sk.partials != NULL);  y = hres[row] * rsqrt(mean(hres[row]^2) + eps) * g.
 // NW warps cooperate; `red` is shared memory for (d + 127) / 128 floats; bar() synchronises those warps.
+// yr_lo (bf16 only, may be NULL): the row of the low-order plane of y.
 template <typename T, int NW, typename Bar>
-__device__ __forceinline__ void resid_norm_row(float* xr, const StreamK& sk, int sk_row, const T* g, T* yr, int d, float eps,
+__device__ __forceinline__ void resid_norm_row(float* xr, const StreamK& sk, int sk_row, const T* g, T* yr, T* yr_lo, int d, float eps,
                                                float* copy_row, float* red, const NormFirst<T>& pf, int warp, int lane, Bar bar) {
     const int ng = (d + TILE_N - 1) / TILE_N;
     constexpr int KEEP = 3;
@@ -81,10 +89,17 @@ __device__ __forceinline__ void resid_norm_row(float* xr, const StreamK& sk, int
             load4(gg, g + j);
         }
         T o[4];
+        if constexpr (sizeof(T) == 2) {
+            T ol[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) o[i] = from_f32<T>(__fmul_rn(__fmul_rn(xv[i], rinv), to_f32(gg[i])));
-        if constexpr (sizeof(T) == 2) *reinterpret_cast<uint2*>(yr + j) = *reinterpret_cast<const uint2*>(o);
-        else *reinterpret_cast<float4*>(yr + j) = *reinterpret_cast<const float4*>(o);
+            for (int i = 0; i < 4; ++i) split_bf16(__fmul_rn(__fmul_rn(xv[i], rinv), to_f32(gg[i])), o[i], ol[i]);
+            *reinterpret_cast<uint2*>(yr + j) = *reinterpret_cast<const uint2*>(o);
+            if (yr_lo) *reinterpret_cast<uint2*>(yr_lo + j) = *reinterpret_cast<const uint2*>(ol);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[i] = from_f32<T>(__fmul_rn(__fmul_rn(xv[i], rinv), to_f32(gg[i])));
+            *reinterpret_cast<float4*>(yr + j) = *reinterpret_cast<const float4*>(o);
+        }
         if (copy_row) *reinterpret_cast<float4*>(copy_row + j) = x;
     }
 }
@@ -184,7 +199,9 @@ __device__ __forceinline__ void qkv_finish_task(const QkvPre<HD>& pf, const QkvA
 // ------------------------------------------------------------------ gate/up: eight features of one row per task
 // A tile holds 64 gate features (columns 0..63) and the matching 64 up features (columns 64..127).
 // en: the contributor entry of tile j0 / 64; act_row: the row's [F] activations; sr: row in the partials.
-__device__ __forceinline__ void swiglu_task(const StreamK& sk, const SkEntry& en, int sr, __nv_bfloat16* act_row, int j0, int F) {
+// act_lo_row (may be NULL): the row of the low-order plane.
+__device__ __forceinline__ void swiglu_task(const StreamK& sk, const SkEntry& en, int sr, __nv_bfloat16* act_row, __nv_bfloat16* act_lo_row,
+                                            int j0, int F) {
     float4 g[2], u[2];
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
@@ -193,15 +210,20 @@ __device__ __forceinline__ void swiglu_task(const StreamK& sk, const SkEntry& en
         g[q] = sk_sum4(sk, en, sr, f);
         u[q] = sk_sum4(sk, en, sr, 64 + f);
     }
-    __nv_bfloat16 o[8];
+    __nv_bfloat16 o[8], ol[8];
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
         const float gv[4] = {g[q].x, g[q].y, g[q].z, g[q].w}, uv[4] = {u[q].x, u[q].y, u[q].z, u[q].w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) o[4 * q + i] = __float2bfloat16_rn(__fmul_rn(gv[i] / __fadd_rn(1.0f, expf(-gv[i])), uv[i]));
+        for (int i = 0; i < 4; ++i) split_bf16(__fmul_rn(gv[i] / __fadd_rn(1.0f, expf(-gv[i])), uv[i]), o[4 * q + i], ol[4 * q + i]);
     }
-    if (j0 + 8 <= F) *reinterpret_cast<uint4*>(act_row + j0) = *reinterpret_cast<const uint4*>(o);
-    else *reinterpret_cast<uint2*>(act_row + j0) = *reinterpret_cast<const uint2*>(o);
+    if (j0 + 8 <= F) {
+        *reinterpret_cast<uint4*>(act_row + j0) = *reinterpret_cast<const uint4*>(o);
+        if (act_lo_row) *reinterpret_cast<uint4*>(act_lo_row + j0) = *reinterpret_cast<const uint4*>(ol);
+    } else {
+        *reinterpret_cast<uint2*>(act_row + j0) = *reinterpret_cast<const uint2*>(o);
+        if (act_lo_row) *reinterpret_cast<uint2*>(act_lo_row + j0) = *reinterpret_cast<const uint2*>(ol);
+    }
 }
 
 }  // namespace esp

@@ -48,22 +48,28 @@ using namespace tc;
 // Ring depth.  The bytes in flight per SM (depth x 16 KB of weights) over the load round trip bound the stream rate,
 // and the ring is also what is requested before the preceding kernel has finished: deeper is better.  The
 // partial-only kernel keeps no accumulator copy in shared memory and spends that room on the ring.
-__host__ __device__ constexpr int stages_of(int epi, int nq, int nrs) {
-    return nrs == 80 ? (nq == 3 ? 4 : (nq == 2 ? 6 : (epi == EPI_PARTIAL ? 8 : 6)))
-                     : (nq == 2 ? 4 : (epi == EPI_PARTIAL ? 7 : 4));
+// Planes (PL).  The activations reach the tensor cores as bf16.  A plan with two planes reads them as a pair
+// x = hi + lo (hi = bf16(x), lo = bf16(x - hi), stored PL * n_seq blocks apart in the same buffer) and issues every
+// MMA twice into the same accumulator, first with hi, then with lo: the product then sees the activation to 2^-17
+// instead of 2^-9, for 10 KB more shared memory per stage and sequence.
+__host__ __device__ constexpr int stages_of(int epi, int nq, int nrs, int pl = 1) {
+    return pl == 2 ? (nrs == 80 ? (nq == 2 ? 4 : 6) : 4)
+                   : (nrs == 80 ? (nq == 3 ? 4 : (nq == 2 ? 6 : (epi == EPI_PARTIAL ? 8 : 6)))
+                                : (nq == 2 ? 4 : (epi == EPI_PARTIAL ? 7 : 4)));
 }
-__host__ __device__ constexpr int b_bytes_of(int nq, int nrs) { return nq * nrs * BK * 2; }   // 10240 per 80-row sequence
-__host__ __device__ constexpr int stage_bytes_of(int nq, int nrs) { return A_BYTES + b_bytes_of(nq, nrs); }
+__host__ __device__ constexpr int b_bytes_of(int nq, int nrs) { return nq * nrs * BK * 2; }   // 10240 per 80-row sequence and plane
+__host__ __device__ constexpr int stage_bytes_of(int nq, int nrs, int pl = 1) { return A_BYTES + pl * b_bytes_of(nq, nrs); }
 // two accumulator buffers in tensor memory: 128 columns each for up to 128 rows, 256 each beyond
 __host__ __device__ constexpr int acc_cols_of(int nr) { return nr <= 128 ? 128 : 256; }
 constexpr int NUM_THREADS = 192;
 constexpr int MAX_NQ = 3;
-__host__ __device__ constexpr int max_nq_of(int nrs) { return nrs == 80 ? 3 : 2; }
+__host__ __device__ constexpr int max_nq_of(int nrs, int pl = 1) { return pl == 2 ? (nrs == 80 ? 2 : 1) : (nrs == 80 ? 3 : 2); }
 
 struct TcParams {
     CUtensorMap map_a[3];
     CUtensorMap map_b;      // activations [sequence][RT][K], box = NQ sequences x NRS rows x 64 (one map per NQ)
     int32_t b_seq0;         // first sequence (block of RT activation rows) of this launch
+    int32_t b_plane_seqs;   // blocks between the hi and the lo plane of the activations (two-plane plans)
     int32_t rows_w[3];
     int32_t n_tiles, KB, grid, epi;
     int32_t map_swiglu;  // tile = 64 rows of w[0] (gate) + the matching 64 rows of w[1] (up)
@@ -84,15 +90,22 @@ __device__ __forceinline__ void tile_source(const TcParams& p, int tile, int hal
     row = feat + half * 64;
 }
 
-template <int EPI, int NQ, int NRS>
+template <int EPI, int NQ, int NRS, int PL>
 __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constant__ TcParams p) {
     static_assert(NQ == 1 || EPI == EPI_PARTIAL, "several sequences per launch: partial-only output");
-    static_assert(NQ * NRS <= 256 && NRS % 16 == 0 && NRS <= RT, "MMA N");
-    constexpr int STAGE_BYTES = stage_bytes_of(NQ, NRS), ACC_COLS = acc_cols_of(NQ * NRS), TMEM_COLS = 2 * ACC_COLS;
-    constexpr uint32_t IDESC = idesc_of(NQ * NRS);
+    static_assert(NQ * NRS <= 256 && (PL == 1 || NQ > 1 || 2 * NRS <= 256) && NRS % 16 == 0 && NRS <= RT, "MMA N");
+    static_assert(PL == 1 || EPI == EPI_PARTIAL, "two activation planes: partial-only output");
+    // One sequence with two planes: hi and lo rows sit back to back in the stage and form ONE B operand of 2 * NRS
+    // rows; the accumulator gets W x_hi in columns [0, NRS) and W x_lo in [NRS, 2 NRS), added by the epilogue.
+    // (One MMA per k-step reads the weight slice once from shared memory; two MMAs would read it twice.)
+    constexpr bool JOINT = PL == 2 && NQ == 1;
+    constexpr int N_MMA = JOINT ? 2 * NRS : NQ * NRS;
+    constexpr int STAGE_BYTES = stage_bytes_of(NQ, NRS, PL), ACC_COLS = acc_cols_of(N_MMA), TMEM_COLS = 2 * ACC_COLS;
+    constexpr int B_PLANE = b_bytes_of(NQ, NRS);
+    constexpr uint32_t IDESC = idesc_of(N_MMA);
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int STAGES = stages_of(EPI, NQ, NRS);
+    constexpr int STAGES = stages_of(EPI, NQ, NRS, PL);
     unsigned char* stages = smem;
     float* s_acc = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES);
     float* s_aux = s_acc + (EPI == EPI_PARTIAL ? 0 : NRS * ACC_LD);
@@ -153,7 +166,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                                 tma_load_2d_hint(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[it], pol_w);
                             }
                         } else {
-                            tma_load_3d_hint(sa + A_BYTES, &p.map_b, kb * BK, 0, p.b_seq0, &full[it], pol_x);
+#pragma unroll
+                            for (int pl = 0; pl < PL; ++pl)
+                                tma_load_3d_hint(sa + A_BYTES + pl * B_PLANE, &p.map_b, kb * BK, 0, p.b_seq0 + pl * p.b_plane_seqs, &full[it], pol_x);
                         }
                     }
                 }
@@ -178,7 +193,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                             tma_load_2d_hint(sa, &p.map_a[m0], kb * BK, r0, &full[stage], pol_w);
                             tma_load_2d_hint(sa + A_BYTES / 2, &p.map_a[m1], kb * BK, r1, &full[stage], pol_w);
                         }
-                        tma_load_3d_hint(sa + A_BYTES, &p.map_b, kb * BK, 0, p.b_seq0, &full[stage], pol_x);
+#pragma unroll
+                        for (int pl = 0; pl < PL; ++pl)
+                            tma_load_3d_hint(sa + A_BYTES + pl * B_PLANE, &p.map_b, kb * BK, 0, p.b_seq0 + pl * p.b_plane_seqs, &full[stage], pol_x);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -203,8 +220,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
                     const uint32_t sa = smem_u32(stages + stage * STAGE_BYTES);
                     const uint64_t da = smem_desc(sa, 16), db = smem_desc(sa + A_BYTES, 16);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
+                    for (int k = 0; k < BK / 16; ++k) {
                         umma(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), IDESC, (kb > sg.kb0 || k > 0) ? 1u : 0u);
+                        if constexpr (PL == 2 && !JOINT)      // several sequences: the same step with their low-order planes
+                            umma(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)((B_PLANE >> 4) + k * 2), IDESC, 1u);
+                    }
                     umma_commit(&empty[stage]);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -257,6 +277,16 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
 #pragma unroll
             for (int c = 0; c < NRS / 16; ++c) tmem_ld16_issue(taddr + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if constexpr (JOINT) {      // + the product with the low-order plane
+#pragma unroll
+                for (int c = 0; c < NRS / 16; ++c) {
+                    uint32_t lo16[16];
+                    tmem_ld16_issue(taddr + NRS + c * 16, lo16);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[c * 16 + j] = __float_as_uint(__fadd_rn(__uint_as_float(v[c * 16 + j]), __uint_as_float(lo16[j])));
+                }
+            }
             // the accumulator is in registers: hand the tensor-memory buffer back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(&tempty[buf]);
@@ -376,8 +406,8 @@ __global__ void __launch_bounds__(128) k_pack_weights(PackArgs g, unsigned char*
     }
 }
 
-constexpr size_t smem_bytes_of(int epi, int nq, int nrs) {
-    return 1024 + (size_t)stages_of(epi, nq, nrs) * stage_bytes_of(nq, nrs) +
+constexpr size_t smem_bytes_of(int epi, int nq, int nrs, int pl = 1) {
+    return 1024 + (size_t)stages_of(epi, nq, nrs, pl) * stage_bytes_of(nq, nrs, pl) +
            (epi == EPI_PARTIAL ? 0 : sizeof(float) * (nrs * ACC_LD + nrs * 4)) + 256;
 }
 
@@ -417,11 +447,12 @@ struct TcGemm {
     CUtensorMap map_b_nq[MAX_NQ];   // activation maps with a box of nrs rows x (i+1) sequences
     int nq_max = 1;
     int nrs = 80;                   // rows of a sequence's block that take part: 80 or RT
+    int planes = 1;                 // 2: the activation buffer holds a hi and a lo plane, x_seqs blocks apart
 };
 
 constexpr int MAX_SLOTS = 4;
 size_t tc_gemm_partial_bytes(int n_sm, int nq, int nrs) { return (size_t)n_sm * MAX_SLOTS * nq * nrs * TILE_N * sizeof(float); }
-int tc_gemm_max_nq(int nrs) { return max_nq_of(nrs); }
+int tc_gemm_max_nq(int nrs, int planes) { return max_nq_of(nrs, planes); }
 int tc_gemm_counter_ints() { return 4096; }
 size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K) {
     const long long total = (long long)rows_w[0] + rows_w[1] + rows_w[2];
@@ -432,14 +463,17 @@ int tc_gemm_tiles(const TcGemm* g) { return g ? g->p.n_tiles : 0; }
 void tc_gemm_geometry(const TcGemm* g, TcGemmGeom* out) {
     out->n_tiles = g->p.n_tiles; out->KB = g->p.KB; out->grid = g->p.grid; out->slots = g->p.slots;
     out->table = g->table; out->packed = g->p.a_packed; out->partials = g->p.partials; out->nrs = g->nrs;
+    out->planes = g->planes; out->plane_seqs = g->p.b_plane_seqs;
     out->map_b = g->map_b_nq[0];
 }
 
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
                    int x_seqs, int nrs, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
-                   int table_entries, void* packed, cudaStream_t stream) {
-    if (!out || (nrs != 80 && nrs != RT) || nq_max < 1 || nq_max > max_nq_of(nrs) || x_seqs < nq_max || K % 8 || n_sm < 1) return -1;
-    if (nq_max > 1 && !defer) return -1;
+                   int table_entries, void* packed, cudaStream_t stream, int planes) {
+    if (!out || (nrs != 80 && nrs != RT) || (planes != 1 && planes != 2) || nq_max < 1 || nq_max > max_nq_of(nrs, planes) ||
+        x_seqs < nq_max || K % 8 || n_sm < 1)
+        return -1;
+    if ((nq_max > 1 || planes > 1) && !defer) return -1;
     if (reinterpret_cast<uintptr_t>(x) % 16) return -1;
     TcGemm* g = new (std::nothrow) TcGemm();
     if (!g) return -1;
@@ -456,9 +490,11 @@ int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], co
         }
     }
     for (int i = 0; i < nq_max; ++i)
-        if (make_map_b(&g->map_b_nq[i], x, x_seqs, K, nrs, i + 1)) { delete g; return -1; }
+        if (make_map_b(&g->map_b_nq[i], x, planes * x_seqs, K, nrs, i + 1)) { delete g; return -1; }
     g->nq_max = nq_max;
     g->nrs = nrs;
+    g->planes = planes;
+    p.b_plane_seqs = x_seqs;
     p.map_b = g->map_b_nq[0];
     p.map_swiglu = epi == EPI_SWIGLU;
     p.epi = defer ? (int)EPI_PARTIAL : epi;
@@ -556,21 +592,28 @@ int tc_gemm_launch(const TcGemm* g, const EpiArgs& a, cudaStream_t s, bool pdl, 
     p.map_b = g->map_b_nq[nq - 1];
     p.b_seq0 = b_seq0;
     cudaError_t e = cudaSuccess;
-#define ESP_TC_CASE(E, Q, N)                                                                                  \
-    {                                                                                                         \
-        if (ensure_dynamic_smem(reinterpret_cast<const void*>(k_gemm_tc<E, Q, N>), (int)smem_bytes_of(E, Q, N))) return ESP_E_CUDA;            \
-        e = launch_k(k_gemm_tc<E, Q, N>, dim3(p.grid), dim3(NUM_THREADS), smem_bytes_of(E, Q, N), s, pdl, p); \
+#define ESP_TC_CASE(E, Q, N, PLN)                                                                                  \
+    {                                                                                                              \
+        if (ensure_dynamic_smem(reinterpret_cast<const void*>(k_gemm_tc<E, Q, N, PLN>), (int)smem_bytes_of(E, Q, N, PLN))) return ESP_E_CUDA; \
+        e = launch_k(k_gemm_tc<E, Q, N, PLN>, dim3(p.grid), dim3(NUM_THREADS), smem_bytes_of(E, Q, N, PLN), s, pdl, p); \
     }
     const bool wide = g->nrs != 80;
-    if (p.epi == EPI_STORE_F32 && !wide) ESP_TC_CASE(EPI_STORE_F32, 1, 80)
-    else if (p.epi == EPI_STORE_F32) ESP_TC_CASE(EPI_STORE_F32, 1, RT)
-    else if (p.epi == EPI_LOGITS && !wide) ESP_TC_CASE(EPI_LOGITS, 1, 80)
-    else if (p.epi == EPI_LOGITS) ESP_TC_CASE(EPI_LOGITS, 1, RT)
-    else if (p.epi == EPI_PARTIAL && !wide && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1, 80)
-    else if (p.epi == EPI_PARTIAL && !wide && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2, 80)
-    else if (p.epi == EPI_PARTIAL && !wide && nq == 3) ESP_TC_CASE(EPI_PARTIAL, 3, 80)
-    else if (p.epi == EPI_PARTIAL && wide && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1, RT)
-    else if (p.epi == EPI_PARTIAL && wide && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2, RT)
+    if (g->planes == 2) {
+        if (p.epi != EPI_PARTIAL) return ESP_E_ARG;
+        if (!wide && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1, 80, 2)
+        else if (!wide && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2, 80, 2)
+        else if (wide && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1, RT, 2)
+        else return ESP_E_ARG;
+    }
+    else if (p.epi == EPI_STORE_F32 && !wide) ESP_TC_CASE(EPI_STORE_F32, 1, 80, 1)
+    else if (p.epi == EPI_STORE_F32) ESP_TC_CASE(EPI_STORE_F32, 1, RT, 1)
+    else if (p.epi == EPI_LOGITS && !wide) ESP_TC_CASE(EPI_LOGITS, 1, 80, 1)
+    else if (p.epi == EPI_LOGITS) ESP_TC_CASE(EPI_LOGITS, 1, RT, 1)
+    else if (p.epi == EPI_PARTIAL && !wide && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1, 80, 1)
+    else if (p.epi == EPI_PARTIAL && !wide && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2, 80, 1)
+    else if (p.epi == EPI_PARTIAL && !wide && nq == 3) ESP_TC_CASE(EPI_PARTIAL, 3, 80, 1)
+    else if (p.epi == EPI_PARTIAL && wide && nq == 1) ESP_TC_CASE(EPI_PARTIAL, 1, RT, 1)
+    else if (p.epi == EPI_PARTIAL && wide && nq == 2) ESP_TC_CASE(EPI_PARTIAL, 2, RT, 1)
     else return ESP_E_ARG;
 #undef ESP_TC_CASE
     return e == cudaSuccess ? ESP_OK : ESP_E_CUDA;

@@ -59,7 +59,7 @@ __device__ __forceinline__ Seg get_seg(const Range& r, int i) {
 
 // What the all-layers kernel needs to know about a GEMM plan (every layer has the same geometry).
 struct TcGemmGeom {
-    int n_tiles, KB, grid, slots, nrs;
+    int n_tiles, KB, grid, slots, nrs, planes, plane_seqs;
     const TileSrc* table;            // contributor table of the consumers
     const unsigned char* packed;     // this plan's repacked weights
     float* partials;

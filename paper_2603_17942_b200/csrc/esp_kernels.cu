@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const SeqState* states, const f
 // One block per row (resid_norm_row); with sk.partials == NULL it is a plain RMSNorm of hres.  The sum order
 // depends only on the GEMM's shape, never on the number of rows in the block.
 template <typename T>
-__global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, float* hres, StreamK sk, const T* g, T* y, int d,
+__global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, float* hres, StreamK sk, const T* g, T* y, T* y_lo, int d,
                                                     float eps, float* copy_out) {
     // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
     // waits for this kernel to complete before it touches anything this kernel or its predecessors write
@@ -157,8 +157,8 @@ __global__ void __launch_bounds__(1024) k_resid_norm(const SeqState* states, flo
     pdl_wait();
     if (idle) return;
     const size_t row = (size_t)(seq * RT + r) * d;
-    resid_norm_row<T, 32>(hres + row, sk, seq * sk.seq_rows + r, g, y + row, d, eps, copy_out ? copy_out + row : nullptr, red, pf,
-                          warp, lane, [] { __syncthreads(); });
+    resid_norm_row<T, 32>(hres + row, sk, seq * sk.seq_rows + r, g, y + row, y_lo ? y_lo + row : nullptr, d, eps,
+                          copy_out ? copy_out + row : nullptr, red, pf, warp, lane, [] { __syncthreads(); });
 }
 
 // Consumer of the split QKV GEMM: sums the partials of one (row, head) in CTA order, then what follows
@@ -191,7 +191,8 @@ __global__ void __launch_bounds__(128) k_qkv_finish(EpiArgs a, StreamK sk) {
 
 // Consumer of the split gate/up GEMM: a tile holds 64 gate features (columns 0..63) and the matching 64 up
 // features (columns 64..127); sums both over the tile's contributors in CTA order and stores silu(gate) * up.
-__global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, int rows_fixed, StreamK sk, __nv_bfloat16* act, int F) {
+__global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, int rows_fixed, StreamK sk, __nv_bfloat16* act,
+                                                      __nv_bfloat16* act_lo, int F) {
     // let the next kernel start its own preamble (for a GEMM: the first weight tiles) while this one runs; it still
     // waits for this kernel to complete before it touches anything this kernel or its predecessors write
     if (threadIdx.x == 0) pdl_launch_dependents();
@@ -204,7 +205,7 @@ __global__ void __launch_bounds__(256) k_swiglu_finish(const SeqState* states, i
     const int n_rows = states ? (states[seq].active ? states[seq].n_rows : 0) : rows_fixed;   // written by an earlier step
     pdl_wait();
     if (r >= n_rows || j0 >= F) return;
-    swiglu_task(sk, en, seq * sk.seq_rows + r, act + (size_t)(seq * RT + r) * F, j0, F);
+    swiglu_task(sk, en, seq * sk.seq_rows + r, act + (size_t)(seq * RT + r) * F, act_lo ? act_lo + (size_t)(seq * RT + r) * F : nullptr, j0, F);
 }
 
 // ------------------------------------------------------------------ CUDA-core GEMM
@@ -479,6 +480,17 @@ __global__ void __launch_bounds__(128) k_attn_tail_merge(AttnArgs a) {
     const float inv = 1.0f / l;
 #pragma unroll
     for (int i = 0; i < HD / 32; ++i) out[lane + 32 * i] = from_f32<T>(o[i] * inv);
+    if constexpr (sizeof(T) == 2) {
+        if (a.out_lo) {      // low-order plane for an O projection that reads the output as hi + lo
+            T* out_lo = reinterpret_cast<T*>(a.out_lo) + ((size_t)(seq * RT + r) * a.Hq + head) * HD;
+#pragma unroll
+            for (int i = 0; i < HD / 32; ++i) {
+                T hi, lo2;
+                split_bf16(o[i] * inv, hi, lo2);
+                out_lo[lane + 32 * i] = lo2;
+            }
+        }
+    }
 }
 
 template <typename T, int HD>
@@ -1084,13 +1096,14 @@ void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g
     if (dtype == 0) launch_k(k_rmsnorm<float>, grid, dim3(256), 0, s, pdl, st, x, (const float*)g, (float*)y, d, eps, copy_out);
     else launch_k(k_rmsnorm<__nv_bfloat16>, grid, dim3(256), 0, s, pdl, st, x, (const __nv_bfloat16*)g, (__nv_bfloat16*)y, d, eps, copy_out);
 }
-void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
+void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, void* y_lo, int d, float eps,
                        float* copy_out, int nq, cudaStream_t s, bool pdl, int rows_cap) {
     launch_k(k_resid_norm<__nv_bfloat16>, dim3(rows_cap, nq), dim3(1024), 0, s, pdl, st, hres, sk, (const __nv_bfloat16*)g,
-             (__nv_bfloat16*)y, d, eps, copy_out);
+             (__nv_bfloat16*)y, (__nv_bfloat16*)y_lo, d, eps, copy_out);
 }
-void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl, int rows_cap) {
-    launch_k(k_swiglu_finish, dim3((F / 8 + 255) / 256, rows_cap, nq), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act, F);
+void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, void* act_lo, int F, int nq, cudaStream_t s, bool pdl, int rows_cap) {
+    launch_k(k_swiglu_finish, dim3((F / 8 + 255) / 256, rows_cap, nq), dim3(256), 0, s, pdl, st, 0, sk, (__nv_bfloat16*)act,
+             (__nv_bfloat16*)act_lo, F);
 }
 int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl, int rows_cap) {
     const int n_heads = a.Hq + 2 * a.Hkv;

@@ -10,6 +10,7 @@ struct AttnArgs {
     const void* kc;       // [batch][Hkv][cap][h]
     const void* vc;
     void* out;            // [batch][RT][Hq][h]
+    void* out_lo;         // optional (tensor-core path): low-order bf16 plane of out, out = hi + lo
     float* part_o;        // [batch*RT][Hq][n_split_max][h]
     float2* part_ml;      // [batch*RT][Hq][n_split_max]
     const SeqState* st;   // NULL -> use the explicit fields below
@@ -47,10 +48,11 @@ void launch_assemble(int dtype, const SeqState* st, const void* embed, const flo
 void launch_rmsnorm(int dtype, const SeqState* st, const float* x, const void* g, void* y, int d, float eps, int batch,
                     float* copy_out, cudaStream_t s, bool pdl);
 // consumers of the split (EPI_PARTIAL) tensor-core GEMMs, bf16 models; nq = sequences the GEMM launch covered
-void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, int d, float eps,
+// y_lo / act_lo: optional low-order planes (the next GEMM then reads the activation as hi + lo)
+void launch_resid_norm(const SeqState* st, float* hres, const StreamK& sk, const void* g, void* y, void* y_lo, int d, float eps,
                        float* copy_out, int nq, cudaStream_t s, bool pdl, int rows_cap = RT);
 int launch_qkv_finish(const EpiArgs& a, const StreamK& sk, int nq, cudaStream_t s, bool pdl, int rows_cap = RT);
-void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, int F, int nq, cudaStream_t s, bool pdl, int rows_cap = RT);
+void launch_swiglu_finish(const SeqState* st, const StreamK& sk, void* act, void* act_lo, int F, int nq, cudaStream_t s, bool pdl, int rows_cap = RT);
 void launch_setup_chain(SeqState* st, int seq, const int32_t* prompt_dev, int off, int n, int last, int k, cudaStream_t s);
 void launch_set_tree(SeqState* st, int seq, const int32_t* tokens, const int32_t* parents, int n, int k, int n_anchor,
                      int* err, cudaStream_t s);
@@ -81,10 +83,11 @@ struct TcGemm;
 // epi selects the tile -> weight-row mapping and the fused epilogue; with defer the kernel only stores partials
 // (EPI_PARTIAL) and the caller runs the matching consumer kernel.  x: activations [x_seqs][RT][K]; nrs = rows of a
 // block that take part (80, or RT for blocks of more than 80 rows); a deferred plan may cover up to nq_max
-// sequences per launch, so that the weights are streamed once for all of them
+// sequences per launch, so that the weights are streamed once for all of them.  planes = 2 (deferred plans only):
+// x holds the activations as hi + lo bf16 pairs, [2][x_seqs][RT][K], and every product is taken with both
 int tc_gemm_create(TcGemm** out, int epi, bool defer, const void* const w[3], const int32_t rows_w[3], int K, const void* x,
                    int x_seqs, int nrs, int nq_max, void* partials, size_t partial_bytes, int* counters, int n_sm, int* err, TileSrc* table_dev,
-                   int table_entries, void* packed, cudaStream_t stream);
+                   int table_entries, void* packed, cudaStream_t stream, int planes = 1);
 // bytes of the repacked copy of a weight set (tc_gemm_create's `packed`; NULL there = stream the caller's matrices)
 size_t tc_gemm_packed_bytes(int epi, const int32_t rows_w[3], int K);
 void tc_gemm_destroy(TcGemm* g);
@@ -93,7 +96,7 @@ StreamK tc_gemm_streamk(const TcGemm* g, int nq = 1);
 int tc_wait_selftest(int* err_dev, cudaStream_t s);
 int tc_gemm_tiles(const TcGemm* g);
 size_t tc_gemm_partial_bytes(int n_sm, int nq = 1, int nrs = 80);
-int tc_gemm_max_nq(int nrs = 80);
+int tc_gemm_max_nq(int nrs = 80, int planes = 1);
 int tc_gemm_counter_ints();
 
 
@@ -106,6 +109,7 @@ struct LayersTcDesc {
     size_t pk_layer;
     float* hres;
     void *xn, *qbuf, *attn_out, *act;
+    void *xn_lo, *attn_out_lo, *act_lo;   // low-order planes of the GEMM inputs
     void *kcache, *vcache;         // [n_layers][batch][Hkv][cap][h]
     size_t layer_kv_stride;        // bytes
     const void* const* norm_attn;  // device arrays of n_layers device pointers

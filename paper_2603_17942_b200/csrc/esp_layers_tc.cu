@@ -35,16 +35,18 @@ namespace {
 
 using namespace tc;
 
-constexpr int STAGES = 8;
+constexpr int STAGES = 6;
 constexpr int NRS = 80;                                  // rows of the block that take part in the GEMMs
-constexpr int B_BYTES = NRS * BK * 2;                    // 10240
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;           // 26624, a multiple of 1024
-constexpr int RING_BYTES = STAGES * STAGE_BYTES;         // 212992; the attention phase reuses it (attn::ITEM_BYTES fit)
-constexpr int ACC_COLS = 128;                            // two accumulators of 128 columns; attention: S0, S1, O
+constexpr int PLANES = 2;                                // the activations arrive as hi + lo bf16 pairs (see esp_gemm_tc.cu)
+constexpr int B_PLANE = NRS * BK * 2;                    // 10240
+constexpr int B_BYTES = PLANES * B_PLANE;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;           // 36864, a multiple of 1024
+constexpr int RING_BYTES = STAGES * STAGE_BYTES;         // 221184; the attention phase reuses it (attn::ITEM_BYTES fit)
+constexpr int ACC_COLS = 256;                            // two accumulators: W x_hi in columns [0, 80), W x_lo in [80, 160); attention: S0, S1, O
 constexpr int NUM_THREADS = 448;                         // producer warp, MMA warp, 12 consumer warps
 constexpr int CONS_WARPS = 12;
 constexpr int CONS_THREADS = CONS_WARPS * 32;
-constexpr uint32_t IDESC = idesc_of(NRS);
+constexpr uint32_t IDESC = idesc_of(PLANES * NRS);     // hi and lo rows form one B operand of 160 rows
 static_assert(attn::ITEM_BYTES <= RING_BYTES, "the attention item must fit into the ring");
 
 enum { G_QKV = 0, G_O = 1, G_GU = 2, G_DOWN = 3 };
@@ -56,7 +58,8 @@ struct GemmDesc {
 };
 
 struct LayersParams {
-    CUtensorMap map_b[4];          // activations of the four GEMMs: [sequence][RT][K], box 64 x 80 x 1
+    CUtensorMap map_b[4];          // activations of the four GEMMs: [plane][sequence][RT][K], box 64 x 80 x 1
+    int32_t b_plane_seqs;          // blocks between the hi and the lo plane
     CUtensorMap map_q, map_k, map_v;   // attention: query buffer; K and V cache of ALL layers as [rows][128]
     GemmDesc g[4];
     const unsigned char* packed;   // layer 0's repacked weights
@@ -66,6 +69,7 @@ struct LayersParams {
     const SeqState* st;
     float* hres;
     __nv_bfloat16 *xn, *qbuf, *attn_out, *act;
+    __nv_bfloat16 *xn_lo, *attn_out_lo, *act_lo;   // low-order planes
     char *kcache, *vcache;         // layer 0, this sequence
     unsigned long long layer_kv_stride;   // bytes
     const void* const* norm_attn;  // [n_layers] device pointers
@@ -100,6 +104,7 @@ struct Shared {                    // behind the ring
 };
 static_assert(offsetof(Shared, s_q) % 16 == 0 && offsetof(Shared, full) % 8 == 0, "vector and barrier alignment");
 constexpr size_t SMEM_BYTES = 1024 + RING_BYTES + sizeof(Shared);
+static_assert(SMEM_BYTES <= 227 * 1024, "dynamic shared memory of one CTA");
 
 __device__ __forceinline__ void cons_bar() { asm volatile("bar.sync 1, %0;" ::"n"(CONS_THREADS) : "memory"); }
 __device__ __forceinline__ void main_bar() { __syncthreads(); }
@@ -210,7 +215,9 @@ __device__ __forceinline__ bool produce_gemm(const LayersParams& p, Shared& sh, 
                 mbar_expect_tx(&sh.full[stage], STAGE_BYTES);
                 bulk_load(sa, base + ((size_t)sg.tile * gd.KB + kb) * A_BYTES, A_BYTES, &sh.full[stage], pol_w);
                 }
-            tma_load_3d_hint(sa + A_BYTES, &p.map_b[g], kb * BK, 0, 0, &sh.full[stage], pol_x);
+#pragma unroll
+            for (int pl = 0; pl < PLANES; ++pl)
+                tma_load_3d_hint(sa + A_BYTES + pl * B_PLANE, &p.map_b[g], kb * BK, 0, pl * p.b_plane_seqs, &sh.full[stage], pol_x);
             ++rg.it;
             if (idx + 1 == rg.pre) trace(p, tr, 2);
         }
@@ -266,6 +273,14 @@ __device__ __forceinline__ bool epilogue_gemm(const LayersParams& p, Shared& sh,
 #pragma unroll
         for (int c = 0; c < NRS / 16; ++c) tmem_ld16_issue(taddr + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&v[c * 16]));
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int c = 0; c < NRS / 16; ++c) {      // + the product with the low-order plane
+            uint32_t lo16[16];
+            tmem_ld16_issue(taddr + NRS + c * 16, lo16);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[c * 16 + j] = __float_as_uint(__fadd_rn(__uint_as_float(v[c * 16 + j]), __uint_as_float(lo16[j])));
+        }
         // the accumulator is in registers: hand the tensor-memory buffer back to the MMA thread
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         mbar_arrive(&sh.tempty[buf]);
@@ -346,8 +361,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
         const __nv_bfloat16* gw = reinterpret_cast<const __nv_bfloat16*>(gain);
         NormFirst<__nv_bfloat16> pf;
         norm_prefetch(pf, sk, gw, p.d, cw, lane);
-        resid_norm_row<__nv_bfloat16, CONS_WARPS>(p.hres + (size_t)cta * p.d, sk, cta, gw, p.xn + (size_t)cta * p.d, p.d, p.rms_eps, nullptr,
-                                                  sh.red, pf, cw, lane, [] { cons_bar(); });
+        resid_norm_row<__nv_bfloat16, CONS_WARPS>(p.hres + (size_t)cta * p.d, sk, cta, gw, p.xn + (size_t)cta * p.d, p.xn_lo + (size_t)cta * p.d,
+                                                  p.d, p.rms_eps, nullptr, sh.red, pf, cw, lane, [] { cons_bar(); });
     };
 
     attn::BulkShared bsm;
@@ -357,7 +372,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
     attn::BulkMaps bmp;
     bmp.q = &p.map_q; bmp.k = &p.map_k; bmp.v = &p.map_v; bmp.group = p.group; bmp.rows_per_tile = p.rows_per_tile;
     AttnArgs aa;
-    aa.q = p.qbuf; aa.out = p.attn_out; aa.part_o = p.part_o; aa.part_ml = p.part_ml; aa.st = st; aa.anc = nullptr; aa.depth = nullptr;
+    aa.q = p.qbuf; aa.out = p.attn_out; aa.out_lo = p.attn_out_lo; aa.part_o = p.part_o; aa.part_ml = p.part_ml; aa.st = st; aa.anc = nullptr; aa.depth = nullptr;
     aa.rows_cap = NRS; aa.cache_in_flight = 0; aa.n_rows_fixed = 0; aa.L_fixed = 0;
     aa.Hq = p.Hq; aa.Hkv = p.Hkv; aa.h = attn::HD; aa.cap = p.cap; aa.split_len = p.split_len; aa.n_split_max = p.n_split_max; aa.dcap = p.dcap;
     aa.scale_log2 = p.scale_log2; aa.err = p.err;
@@ -463,7 +478,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
             const long long total = (long long)n_rows * groups;
             for (long long t = (long long)cta * CONS_THREADS + (threadIdx.x - 64); t < total; t += (long long)G * CONS_THREADS) {
                 const int r = (int)(t / groups), j0 = (int)(t % groups) * 8;
-                swiglu_task(sk, sk_entry(sk, j0 / 64), r, p.act + (size_t)r * p.F, j0, p.F);
+                swiglu_task(sk, sk_entry(sk, j0 / 64), r, p.act + (size_t)r * p.F, p.act_lo + (size_t)r * p.F, j0, p.F);
             }
         }
         if (!(ok = grid_sync(p, sh, epoch, stamp))) break;
@@ -514,7 +529,8 @@ int layers_tc_create(LayersTc** out, const LayersTcDesc& d) {
     for (int i = 0; i < 4; ++i) {
         TcGemmGeom gg;
         tc_gemm_geometry(d.gemm[i], &gg);
-        if (gg.nrs != NRS || !gg.packed || !gg.table) { delete t; return -1; }
+        if (gg.nrs != NRS || gg.planes != PLANES || !gg.packed || !gg.table) { delete t; return -1; }
+        p.b_plane_seqs = gg.plane_seqs;
         p.g[i].n_tiles = gg.n_tiles; p.g[i].KB = gg.KB; p.g[i].G = gg.grid; p.g[i].slots = gg.slots; p.g[i].table = gg.table;
         p.g[i].pk_off = (unsigned long long)(gg.packed - reinterpret_cast<const unsigned char*>(d.packed));
         p.map_b[i] = gg.map_b;
@@ -529,6 +545,9 @@ int layers_tc_create(LayersTc** out, const LayersTcDesc& d) {
     p.hres = d.hres;
     p.xn = reinterpret_cast<__nv_bfloat16*>(d.xn); p.qbuf = reinterpret_cast<__nv_bfloat16*>(d.qbuf);
     p.attn_out = reinterpret_cast<__nv_bfloat16*>(d.attn_out); p.act = reinterpret_cast<__nv_bfloat16*>(d.act);
+    p.xn_lo = reinterpret_cast<__nv_bfloat16*>(d.xn_lo); p.attn_out_lo = reinterpret_cast<__nv_bfloat16*>(d.attn_out_lo);
+    p.act_lo = reinterpret_cast<__nv_bfloat16*>(d.act_lo);
+    if (!p.xn_lo || !p.attn_out_lo || !p.act_lo) { delete t; return -1; }
     p.layer_kv_stride = d.layer_kv_stride;
     p.norm_attn = d.norm_attn; p.norm_ffn = d.norm_ffn; p.q_norm = d.q_norm; p.k_norm = d.k_norm;
     p.rope_cos = d.rope_cos; p.rope_sin = d.rope_sin;

@@ -54,3 +54,23 @@ def test_reference_arm_prints_the_contract_line():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"], env=env,
                          capture_output=True, text=True, timeout=120)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_reference_arm_runs_whole_steps_and_reports_what_it_ran():
+    """Rank 0 of `--impl reference` on a one-layer cut of the shape: the line carries the contract's keys, the
+    `config` object has exactly the keys and values the GPU arm prints for the same workload, and steps x
+    ms_per_step is the time the steps really took (nothing extrapolated)."""
+    import time
+    t0 = time.time()
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--layers", "1",
+                          "--steps", "2", "--warmup", "0"], env=dict(os.environ, RANK="0", WORLD_SIZE="1"),
+                         capture_output=True, text=True, timeout=600)
+    wall = time.time() - t0
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["metric"] == bench.METRIC and line["unit"] == bench.UNIT
+    assert line["steps"] == 2 and line["warmup"] == 0 and line["higher_is_better"] is True
+    assert line["config"] == bench.workload_config("llama3-8b", 1024, 1, 0.0, 4, 10, 64, 68, 1)
+    assert line["steps"] * line["ms_per_step"] * 1e-3 < wall
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
+    assert line["e2e"] == {"value": line["value"], "unit": bench.UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
