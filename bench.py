@@ -41,7 +41,7 @@ UNIT = "tok/s"
 
 # DRAM bytes (read + written) of one gate/up GEMM launch from the ncu capture summarised under profiles/
 # (Llama-3-8B shape, 68 rows, one sequence); None for workloads without a capture of the current kernel.
-GATEUP_DRAM_TRAFFIC = {"llama3-8b": 241.9e6}
+GATEUP_DRAM_TRAFFIC = {"llama3-8b": 242.8e6}
 
 WORKLOADS = {
     # name: (shape attr in synth, prompt length, probes, topk, max_nodes)
@@ -258,13 +258,18 @@ def replay_leg(P, shape, w, prompt, stream, k, B, n_steps, probs, seed=0):
     out = [h.prefill(prompt)]
     rng = np.random.default_rng(seed)
     per_level = (B - 1) // k
+    # the schedule holds each accepted length exactly in its proportion (so that tau comes out at the operating point
+    # whatever the seed), in a random order
+    counts = [int(round(q * n_steps)) for q in probs]
+    counts[0] += n_steps - sum(counts)
+    schedule = rng.permutation(np.repeat(np.arange(len(probs)), counts))
     steps = 0
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     L_start = h.state()["L"]
     while steps < n_steps and len(out) + k + 1 < len(truth):
         n = len(out)
-        a = int(min(rng.choice(len(probs), p=probs), k))
+        a = int(min(schedule[steps], k))
         toks, pars, main = [out[-1]], [-1], 0
         for d in range(1, k + 1):
             level = []
@@ -581,6 +586,60 @@ def run_attention_op(args):
     print(json.dumps(line), flush=True)
 
 
+def run_layer_kernel_trace(args, shape, plen, k, K, B):
+    """The all-layers persistent kernel (esp_debug_set_layer_kernel mode 0) against the default path of one kernel
+    per operation, on the same workload: device ms per step of both, and where the persistent kernel's time goes
+    per layer -- for each of its ten phases the time its first CTA spends in the phase and then in the grid
+    barrier behind it (averages over the layers after the first and over 5 traced steps)."""
+    import torch
+    import synth
+    import paper_2603_17942_b200 as P
+    from paper_2603_17942_b200 import build as esp_build
+    esp_build.build()
+    torch.cuda.set_device(0)
+    w = synth.make_weights(shape, seed=0, device="cuda")
+    prompt = synth.make_prompt(shape.vocab, plen, 0)
+    spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1)
+    stream = torch.cuda.Stream()
+    steps = min(args.steps, P.ESP_MAX_UNREAD_STEPS)
+    h = P.Handle(shape, spec, w, max_seq_len=plen + (k + 1) * (2 * steps + 40) + 64, stream=stream)
+    h.prefill(prompt)
+    out = {}
+    for mode, name in ((1, "kernel_per_operation"), (0, "all_layers_kernel")):
+        P.esp_debug_set_layer_kernel(h.h, mode)
+        for _ in range(max(args.warmup, 3)):
+            h.step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record()
+            for _ in range(steps):
+                h.step_async()
+            e1.record()
+        torch.cuda.synchronize()
+        for _ in range(steps):
+            h.read()
+        out[name + "_ms_per_step"] = e0.elapsed_time(e1) / steps
+    names = ["attention norm", "QKV GEMM", "q/k/v finish", "attention over the cache", "attention tail + merge", "O GEMM",
+             "FFN norm", "gate/up GEMM", "SiLU*up", "down GEMM"]
+    acc = np.zeros((10, 2))
+    n_tr = 5
+    for _ in range(n_tr):
+        P.esp_step_profiled(h.h, h.tokens_out, h.n_out)
+        tl = P.esp_debug_layer_timeline(h.h, shape.n_layers).astype(np.int64).reshape(-1, 8)
+        body = np.concatenate([[0], tl[1:, 0] - tl[:-1, 1]]).reshape(-1, 10)
+        wait = (tl[:, 1] - tl[:, 0]).reshape(-1, 10)
+        acc[:, 0] += body[1:].mean(axis=0) / n_tr
+        acc[:, 1] += wait[1:].mean(axis=0) / n_tr
+    out["phase_us"] = {nm: {"phase": round(float(a[0]) / 1e3, 2), "barrier": round(float(a[1]) / 1e3, 2)} for nm, a in zip(names, acc)}
+    out["layer_us"] = round(float(acc.sum()) / 1e3, 2)
+    err = h.stats().device_error
+    h.close()
+    if err:
+        raise SystemExit("device error word set")
+    print(json.dumps({"metric": "all_layers_kernel_trace", "config": workload_config(args.config, plen, 1, 0.0, k, K, B, B + k, 1),
+                      "steps": steps, **out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -595,6 +654,8 @@ def main():
     ap.add_argument("--per-node-probes", action="store_true",
                     help="k = 3 probes behind each of 30 tree nodes (block complexity 120) instead of the default block")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer count (smaller captures under a profiler)")
+    ap.add_argument("--trace-layer-kernel", action="store_true",
+                    help="time the all-layers persistent kernel against the default path and print its per-phase trace")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-greedy", action="store_true", help="skip the greedy-decoding leg")
     args = ap.parse_args()
@@ -609,7 +670,10 @@ def main():
     shape = getattr(synth, name)
     if args.layers > 0:
         shape = shape.replace(n_layers=args.layers)
-    if args.impl == "reference":
+    if args.trace_layer_kernel:
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_layer_kernel_trace(args, shape, plen, k, K, B)
+    elif args.impl == "reference":
         run_reference(args, shape, plen, k, K, B)
     else:
         run_ours(args, shape, plen, k, K, B)
