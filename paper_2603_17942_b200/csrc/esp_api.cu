@@ -127,8 +127,7 @@ int check_cfg(const esp_model_cfg* m, const esp_spec_cfg* s, Dims* D) {
         D->F = m->d_ffn; D->V = m->vocab; D->qk_norm = m->qk_norm;
         D->cap = m->max_seq_len + RT;
         D->batch = m->max_batch;
-        int S = 256;
-        while ((m->max_seq_len + S - 1) / S > 16) S *= 2;   // at most 16 splits: the partials stay small next to the cache
+        const int S = attn_split_len(m->max_seq_len, m->max_batch, m->n_kv_heads);
         D->split_len = S;
         D->n_split_max = (m->max_seq_len + RT + S - 1) / S + 1;   // a prefill block's own rows count as cache positions
         D->rms_eps = m->rms_eps;
@@ -1000,9 +999,8 @@ void esp_free(esp_handle* h) {
 // ------------------------------------------------------------------ stand-alone operators
 int esp_tree_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t cap, size_t* bytes_out) {
     if (!bytes_out || batch < 1 || n_q_heads < 1 || cap < RT) return ESP_E_ARG;
-    int S = 256;
-    while ((cap - RT + S - 1) / S > 16) S *= 2;
-    const size_t ns = (cap + S - 1) / S + 1;
+    const int S = attn_split_len(cap - RT, 1, 1);   // the finest split of this capacity: covers every batch
+    const size_t ns = ((size_t)cap + S - 1) / S + 1;
     const size_t rows = (size_t)batch * RT * n_q_heads * ns;
     *bytes_out = align_up(rows * head_dim * sizeof(float), 256) + align_up(rows * sizeof(float2), 256) + 256;
     return ESP_OK;
@@ -1021,9 +1019,8 @@ int esp_tree_attention(int32_t dtype, int32_t batch, int32_t n_rows, int32_t L, 
     size_t need = 0;
     esp_tree_attention_scratch_bytes(batch, n_q_heads, head_dim, cap, &need);
     if (scratch_bytes < need || reinterpret_cast<uintptr_t>(scratch) % 256) return ESP_E_WORKSPACE;
-    int S = 256;
-    while ((cap - RT + S - 1) / S > 16) S *= 2;
-    const size_t ns = (cap + S - 1) / S + 1;
+    const int S = attn_split_len(cap - RT, batch, n_kv_heads);
+    const size_t ns = ((size_t)cap + S - 1) / S + 1;
     const size_t rows = (size_t)batch * RT * n_q_heads * ns;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
     char* sc = reinterpret_cast<char*>(scratch);

@@ -67,9 +67,11 @@ __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __g
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     BulkShared sm;
     sm.buf = smem;
-    sm.kv_full = reinterpret_cast<uint64_t*>(smem + ONCE_OFF_BAR);   // [2]
-    sm.kv_empty = sm.kv_full + 2;                                    // [2]
-    sm.s_full = sm.kv_empty + 2;                                     // [2]
+    sm.k_full = reinterpret_cast<uint64_t*>(smem + ONCE_OFF_BAR);    // [2]
+    sm.k_empty = sm.k_full + 2;                                      // [2]
+    sm.v_full = sm.k_empty + 2;                                      // [2]
+    sm.v_empty = sm.v_full + 2;                                      // [2]
+    sm.s_full = sm.v_empty + 2;                                      // [2]
     sm.q_full = sm.s_full + 2;
     sm.p_ready = sm.q_full + 1;
     sm.pv_done = sm.p_ready + 1;
@@ -157,9 +159,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
     __shared__ int2 s_seq[MAX_T0_ENTRIES];  // [sequence]: (rows in its block, cached positions L)
     __shared__ float s_xchg[2][2 * MP];   // [exchange parity][half][pair]
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);   // [2]
-    uint64_t* kv_empty = kv_full + 2;                                  // [2]
-    uint64_t* s_full = kv_empty + 2;                                   // [2]
+    uint64_t* k_full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);    // [2] a stage's K half has landed
+    uint64_t* k_empty = k_full + 2;                                    // [2] ... its Q K^T has completed
+    uint64_t* v_full = k_empty + 2;                                    // [2] a stage's V half has landed
+    uint64_t* v_empty = v_full + 2;                                    // [2] ... its P V has completed
+    uint64_t* s_full = v_empty + 2;                                    // [2]
     uint64_t* o_free = s_full + 2;                                     // [2] an O accumulator has been read out
     uint64_t* o_full = o_free + 2;                                     // [2] an item's last P V has completed
     uint64_t* q_full = o_full + 2;
@@ -192,7 +196,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
     }
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
-            mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); mbar_init(&s_full[i], 1); mbar_init(&o_free[i], 128);
+            mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
+            mbar_init(&s_full[i], 1); mbar_init(&o_free[i], 128);
             mbar_init(&o_full[i], 1);
         }
         mbar_init(q_full, 1);
@@ -240,44 +245,75 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
-            bool ok = true, first = true;
-            uint32_t gc = 0, n_it = 0;       // chunks and items issued so far
-            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
-                Item it;
-                if (!get_item(idx, it)) continue;
-                const int kvrow0 = (it.seq * a.Hkv + it.kvh) * a.cap + it.beg;
-                auto load_chunk = [&](int c) -> bool {
-                    const uint32_t g = gc + c;
-                    // a fresh barrier passes a wait on parity 1: the first use of a stage does not block
-                    if (!mbar_wait(&kv_empty[g & 1], ((g >> 1) & 1) ^ 1, s_abort)) return false;
-                    unsigned char* st = smem + OFF_KV + (g & 1) * KV_STAGE;
-                    mbar_expect_tx(&kv_full[g & 1], KV_STAGE);
-                    tma_load_2d(st, &p.map_k, 0, kvrow0 + c * CK, &kv_full[g & 1]);
-                    tma_load_2d(st + HALF_BYTES, &p.map_k, 64, kvrow0 + c * CK, &kv_full[g & 1]);
-                    tma_load_2d(st + K_BYTES, &p.map_v, 0, kvrow0 + c * CK, &kv_full[g & 1]);
-                    tma_load_2d(st + K_BYTES + HALF_BYTES, &p.map_v, 64, kvrow0 + c * CK, &kv_full[g & 1]);
-                    return true;
-                };
-                int c0 = 0;
-                if (first) {
-                    // the cache does not depend on the kernel before this one, the queries do
-                    if (a.cache_in_flight) trigger_after_wait();
-                    for (; c0 < it.n_chunks && c0 < 2 && ok; ++c0) ok = load_chunk(c0);
-                    if (!a.cache_in_flight) trigger_after_wait();
-                    first = false;
-                } else {
-                    // Q is single buffered: the previous item's last Q K^T must have completed
-                    ok = mbar_wait(q_free, (n_it - 1) & 1, s_abort);
-                }
-                if (!ok) break;
+            // Two cursors walk the CTA's chunks (item after item): K, which also requests an item's Q, and V.  A K
+            // half is free again when its Q K^T has completed, about a chunk period before the V half (free when
+            // P V has), so K runs one chunk ahead of V and both have two chunk periods for their trip from HBM.
+            struct Cursor { int idx, c; uint32_t g; bool live; Item it; };
+            auto seek = [&](Cursor& k, int from) {
+                k.live = false;
+                for (int idx = from; idx < n_items; idx += gridDim.x)
+                    if (get_item(idx, k.it)) { k.idx = idx; k.c = 0; k.live = true; return; }
+            };
+            auto advance = [&](Cursor& k) {
+                ++k.g;
+                if (++k.c == k.it.n_chunks) seek(k, k.idx + gridDim.x);
+            };
+            auto load_half = [&](const Cursor& k, bool is_k) -> bool {
+                uint64_t* empty = is_k ? k_empty : v_empty;
+                uint64_t* full = is_k ? k_full : v_full;
+                // a fresh barrier passes a wait on parity 1: the first use of a stage does not block
+                if (!mbar_wait(&empty[k.g & 1], ((k.g >> 1) & 1) ^ 1, s_abort)) return false;
+                const int row = (k.it.seq * a.Hkv + k.it.kvh) * a.cap + k.it.beg + k.c * CK;
+                unsigned char* st = smem + OFF_KV + (k.g & 1) * KV_STAGE + (is_k ? 0 : K_BYTES);
+                const CUtensorMap* map = is_k ? &p.map_k : &p.map_v;
+                mbar_expect_tx(&full[k.g & 1], K_BYTES);
+                tma_load_2d(st, map, 0, row, &full[k.g & 1]);
+                tma_load_2d(st + HALF_BYTES, map, 64, row, &full[k.g & 1]);
+                return true;
+            };
+            auto load_q = [&](const Item& it) {
                 mbar_expect_tx(q_full, Q_BYTES);
                 tma_load_3d(sQ, &p.map_q, 0, it.kvh * p.group, it.seq * RT + it.row0, q_full);
                 tma_load_3d(sQ + HALF_BYTES, &p.map_q, 64, it.kvh * p.group, it.seq * RT + it.row0, q_full);
-                for (int c = c0; c < it.n_chunks && ok; ++c) ok = load_chunk(c);
-                gc += it.n_chunks;
-                ++n_it;
+            };
+            bool ok = true;
+            uint32_t n_q = 0;                // items whose Q has been requested
+            Cursor ck, cv;
+            ck.g = 0;
+            seek(ck, blockIdx.x);
+            cv = ck;
+            if (!ck.live) {
+                trigger_after_wait();
+            } else {
+                // the first item: the cache does not depend on the kernel before this one, the queries do
+                const Item it0 = ck.it;
+                if (a.cache_in_flight) trigger_after_wait();
+                const int pre = it0.n_chunks < 2 ? 1 : 2;
+                for (int i = 0; i < pre && ok; ++i) { ok = load_half(ck, true); advance(ck); }
+                for (int i = 0; i < pre && ok; ++i) { ok = load_half(cv, false); advance(cv); }
+                if (!a.cache_in_flight) trigger_after_wait();
+                load_q(it0);
+                n_q = 1;
+                auto k_step = [&]() -> bool {
+                    if (!ck.live) return true;
+                    if (ck.c == 0) {
+                        // Q is single buffered: the previous item's last Q K^T must have completed
+                        if (!mbar_wait(q_free, (n_q - 1) & 1, s_abort)) return false;
+                        load_q(ck.it);
+                        ++n_q;
+                    }
+                    const bool done = load_half(ck, true);
+                    advance(ck);
+                    return done;
+                };
+                ok = ok && k_step();                      // K one chunk ahead of V from here on
+                while (ok && cv.live) {
+                    ok = k_step();
+                    if (!ok) break;
+                    ok = load_half(cv, false);
+                    advance(cv);
+                }
             }
-            if (first) trigger_after_wait();
             if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
         }
     } else if (warp == 1) {
@@ -300,9 +336,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                         umma(tmem_s, smem_desc(q_addr + off, 16), smem_desc(k_addr + off, 16), IDESC_QK, kk > 0 ? 1u : 0u);
                     }
                     umma_commit(&s_full[g & 1]);
+                    umma_commit(&k_empty[g & 1]);
                     if (c == it.n_chunks - 1) umma_commit(q_free);
                 };
-                ok = mbar_wait(q_full, n_it & 1, s_abort) && mbar_wait(&kv_full[gc & 1], (gc >> 1) & 1, s_abort) &&
+                ok = mbar_wait(q_full, n_it & 1, s_abort) && mbar_wait(&k_full[gc & 1], (gc >> 1) & 1, s_abort) &&
                      mbar_wait(&o_free[n_it & 1], ((n_it >> 1) & 1) ^ 1, s_abort);   // this O buffer's previous item was read out
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -310,11 +347,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                 for (int c = 0; c < it.n_chunks && ok; ++c) {
                     const uint32_t g = gc + c;
                     if (c + 1 < it.n_chunks) {     // S of the next chunk while the softmax of this one runs
-                        if (!mbar_wait(&kv_full[(g + 1) & 1], ((g + 1) >> 1) & 1, s_abort)) { ok = false; break; }
+                        if (!mbar_wait(&k_full[(g + 1) & 1], ((g + 1) >> 1) & 1, s_abort)) { ok = false; break; }
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         issue_qk(c + 1);
                     }
-                    if (!mbar_wait(p_ready, g & 1, s_abort)) { ok = false; break; }
+                    if (!mbar_wait(p_ready, g & 1, s_abort) || !mbar_wait(&v_full[g & 1], (g >> 1) & 1, s_abort)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t v_addr = smem_u32(smem + OFF_KV + (g & 1) * KV_STAGE + K_BYTES);
 #pragma unroll
@@ -325,7 +362,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                              (c > 0 || kk > 0) ? 1u : 0u);
                     }
                     umma_commit(pv_done);
-                    umma_commit(&kv_empty[g & 1]);
+                    umma_commit(&v_empty[g & 1]);
                     if (c == it.n_chunks - 1) umma_commit(&o_full[n_it & 1]);
                 }
                 gc += it.n_chunks;

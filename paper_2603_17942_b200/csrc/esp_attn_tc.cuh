@@ -75,7 +75,13 @@ __device__ __forceinline__ bool softmax_chunk(uint32_t s_addr, uint32_t o_addr, 
     mbar_arrive(xchg);
     if (!__all_sync(0xffffffffu, mbar_wait(xchg, xchg_parity, s_abort))) return false;
     cmax = fmaxf(xch[pair], xch[MP + pair]);
-    const float m_new = fmaxf(m_run, cmax);
+    // The running reference follows the maximum lazily: it moves only when the maximum has grown by more than
+    // 2^8 over it (or there was none yet).  Until then alpha is exactly 1, O needs no rescaling, and the
+    // probabilities of this chunk are at most 2^8, exact in fp32 and as precise as ever in bf16.  The decision is
+    // the row's own (both threads of the pair see the same maximum), so a row's bits stay independent of its
+    // neighbours; whoever merges the partial takes m_run as what it is, the reference of l and O.
+    const float m_max = fmaxf(m_run, cmax);
+    const float m_new = (m_run == -INFINITY || __fsub_rn(m_max, m_run) > 8.f) ? m_max : m_run;
     const float m_use = m_new == -INFINITY ? 0.f : m_new;
     const float alpha = exp2f(__fsub_rn(m_run, m_use));
     // P of the previous chunk must have been consumed before it is overwritten, and O must be final
@@ -137,14 +143,17 @@ struct BulkItem {
 };
 struct BulkShared {
     unsigned char* buf;     // 1024-byte aligned, ITEM_BYTES
-    uint64_t *kv_full, *kv_empty, *s_full;   // [2] each, count 1
+    uint64_t *k_full, *k_empty, *v_full, *v_empty, *s_full;   // [2] each, count 1
     uint64_t *q_full, *pv_done;              // count 1
     uint64_t *p_ready, *xchg;                // count 256
     float* s_xchg;          // [2][2 * MP]
     volatile int* s_abort;
 };
 __device__ __forceinline__ void bulk_init_barriers(const BulkShared& sm) {
-    for (int i = 0; i < 2; ++i) { mbar_init(&sm.kv_full[i], 1); mbar_init(&sm.kv_empty[i], 1); mbar_init(&sm.s_full[i], 1); }
+    for (int i = 0; i < 2; ++i) {
+        mbar_init(&sm.k_full[i], 1); mbar_init(&sm.k_empty[i], 1); mbar_init(&sm.v_full[i], 1); mbar_init(&sm.v_empty[i], 1);
+        mbar_init(&sm.s_full[i], 1);
+    }
     mbar_init(sm.q_full, 1);
     mbar_init(sm.p_ready, 256);
     mbar_init(sm.pv_done, 1);
@@ -167,25 +176,35 @@ __device__ __forceinline__ void bulk_item_roles(const BulkMaps& mp, const AttnAr
         if (lane == 0) {
             const int kvrow0 = it.kv_row0 + it.beg;
             bool ok = true;
-            auto load_chunk = [&](int c) {
+            // K and V of a chunk have a stage half and a barrier pair each: a K half is free again when its Q K^T has
+            // completed, about one chunk period before the V half (free when P V has), so K runs one chunk ahead of V
+            // and both have two chunk periods for their trip from HBM
+            auto load_k = [&](int c) -> bool {
+                if (!mbar_wait(&sm.k_empty[c & 1], ((c >> 1) & 1) ^ 1, s_abort)) return false;   // a fresh barrier passes parity 1
                 unsigned char* st = smem + OFF_KV + (c & 1) * KV_STAGE;
-                mbar_expect_tx(&sm.kv_full[c & 1], KV_STAGE);
-                tma_load_2d(st, mp.k, 0, kvrow0 + c * CK, &sm.kv_full[c & 1]);
-                tma_load_2d(st + HALF_BYTES, mp.k, 64, kvrow0 + c * CK, &sm.kv_full[c & 1]);
-                tma_load_2d(st + K_BYTES, mp.v, 0, kvrow0 + c * CK, &sm.kv_full[c & 1]);
-                tma_load_2d(st + K_BYTES + HALF_BYTES, mp.v, 64, kvrow0 + c * CK, &sm.kv_full[c & 1]);
+                mbar_expect_tx(&sm.k_full[c & 1], K_BYTES);
+                tma_load_2d(st, mp.k, 0, kvrow0 + c * CK, &sm.k_full[c & 1]);
+                tma_load_2d(st + HALF_BYTES, mp.k, 64, kvrow0 + c * CK, &sm.k_full[c & 1]);
+                return true;
+            };
+            auto load_v = [&](int c) -> bool {
+                if (!mbar_wait(&sm.v_empty[c & 1], ((c >> 1) & 1) ^ 1, s_abort)) return false;
+                unsigned char* st = smem + OFF_KV + (c & 1) * KV_STAGE + K_BYTES;
+                mbar_expect_tx(&sm.v_full[c & 1], V_BYTES);
+                tma_load_2d(st, mp.v, 0, kvrow0 + c * CK, &sm.v_full[c & 1]);
+                tma_load_2d(st + HALF_BYTES, mp.v, 64, kvrow0 + c * CK, &sm.v_full[c & 1]);
+                return true;
             };
             // the cache below T0 is settled in a decode step: request it before waiting for the kernel that wrote the queries
             if (PDL && a.cache_in_flight) trigger_after_wait();
-            for (int c = 0; c < it.n_chunks && c < 2; ++c) load_chunk(c);
+            const int n = it.n_chunks;
+            ok = load_k(0) && (n < 2 || load_k(1)) && load_v(0) && (n < 2 || load_v(1));    // both stages are free
             if (PDL && !a.cache_in_flight) trigger_after_wait();
             mbar_expect_tx(sm.q_full, Q_BYTES);
             tma_load_3d(sQ, mp.q, 0, it.kvh * mp.group, it.seq * RT + it.row0, sm.q_full);
             tma_load_3d(sQ + HALF_BYTES, mp.q, 64, it.kvh * mp.group, it.seq * RT + it.row0, sm.q_full);
-            for (int c = 2; c < it.n_chunks && ok; ++c) {
-                if (!mbar_wait(&sm.kv_empty[c & 1], ((c >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
-                load_chunk(c);
-            }
+            if (ok && n > 2) ok = load_k(2);
+            for (int c = 2; c < n && ok; ++c) ok = (c + 1 >= n || load_k(c + 1)) && load_v(c);
             if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
         }
     } else if (warp == 1) {
@@ -202,19 +221,20 @@ __device__ __forceinline__ void bulk_item_roles(const BulkMaps& mp, const AttnAr
                     umma(tmem_s, smem_desc(q_addr + off, 16), smem_desc(k_addr + off, 16), IDESC_QK, kk > 0 ? 1u : 0u);
                 }
                 umma_commit(&sm.s_full[c & 1]);
+                umma_commit(&sm.k_empty[c & 1]);
             };
-            ok = mbar_wait(sm.q_full, 0, s_abort) && mbar_wait(&sm.kv_full[0], 0, s_abort);
+            ok = mbar_wait(sm.q_full, 0, s_abort) && mbar_wait(&sm.k_full[0], 0, s_abort);
             if (ok) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 issue_qk(0);
             }
             for (int c = 0; c < it.n_chunks && ok; ++c) {
                 if (c + 1 < it.n_chunks) {     // S of the next chunk while the softmax of this one runs
-                    if (!mbar_wait(&sm.kv_full[(c + 1) & 1], ((c + 1) >> 1) & 1, s_abort)) { ok = false; break; }
+                    if (!mbar_wait(&sm.k_full[(c + 1) & 1], ((c + 1) >> 1) & 1, s_abort)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     issue_qk(c + 1);
                 }
-                if (!mbar_wait(sm.p_ready, c & 1, s_abort)) { ok = false; break; }
+                if (!mbar_wait(sm.p_ready, c & 1, s_abort) || !mbar_wait(&sm.v_full[c & 1], (c >> 1) & 1, s_abort)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t v_addr = smem_u32(smem + OFF_KV + (c & 1) * KV_STAGE + K_BYTES);
 #pragma unroll
@@ -225,12 +245,12 @@ __device__ __forceinline__ void bulk_item_roles(const BulkMaps& mp, const AttnAr
                          (c > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(sm.pv_done);
-                umma_commit(&sm.kv_empty[c & 1]);
+                umma_commit(&sm.v_empty[c & 1]);
             }
             // the arrivals on the K/V stage barriers are the item's last asynchronous ones: see them land, so that
             // a kernel that runs several items may initialise the barriers again
             for (int c = it.n_chunks - 2 < 0 ? 0 : it.n_chunks - 2; c < it.n_chunks && ok; ++c)
-                ok = mbar_wait(&sm.kv_empty[c & 1], (c >> 1) & 1, s_abort);
+                ok = mbar_wait(&sm.k_empty[c & 1], (c >> 1) & 1, s_abort) && mbar_wait(&sm.v_empty[c & 1], (c >> 1) & 1, s_abort);
             if (!ok) { set_error(a.err, DEV_E_WAIT_TIMEOUT); *s_abort = 1; }
         }
     } else if (warp < 10) {

@@ -115,6 +115,14 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
         const int Mtot = a.batch * RT;
         uint32_t noise_pos = 0xffffffffu;   // rows come in breadth-first order: equal depths are neighbours and
         float noise[4] = {0.f, 0.f, 0.f, 0.f};   // share their noise, which is a function of (position, token)
+        // The rows' floors (see below) are fetched once per tile, all rows at a time, and the floors this tile
+        // establishes go back in one batch at the end: no L2 round trip or atomic inside the row loop.
+        uint32_t* s_floor = reinterpret_cast<uint32_t*>(s_aux);          // [RT] in, [RT] out
+        for (int r = f; r < n_rows; r += 128) {
+            s_floor[r] = (r >= n_nodes && a.cand_floor) ? __ldcg(a.cand_floor + grow0 + r) : 0u;
+            s_floor[RT + r] = 0u;
+        }
+        epi_bar(bar_id);
         for (int r = warp; r < n_rows; r += 4) {
             float v[4];
             int id[4];
@@ -149,9 +157,10 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
             }
             // what other tiles have already established about this row's K'-th largest logit: a tile's own K'-th
             // best is a lower bound of it, so an entry strictly below the bound cannot make the final list
-            uint32_t floor_key = 0;
-            if (probe && a.cand_floor) floor_key = __ldcg(a.cand_floor + grow0 + r);
+            const uint32_t floor_key = s_floor[r];
             unsigned used = 0;
+            float keep_v = -INFINITY;          // lane j keeps the j-th entry (K' <= 32); one coalesced store per row
+            int keep_i = -1;
             for (int j = 0; j < kp; ++j) {
                 // lane-local best among unused, then warp-wide best by (value desc, id asc)
                 float bv = -INFINITY;
@@ -167,15 +176,16 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
                 const int wi = wkey == 0u ? 0x7fffffff : (int)wid;
                 const float wv = wkey == 0u ? -INFINITY : float_from_order_key(wkey);
                 if (wi == bi && bslot >= 0) used |= 1u << bslot;
-                if (probe && wi != 0x7fffffff && float_order_key(wv) < floor_key) {   // warp-uniform: this and all later entries are out
-                    if (lane == 0) for (int jj = j; jj < kp; ++jj) { out[jj].val = -INFINITY; out[jj].id = -1; }
-                    break;
-                }
-                if (lane == 0) { out[j].val = wv; out[j].id = wi == 0x7fffffff ? -1 : wi; }
+                if (probe && wi != 0x7fffffff && wkey < floor_key) break;   // warp-uniform: this and all later entries are out
+                if (lane == j) { keep_v = wv; keep_i = wi == 0x7fffffff ? -1 : wi; }
                 if (probe && a.cand_floor && j == kp - 1 && wi != 0x7fffffff && lane == 0)
-                    atomicMax(a.cand_floor + grow0 + r, float_order_key(wv));          // this tile holds kp entries >= wv
+                    s_floor[RT + r] = wkey;                                   // this tile holds kp entries >= wv
             }
+            if (lane < kp) { out[lane].val = keep_v; out[lane].id = keep_i; }
         }
+        epi_bar(bar_id);
+        for (int r = f; r < n_rows; r += 128)
+            if (s_floor[RT + r] > s_floor[r]) atomicMax(a.cand_floor + grow0 + r, s_floor[RT + r]);
     }
 }
 

@@ -71,6 +71,31 @@ int launch_attn_simt(int dtype, const AttnArgs& a, int batch, int n_split_launch
 // A plan holds the TMA descriptors of one query buffer and one layer's KV cache.
 struct AttnTc;
 bool attn_tc_supported(int h, int Hq, int Hkv);
+
+// Length of the cache splits of tree attention: a power of two >= 256 positions, at most 16 splits of max_len.
+// A split is one work item per (sequence, KV head, row tile) and leaves one partial per (row, head), so the
+// choice trades items for partial traffic.  One sequence keeps the finest split (the items are what fills the
+// SMs).  With several sequences the groups alone fill them, and the length is the one a small cost model prefers:
+// waves of items over the SMs x (1.45 us per 128-key chunk + 2.6 us per item) + the items' partial traffic.
+// It depends on nothing but the handle's capacity, batch and head count, so every row of a handle sees one
+// split grid, whatever the block it arrives in.
+inline int attn_split_len(int max_len, int batch, int Hkv) {
+    int S = 256;
+    while ((max_len + S - 1) / S > 16) S *= 2;
+    if (batch <= 1) return S;
+    const double groups = (double)batch * Hkv * 3;   // 3 row tiles: up to 96 rows x 4 heads of a group
+    int best = S;
+    double best_t = 0;
+    for (int c = S;; c *= 2) {
+        const int splits = (max_len + c - 1) / c;
+        const double items = splits * groups;
+        const double waves = (double)(long long)((items + 147) / 148);
+        const double t = waves * ((c / 128) * 1.45 + 2.6) + items * 0.02;
+        if (c == S || t < best_t) { best = c; best_t = t; }
+        if (splits == 1) break;
+    }
+    return best;
+}
 int attn_tc_create(AttnTc** out, const void* q, const void* kcache, const void* vcache, int batch, int Hq, int Hkv, int cap);
 void attn_tc_destroy(AttnTc* t);
 int attn_tc_launch(const AttnTc* t, const AttnArgs& a, int batch, int n_split_launch, cudaStream_t s, bool pdl);

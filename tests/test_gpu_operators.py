@@ -191,28 +191,39 @@ def test_tree_attention_rows_equal_decoding_each_path_alone():
 
 def test_tree_attention_one_item_and_persistent_kernels_agree_bitwise():
     """The cache below T0 is summed by one of two tensor-core kernels, picked by the number of (split, KV head,
-    row tile, sequence) items in the launch.  One sequence at KV 2048 stays below the switch (8 x 24 = 192 items),
-    three copies of it in one call are above it (576 items): every copy must come out bit for bit like the single
-    one, and a different sequence in the same call must not disturb them."""
-    Hq, Hkv, h, n_nodes, n_probes, L = 32, 8, 128, 64, 4, 2048
+    row tile, sequence) items in the launch.  The split length is a function of capacity, batch and head count, so
+    the two are compared inside one batch: 12 sequences at KV 2048 get one split each; with 68 rows (3 row tiles)
+    that is 288 items, above the switch, with the block cut to its first 20 rows (1 row tile, ancestors are
+    earlier rows) 96 items, below it.  The 20 rows must come out bit for bit alike from both calls, every copy of
+    a sequence like the others, and a different sequence in the same call must not disturb them."""
+    Hq, Hkv, h, n_nodes, n_probes, L, few = 32, 8, 128, 64, 4, 2048, 20
     M = n_nodes + n_probes
     cap = L + R
     q, kc, vc, kb, vb = synth.random_qkv((1, R, Hq, h), (1, Hkv, cap, h), (1, Hkv, M, h), seed=77, device="cuda")
     kc[:, :, L:L + M] = kb
     vc[:, :, L:L + M] = vb
     _, d, vis = _tree_block(n_nodes, n_probes, 5, seed=5)
+    assert not vis[:few, few:].any()
     anc = _anc_words(vis)[None]
     depth = np.zeros((1, R), np.int32)
     depth[0, :M] = d
-    single = _run_attention(1, q, kc, vc, anc, depth, M, L, Hq, Hkv, h)
     q2, kc2, vc2, _, _ = synth.random_qkv((1, R, Hq, h), (1, Hkv, cap, h), (1, Hkv, M, h), seed=78, device="cuda")
-    qq = torch.cat([q, q2, q, q]).contiguous()
-    kk = torch.cat([kc, kc2, kc, kc]).contiguous()
-    vv = torch.cat([vc, vc2, vc, vc]).contiguous()
-    many = _run_attention(1, qq, kk, vv, np.repeat(anc, 4, 0), np.repeat(depth, 4, 0), M, L, Hq, Hkv, h)
-    for s in (0, 2, 3):
-        assert torch.equal(many[s, :M], single[0, :M]), f"copy {s}"
-    assert not torch.equal(many[1, :M], single[0, :M])
+    order = [0, 1] + [0] * 10
+    qq = torch.cat([(q, q2)[i] for i in order]).contiguous()
+    kk = torch.cat([(kc, kc2)[i] for i in order]).contiguous()
+    vv = torch.cat([(vc, vc2)[i] for i in order]).contiguous()
+    ancs, depths = np.repeat(anc, len(order), 0), np.repeat(depth, len(order), 0)
+    many = _run_attention(1, qq, kk, vv, ancs, depths, M, L, Hq, Hkv, h)
+    anc_few = ancs.copy()
+    for r in range(few, M):
+        anc_few[:, r] = 0
+        anc_few[:, r, r // 64] = np.uint64(1) << np.uint64(r % 64)
+    fewer = _run_attention(1, qq, kk, vv, anc_few, depths, few, L, Hq, Hkv, h)
+    for s in range(len(order)):
+        assert torch.equal(many[s, :few], fewer[s, :few]), f"sequence {s}: the two kernels differ"
+        if s >= 2:
+            assert torch.equal(many[s, :M], many[0, :M]), f"copy {s}"
+    assert not torch.equal(many[1, :M], many[0, :M])
 
 
 def test_tree_attention_long_context_against_oracle():
