@@ -12,8 +12,9 @@ from HBM every step, far more than the L2 holds, so no cache flush is needed bet
 Prints ONE JSON line.  `value` is accepted tokens per second with everything resident on the device
 (K esp_step_async calls between two CUDA events on the library's stream; their tokens are read afterwards from
 the per-step result records and must equal greedy decoding with the same kernels); `e2e` is the same metric
-over a whole request through the public calls -- the prompt from host memory into esp_prefill, then K
-synchronous esp_step calls that return their tokens in host memory -- and `e2e_step` that request's steps
+over a whole request of the workload through the public calls -- the prompt from host memory into esp_prefill,
+then synchronous esp_step calls, each returning its tokens in host memory, until the workload's number of new
+tokens (256; 128 in the batch / long-context sweep) has been emitted -- and `e2e_step` that request's steps
 alone.  With N > 1 every rank runs an independent replica of the whole job (the method has no cross-GPU
 exchange); `value` sums the replicas' tokens over the slowest rank's time.
 
@@ -43,6 +44,8 @@ UNIT = "tok/s"
 # (Llama-3-8B shape, 68 rows, one sequence); None for workloads without a capture of the current kernel.
 GATEUP_DRAM_TRAFFIC = {"llama3-8b": 242.8e6}
 
+GEN_TOKENS = 256          # new tokens per request of the two model workloads
+GEN_TOKENS_SWEEP = 128    # ... of the batch / long-context sweep (--batch, --prompt-len)
 WORKLOADS = {
     # name: (shape attr in synth, prompt length, probes, topk, max_nodes)
     "llama3-8b": ("LLAMA3_8B", 1024, 4, 10, 64),
@@ -347,7 +350,8 @@ def run_ours(args, shape, plen, k, K, B):
     else:
         spec = P.spec_cfg(n_probes=k, topk=K, max_nodes=B, expand_width=0, n_anchor=1, temperature=args.temperature, seed=1)
     # room for one leg (at most k+1 tokens per step): the end-to-end leg starts again from the prompt
-    max_seq = plen + (k + 1) * (steps + warm + 20 + 16) + 64
+    gen = GEN_TOKENS_SWEEP if (args.batch > 1 or args.prompt_len > 0) else GEN_TOKENS
+    max_seq = max(plen + (k + 1) * (steps + warm + 20 + 16) + 64, plen + gen + (k + 1) * 24 + 64)   # the request, then up to 20 profiled steps
     stream = torch.cuda.Stream()
     nbatch = max(1, args.batch)
     h = P.Handle(shape, spec, w, max_seq_len=max_seq, max_batch=nbatch, stream=stream)
@@ -401,7 +405,7 @@ def run_ours(args, shape, plen, k, K, B):
     esp_stream.extend(timed_stream)
 
     # ---- end to end, a whole request through the public calls: the prompt goes from host memory into esp_prefill,
-    # then `steps` synchronous esp_step calls, each returning its tokens in host memory
+    # then synchronous esp_step calls, each returning its tokens in host memory, until every sequence has `gen` new tokens
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
@@ -409,14 +413,17 @@ def run_ours(args, shape, plen, k, K, B):
     prefill_all()
     torch.cuda.synchronize()
     prefill_ms = (time.perf_counter() - te0) * 1e3
-    e2e_tokens = nbatch                # the prefill emits every sequence's first token
-    for _ in range(steps):
+    emitted_seq = np.ones(nbatch, np.int64)       # the prefill emits every sequence's first token
+    e2e_steps = 0
+    while int(emitted_seq.min()) < gen and e2e_steps < 2 * gen:
         h.step()
-        e2e_tokens += int(h.n_out.sum())
+        emitted_seq += h.n_out[:nbatch].astype(np.int64)
+        e2e_steps += 1
+    e2e_tokens = int(emitted_seq.sum())
     torch.cuda.synchronize()
     te1 = time.perf_counter()
     e2e_ms = (te1 - te0) * 1e3
-    e2e_step_ms = (e2e_ms - prefill_ms) / steps
+    e2e_step_ms = (e2e_ms - prefill_ms) / max(e2e_steps, 1)
     h2d_request = nbatch * plen * 4                              # the prompts (int32 ids)
     d2h_step = nbatch * (P.ESP_MAX_PROBES + 4) * 4 + 4           # every sequence's result record + the status word
 
@@ -486,11 +493,13 @@ def run_ours(args, shape, plen, k, K, B):
             "kv_len": {"timed_start": L0, "timed_end": L1},
             "clocks": clocks,
             "e2e": {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": UNIT,
-                    "h2d_bytes_per_step": h2d_request / steps, "d2h_bytes_per_step": d2h_step,
+                    "h2d_bytes_per_step": h2d_request / max(e2e_steps, 1), "d2h_bytes_per_step": d2h_step,
                     "h2d_bytes_per_request": h2d_request, "request_ms": e2e_ms, "request_tokens": e2e_tokens,
-                    "note": "whole requests through the public calls, every rank: the prompt from host memory into "
-                            "esp_prefill, then `steps` synchronous esp_step calls that return their tokens in host "
-                            "memory; the prefill time is inside the timed region and its bytes are spread over the steps"},
+                    "request_steps": e2e_steps,
+                    "note": "whole requests of the workload through the public calls, every rank: the prompt from host "
+                            "memory into esp_prefill, then synchronous esp_step calls that return their tokens in host "
+                            f"memory until {gen} new tokens per sequence; the prefill time is inside the timed region "
+                            "and its bytes are spread over the steps"},
             "e2e_step": {"value": (e2e_tokens - nbatch * world) / ((e2e_ms - prefill_ms) * 1e-3), "unit": UNIT, "ms_per_step": e2e_step_ms,
                          "note": "the synchronous esp_step calls of that request alone (a step's inputs are the device "
                                  "state the step before left; its tokens land in host memory)"},
