@@ -20,13 +20,14 @@
 //               shared memory in the A-operand layout;
 //   O += P V    tcgen05.mma with V as the MN-major B operand (the cache keeps
 //               values as [key][dim]); O (128 x 128 fp32) stays in tensor
-//               memory and is rescaled there when the running max moves.
+//               memory; the softmax reference follows the running max lazily
+//               (it moves, and O is rescaled, only after a growth of 2^8).
 // Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 softmax (two threads per pair, 64 keys each).  S and the
 // K/V stages are double buffered, so Q K^T of chunk c+1 overlaps the softmax of
-// chunk c.  Every mbarrier wait is bounded; on a timeout the kernel records
-// DEV_E_WAIT_TIMEOUT, frees its tensor memory and returns.
-#include <new>
-#include <string.h>
+// chunk c; a stage's K half is released by its Q K^T and its V half by its P V,
+// and the producer keeps K one chunk ahead of V.  Every mbarrier wait is bounded;
+// on a timeout the kernel records DEV_E_WAIT_TIMEOUT, frees its tensor memory
+// and returns.
 #include <new>
 #include <string.h>
 
@@ -75,8 +76,8 @@ __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __g
     sm.q_full = sm.s_full + 2;
     sm.p_ready = sm.q_full + 1;
     sm.pv_done = sm.p_ready + 1;
-    sm.xchg = sm.pv_done + 1;                                        // the two threads of a pair exchanged a value
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm.xchg + 1);
+    sm.xchg = sm.pv_done + 1;                                        // [4] the two threads of a pair exchanged a value
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sm.xchg + 4);
     sm.s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
     sm.s_xchg = &s_xchg[0][0];
 
@@ -112,6 +113,9 @@ __global__ void __launch_bounds__(ONCE_THREADS, 1) k_attn_bulk_tc_once(const __g
         if (lane == 0) s_T0max = t0;
     }
     if (threadIdx.x == 0) {
+        prefetch_tensormap(&p.map_k);
+        prefetch_tensormap(&p.map_v);
+        prefetch_tensormap(&p.map_q);
         bulk_init_barriers(sm);
         *sm.s_abort = 0;
     }
@@ -170,8 +174,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
     uint64_t* q_free = q_full + 1;                                     // the item's last Q K^T has completed
     uint64_t* p_ready = q_free + 1;
     uint64_t* pv_done = p_ready + 1;
-    uint64_t* xchg = pv_done + 1;                                      // the two threads of a pair exchanged a value
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(xchg + 1);
+    uint64_t* xchg = pv_done + 1;                                      // [4] the two threads of a pair exchanged a value (per lane quadrant)
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(xchg + 4);
     volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
     const AttnArgs& a = p.a;
@@ -195,6 +199,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
         }
     }
     if (threadIdx.x == 0) {
+        prefetch_tensormap(&p.map_k);
+        prefetch_tensormap(&p.map_v);
+        prefetch_tensormap(&p.map_q);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
             mbar_init(&s_full[i], 1); mbar_init(&o_free[i], 128);
@@ -202,9 +209,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
         }
         mbar_init(q_full, 1);
         mbar_init(q_free, 1);
-        mbar_init(p_ready, 256);
+        mbar_init(p_ready, 8);
         mbar_init(pv_done, 1);
-        mbar_init(xchg, 256);
+        for (int i = 0; i < 4; ++i) mbar_init(&xchg[i], 2);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -395,7 +402,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
                 if (!__all_sync(0xffffffffu, mbar_wait(&s_full[g & 1], (g >> 1) & 1, s_abort))) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 ok = softmax_chunk(lane_addr + (g & 1) * 128, o_addr, it.beg + c * CK + hf * 64, T0row, a.scale_log2, m_run, l_run,
-                                   &s_xchg[xc & 1][0], xchg, xc & 1, g > 0, pv_done, (g - 1) & 1, c > 0,
+                                   &s_xchg[xc & 1][0], xchg + q4, xc & 1, g > 0, pv_done, (g - 1) & 1, c > 0,
                                    sP + hf * HALF_BYTES + pair * 128, pair, hf, p_ready, s_abort);
                 ++xc;
             }
@@ -403,8 +410,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_attn_bulk_tc(const __grid_co
             gc += it.n_chunks;
             // the row sum = first half's share + second half's share; the output warps take care of O
             s_xchg[xc & 1][hf * MP + pair] = l_run;
-            mbar_arrive(xchg);
-            if (!__all_sync(0xffffffffu, mbar_wait(xchg, xc & 1, s_abort))) { ok = false; break; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(xchg + q4);
+            if (!__all_sync(0xffffffffu, mbar_wait(xchg + q4, xc & 1, s_abort))) { ok = false; break; }
             const float l_tot = __fadd_rn(s_xchg[xc & 1][pair], s_xchg[xc & 1][MP + pair]);
             ++xc;
             if (pv && hf == 0) __stcg(a.part_ml + ((size_t)(it.seq * RT + r) * a.Hq + head) * a.n_split_max + it.split, make_float2(m_run, l_tot));

@@ -124,6 +124,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_gemm_tc(const __grid_constan
 
     if (threadIdx.x == 0) {
         pdl_launch_dependents();
+        prefetch_tensormap(&p.map_b);
+        if (!p.a_packed)
+            for (int i = 0; i < 3; ++i)
+                if (p.rows_w[i] > 0) prefetch_tensormap(&p.map_a[i]);
         for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], 128); }
         *s_abort = 0;

@@ -95,7 +95,7 @@ struct LayersParams {
 
 struct Shared {                    // behind the ring
     uint64_t full[STAGES], empty[STAGES], tfull[2], tempty[2];                         // GEMM ring and accumulators
-    uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], q_full, p_ready, pv_done, xchg;   // attention item
+    uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], q_full, p_ready, pv_done, xchg[4];   // attention item
     uint32_t tmem;
     int abort_flag, T0max, sync_ok;
     alignas(16) float red[128];
@@ -309,6 +309,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
     const int cw = warp - 2;                // consumer warp index (warps 2..13)
 
     if (threadIdx.x == 0) {
+        for (int i = 0; i < 4; ++i) prefetch_tensormap(&p.map_b[i]);
+        prefetch_tensormap(&p.map_q);
+        prefetch_tensormap(&p.map_k);
+        prefetch_tensormap(&p.map_v);
         for (int i = 0; i < STAGES; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 128); }
         sh.abort_flag = 0;
@@ -368,7 +372,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) k_layers_tc(const __grid_const
     attn::BulkShared bsm;
     bsm.buf = ring;
     bsm.k_full = sh.k_full; bsm.k_empty = sh.k_empty; bsm.v_full = sh.v_full; bsm.v_empty = sh.v_empty; bsm.s_full = sh.s_full; bsm.q_full = &sh.q_full; bsm.p_ready = &sh.p_ready;
-    bsm.pv_done = &sh.pv_done; bsm.xchg = &sh.xchg; bsm.s_xchg = &sh.xch[0][0]; bsm.s_abort = &sh.abort_flag;
+    bsm.pv_done = &sh.pv_done; bsm.xchg = sh.xchg; bsm.s_xchg = &sh.xch[0][0]; bsm.s_abort = &sh.abort_flag;
     attn::BulkMaps bmp;
     bmp.q = &p.map_q; bmp.k = &p.map_k; bmp.v = &p.map_v; bmp.group = p.group; bmp.rows_per_tile = p.rows_per_tile;
     AttnArgs aa;
