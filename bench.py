@@ -42,7 +42,7 @@ UNIT = "tok/s"
 
 # DRAM bytes (read + written) of one gate/up GEMM launch from the ncu capture summarised under profiles/
 # (Llama-3-8B shape, 68 rows, one sequence); None for workloads without a capture of the current kernel.
-GATEUP_DRAM_TRAFFIC = {"llama3-8b": 242.8e6}
+GATEUP_DRAM_TRAFFIC = {"llama3-8b": 242.9e6}
 
 GEN_TOKENS = 256          # new tokens per request of the two model workloads
 GEN_TOKENS_SWEEP = 128    # ... of the batch / long-context sweep (--batch, --prompt-len)
