@@ -117,10 +117,35 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
         float noise[4] = {0.f, 0.f, 0.f, 0.f};   // share their noise, which is a function of (position, token)
         // The rows' floors (see below) are fetched once per tile, all rows at a time, and the floors this tile
         // establishes go back in one batch at the end: no L2 round trip or atomic inside the row loop.
-        uint32_t* s_floor = reinterpret_cast<uint32_t*>(s_aux);          // [RT] in, [RT] out
+        const int S = n_rows <= 80 ? 80 : RT;                             // s_aux holds at least 3 * S words
+        uint32_t* s_floor = reinterpret_cast<uint32_t*>(s_aux);          // [S] in, [S] out, [S] "this probe row has entries at or above its floor"
+        uint32_t* s_need = s_floor + 2 * S;
         for (int r = f; r < n_rows; r += 128) {
             s_floor[r] = (r >= n_nodes && a.cand_floor) ? __ldcg(a.cand_floor + grow0 + r) : 0u;
-            s_floor[RT + r] = 0u;
+            s_floor[S + r] = 0u;
+        }
+        epi_bar(bar_id);
+        // Probe rows, one thread per row (the padded row stride keeps the threads on different banks): the tile's
+        // (max, sum-exp) for the row's log-sum-exp, and whether anything of the tile can still reach the row's final
+        // list.  A row whose maximum lies below its floor is done: its K' entries of this tile are empty.  With many
+        // probe rows per block nearly all rows of nearly all tiles end here, without one warp-wide reduction.
+        {
+            const int r = n_nodes + f;
+            if (r < n_rows) {
+                const int n_valid = a.n_out - n0 < TILE_N ? a.n_out - n0 : TILE_N;
+                const float* row = s_acc + r * ACC_LD;
+                float tmax = -INFINITY;
+                for (int i = 0; i < n_valid; ++i) tmax = fmaxf(tmax, row[i]);
+                float sum = 0.f;
+                for (int i = 0; i < n_valid; ++i) sum += expf(row[i] - tmax);
+                a.cand_ms[(size_t)tile * Mtot + grow0 + r] = make_float2(tmax, sum);
+                const bool need = float_order_key(tmax) >= s_floor[r];
+                s_need[r] = need ? 1u : 0u;
+                if (!need) {
+                    Cand* out = a.cand + ((size_t)tile * Mtot + grow0 + r) * a.KP;
+                    for (int j = 0; j < a.KP; ++j) { out[j].val = -INFINITY; out[j].id = -1; }
+                }
+            }
         }
         epi_bar(bar_id);
         for (int r = warp; r < n_rows; r += 4) {
@@ -132,6 +157,7 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
                 v[i] = id[i] < a.n_out ? s_acc[r * ACC_LD + lane + 32 * i] : -INFINITY;
                 if (a.logits_dump && id[i] < a.n_out) a.logits_dump[(size_t)(grow0 + r) * a.n_out + id[i]] = v[i];
             }
+            if (r >= n_nodes && !s_need[r]) continue;       // warp-uniform
             const bool probe = r >= n_nodes;
             const int kp = probe ? a.KP : 1;
             Cand* out = a.cand + ((size_t)tile * Mtot + grow0 + r) * a.KP;
@@ -146,14 +172,6 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     if (id[i] < a.n_out) v[i] = sample_score(v[i], a.samp_inv_temp, noise[i]);
-            }
-            if (probe) {
-                float tmax = warp_max(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])));
-                float s = 0.f;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) s += id[i] < a.n_out ? expf(v[i] - tmax) : 0.f;
-                s = warp_sum(s);
-                if (lane == 0) a.cand_ms[(size_t)tile * Mtot + grow0 + r] = make_float2(tmax, s);
             }
             // what other tiles have already established about this row's K'-th largest logit: a tile's own K'-th
             // best is a lower bound of it, so an entry strictly below the bound cannot make the final list
@@ -179,13 +197,13 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
                 if (probe && wi != 0x7fffffff && wkey < floor_key) break;   // warp-uniform: this and all later entries are out
                 if (lane == j) { keep_v = wv; keep_i = wi == 0x7fffffff ? -1 : wi; }
                 if (probe && a.cand_floor && j == kp - 1 && wi != 0x7fffffff && lane == 0)
-                    s_floor[RT + r] = wkey;                                   // this tile holds kp entries >= wv
+                    s_floor[S + r] = wkey;                                    // this tile holds kp entries >= wv
             }
             if (lane < kp) { out[lane].val = keep_v; out[lane].id = keep_i; }
         }
         epi_bar(bar_id);
         for (int r = f; r < n_rows; r += 128)
-            if (s_floor[RT + r] > s_floor[r]) atomicMax(a.cand_floor + grow0 + r, s_floor[RT + r]);
+            if (s_floor[S + r] > s_floor[r]) atomicMax(a.cand_floor + grow0 + r, s_floor[S + r]);
     }
 }
 
