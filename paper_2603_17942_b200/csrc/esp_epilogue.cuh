@@ -129,7 +129,8 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
         // (max, sum-exp) for the row's log-sum-exp, and whether anything of the tile can still reach the row's final
         // list.  A row whose maximum lies below its floor is done: its K' entries of this tile are empty.  With many
         // probe rows per block nearly all rows of nearly all tiles end here, without one warp-wide reduction.
-        {
+        const bool many_probes = n_rows - n_nodes >= 16;     // block-uniform; a handful of probe rows is cheaper warp by warp
+        if (many_probes) {
             const int r = n_nodes + f;
             if (r < n_rows) {
                 const int n_valid = a.n_out - n0 < TILE_N ? a.n_out - n0 : TILE_N;
@@ -157,7 +158,7 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
                 v[i] = id[i] < a.n_out ? s_acc[r * ACC_LD + lane + 32 * i] : -INFINITY;
                 if (a.logits_dump && id[i] < a.n_out) a.logits_dump[(size_t)(grow0 + r) * a.n_out + id[i]] = v[i];
             }
-            if (r >= n_nodes && !s_need[r]) continue;       // warp-uniform
+            if (many_probes && r >= n_nodes && !s_need[r]) continue;       // warp-uniform
             const bool probe = r >= n_nodes;
             const int kp = probe ? a.KP : 1;
             Cand* out = a.cand + ((size_t)tile * Mtot + grow0 + r) * a.KP;
@@ -172,6 +173,14 @@ __device__ void run_epilogue(float* s_acc, float* s_aux, int tile, int seq, cons
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     if (id[i] < a.n_out) v[i] = sample_score(v[i], a.samp_inv_temp, noise[i]);
+            }
+            if (probe && !many_probes) {
+                float tmax = warp_max(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])));
+                float s = 0.f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) s += id[i] < a.n_out ? expf(v[i] - tmax) : 0.f;
+                s = warp_sum(s);
+                if (lane == 0) a.cand_ms[(size_t)tile * Mtot + grow0 + r] = make_float2(tmax, s);
             }
             // what other tiles have already established about this row's K'-th largest logit: a tile's own K'-th
             // best is a lower bound of it, so an entry strictly below the bound cannot make the final list
